@@ -1,0 +1,176 @@
+/*
+ * cake_kmeans.h -- C ABI of the B200 (sm_100a) Flash-KMeans Lloyd hot path.
+ *
+ * The operations are the two kernels of the paper's Section 5, paragraph "Flash-KMeans
+ * clean-start workload", and the Lloyd iteration they make up:
+ *   assign           squared Euclidean distance from every point to all K centroids, arg-min
+ *                    (bf16 inputs, fp32 accumulation; the N x K distance matrix is never stored);
+ *   centroid_update  per-cluster sums and counts of the assigned points (then, in this library,
+ *                    the division into means, with empty clusters keeping their previous centroid);
+ *   lloyd            iters x (assign, update).
+ *
+ * Conventions shared by every entry point
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer on the current device.
+ *     The caller owns all buffers; the library allocates nothing and frees nothing.
+ *   - cake_bf16 is a raw bfloat16 bit pattern.  Matrices are row-major and contiguous:
+ *     X[B][N][D], C[B][K][D], idx[B][N], counts[B][K].  The un-batched calls are B = 1.
+ *     Base pointers must be 16-byte aligned.  Inputs must be finite.
+ *   - `ws` is caller-provided scratch of at least cake_kmeans_workspace_bytes(...) bytes,
+ *     256-byte aligned.  Its first word is a sticky device status (see cake_kmeans_device_status);
+ *     the caller zeroes the first 256 bytes once, before the first call that uses the buffer.
+ *     Calls that run concurrently must use distinct workspaces.
+ *   - Work is enqueued on `stream` (a cudaStream_t; NULL = the legacy default stream) and the
+ *     call returns without synchronising.  The return value reports what the host could check:
+ *     CAKE_OK or a negative CAKE_ERR_* code; on error nothing was enqueued.
+ *   - N = 0 is valid and does nothing (update then treats every cluster as empty).
+ *   - Ties in the arg-min go to the lowest centroid index.  Indices and counts are int32.
+ *   - `flags` selects a code path for testing; 0 lets the library choose.
+ */
+#ifndef CAKE_KMEANS_H_
+#define CAKE_KMEANS_H_
+
+#include <stddef.h>
+
+#if defined(__GNUC__)
+#define CAKE_API __attribute__((visibility("default")))
+#else
+#define CAKE_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* cake_stream_t;
+typedef unsigned short cake_bf16;
+
+enum {
+    CAKE_OK = 0,
+    CAKE_ERR_NULL = -1,        /* a required pointer is NULL                                   */
+    CAKE_ERR_SHAPE = -2,       /* B < 1, N < 0, D < 1, K < 1, iters < 0, or sizes over int32    */
+    CAKE_ERR_ALIGN = -3,       /* a base pointer is not 16-byte aligned (ws: 256)              */
+    CAKE_ERR_UNSUPPORTED = -4, /* the requested path cannot run this shape                     */
+    CAKE_ERR_WORKSPACE = -5,   /* ws_bytes too small                                           */
+    CAKE_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed                          */
+    CAKE_ERR_BAD_INDEX = -7,   /* device status: an idx value was outside [0,K) and was skipped */
+    CAKE_ERR_TIMEOUT = -8,     /* device status: a bounded in-kernel wait expired              */
+    CAKE_ERR_DEVICE = -9       /* no CUDA device, or not compute capability 10.x               */
+};
+
+enum {
+    CAKE_ASSIGN_AUTO = 0,
+    CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 256 */
+    CAKE_ASSIGN_SIMT = 2,      /* plain CUDA-core fallback, any D                               */
+    CAKE_ASSIGN_MASK = 0xF,
+    CAKE_UPDATE_AUTO = 0,
+    CAKE_UPDATE_SMEM = 1 << 4, /* shared-memory partial sums; needs K*D*4 + K*4 bytes of smem   */
+    CAKE_UPDATE_SORT = 2 << 4, /* counting sort by cluster + segmented reduction, any K         */
+    CAKE_UPDATE_MASK = 0xF << 4
+};
+
+/* Library version (major*10000 + minor*100 + patch).  No paper counterpart. */
+CAKE_API int cake_version(void);
+
+/* Static, human-readable text for a CAKE_* code.  Never NULL.  No paper counterpart. */
+CAKE_API const char* cake_strerror(int code);
+
+/*
+ * Bytes of device scratch that any of the calls below needs for B problems of N points,
+ * D features and K clusters (one figure covers assign, update and lloyd).
+ *   out_bytes  host pointer, receives the size.
+ * Returns CAKE_OK, CAKE_ERR_NULL or CAKE_ERR_SHAPE.  Touches no device.
+ */
+CAKE_API int cake_kmeans_workspace_bytes(long long B, long long N, int D, int K, size_t* out_bytes);
+
+/*
+ * assign (Section 5, "Flash-KMeans clean-start workload": squared Euclidean distances to all K
+ * centroids and the arg-min).  Computed as ||x||^2 - 2 x.c + ||c||^2 with x.c on the tensor
+ * cores in fp32; the row constant ||x||^2 does not enter the comparison.
+ *   X        [B][N][D] bf16, in
+ *   C        [B][K][D] bf16, in
+ *   out_idx  [B][N] int32, out: arg-min_k, lowest k on ties
+ *   out_dist [B][N] fp32, out, may be NULL: max(0, squared distance to the chosen centroid)
+ */
+CAKE_API int cake_kmeans_assign(const cake_bf16* X, const cake_bf16* C, long long N, int D, int K,
+                       int* out_idx, float* out_dist, void* ws, size_t ws_bytes,
+                       cake_stream_t stream, unsigned flags);
+CAKE_API int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, long long B, long long N,
+                               int D, int K, int* out_idx, float* out_dist, void* ws,
+                               size_t ws_bytes, cake_stream_t stream, unsigned flags);
+
+/*
+ * centroid_update (same paragraph: per-cluster sums and counts), followed by the division.
+ *   X          [B][N][D] bf16, in
+ *   idx        [B][N] int32, in; values outside [0,K) are skipped and raise the device status
+ *              CAKE_ERR_BAD_INDEX
+ *   C_prev     [B][K][D] bf16, in, may be NULL: centroid kept by an empty cluster (zeros if NULL)
+ *   out_C      [B][K][D] fp32, out: sums / counts in fp32
+ *   out_C_bf16 [B][K][D] bf16, out, may be NULL: out_C rounded to nearest even
+ *   out_counts [B][K] int32, out
+ * fp32 summation order is unspecified (results agree to fp32 rounding between calls).
+ */
+CAKE_API int cake_kmeans_update(const cake_bf16* X, const int* idx, long long N, int D, int K,
+                       const cake_bf16* C_prev, float* out_C, cake_bf16* out_C_bf16,
+                       int* out_counts, void* ws, size_t ws_bytes, cake_stream_t stream,
+                       unsigned flags);
+CAKE_API int cake_kmeans_update_batched(const cake_bf16* X, const int* idx, long long B, long long N, int D,
+                               int K, const cake_bf16* C_prev, float* out_C,
+                               cake_bf16* out_C_bf16, int* out_counts, void* ws, size_t ws_bytes,
+                               cake_stream_t stream, unsigned flags);
+
+/*
+ * lloyd (same paragraph: a Lloyd iteration is assign followed by centroid_update).
+ * For t = 0 .. iters-1: assign against C_t (C_0 = C0), out_inertia[t] = sum_i out_dist_t[i],
+ * then update -> C_{t+1}; the next assign reads C_{t+1} rounded to bf16.  Exactly `iters`
+ * iterations run; there is no convergence test.
+ *   out_C       [B][K][D] fp32: C_iters (fp32 means of the last update)
+ *   out_C_bf16  [B][K][D] bf16, may be NULL: its bf16 rounding
+ *   out_idx     [B][N], out_dist [B][N] (may be NULL): those of the LAST assign (against C_{iters-1})
+ *   out_counts  [B][K]: counts of the last update
+ *   out_inertia [B][iters] fp64, may be NULL
+ * iters = 0 copies C0 to the outputs and leaves idx / dist / counts untouched.
+ */
+CAKE_API int cake_kmeans_lloyd(const cake_bf16* X, const cake_bf16* C0, long long N, int D, int K, int iters,
+                      float* out_C, cake_bf16* out_C_bf16, int* out_idx, float* out_dist,
+                      int* out_counts, double* out_inertia, void* ws, size_t ws_bytes,
+                      cake_stream_t stream, unsigned flags);
+CAKE_API int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long B, long long N,
+                              int D, int K, int iters, float* out_C, cake_bf16* out_C_bf16,
+                              int* out_idx, float* out_dist, int* out_counts, double* out_inertia,
+                              void* ws, size_t ws_bytes, cake_stream_t stream, unsigned flags);
+
+/*
+ * lloyd with HOST buffers (same operation; measures the end-to-end cost a caller with data in
+ * host memory sees).  X_host, C0_host and every out_*_host pointer are HOST pointers (pinned
+ * memory makes the copies asynchronous); `dev` is device scratch of at least
+ * cake_kmeans_lloyd_host_device_bytes(...) bytes, 256-byte aligned, into which the library copies
+ * the inputs, runs cake_kmeans_lloyd_batched and from which it copies the results back, all on
+ * `stream`.  The call returns after enqueueing; synchronise the stream before reading outputs.
+ * Nullable outputs as in cake_kmeans_lloyd.
+ */
+CAKE_API int cake_kmeans_lloyd_host_device_bytes(long long B, long long N, int D, int K, int iters,
+                                        size_t* out_bytes);
+CAKE_API int cake_kmeans_lloyd_host(const cake_bf16* X_host, const cake_bf16* C0_host, long long B,
+                           long long N, int D, int K, int iters, float* out_C_host,
+                           cake_bf16* out_C_bf16_host, int* out_idx_host, float* out_dist_host,
+                           int* out_counts_host, double* out_inertia_host, void* dev,
+                           size_t dev_bytes, cake_stream_t stream, unsigned flags);
+
+/*
+ * Reads the sticky device status word of a workspace: synchronises `stream`, copies the word to
+ * *host_out (host pointer) and clears it.  *host_out is CAKE_OK, CAKE_ERR_BAD_INDEX or
+ * CAKE_ERR_TIMEOUT.  No paper counterpart.
+ */
+CAKE_API int cake_kmeans_device_status(void* ws, cake_stream_t stream, int* host_out);
+
+/*
+ * Self-test of the bounded in-kernel wait: one thread waits on an mbarrier that nothing ever
+ * completes, for at most `limit_ms` milliseconds, then records CAKE_ERR_TIMEOUT in the status
+ * word of `ws` and returns normally (the context stays usable).  No paper counterpart.
+ */
+CAKE_API int cake_kmeans_selftest_bounded_wait(void* ws, size_t ws_bytes, int limit_ms, cake_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAKE_KMEANS_H_ */

@@ -1,0 +1,320 @@
+// The C ABI: argument checks, workspace carving, path selection and the Lloyd loop.
+// Every step of the path runs in this library's kernels; nothing here allocates.
+#include <limits.h>
+
+#include "internal.h"
+
+namespace cake {
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct Workspace {
+    int* status;          // [64] header, word 0 = sticky device status
+    float* cn;            // [B][Kpad]
+    float* sums;          // [B][K][D]
+    int* offsets;         // [B][K+1]
+    int* cursor;          // [B][K]
+    int* perm;            // [B][N]
+    cake_bf16* cbuf[2];   // [B][K][D] each
+    float* dist;          // [B][N]
+    size_t bytes;
+};
+
+Workspace carve(void* base, i64 B, i64 N, int D, int K) {
+    Workspace w;
+    size_t o = 0;
+    char* p = static_cast<char*>(base);
+    auto take = [&](size_t n) { char* r = p ? p + o : nullptr; o += up(n); return r; };
+    const size_t kd = static_cast<size_t>(B) * K * D;
+    w.status = reinterpret_cast<int*>(take(256));
+    w.cn = reinterpret_cast<float*>(take(static_cast<size_t>(B) * padded_k(K) * 4));
+    w.sums = reinterpret_cast<float*>(take(kd * 4));
+    w.offsets = reinterpret_cast<int*>(take(static_cast<size_t>(B) * (K + 1) * 4));
+    w.cursor = reinterpret_cast<int*>(take(static_cast<size_t>(B) * K * 4));
+    w.perm = reinterpret_cast<int*>(take(static_cast<size_t>(B) * N * 4));
+    w.cbuf[0] = reinterpret_cast<cake_bf16*>(take(kd * 2));
+    w.cbuf[1] = reinterpret_cast<cake_bf16*>(take(kd * 2));
+    w.dist = reinterpret_cast<float*>(take(static_cast<size_t>(B) * N * 4));
+    w.bytes = o;
+    return w;
+}
+
+int check_shape(i64 B, i64 N, int D, int K) {
+    if (B < 1 || N < 0 || D < 1 || K < 1) return CAKE_ERR_SHAPE;
+    if (B > 65535 || N > INT_MAX - 1024 || static_cast<i64>(K) > INT_MAX - 1024) return CAKE_ERR_SHAPE;
+    if (static_cast<double>(B) * K * D > 4.0e12 || static_cast<double>(B) * N * D > 4.0e13) return CAKE_ERR_SHAPE;
+    return CAKE_OK;
+}
+inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
+
+int check_ws(void* ws, size_t ws_bytes, i64 B, i64 N, int D, int K, Workspace* out) {
+    if (!ws) return CAKE_ERR_NULL;
+    if (misaligned(ws, kAlign)) return CAKE_ERR_ALIGN;
+    *out = carve(ws, B, N, D, K);
+    if (ws_bytes < out->bytes) return CAKE_ERR_WORKSPACE;
+    return CAKE_OK;
+}
+
+int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, int* out_idx,
+              float* out_dist, const Workspace& w, cudaStream_t s, unsigned flags) {
+    unsigned path = flags & CAKE_ASSIGN_MASK;
+    if (path == CAKE_ASSIGN_AUTO) path = assign_tc_supports(D) ? CAKE_ASSIGN_TCGEN05 : CAKE_ASSIGN_SIMT;
+    if (path == CAKE_ASSIGN_SIMT) return launch_assign_simt(X, C, B, N, D, K, out_idx, out_dist, s);
+    if (path != CAKE_ASSIGN_TCGEN05) return CAKE_ERR_UNSUPPORTED;
+    if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
+    if (N == 0) return CAKE_OK;
+    const int Kpad = padded_k(K);
+    if (launch_centroid_norms(C, B, K, D, Kpad, w.cn, s) != cudaSuccess) return CAKE_ERR_CUDA;
+    return launch_assign_tc(X, C, B, N, D, K, w.cn, Kpad, out_idx, out_dist, w.status, s);
+}
+
+int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, const cake_bf16* C_prev,
+              float* out_C, cake_bf16* out_C_bf16, int* out_counts, const Workspace& w, cudaStream_t s,
+              unsigned flags) {
+    DeviceInfo di;
+    int rc = current_device_info(&di);
+    if (rc != CAKE_OK) return rc;
+    unsigned path = flags & CAKE_UPDATE_MASK;
+    if (path == CAKE_UPDATE_AUTO)
+        path = update_smem_supports(D, K, di.smem_optin) ? CAKE_UPDATE_SMEM : CAKE_UPDATE_SORT;
+    if (path == CAKE_UPDATE_SMEM) {
+        rc = launch_update_smem(X, idx, B, N, D, K, w.sums, out_counts, w.status, s);
+    } else if (path == CAKE_UPDATE_SORT) {
+        UpdateScratch scr{w.sums, w.offsets, w.cursor, w.perm};
+        rc = launch_update_sort(X, idx, B, N, D, K, scr, out_counts, w.status, s);
+    } else {
+        rc = CAKE_ERR_UNSUPPORTED;
+    }
+    if (rc != CAKE_OK) return rc;
+    if (launch_finalize(w.sums, out_counts, C_prev, B, K, D, out_C, out_C_bf16, s) != cudaSuccess)
+        return CAKE_ERR_CUDA;
+    return CAKE_OK;
+}
+
+}  // namespace
+}  // namespace cake
+
+using namespace cake;
+
+extern "C" {
+
+int cake_version(void) { return 100; }
+
+const char* cake_strerror(int code) {
+    switch (code) {
+        case CAKE_OK: return "ok";
+        case CAKE_ERR_NULL: return "a required pointer is NULL";
+        case CAKE_ERR_SHAPE: return "invalid or too large shape";
+        case CAKE_ERR_ALIGN: return "a base pointer is not sufficiently aligned";
+        case CAKE_ERR_UNSUPPORTED: return "the requested path does not support this shape";
+        case CAKE_ERR_WORKSPACE: return "workspace too small";
+        case CAKE_ERR_CUDA: return "a CUDA call failed";
+        case CAKE_ERR_BAD_INDEX: return "an index was outside [0,K) and was skipped";
+        case CAKE_ERR_TIMEOUT: return "a bounded in-kernel wait expired";
+        case CAKE_ERR_DEVICE: return "no usable CUDA device (compute capability 10.x needed)";
+        default: return "unknown cake_kmeans code";
+    }
+}
+
+int cake_kmeans_workspace_bytes(long long B, long long N, int D, int K, size_t* out_bytes) {
+    if (!out_bytes) return CAKE_ERR_NULL;
+    int rc = check_shape(B, N, D, K);
+    if (rc != CAKE_OK) return rc;
+    *out_bytes = carve(nullptr, B, N, D, K).bytes;
+    return CAKE_OK;
+}
+
+int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, long long B, long long N, int D,
+                               int K, int* out_idx, float* out_dist, void* ws, size_t ws_bytes,
+                               cake_stream_t stream, unsigned flags) {
+    int rc = check_shape(B, N, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (!C || !ws || (N > 0 && (!X || !out_idx))) return CAKE_ERR_NULL;
+    if (misaligned(X, 16) || misaligned(C, 16) || misaligned(out_idx, 4) || misaligned(out_dist, 4))
+        return CAKE_ERR_ALIGN;
+    Workspace w;
+    rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
+    if (rc != CAKE_OK) return rc;
+    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, w,
+                     reinterpret_cast<cudaStream_t>(stream), flags);
+}
+
+int cake_kmeans_assign(const cake_bf16* X, const cake_bf16* C, long long N, int D, int K, int* out_idx,
+                       float* out_dist, void* ws, size_t ws_bytes, cake_stream_t stream, unsigned flags) {
+    return cake_kmeans_assign_batched(X, C, 1, N, D, K, out_idx, out_dist, ws, ws_bytes, stream, flags);
+}
+
+int cake_kmeans_update_batched(const cake_bf16* X, const int* idx, long long B, long long N, int D, int K,
+                               const cake_bf16* C_prev, float* out_C, cake_bf16* out_C_bf16,
+                               int* out_counts, void* ws, size_t ws_bytes, cake_stream_t stream,
+                               unsigned flags) {
+    int rc = check_shape(B, N, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (!out_C || !out_counts || !ws || (N > 0 && (!X || !idx))) return CAKE_ERR_NULL;
+    if (misaligned(X, 16) || misaligned(C_prev, 16) || misaligned(out_C, 16) || misaligned(out_C_bf16, 16) ||
+        misaligned(idx, 4) || misaligned(out_counts, 4))
+        return CAKE_ERR_ALIGN;
+    Workspace w;
+    rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
+    if (rc != CAKE_OK) return rc;
+    return do_update(X, idx, static_cast<int>(B), N, D, K, C_prev, out_C, out_C_bf16, out_counts, w,
+                     reinterpret_cast<cudaStream_t>(stream), flags);
+}
+
+int cake_kmeans_update(const cake_bf16* X, const int* idx, long long N, int D, int K,
+                       const cake_bf16* C_prev, float* out_C, cake_bf16* out_C_bf16, int* out_counts,
+                       void* ws, size_t ws_bytes, cake_stream_t stream, unsigned flags) {
+    return cake_kmeans_update_batched(X, idx, 1, N, D, K, C_prev, out_C, out_C_bf16, out_counts, ws,
+                                      ws_bytes, stream, flags);
+}
+
+int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long B, long long N, int D,
+                              int K, int iters, float* out_C, cake_bf16* out_C_bf16, int* out_idx,
+                              float* out_dist, int* out_counts, double* out_inertia, void* ws,
+                              size_t ws_bytes, cake_stream_t stream, unsigned flags) {
+    int rc = check_shape(B, N, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (iters < 0) return CAKE_ERR_SHAPE;
+    if (!C0 || !out_C || !ws) return CAKE_ERR_NULL;
+    if (iters > 0 && (!out_counts || (N > 0 && (!X || !out_idx)))) return CAKE_ERR_NULL;
+    if (misaligned(X, 16) || misaligned(C0, 16) || misaligned(out_C, 16) || misaligned(out_C_bf16, 16) ||
+        misaligned(out_idx, 4) || misaligned(out_dist, 4) || misaligned(out_counts, 4) ||
+        misaligned(out_inertia, 8))
+        return CAKE_ERR_ALIGN;
+    Workspace w;
+    rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
+    if (rc != CAKE_OK) return rc;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int Bi = static_cast<int>(B);
+    const size_t kd = static_cast<size_t>(B) * K * D;
+
+    if (cudaMemcpyAsync(w.cbuf[0], C0, kd * 2, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return CAKE_ERR_CUDA;
+    if (out_inertia && iters > 0 &&
+        cudaMemsetAsync(out_inertia, 0, static_cast<size_t>(B) * iters * sizeof(double), s) != cudaSuccess)
+        return CAKE_ERR_CUDA;
+    int cur = 0;
+    if (iters == 0) {
+        // out_C = C0 widened: the division kernel with all-zero counts takes the keep-previous branch
+        if (cudaMemsetAsync(w.cursor, 0, static_cast<size_t>(B) * K * 4, s) != cudaSuccess) return CAKE_ERR_CUDA;
+        if (launch_finalize(w.sums, w.cursor, w.cbuf[0], Bi, K, D, out_C, nullptr, s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
+    }
+    float* dist = out_dist ? out_dist : (out_inertia ? w.dist : nullptr);
+    for (int t = 0; t < iters; ++t) {
+        rc = do_assign(X, w.cbuf[cur], Bi, N, D, K, out_idx, dist, w, s, flags);
+        if (rc != CAKE_OK) return rc;
+        if (out_inertia && launch_inertia(dist, Bi, N, out_inertia + t, iters, s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
+        rc = do_update(X, out_idx, Bi, N, D, K, w.cbuf[cur], out_C, w.cbuf[cur ^ 1], out_counts, w, s, flags);
+        if (rc != CAKE_OK) return rc;
+        cur ^= 1;
+    }
+    if (out_C_bf16 &&
+        cudaMemcpyAsync(out_C_bf16, w.cbuf[cur], kd * 2, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return CAKE_ERR_CUDA;
+    return CAKE_OK;
+}
+
+int cake_kmeans_lloyd(const cake_bf16* X, const cake_bf16* C0, long long N, int D, int K, int iters,
+                      float* out_C, cake_bf16* out_C_bf16, int* out_idx, float* out_dist, int* out_counts,
+                      double* out_inertia, void* ws, size_t ws_bytes, cake_stream_t stream, unsigned flags) {
+    return cake_kmeans_lloyd_batched(X, C0, 1, N, D, K, iters, out_C, out_C_bf16, out_idx, out_dist,
+                                     out_counts, out_inertia, ws, ws_bytes, stream, flags);
+}
+
+namespace {
+struct HostDev {
+    cake_bf16 *X, *C0, *Cb;
+    float *C, *dist;
+    int *idx, *counts;
+    double* inertia;
+    void* ws;
+    size_t ws_bytes, bytes;
+};
+HostDev carve_host(void* base, i64 B, i64 N, int D, int K, int iters) {
+    HostDev h;
+    size_t o = 0;
+    char* p = static_cast<char*>(base);
+    auto take = [&](size_t n) { char* r = p ? p + o : nullptr; o += up(n); return r; };
+    const size_t kd = static_cast<size_t>(B) * K * D, nd = static_cast<size_t>(B) * N * D;
+    h.X = reinterpret_cast<cake_bf16*>(take(nd * 2));
+    h.C0 = reinterpret_cast<cake_bf16*>(take(kd * 2));
+    h.Cb = reinterpret_cast<cake_bf16*>(take(kd * 2));
+    h.C = reinterpret_cast<float*>(take(kd * 4));
+    h.dist = reinterpret_cast<float*>(take(static_cast<size_t>(B) * N * 4));
+    h.idx = reinterpret_cast<int*>(take(static_cast<size_t>(B) * N * 4));
+    h.counts = reinterpret_cast<int*>(take(static_cast<size_t>(B) * K * 4));
+    h.inertia = reinterpret_cast<double*>(take(static_cast<size_t>(B) * (iters > 0 ? iters : 1) * 8));
+    h.ws_bytes = carve(nullptr, B, N, D, K).bytes;
+    h.ws = take(h.ws_bytes);
+    h.bytes = o;
+    return h;
+}
+}  // namespace
+
+int cake_kmeans_lloyd_host_device_bytes(long long B, long long N, int D, int K, int iters, size_t* out_bytes) {
+    if (!out_bytes) return CAKE_ERR_NULL;
+    int rc = check_shape(B, N, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (iters < 0) return CAKE_ERR_SHAPE;
+    *out_bytes = carve_host(nullptr, B, N, D, K, iters).bytes;
+    return CAKE_OK;
+}
+
+int cake_kmeans_lloyd_host(const cake_bf16* X_host, const cake_bf16* C0_host, long long B, long long N,
+                           int D, int K, int iters, float* out_C_host, cake_bf16* out_C_bf16_host,
+                           int* out_idx_host, float* out_dist_host, int* out_counts_host,
+                           double* out_inertia_host, void* dev, size_t dev_bytes, cake_stream_t stream,
+                           unsigned flags) {
+    int rc = check_shape(B, N, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (iters < 0) return CAKE_ERR_SHAPE;
+    if (!C0_host || !out_C_host || !dev || (N > 0 && !X_host)) return CAKE_ERR_NULL;
+    if (misaligned(dev, kAlign)) return CAKE_ERR_ALIGN;
+    HostDev h = carve_host(dev, B, N, D, K, iters);
+    if (dev_bytes < h.bytes) return CAKE_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t kd = static_cast<size_t>(B) * K * D, nd = static_cast<size_t>(B) * N * D;
+    const size_t bn = static_cast<size_t>(B) * N, bk = static_cast<size_t>(B) * K;
+    if (nd && cudaMemcpyAsync(h.X, X_host, nd * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return CAKE_ERR_CUDA;
+    if (cudaMemcpyAsync(h.C0, C0_host, kd * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return CAKE_ERR_CUDA;
+    if (cudaMemsetAsync(h.ws, 0, 256, s) != cudaSuccess) return CAKE_ERR_CUDA;
+    rc = cake_kmeans_lloyd_batched(h.X, h.C0, B, N, D, K, iters, h.C, out_C_bf16_host ? h.Cb : nullptr, h.idx,
+                                   out_dist_host ? h.dist : nullptr, h.counts,
+                                   out_inertia_host ? h.inertia : nullptr, h.ws, h.ws_bytes, stream, flags);
+    if (rc != CAKE_OK) return rc;
+    bool ok = cudaMemcpyAsync(out_C_host, h.C, kd * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    if (out_C_bf16_host) ok = ok && cudaMemcpyAsync(out_C_bf16_host, h.Cb, kd * 2, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    if (iters > 0) {
+        if (out_idx_host && bn) ok = ok && cudaMemcpyAsync(out_idx_host, h.idx, bn * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+        if (out_dist_host && bn) ok = ok && cudaMemcpyAsync(out_dist_host, h.dist, bn * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+        if (out_counts_host) ok = ok && cudaMemcpyAsync(out_counts_host, h.counts, bk * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+        if (out_inertia_host) ok = ok && cudaMemcpyAsync(out_inertia_host, h.inertia, static_cast<size_t>(B) * iters * 8, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    }
+    return ok ? CAKE_OK : CAKE_ERR_CUDA;
+}
+
+int cake_kmeans_device_status(void* ws, cake_stream_t stream, int* host_out) {
+    if (!ws || !host_out) return CAKE_ERR_NULL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    int v = 0;
+    if (cudaMemcpyAsync(&v, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return CAKE_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, sizeof(int), s) != cudaSuccess) return CAKE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return CAKE_ERR_CUDA;
+    *host_out = v;
+    return CAKE_OK;
+}
+
+int cake_kmeans_selftest_bounded_wait(void* ws, size_t ws_bytes, int limit_ms, cake_stream_t stream) {
+    if (!ws) return CAKE_ERR_NULL;
+    if (ws_bytes < 256) return CAKE_ERR_WORKSPACE;
+    if (limit_ms < 1 || limit_ms > 1000) return CAKE_ERR_SHAPE;
+    if (launch_bounded_wait_selftest(static_cast<int*>(ws), limit_ms, reinterpret_cast<cudaStream_t>(stream)) !=
+        cudaSuccess)
+        return CAKE_ERR_CUDA;
+    return CAKE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,64 @@
+// Host-side declarations shared by the translation units of the library (not a public header).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/cake_kmeans.h"
+
+namespace cake {
+
+typedef long long i64;
+
+struct DeviceInfo {
+    int device;
+    int sm_count;
+    int smem_optin;   // max dynamic shared memory per block (opt-in), bytes
+    int cc_major;
+};
+// Properties of the current device (cached per device). Returns CAKE_OK / CAKE_ERR_DEVICE / CAKE_ERR_CUDA.
+int current_device_info(DeviceInfo* out);
+
+inline i64 round_up(i64 a, i64 b) { return (a + b - 1) / b * b; }
+
+// Centroid tiles of the tensor-core assign kernel are 256 wide; ||c||^2 is padded to that with +inf.
+constexpr int kAssignBlockN = 256;
+inline int padded_k(int K) { return (int)round_up(K, kAssignBlockN); }
+
+// ---- prologue: cn[b][k] = sum_d C[b][k][d]^2 (fp32), +inf for K <= k < Kpad
+cudaError_t launch_centroid_norms(const cake_bf16* C, int B, int K, int D, int Kpad, float* cn,
+                                  cudaStream_t s);
+
+// ---- assign
+bool assign_tc_supports(int D);
+int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
+                     const float* cn, int Kpad, int* out_idx, float* out_dist, int* status,
+                     cudaStream_t s);
+int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
+                       int* out_idx, float* out_dist, cudaStream_t s);
+
+// ---- update
+struct UpdateScratch {
+    float* sums;      // [B][K][D]
+    int* offsets;     // [B][K+1]   (sort path)
+    int* cursor;      // [B][K]     (sort path)
+    int* perm;        // [B][N]     (sort path)
+};
+bool update_smem_supports(int D, int K, int smem_optin);
+int launch_update_smem(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, float* sums,
+                       int* counts, int* status, cudaStream_t s);
+int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K,
+                       const UpdateScratch& scr, int* counts, int* status, cudaStream_t s);
+// out_C = counts>0 ? sums/counts : C_prev (or 0); optional bf16 copy
+cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B,
+                            int K, int D, float* out_C, cake_bf16* out_C_bf16, cudaStream_t s);
+
+// ---- inertia: acc[b] += sum_i dist[b][i] (fp64 atomics); acc stride given in elements
+cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc_stride,
+                           cudaStream_t s);
+
+// ---- bounded-wait self test
+cudaError_t launch_bounded_wait_selftest(int* status, int limit_ms, cudaStream_t s);
+
+}  // namespace cake

@@ -1,0 +1,439 @@
+// Centroid update: per-cluster sums and counts of the assigned points (paper Section 5,
+// "Flash-KMeans clean-start workload": centroid_update), then the division into means.
+//
+// Two routes produce sums[B][K][D] (fp32) and counts[B][K]:
+//   smem route : every CTA keeps a private K x D table of partial sums in shared memory, streams a
+//                slab of rows through it with shared-memory atomics and adds its table to the
+//                global one at the end.  For K*D*4 bytes that fit in one SM's shared memory.
+//   sort route : counting sort by cluster (histogram, exclusive scan, scatter of row numbers) and a
+//                segmented reduction in which each warp sums a fixed-size run of the sorted order
+//                in registers and adds one partial per cluster it touches.  Any K.
+// Both stream X exactly once with 16-byte (smem route: 4-byte) loads; HBM bandwidth is the bound.
+#include "internal.h"
+
+namespace cake {
+namespace {
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// ======================================================================= smem route
+// Table layout per cluster: the D/2 even columns first, then the D/2 odd ones, so that the 32 lanes
+// of a warp (lane l holds columns 2l, 2l+1 of a 64-column group) hit 32 different banks.
+constexpr int SMEM_THREADS = 512;
+constexpr int SMEM_ROWS_PER_ITER = 8;  // rows in flight per warp
+
+__global__ void __launch_bounds__(SMEM_THREADS)
+update_smem_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx, i64 N, int D, int K,
+                   float* __restrict__ sums, int* __restrict__ counts, int* status) {
+    extern __shared__ float tab[];                 // [K][D] permuted, then int cnt[K]
+    int* cnt = reinterpret_cast<int*>(tab + static_cast<size_t>(K) * D);
+    const int b = blockIdx.y;
+    const int half = D >> 1;
+    for (int e = threadIdx.x; e < K * D; e += blockDim.x) tab[e] = 0.f;
+    for (int e = threadIdx.x; e < K; e += blockDim.x) cnt[e] = 0;
+    __syncthreads();
+
+    const uint32_t* Xw = reinterpret_cast<const uint32_t*>(X) + static_cast<size_t>(b) * N * half;
+    const int* idx_b = idx + static_cast<size_t>(b) * N;
+    const i64 per_cta = (N + gridDim.x - 1) / gridDim.x;
+    const i64 r0 = per_cta * blockIdx.x;
+    const i64 r1 = (r0 + per_cta < N) ? r0 + per_cta : N;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    bool bad = false;
+
+    for (i64 base = r0 + static_cast<i64>(warp) * 32; base < r1; base += static_cast<i64>(nwarps) * 32) {
+        const i64 mine = base + lane;
+        int k_lane = -1;
+        if (mine < r1) {
+            k_lane = idx_b[mine];
+            if (k_lane < 0 || k_lane >= K) { bad = true; k_lane = -1; }
+            else atomicAdd(&cnt[k_lane], 1);
+        }
+        const int rows_here = (r1 - base < 32) ? static_cast<int>(r1 - base) : 32;
+        for (int j0 = 0; j0 < rows_here; j0 += SMEM_ROWS_PER_ITER) {
+            for (int c0 = 0; c0 < half; c0 += 32) {
+                const int c = c0 + lane;
+                uint32_t w[SMEM_ROWS_PER_ITER];
+                int kk[SMEM_ROWS_PER_ITER];
+#pragma unroll
+                for (int u = 0; u < SMEM_ROWS_PER_ITER; ++u) {
+                    kk[u] = __shfl_sync(0xffffffffu, k_lane, (j0 + u) & 31);
+                    if (j0 + u >= rows_here) kk[u] = -1;
+                    w[u] = 0;
+                    if (kk[u] >= 0 && c < half) w[u] = __ldg(Xw + (base + j0 + u) * half + c);
+                }
+#pragma unroll
+                for (int u = 0; u < SMEM_ROWS_PER_ITER; ++u) {
+                    if (kk[u] >= 0 && c < half) {
+                        float* row = tab + static_cast<size_t>(kk[u]) * D;
+                        atomicAdd(row + c, bf16lo(w[u]));
+                        atomicAdd(row + half + c, bf16hi(w[u]));
+                    }
+                }
+            }
+        }
+    }
+    if (bad) atomicCAS(status, CAKE_OK, CAKE_ERR_BAD_INDEX);
+    __syncthreads();
+    float* sums_b = sums + static_cast<size_t>(b) * K * D;
+    for (int e = threadIdx.x; e < K * D; e += blockDim.x) {
+        const float v = tab[e];
+        if (v != 0.f) {
+            const int k = e / D, pc = e - k * D;
+            const int col = pc < half ? 2 * pc : 2 * (pc - half) + 1;
+            atomicAdd(sums_b + static_cast<size_t>(k) * D + col, v);
+        }
+    }
+    for (int e = threadIdx.x; e < K; e += blockDim.x)
+        if (cnt[e]) atomicAdd(counts + static_cast<size_t>(b) * K + e, cnt[e]);
+}
+
+// ======================================================================= sort route
+constexpr int HIST_THREADS = 512;
+constexpr int HIST_SMEM_MAX_K = 8192;
+
+__global__ void __launch_bounds__(HIST_THREADS)
+hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts, int* status) {
+    extern __shared__ int h[];
+    const int b = blockIdx.y;
+    const bool use_smem = K <= HIST_SMEM_MAX_K;
+    if (use_smem) {
+        for (int e = threadIdx.x; e < K; e += blockDim.x) h[e] = 0;
+        __syncthreads();
+    }
+    const int* idx_b = idx + static_cast<size_t>(b) * N;
+    int* counts_b = counts + static_cast<size_t>(b) * K;
+    bool bad = false;
+    for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < N;
+         i += static_cast<i64>(gridDim.x) * blockDim.x) {
+        const int k = idx_b[i];
+        if (k < 0 || k >= K) { bad = true; continue; }
+        if (use_smem) atomicAdd(&h[k], 1);
+        else atomicAdd(counts_b + k, 1);
+    }
+    if (bad) atomicCAS(status, CAKE_OK, CAKE_ERR_BAD_INDEX);
+    if (use_smem) {
+        __syncthreads();
+        for (int e = threadIdx.x; e < K; e += blockDim.x)
+            if (h[e]) atomicAdd(counts_b + e, h[e]);
+    }
+}
+
+// offsets[b][k] = sum_{j<k} counts[b][j], offsets[b][K] = total; cursor = offsets[0..K)
+__global__ void __launch_bounds__(1024)
+scan_kernel(const int* __restrict__ counts, int K, int* __restrict__ offsets, int* __restrict__ cursor) {
+    __shared__ int warp_tot[32];
+    const int b = blockIdx.x;
+    const int* c = counts + static_cast<size_t>(b) * K;
+    int* off = offsets + static_cast<size_t>(b) * (K + 1);
+    int* cur = cursor + static_cast<size_t>(b) * K;
+    const int per = (K + blockDim.x - 1) / blockDim.x;
+    const int k0 = threadIdx.x * per, k1 = (k0 + per < K) ? k0 + per : K;
+    int local = 0;
+    for (int k = k0; k < k1; ++k) local += c[k];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int t = warp_tot[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, t, o);
+            if (lane >= o) t += u;
+        }
+        warp_tot[lane] = t;  // inclusive over warps
+    }
+    __syncthreads();
+    int run = incl - local + (warp ? warp_tot[warp - 1] : 0);
+    for (int k = k0; k < k1; ++k) {
+        off[k] = run;
+        cur[k] = run;
+        run += c[k];
+    }
+    if (threadIdx.x == blockDim.x - 1) off[K] = warp_tot[31];
+}
+
+// perm[b][pos] = i, pos taken from the cluster's cursor; lanes of a warp that hit the same cluster
+// take their slots with a single atomic.
+__global__ void __launch_bounds__(256)
+scatter_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ cursor, int* __restrict__ perm) {
+    const int b = blockIdx.y;
+    const int* idx_b = idx + static_cast<size_t>(b) * N;
+    int* cur = cursor + static_cast<size_t>(b) * K;
+    int* perm_b = perm + static_cast<size_t>(b) * N;
+    const int lane = threadIdx.x & 31;
+    const i64 span = static_cast<i64>(gridDim.x) * blockDim.x;
+    const i64 n_round = (N + 31) / 32 * 32;  // keep whole warps in the loop for the match
+    for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_round; i += span) {
+        int k = -1;
+        if (i < N) {
+            k = idx_b[i];
+            if (k < 0 || k >= K) k = -1;
+        }
+        const unsigned peers = __match_any_sync(0xffffffffu, k);
+        if (k >= 0) {
+            const int leader = __ffs(peers) - 1;
+            const int rank = __popc(peers & ((1u << lane) - 1u));
+            int base = 0;
+            if (lane == leader) base = atomicAdd(cur + k, __popc(peers));
+            base = __shfl_sync(peers, base, leader);
+            perm_b[base + rank] = static_cast<int>(i);
+        }
+    }
+}
+
+// Segmented reduction over the sorted order. Each warp owns SEG_ROWS consecutive sorted positions.
+// A row is read as 16-byte granules (8 bf16); LPR lanes share a row, 32/LPR rows are read at once.
+constexpr int SEG_ROWS = 64;
+constexpr int SEG_WARPS = 8;
+constexpr int SEG_UNROLL = 4;
+
+template <int GPL>  // granules per lane (D <= 256*GPL)
+__global__ void __launch_bounds__(SEG_WARPS * 32)
+segreduce_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ perm,
+                 const int* __restrict__ offsets, i64 N, int D, int K, int lpr,
+                 float* __restrict__ sums) {
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const i64 w = static_cast<i64>(blockIdx.x) * SEG_WARPS + (threadIdx.x >> 5);
+    const int* off = offsets + static_cast<size_t>(b) * (K + 1);
+    const int n_valid = off[K];
+    const i64 p0 = w * SEG_ROWS;
+    if (p0 >= n_valid) return;
+    const int p1 = static_cast<int>((p0 + SEG_ROWS < n_valid) ? p0 + SEG_ROWS : n_valid);
+    const int* perm_b = perm + static_cast<size_t>(b) * N;
+    const uint4* Xg = reinterpret_cast<const uint4*>(X) + static_cast<size_t>(b) * N * (D >> 3);
+    float* sums_b = sums + static_cast<size_t>(b) * K * D;
+    const int G = D >> 3;           // granules per row
+    const int rpp = 32 / lpr;       // rows per pass
+    const int sl = lane % lpr;      // granule slot inside the row
+    const int rs = lane / lpr;      // row slot
+
+    // cluster containing position p0: largest k with off[k] <= p0
+    int lo = 0, hi = K;             // invariant: off[lo] <= p0 < off[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (off[mid] <= static_cast<int>(p0)) lo = mid; else hi = mid;
+    }
+    int k = lo;
+    int p = static_cast<int>(p0);
+    while (p < p1) {
+        const int kend = off[k + 1];
+        if (kend <= p) { ++k; continue; }
+        const int e = kend < p1 ? kend : p1;
+        float acc[GPL][8];
+#pragma unroll
+        for (int g = 0; g < GPL; ++g)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
+        for (int q = p; q < e; q += rpp * SEG_UNROLL) {
+            uint4 v[SEG_UNROLL][GPL];
+#pragma unroll
+            for (int u = 0; u < SEG_UNROLL; ++u) {
+                const int pos = q + u * rpp + rs;
+                const bool on = pos < e;
+                const int row = on ? __ldg(perm_b + pos) : 0;
+#pragma unroll
+                for (int g = 0; g < GPL; ++g) {
+                    const int gi = sl + g * lpr;
+                    v[u][g] = make_uint4(0, 0, 0, 0);
+                    if (on && gi < G) v[u][g] = __ldg(Xg + static_cast<size_t>(row) * G + gi);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < SEG_UNROLL; ++u)
+#pragma unroll
+                for (int g = 0; g < GPL; ++g) {
+                    acc[g][0] += bf16lo(v[u][g].x); acc[g][1] += bf16hi(v[u][g].x);
+                    acc[g][2] += bf16lo(v[u][g].y); acc[g][3] += bf16hi(v[u][g].y);
+                    acc[g][4] += bf16lo(v[u][g].z); acc[g][5] += bf16hi(v[u][g].z);
+                    acc[g][6] += bf16lo(v[u][g].w); acc[g][7] += bf16hi(v[u][g].w);
+                }
+        }
+        // fold the row slots together, then one vector add per granule
+#pragma unroll
+        for (int g = 0; g < GPL; ++g)
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                for (int o = lpr; o < 32; o <<= 1) acc[g][j] += __shfl_xor_sync(0xffffffffu, acc[g][j], o);
+        if (rs == 0) {
+#pragma unroll
+            for (int g = 0; g < GPL; ++g) {
+                const int gi = sl + g * lpr;
+                if (gi < G) {
+                    float4* dst = reinterpret_cast<float4*>(sums_b + static_cast<size_t>(k) * D + gi * 8);
+                    atomicAdd(dst, make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]));
+                    atomicAdd(dst + 1, make_float4(acc[g][4], acc[g][5], acc[g][6], acc[g][7]));
+                }
+            }
+        }
+        p = e;
+    }
+}
+
+// Scalar variant for D not a multiple of 8 (or very large D): one warp per run, lanes stride columns.
+__global__ void __launch_bounds__(SEG_WARPS * 32)
+segreduce_scalar_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ perm,
+                        const int* __restrict__ offsets, i64 N, int D, int K, float* __restrict__ sums) {
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const i64 w = static_cast<i64>(blockIdx.x) * SEG_WARPS + (threadIdx.x >> 5);
+    const int* off = offsets + static_cast<size_t>(b) * (K + 1);
+    const int n_valid = off[K];
+    const i64 p0 = w * SEG_ROWS;
+    if (p0 >= n_valid) return;
+    const int p1 = static_cast<int>((p0 + SEG_ROWS < n_valid) ? p0 + SEG_ROWS : n_valid);
+    const int* perm_b = perm + static_cast<size_t>(b) * N;
+    const cake_bf16* Xb = X + static_cast<size_t>(b) * N * D;
+    float* sums_b = sums + static_cast<size_t>(b) * K * D;
+    int lo = 0, hi = K;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (off[mid] <= static_cast<int>(p0)) lo = mid; else hi = mid;
+    }
+    int k = lo, p = static_cast<int>(p0);
+    while (p < p1) {
+        const int kend = off[k + 1];
+        if (kend <= p) { ++k; continue; }
+        const int e = kend < p1 ? kend : p1;
+        for (int c = lane; c < D; c += 32) {
+            float a = 0.f;
+            for (int q = p; q < e; ++q)
+                a += __uint_as_float(static_cast<uint32_t>(Xb[static_cast<size_t>(perm_b[q]) * D + c]) << 16);
+            atomicAdd(sums_b + static_cast<size_t>(k) * D + c, a);
+        }
+        p = e;
+    }
+}
+
+// ======================================================================= division
+__device__ __forceinline__ cake_bf16 f32_to_bf16_rne(float f) {
+    uint32_t u = __float_as_uint(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<cake_bf16>((u >> 16) | 0x40u);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return static_cast<cake_bf16>(u >> 16);
+}
+
+__global__ void __launch_bounds__(256)
+finalize_kernel(const float* __restrict__ sums, const int* __restrict__ counts,
+                const cake_bf16* __restrict__ C_prev, i64 total, int D, float* __restrict__ out_C,
+                cake_bf16* __restrict__ out_C_bf16) {
+    for (i64 e = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; e < total;
+         e += static_cast<i64>(gridDim.x) * blockDim.x) {
+        const i64 row = e / D;  // b*K + k
+        const int n = counts[row];
+        float v;
+        if (n > 0) v = sums[e] / static_cast<float>(n);
+        else v = C_prev ? __uint_as_float(static_cast<uint32_t>(C_prev[e]) << 16) : 0.f;
+        out_C[e] = v;
+        if (out_C_bf16) out_C_bf16[e] = f32_to_bf16_rne(v);
+    }
+}
+
+}  // namespace
+
+// ======================================================================= host side
+bool update_smem_supports(int D, int K, int smem_optin) {
+    if (D % 2 != 0) return false;
+    const i64 need = static_cast<i64>(K) * D * 4 + static_cast<i64>(K) * 4;
+    return need <= smem_optin;
+}
+
+int launch_update_smem(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, float* sums,
+                       int* counts, int* status, cudaStream_t s) {
+    DeviceInfo di;
+    int rc = current_device_info(&di);
+    if (rc != CAKE_OK) return rc;
+    if (!update_smem_supports(D, K, di.smem_optin)) return CAKE_ERR_UNSUPPORTED;
+    const size_t kd = static_cast<size_t>(B) * K * D;
+    if (cudaMemsetAsync(sums, 0, kd * sizeof(float), s) != cudaSuccess) return CAKE_ERR_CUDA;
+    if (cudaMemsetAsync(counts, 0, static_cast<size_t>(B) * K * sizeof(int), s) != cudaSuccess)
+        return CAKE_ERR_CUDA;
+    if (N == 0) return CAKE_OK;
+    const size_t smem = static_cast<size_t>(K) * D * 4 + static_cast<size_t>(K) * 4;
+    static int attr_done_for_device = -1;
+    if (attr_done_for_device != di.device) {
+        if (cudaFuncSetAttribute(update_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 di.smem_optin) != cudaSuccess)
+            return CAKE_ERR_CUDA;
+        attr_done_for_device = di.device;
+    }
+    // CTAs per SM limited by shared memory (228 KiB per SM, 1 KiB reserved per CTA) and threads
+    int per_sm = static_cast<int>((228 * 1024) / (smem + 1024));
+    if (per_sm > 2048 / SMEM_THREADS) per_sm = 2048 / SMEM_THREADS;
+    if (per_sm < 1) per_sm = 1;
+    i64 ctas = (static_cast<i64>(di.sm_count) * per_sm + B - 1) / B;
+    const i64 max_useful = (N + 255) / 256;  // at least 256 rows per CTA
+    if (ctas > max_useful) ctas = max_useful;
+    if (ctas < 1) ctas = 1;
+    dim3 grid(static_cast<unsigned>(ctas), static_cast<unsigned>(B));
+    update_smem_kernel<<<grid, SMEM_THREADS, smem, s>>>(X, idx, N, D, K, sums, counts, status);
+    return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
+}
+
+int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K,
+                       const UpdateScratch& scr, int* counts, int* status, cudaStream_t s) {
+    DeviceInfo di;
+    int rc = current_device_info(&di);
+    if (rc != CAKE_OK) return rc;
+    const size_t kd = static_cast<size_t>(B) * K * D;
+    if (cudaMemsetAsync(scr.sums, 0, kd * sizeof(float), s) != cudaSuccess) return CAKE_ERR_CUDA;
+    if (cudaMemsetAsync(counts, 0, static_cast<size_t>(B) * K * sizeof(int), s) != cudaSuccess)
+        return CAKE_ERR_CUDA;
+    if (N == 0) return CAKE_OK;
+    {
+        i64 ctas = (N + HIST_THREADS * 8 - 1) / (HIST_THREADS * 8);
+        const i64 cap = (static_cast<i64>(di.sm_count) * 4 + B - 1) / B;
+        if (ctas > cap) ctas = cap;
+        if (ctas < 1) ctas = 1;
+        const size_t smem = K <= HIST_SMEM_MAX_K ? static_cast<size_t>(K) * 4 : 0;
+        hist_kernel<<<dim3(static_cast<unsigned>(ctas), B), HIST_THREADS, smem, s>>>(idx, N, K, counts, status);
+    }
+    scan_kernel<<<B, 1024, 0, s>>>(counts, K, scr.offsets, scr.cursor);
+    {
+        i64 ctas = (N + 256 * 4 - 1) / (256 * 4);
+        const i64 cap = (static_cast<i64>(di.sm_count) * 8 + B - 1) / B;
+        if (ctas > cap) ctas = cap;
+        if (ctas < 1) ctas = 1;
+        scatter_kernel<<<dim3(static_cast<unsigned>(ctas), B), 256, 0, s>>>(idx, N, K, scr.cursor, scr.perm);
+    }
+    {
+        const i64 warps = (N + SEG_ROWS - 1) / SEG_ROWS;
+        const unsigned ctas = static_cast<unsigned>((warps + SEG_WARPS - 1) / SEG_WARPS);
+        dim3 grid(ctas, B);
+        if (D % 8 == 0 && D <= 1024) {
+            const int G = D / 8;
+            int lpr = 1;
+            while (lpr < G && lpr < 32) lpr <<= 1;
+            const int gpl = (G + lpr - 1) / lpr;
+            if (gpl == 1)
+                segreduce_kernel<1><<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.perm, scr.offsets, N, D, K, lpr, scr.sums);
+            else if (gpl == 2)
+                segreduce_kernel<2><<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.perm, scr.offsets, N, D, K, lpr, scr.sums);
+            else
+                segreduce_kernel<4><<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.perm, scr.offsets, N, D, K, lpr, scr.sums);
+        } else {
+            segreduce_scalar_kernel<<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.perm, scr.offsets, N, D, K, scr.sums);
+        }
+    }
+    return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
+}
+
+cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B, int K,
+                            int D, float* out_C, cake_bf16* out_C_bf16, cudaStream_t s) {
+    const i64 total = static_cast<i64>(B) * K * D;
+    i64 ctas = (total + 256 * 4 - 1) / (256 * 4);
+    if (ctas > 148 * 16) ctas = 148 * 16;
+    if (ctas < 1) ctas = 1;
+    finalize_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(sums, counts, C_prev, total, D, out_C, out_C_bf16);
+    return cudaGetLastError();
+}
+
+}  // namespace cake

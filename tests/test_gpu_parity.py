@@ -1,0 +1,333 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle.
+
+Small shapes are compared element by element; the full-size workloads are compared on sampled rows
+(assign is independent per row) and in full for update (linear cost).  Tolerances: tests/grading.py.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_12629_b200 as cake
+from oracle import kmeans_oracle as orc
+from paper_2608_12629_b200 import inputs
+from tests import grading
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def problem(N, D, K, seed, comps=None, mean_std=1.0, sigma=0.5):
+    X, _ = inputs.gaussian_mixture(N, D, comps or max(1, min(K, 64)), mean_std, sigma, seed)
+    C = inputs.sample_init(X, K, seed)
+    return X, C
+
+
+def check_status(ws, want=cake.CAKE_OK):
+    assert cake.cake_kmeans_device_status(ws) == want
+
+
+# ------------------------------------------------------------------------------------ assign
+
+TC_SHAPES = [
+    # N, D, K : single tile, ragged rows, ragged K, several K tiles, D tails (96, 72, 8), D=256
+    (1, 64, 1), (127, 64, 2), (128, 64, 256), (129, 128, 257), (1000, 128, 1000), (777, 96, 65),
+    (4096, 128, 300), (300, 256, 700), (257, 16, 5), (1000, 8, 3), (2000, 72, 260), (333, 192, 513),
+    (20000, 64, 128), (50, 128, 2048),
+]
+
+
+@pytest.mark.parametrize("N,D,K", TC_SHAPES)
+def test_assign_tcgen05_small_shapes(N, D, K):
+    X, C = problem(N, D, K, seed=N + D + K)
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), ws=ws, flags=cake.CAKE_ASSIGN_TCGEN05)
+    torch.cuda.synchronize()
+    check_status(ws)
+    rep = grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx.cpu().numpy(), dist.cpu().numpy())
+    assert rep["mismatch"] <= max(2, N // 1000), rep
+
+
+@pytest.mark.parametrize("N,D,K", [(100, 5, 7), (300, 33, 40), (64, 130, 3), (1000, 64, 100)])
+def test_assign_simt_fallback(N, D, K):
+    X, C = problem(N, D, K, seed=N * 3 + D)
+    idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_SIMT)
+    grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx.cpu().numpy(), dist.cpu().numpy())
+    if D % 8:  # the automatic choice must take the fallback for such D, and the tensor path must refuse
+        idx2, _ = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV))
+        assert torch.equal(idx, idx2)
+        with pytest.raises(cake.CakeError) as e:
+            cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_TCGEN05)
+        assert e.value.code == cake.CAKE_ERR_UNSUPPORTED
+
+
+def test_assign_exact_ties_lowest_index():
+    """Small integers: every product, norm and sum is exact in fp32, so ties are exact on the GPU too."""
+    g = torch.Generator().manual_seed(4)
+    N, D, K = 3000, 64, 600
+    X = torch.randint(-2, 3, (N, D), generator=g).to(torch.bfloat16)
+    C = torch.randint(-2, 3, (K, D), generator=g).to(torch.bfloat16)
+    C[300:600] = C[0:300]            # every centroid duplicated across the two K tiles and column halves
+    C[17] = C[5]
+    idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_TCGEN05)
+    idx_o, dist_o, _ = orc.assign(inputs.to_bits(X), inputs.to_bits(C))
+    assert np.array_equal(idx.cpu().numpy(), idx_o)
+    assert np.array_equal(dist.cpu().numpy().astype(np.float64), dist_o)
+    assert idx_o.max() < 300
+
+
+def test_assign_batched_matches_per_problem_and_oracle():
+    B, N, D, K = 5, 700, 128, 300
+    Xs, Cs = zip(*(problem(N, D, K, seed=50 + b) for b in range(B)))
+    X, C = torch.stack(Xs).to(DEV), torch.stack(Cs).to(DEV)
+    ws = cake.alloc_workspace(B, N, D, K, DEV)
+    idx, dist = cake.cake_kmeans_assign(X, C, ws=ws)
+    check_status(ws)
+    for b in range(B):
+        grading.grade_assign(inputs.to_bits(Xs[b]), inputs.to_bits(Cs[b]), idx[b].cpu().numpy(),
+                             dist[b].cpu().numpy())
+        i1, d1 = cake.cake_kmeans_assign(X[b].contiguous(), C[b].contiguous())
+        assert torch.equal(i1, idx[b]) and torch.equal(d1, dist[b])
+
+
+def test_assign_edge_cases():
+    X, C = problem(64, 64, 4, seed=1)
+    # N = 0
+    idx, dist = cake.cake_kmeans_assign(X[:0].to(DEV), C.to(DEV))
+    assert idx.numel() == 0
+    # K > N, and C = X gives the identity with zero distance
+    Xd = X.to(DEV)
+    idx, dist = cake.cake_kmeans_assign(Xd, Xd.clone())
+    rows = inputs.to_bits(X)
+    first = {}
+    for i, r in enumerate(rows):
+        first.setdefault(r.tobytes(), i)
+    want = np.array([first[r.tobytes()] for r in rows])
+    assert np.array_equal(idx.cpu().numpy(), want)
+    assert float(dist.max()) <= 1e-3 * float((X.float() ** 2).sum(1).max()) * 2
+    # no dist requested
+    idx2, none = cake.cake_kmeans_assign(Xd, C.to(DEV), want_dist=False)
+    assert none is None
+    # workspace too small / misaligned / null
+    ws = cake.alloc_workspace(1, 64, 64, 4, DEV)
+    with pytest.raises(cake.CakeError) as e:
+        cake.cake_kmeans_assign(Xd, C.to(DEV), ws=ws[:1024])
+    assert e.value.code == cake.CAKE_ERR_WORKSPACE
+    with pytest.raises(cake.CakeError) as e:
+        cake.cake_kmeans_assign(Xd, C.to(DEV), ws=ws[8:])
+    assert e.value.code == cake.CAKE_ERR_ALIGN
+
+
+# ------------------------------------------------------------------------------------ update
+
+UPD_SHAPES = [(1, 64, 1), (1000, 64, 128), (5000, 128, 256), (333, 96, 17), (4097, 256, 64), (2500, 8, 3),
+              (3000, 128, 3000)]
+
+
+@pytest.mark.parametrize("path", ["smem", "sort"])
+@pytest.mark.parametrize("N,D,K", UPD_SHAPES)
+def test_update_paths(path, N, D, K):
+    flag = cake.CAKE_UPDATE_SMEM if path == "smem" else cake.CAKE_UPDATE_SORT
+    if path == "smem" and K * D * 4 + K * 4 > 227 * 1024:
+        pytest.skip("table does not fit in shared memory")
+    X, C = problem(N, D, K, seed=N + K)
+    g = torch.Generator().manual_seed(N)
+    idx = torch.randint(0, K, (N,), generator=g, dtype=torch.int32)
+    if K > 4:
+        idx[idx == 1] = 0                      # cluster 1 empty, cluster 0 heavy
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=C.to(DEV), ws=ws, flags=flag)
+    check_status(ws)
+    grading.grade_update(inputs.to_bits(X), idx.numpy(), K, inputs.to_bits(C), Cf.cpu().numpy(),
+                         inputs.to_bits(Cb), counts.cpu().numpy())
+
+
+def test_update_odd_feature_count_and_null_prev():
+    N, D, K = 500, 7, 9
+    X, _ = problem(N, D, K, seed=2)
+    idx = (torch.arange(N) % (K - 1)).to(torch.int32)          # last cluster empty
+    Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=None)
+    grading.grade_update(inputs.to_bits(X), idx.numpy(), K, None, Cf.cpu().numpy(), inputs.to_bits(Cb),
+                         counts.cpu().numpy())
+    assert not Cf[K - 1].any()
+
+
+@pytest.mark.parametrize("path", ["smem", "sort"])
+def test_update_bad_index_is_skipped_and_reported(path):
+    flag = cake.CAKE_UPDATE_SMEM if path == "smem" else cake.CAKE_UPDATE_SORT
+    N, D, K = 1000, 64, 10
+    X, C = problem(N, D, K, seed=3)
+    idx = (torch.arange(N) % K).to(torch.int32)
+    idx[5], idx[77] = K, -3
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    Cf, _, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=C.to(DEV), ws=ws, flags=flag)
+    check_status(ws, cake.CAKE_ERR_BAD_INDEX)
+    check_status(ws)                                            # reading clears it
+    keep = (idx >= 0) & (idx < K)
+    C_o, counts_o = orc.update(inputs.to_bits(X)[keep.numpy()], idx[keep].numpy(), K, inputs.to_bits(C))
+    assert np.array_equal(counts.cpu().numpy(), counts_o)
+    np.testing.assert_allclose(Cf.cpu().numpy(), C_o, rtol=1e-4, atol=1e-5)
+
+
+def test_update_batched_and_n_zero():
+    B, N, D, K = 3, 900, 64, 20
+    Xs, Cs = zip(*(problem(N, D, K, seed=70 + b) for b in range(B)))
+    X, C = torch.stack(Xs), torch.stack(Cs)
+    g = torch.Generator().manual_seed(0)
+    idx = torch.randint(0, K, (B, N), generator=g, dtype=torch.int32)
+    for flag in (cake.CAKE_UPDATE_SMEM, cake.CAKE_UPDATE_SORT):
+        Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=C.to(DEV), flags=flag)
+        for b in range(B):
+            grading.grade_update(inputs.to_bits(Xs[b]), idx[b].numpy(), K, inputs.to_bits(Cs[b]),
+                                 Cf[b].cpu().numpy(), inputs.to_bits(Cb[b]), counts[b].cpu().numpy())
+    Cf, Cb, counts = cake.cake_kmeans_update(X[0, :0].to(DEV), idx[0, :0].to(DEV), K, C_prev=C[0].to(DEV))
+    assert not counts.any() and torch.equal(Cb.cpu(), C[0])
+
+
+# ------------------------------------------------------------------------------------ Lloyd
+
+def teacher_forced(X, C0, iters, flags=0):
+    """Runs iteration by iteration on the GPU; the oracle re-derives each step from the GPU's own state."""
+    Xb = inputs.to_bits(X)
+    Xd = X.to(DEV)
+    cur = C0.to(DEV)
+    N, D = X.shape
+    K = C0.shape[0]
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    inertia, near_ties = [], 0
+    for t in range(iters):
+        out = cake.cake_kmeans_lloyd(Xd, cur, 1, ws=ws, flags=flags)
+        torch.cuda.synchronize()
+        check_status(ws)
+        cur_bits = inputs.to_bits(cur)
+        idx = out.idx.cpu().numpy()
+        rep = grading.grade_assign(Xb, cur_bits, idx, out.dist.cpu().numpy())
+        near_ties += rep["mismatch"]
+        _, dist_o, _ = orc.assign(Xb, cur_bits)
+        assert abs(float(out.inertia[0]) - dist_o.sum()) <= grading.INERTIA_TOL * dist_o.sum()
+        grading.grade_update(Xb, idx, K, cur_bits, out.C.cpu().numpy(), inputs.to_bits(out.C_bf16),
+                             out.counts.cpu().numpy())
+        inertia.append(float(out.inertia[0]))
+        cur = out.C_bf16
+    return cur, inertia, near_ties
+
+
+def test_lloyd_c1_teacher_forced_and_free_run():
+    w = inputs.WORKLOADS["c1"]
+    X, C0 = inputs.make_problem(w)
+    cur, inertia, near = teacher_forced(X, C0, w.iters)
+    assert near <= 5
+    # one call for all iterations follows the same trajectory up to fp32 summation order
+    out = cake.cake_kmeans_lloyd(X.to(DEV), C0.to(DEV), w.iters)
+    np.testing.assert_allclose(out.inertia.cpu().numpy(), inertia, rtol=1e-4)
+    # free-running oracle (its own bf16-rounded trajectory)
+    r = orc.lloyd(inputs.to_bits(X), inputs.to_bits(C0), w.iters, round_centroids=True)
+    np.testing.assert_allclose(out.inertia.cpu().numpy(), r.inertia, rtol=grading.INERTIA_TOL)
+    assert int(out.counts.sum()) == w.N
+    assert (np.diff(out.inertia.cpu().numpy()) <= 1e-4 * out.inertia.cpu().numpy()[:-1]).all()
+
+
+@pytest.mark.parametrize("flags", [cake.CAKE_UPDATE_SMEM, cake.CAKE_UPDATE_SORT,
+                                   cake.CAKE_ASSIGN_SIMT | cake.CAKE_UPDATE_SORT])
+def test_lloyd_small_all_paths(flags):
+    X, C0 = problem(3000, 64, 50, seed=12, comps=50, mean_std=2.0, sigma=1.0)
+    teacher_forced(X, C0, 4, flags=flags)
+
+
+def test_lloyd_handworked_example_on_gpu():
+    """The six-point example (golden/handworked_2d.json), padded to D=8 with zero columns."""
+    pts = [[0, 0], [0, 2], [2, 0], [10, 10], [10, 12], [12, 10]]
+    X = torch.zeros(6, 8)
+    X[:, :2] = torch.tensor(pts, dtype=torch.float32)
+    X = X.to(torch.bfloat16)
+    C0 = X[[0, 2]].contiguous()
+    out = cake.cake_kmeans_lloyd(X.to(DEV), C0.to(DEV), 4)
+    assert out.idx.cpu().tolist() == [0, 0, 0, 1, 1, 1]
+    assert out.counts.cpu().tolist() == [3, 3]
+    np.testing.assert_allclose(out.inertia.cpu().numpy(), [576.0, 47.75, 349611 / 32768, 349611 / 32768], rtol=1e-5)
+    np.testing.assert_allclose(out.C.cpu().numpy()[:, :2], [[2 / 3, 2 / 3], [32 / 3, 32 / 3]], rtol=1e-6)
+    assert out.C_bf16.float().cpu()[:, :2].tolist() == [[171 / 256, 171 / 256], [171 / 16, 171 / 16]]
+
+
+def test_lloyd_iters_zero_and_batched():
+    B, N, D, K = 3, 1500, 64, 24
+    Xs, Cs = zip(*(problem(N, D, K, seed=90 + b, comps=24, mean_std=2.0, sigma=1.0) for b in range(B)))
+    X, C0 = torch.stack(Xs).to(DEV), torch.stack(Cs).to(DEV)
+    out0 = cake.cake_kmeans_lloyd(X, C0, 0)
+    assert torch.equal(out0.C_bf16, C0) and torch.equal(out0.C, C0.float())
+    out = cake.cake_kmeans_lloyd(X, C0, 5)
+    for b in range(B):
+        one = cake.cake_kmeans_lloyd(X[b].contiguous(), C0[b].contiguous(), 5)
+        np.testing.assert_allclose(out.inertia[b].cpu().numpy(), one.inertia.cpu().numpy(), rtol=1e-4)
+        r = orc.lloyd(inputs.to_bits(Xs[b]), inputs.to_bits(Cs[b]), 5, round_centroids=True)
+        np.testing.assert_allclose(out.inertia[b].cpu().numpy(), r.inertia, rtol=grading.INERTIA_TOL)
+
+
+def test_lloyd_host_buffers_match_device_call():
+    X, C0 = problem(5000, 128, 40, seed=33, comps=40, mean_std=2.0, sigma=1.0)
+    iters = 3
+    dev_out = cake.cake_kmeans_lloyd(X.to(DEV), C0.to(DEV), iters)
+    Xh, Ch = X.pin_memory(), C0.pin_memory()
+    host_out = cake.alloc_lloyd_outputs(Xh, Ch, iters, pin_host=True)
+    scratch = torch.empty(cake.cake_kmeans_lloyd_host_device_bytes(1, 5000, 128, 40, iters), dtype=torch.uint8,
+                          device=DEV)
+    cake.cake_kmeans_lloyd_host(Xh, Ch, iters, host_out, scratch)
+    torch.cuda.synchronize()
+    assert torch.equal(host_out.idx, dev_out.idx.cpu())
+    np.testing.assert_allclose(host_out.inertia.numpy(), dev_out.inertia.cpu().numpy(), rtol=1e-5)
+    np.testing.assert_allclose(host_out.C.numpy(), dev_out.C.cpu().numpy(), rtol=1e-4, atol=1e-5)
+    assert torch.equal(host_out.counts, dev_out.counts.cpu())
+
+
+# ------------------------------------------------------------------------------------ full-size workloads
+
+def sampled_rows(N, n, seed):
+    return np.sort(np.random.default_rng(seed).choice(N, size=min(n, N), replace=False))
+
+
+@pytest.mark.parametrize("name,sample", [("c2", 4096), ("c4", 1024)])
+def test_full_size_workload_sampled(name, sample):
+    """The benchmark's launch configuration: one Lloyd iteration at full size, graded on sampled rows
+    (assign) and in full (update)."""
+    w = inputs.WORKLOADS[name]
+    X, C0 = inputs.make_problem(w, device=DEV)
+    ws = cake.alloc_workspace(1, w.N, w.D, w.K, DEV)
+    out = cake.cake_kmeans_lloyd(X, C0, 1, ws=ws)
+    torch.cuda.synchronize()
+    check_status(ws)
+    Xb, Cb = inputs.to_bits(X), inputs.to_bits(C0)
+    idx = out.idx.cpu().numpy()
+    rows = sampled_rows(w.N, sample, w.seed)
+    rep = grading.grade_assign(Xb, Cb, idx, out.dist.cpu().numpy(), rows=rows)
+    assert rep["mismatch"] <= max(2, sample // 500), rep
+    assert int(out.counts.sum()) == w.N
+    grading.grade_update(Xb, idx, w.K, Cb, out.C.cpu().numpy(), inputs.to_bits(out.C_bf16), out.counts.cpu().numpy())
+    # inertia equals the sum of the per-point distances the same call returned
+    assert abs(float(out.inertia[0]) - float(out.dist.double().sum())) <= 1e-6 * float(out.inertia[0])
+
+
+def test_full_size_batched_workload_sampled():
+    w = inputs.WORKLOADS["c3"]
+    X, C0 = inputs.make_batch(w, device=DEV)
+    ws = cake.alloc_workspace(w.B, w.N, w.D, w.K, DEV)
+    out = cake.cake_kmeans_lloyd(X, C0, 1, ws=ws)
+    torch.cuda.synchronize()
+    check_status(ws)
+    for b in (0, 13, 31):
+        Xb, Cb = inputs.to_bits(X[b]), inputs.to_bits(C0[b])
+        idx = out.idx[b].cpu().numpy()
+        grading.grade_assign(Xb, Cb, idx, out.dist[b].cpu().numpy(), rows=sampled_rows(w.N, 2048, b))
+        grading.grade_update(Xb, idx, w.K, Cb, out.C[b].cpu().numpy(), inputs.to_bits(out.C_bf16[b]),
+                             out.counts[b].cpu().numpy())
+
+
+# ------------------------------------------------------------------------------------ bounded waits
+
+def test_bounded_wait_expires_and_context_survives():
+    ws = cake.alloc_workspace(1, 16, 8, 2, DEV)
+    cake.cake_kmeans_selftest_bounded_wait(ws, 20)
+    assert cake.cake_kmeans_device_status(ws) == cake.CAKE_ERR_TIMEOUT
+    assert cake.cake_kmeans_device_status(ws) == cake.CAKE_OK
+    X, C = problem(256, 64, 8, seed=5)
+    idx, _ = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), ws=ws)
+    idx_o, _, _ = orc.assign(inputs.to_bits(X), inputs.to_bits(C))
+    assert np.array_equal(idx.cpu().numpy(), idx_o)
