@@ -71,6 +71,12 @@ enum {
 /* Library version (major*10000 + minor*100 + patch).  No paper counterpart. */
 CAKE_API int cake_version(void);
 
+/*
+ * Number of CUDA kernels this library has launched since it was loaded (memsets and copies are
+ * not counted).  For accounting in benchmarks.  No paper counterpart.
+ */
+CAKE_API unsigned long long cake_kmeans_kernel_launches(void);
+
 /* Static, human-readable text for a CAKE_* code.  Never NULL.  No paper counterpart. */
 CAKE_API const char* cake_strerror(int code);
 

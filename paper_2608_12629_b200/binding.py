@@ -23,7 +23,7 @@ CAKE_ASSIGN_AUTO, CAKE_ASSIGN_TCGEN05, CAKE_ASSIGN_SIMT = 0, 1, 2
 CAKE_UPDATE_AUTO, CAKE_UPDATE_SMEM, CAKE_UPDATE_SORT = 0, 1 << 4, 2 << 4
 
 EXPORTS = [
-    "cake_version", "cake_strerror", "cake_kmeans_workspace_bytes", "cake_kmeans_assign",
+    "cake_version", "cake_kmeans_kernel_launches", "cake_strerror", "cake_kmeans_workspace_bytes", "cake_kmeans_assign",
     "cake_kmeans_assign_batched", "cake_kmeans_update", "cake_kmeans_update_batched", "cake_kmeans_lloyd",
     "cake_kmeans_lloyd_batched", "cake_kmeans_lloyd_host_device_bytes", "cake_kmeans_lloyd_host",
     "cake_kmeans_device_status", "cake_kmeans_selftest_bounded_wait",
@@ -62,8 +62,9 @@ def lib() -> ctypes.CDLL:
         L.cake_kmeans_device_status.argtypes = [vp, vp, ctypes.POINTER(i)]
         L.cake_kmeans_selftest_bounded_wait.argtypes = [vp, sz, i, vp]
         for name in EXPORTS:
-            if name not in ("cake_strerror",):
+            if name not in ("cake_strerror", "cake_kmeans_kernel_launches"):
                 getattr(L, name).restype = i
+        L.cake_kmeans_kernel_launches.restype = ctypes.c_ulonglong
         _lib = L
     return _lib
 
@@ -74,6 +75,10 @@ def strerror(code: int) -> str:
 
 def cake_version() -> int:
     return int(lib().cake_version())
+
+
+def cake_kmeans_kernel_launches() -> int:
+    return int(lib().cake_kmeans_kernel_launches())
 
 
 def _check(rc: int, where: str):

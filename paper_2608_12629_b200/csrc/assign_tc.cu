@@ -435,6 +435,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     }
     const i64 grid = p.total_tiles < di.sm_count ? p.total_tiles : di.sm_count;
     assign_tc_kernel<<<static_cast<unsigned>(grid), NUM_THREADS, smem_bytes, s>>>(tx, tc, p);
+    note_launches(1);
     return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
 }
 

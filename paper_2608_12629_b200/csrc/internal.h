@@ -20,6 +20,10 @@ struct DeviceInfo {
 // Properties of the current device (cached per device). Returns CAKE_OK / CAKE_ERR_DEVICE / CAKE_ERR_CUDA.
 int current_device_info(DeviceInfo* out);
 
+// Number of kernels this library has launched since it was loaded (all devices, all streams).
+void note_launches(int n);
+unsigned long long launches_so_far();
+
 inline i64 round_up(i64 a, i64 b) { return (a + b - 1) / b * b; }
 
 // Centroid tiles of the tensor-core assign kernel are 256 wide; ||c||^2 is padded to that with +inf.

@@ -1,11 +1,16 @@
 // Small kernels around the two hot ones: the ||c||^2 prologue, the CUDA-core assign fallback,
 // the inertia reduction and the bounded-wait self test; plus the cached device query.
+#include <atomic>
 #include <mutex>
 
 #include "internal.h"
 #include "ptx.cuh"
 
 namespace cake {
+
+static std::atomic<unsigned long long> g_launches{0};
+void note_launches(int n) { g_launches.fetch_add(static_cast<unsigned long long>(n), std::memory_order_relaxed); }
+unsigned long long launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
 
 int current_device_info(DeviceInfo* out) {
     static std::mutex mu;
@@ -142,6 +147,7 @@ cudaError_t launch_centroid_norms(const cake_bf16* C, int B, int K, int D, int K
     const i64 rows = static_cast<i64>(B) * Kpad;
     const i64 ctas = (rows * 32 + 255) / 256;
     centroid_norms_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(C, K, D, Kpad, rows, cn);
+    note_launches(1);
     return cudaGetLastError();
 }
 
@@ -152,6 +158,7 @@ int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int
     i64 ctas = (rows + 7) / 8;
     if (ctas > 148 * 64) ctas = 148 * 64;
     assign_simt_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(X, C, B, N, D, K, out_idx, out_dist);
+    note_launches(1);
     return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
 }
 
@@ -160,11 +167,13 @@ cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc
     i64 ctas = (N + 256 * 8 - 1) / (256 * 8);
     if (ctas > 296) ctas = 296;
     inertia_kernel<<<dim3(static_cast<unsigned>(ctas), B), 256, 0, s>>>(dist, N, acc, acc_stride);
+    note_launches(1);
     return cudaGetLastError();
 }
 
 cudaError_t launch_bounded_wait_selftest(int* status, int limit_ms, cudaStream_t s) {
     bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(status, static_cast<unsigned long long>(limit_ms) * 1000000ull);
+    note_launches(1);
     return cudaGetLastError();
 }
 

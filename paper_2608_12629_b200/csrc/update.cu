@@ -375,6 +375,7 @@ int launch_update_smem(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
     if (ctas < 1) ctas = 1;
     dim3 grid(static_cast<unsigned>(ctas), static_cast<unsigned>(B));
     update_smem_kernel<<<grid, SMEM_THREADS, smem, s>>>(X, idx, N, D, K, sums, counts, status);
+    note_launches(1);
     return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
 }
 
@@ -423,6 +424,7 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
             segreduce_scalar_kernel<<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.perm, scr.offsets, N, D, K, scr.sums);
         }
     }
+    note_launches(4);  // histogram, scan, scatter, segmented reduction
     return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
 }
 
@@ -433,6 +435,7 @@ cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf1
     if (ctas > 148 * 16) ctas = 148 * 16;
     if (ctas < 1) ctas = 1;
     finalize_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(sums, counts, C_prev, total, D, out_C, out_C_bf16);
+    note_launches(1);
     return cudaGetLastError();
 }
 

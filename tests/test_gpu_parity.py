@@ -66,8 +66,8 @@ def test_assign_exact_ties_lowest_index():
     N, D, K = 3000, 64, 600
     X = torch.randint(-2, 3, (N, D), generator=g).to(torch.bfloat16)
     C = torch.randint(-2, 3, (K, D), generator=g).to(torch.bfloat16)
-    C[300:600] = C[0:300]            # every centroid duplicated across the two K tiles and column halves
     C[17] = C[5]
+    C[300:600] = C[0:300]            # every centroid duplicated across the two K tiles and column halves
     idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_TCGEN05)
     idx_o, dist_o, _ = orc.assign(inputs.to_bits(X), inputs.to_bits(C))
     assert np.array_equal(idx.cpu().numpy(), idx_o)
@@ -323,7 +323,7 @@ def test_full_size_batched_workload_sampled():
 # ------------------------------------------------------------------------------------ bounded waits
 
 def test_bounded_wait_expires_and_context_survives():
-    ws = cake.alloc_workspace(1, 16, 8, 2, DEV)
+    ws = cake.alloc_workspace(1, 256, 64, 8, DEV)
     cake.cake_kmeans_selftest_bounded_wait(ws, 20)
     assert cake.cake_kmeans_device_status(ws) == cake.CAKE_ERR_TIMEOUT
     assert cake.cake_kmeans_device_status(ws) == cake.CAKE_OK
