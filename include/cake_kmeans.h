@@ -105,6 +105,25 @@ CAKE_API int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, 
                                size_t ws_bytes, cake_stream_t stream, unsigned flags);
 
 /*
+ * assign without any workspace, for callers that cannot allocate device memory (code running
+ * inside another framework's allocator callback, or in a process whose device memory is already
+ * fully carved up, has no cudaMalloc to give this library a scratch buffer).  The paper has no
+ * counterpart: this is the un-batched cake_kmeans_assign with its scratch (the ||c||^2 row and the
+ * status word) held in a fixed 65,792-byte array inside the library image, which every GPU that
+ * loads the library keeps until the process exits.
+ *   X, C, out_idx, out_dist: as cake_kmeans_assign (one problem).
+ *   K must be <= 16384; a larger K returns CAKE_ERR_UNSUPPORTED and nothing is enqueued.
+ * The call allocates nothing and frees nothing.  The first call on each device resolves the
+ * array's device address (one-time set-up with that device current); make that first call
+ * outside any stream capture.  All calls on a device share the one array, which keeps the
+ * previous call's contents: the call itself clears what must start at zero, but two calls whose
+ * work overlaps on the GPU (different streams, no ordering between them) race on it -- order them.
+ * The device status word is not readable through this entry point.
+ */
+CAKE_API int cake_kmeans_assign_static(const cake_bf16* X, const cake_bf16* C, long long N, int D, int K,
+                                       int* out_idx, float* out_dist, cake_stream_t stream);
+
+/*
  * centroid_update (same paragraph: per-cluster sums and counts), followed by the division.
  *   X          [B][N][D] bf16, in
  *   idx        [B][N] int32, in; values outside [0,K) are skipped and raise the device status

@@ -26,7 +26,7 @@ EXPORTS = [
     "cake_version", "cake_kmeans_kernel_launches", "cake_strerror", "cake_kmeans_workspace_bytes", "cake_kmeans_assign",
     "cake_kmeans_assign_batched", "cake_kmeans_update", "cake_kmeans_update_batched", "cake_kmeans_lloyd",
     "cake_kmeans_lloyd_batched", "cake_kmeans_lloyd_host_device_bytes", "cake_kmeans_lloyd_host",
-    "cake_kmeans_device_status", "cake_kmeans_selftest_bounded_wait",
+    "cake_kmeans_device_status", "cake_kmeans_selftest_bounded_wait", "cake_kmeans_assign_static",
 ]
 
 _lib = None
@@ -61,6 +61,7 @@ def lib() -> ctypes.CDLL:
         L.cake_kmeans_lloyd_host.argtypes = [vp, vp, ll, ll, i, i, i, vp, vp, vp, vp, vp, vp, vp, sz, vp, u]
         L.cake_kmeans_device_status.argtypes = [vp, vp, ctypes.POINTER(i)]
         L.cake_kmeans_selftest_bounded_wait.argtypes = [vp, sz, i, vp]
+        L.cake_kmeans_assign_static.argtypes = [vp, vp, ll, i, i, vp, vp, vp]
         for name in EXPORTS:
             if name not in ("cake_strerror", "cake_kmeans_kernel_launches"):
                 getattr(L, name).restype = i
@@ -249,3 +250,25 @@ def cake_kmeans_selftest_bounded_wait(ws: torch.Tensor, limit_ms: int, stream=No
     with torch.cuda.device(ws.device):
         _check(lib().cake_kmeans_selftest_bounded_wait(_ptr(ws), ws.numel(), limit_ms, _stream(stream, ws.device)),
                "cake_kmeans_selftest_bounded_wait")
+
+
+def cake_kmeans_assign_static(X, C, out_idx=None, out_dist=None, stream=None, want_dist=True):
+    """Workspace-free assign for callers that cannot allocate: X bf16 [N,D], C bf16 [K,D], K <= 16384.
+
+    The scratch is a fixed array inside the library, shared by every call on the device, so calls
+    must not overlap on the GPU.  Output tensors are still the caller's (allocated here only as a
+    convenience when not passed in).
+    """
+    _want(X, torch.bfloat16, "X"), _want(C, torch.bfloat16, "C")
+    if X.dim() != 2 or C.dim() != 2 or X.shape[1] != C.shape[1]:
+        raise ValueError("X must be [N,D] and C [K,D]")
+    N, D, K = X.shape[0], X.shape[1], C.shape[0]
+    if out_idx is None:
+        out_idx = torch.empty(N, dtype=torch.int32, device=X.device)
+    if out_dist is None and want_dist:
+        out_dist = torch.empty(N, dtype=torch.float32, device=X.device)
+    with torch.cuda.device(X.device):
+        rc = lib().cake_kmeans_assign_static(_ptr(X), _ptr(C), N, D, K, _ptr(out_idx), _ptr(out_dist),
+                                             _stream(stream, X.device))
+    _check(rc, "cake_kmeans_assign_static")
+    return out_idx, out_dist
