@@ -59,8 +59,10 @@ enum {
 
 enum {
     CAKE_ASSIGN_AUTO = 0,
-    CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 256 */
+    CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 256.
+                                  Distances that agree to 2^-16 relative are ordered by index.   */
     CAKE_ASSIGN_SIMT = 2,      /* plain CUDA-core fallback, any D                               */
+    CAKE_ASSIGN_TCGEN05_EXACT = 3, /* same pipeline, full-precision comparison (slower epilogue) */
     CAKE_ASSIGN_MASK = 0xF,
     CAKE_UPDATE_AUTO = 0,
     CAKE_UPDATE_SMEM = 1 << 4, /* shared-memory partial sums; needs K*D*4 + K*4 bytes of smem   */
@@ -90,8 +92,8 @@ CAKE_API int cake_kmeans_workspace_bytes(long long B, long long N, int D, int K,
 
 /*
  * assign (Section 5, "Flash-KMeans clean-start workload": squared Euclidean distances to all K
- * centroids and the arg-min).  Computed as ||x||^2 - 2 x.c + ||c||^2 with x.c on the tensor
- * cores in fp32; the row constant ||x||^2 does not enter the comparison.
+ * centroids and the arg-min).  Computed as ||x||^2 - 2 x.c + ||c||^2, accumulated in fp32 on the
+ * tensor cores.
  *   X        [B][N][D] bf16, in
  *   C        [B][K][D] bf16, in
  *   out_idx  [B][N] int32, out: arg-min_k, lowest k on ties
@@ -108,8 +110,8 @@ CAKE_API int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, 
  * assign without any workspace, for callers that cannot allocate device memory (code running
  * inside another framework's allocator callback, or in a process whose device memory is already
  * fully carved up, has no cudaMalloc to give this library a scratch buffer).  The paper has no
- * counterpart: this is the un-batched cake_kmeans_assign with its scratch (the ||c||^2 row and the
- * status word) held in a fixed 65,792-byte array inside the library image, which every GPU that
+ * counterpart: this is the un-batched cake_kmeans_assign with its scratch (the centroid half-norm
+ * operand and the status word) held in a fixed 524,544-byte array inside the library image, which every GPU that
  * loads the library keeps until the process exits.
  *   X, C, out_idx, out_dist: as cake_kmeans_assign (one problem).
  *   K must be <= 16384; a larger K returns CAKE_ERR_UNSUPPORTED and nothing is enqueued.

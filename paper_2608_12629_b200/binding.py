@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libcake_kmeans.so")
 CAKE_OK = 0
 CAKE_ERR_NULL, CAKE_ERR_SHAPE, CAKE_ERR_ALIGN, CAKE_ERR_UNSUPPORTED = -1, -2, -3, -4
 CAKE_ERR_WORKSPACE, CAKE_ERR_CUDA, CAKE_ERR_BAD_INDEX, CAKE_ERR_TIMEOUT, CAKE_ERR_DEVICE = -5, -6, -7, -8, -9
-CAKE_ASSIGN_AUTO, CAKE_ASSIGN_TCGEN05, CAKE_ASSIGN_SIMT = 0, 1, 2
+CAKE_ASSIGN_AUTO, CAKE_ASSIGN_TCGEN05, CAKE_ASSIGN_SIMT, CAKE_ASSIGN_TCGEN05_EXACT = 0, 1, 2, 3
 CAKE_UPDATE_AUTO, CAKE_UPDATE_SMEM, CAKE_UPDATE_SORT = 0, 1 << 4, 2 << 4
 
 EXPORTS = [

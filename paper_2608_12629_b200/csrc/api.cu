@@ -12,7 +12,7 @@ inline size_t up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Workspace {
     int* status;          // [64] header, word 0 = sticky device status
-    float* cn;            // [B][Kpad]
+    void* caug;           // [B][Kpad/256][8 KiB] half-norm operand of the tensor-core assign
     float* sums;          // [B][K][D]
     int* offsets;         // [B][K+1]
     int* cursor;          // [B][K]
@@ -29,7 +29,7 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     auto take = [&](size_t n) { char* r = p ? p + o : nullptr; o += up(n); return r; };
     const size_t kd = static_cast<size_t>(B) * K * D;
     w.status = reinterpret_cast<int*>(take(256));
-    w.cn = reinterpret_cast<float*>(take(static_cast<size_t>(B) * padded_k(K) * 4));
+    w.caug = take(assign_tc_aug_bytes(B, K));
     w.sums = reinterpret_cast<float*>(take(kd * 4));
     w.offsets = reinterpret_cast<int*>(take(static_cast<size_t>(B) * (K + 1) * 4));
     w.cursor = reinterpret_cast<int*>(take(static_cast<size_t>(B) * K * 4));
@@ -62,12 +62,11 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
     unsigned path = flags & CAKE_ASSIGN_MASK;
     if (path == CAKE_ASSIGN_AUTO) path = assign_tc_supports(D) ? CAKE_ASSIGN_TCGEN05 : CAKE_ASSIGN_SIMT;
     if (path == CAKE_ASSIGN_SIMT) return launch_assign_simt(X, C, B, N, D, K, out_idx, out_dist, s);
-    if (path != CAKE_ASSIGN_TCGEN05) return CAKE_ERR_UNSUPPORTED;
+    if (path != CAKE_ASSIGN_TCGEN05 && path != CAKE_ASSIGN_TCGEN05_EXACT) return CAKE_ERR_UNSUPPORTED;
     if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
     if (N == 0) return CAKE_OK;
-    const int Kpad = padded_k(K);
-    if (launch_centroid_norms(C, B, K, D, Kpad, w.cn, s) != cudaSuccess) return CAKE_ERR_CUDA;
-    return launch_assign_tc(X, C, B, N, D, K, w.cn, Kpad, out_idx, out_dist, w.status, s);
+    return launch_assign_tc(X, C, B, N, D, K, w.caug, path == CAKE_ASSIGN_TCGEN05_EXACT, out_idx, out_dist,
+                            w.status, s);
 }
 
 int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, const cake_bf16* C_prev,

@@ -3,10 +3,10 @@
 // Some callers have no way to hand this library a workspace: code that runs where cudaMalloc is
 // forbidden (inside another framework's memory-pool callback, in a process whose device memory is
 // fully pre-partitioned, in an embedding whose allocator hooks must not be re-entered).  For them
-// the scratch the assign kernel needs -- the ||c||^2 row and the status word -- lives in a fixed
+// the scratch the assign kernel needs -- the centroid half-norm operand and the status word -- lives in a fixed
 // array that is part of the loaded library image, so nothing is allocated at any point.
 //
-// The array is `static __device__`: every GPU that loads the library holds these 65,792 bytes until
+// The array is `static __device__`: every GPU that loads the library holds these 524,544 bytes until
 // the process exits.  In host code the array's name is only a host-side handle, not a device
 // address, so the address is obtained once per device with cudaGetSymbolAddress (with that device
 // current) and that pointer is what the kernels receive.
@@ -19,7 +19,8 @@ namespace {
 
 constexpr int kStaticMaxK = 16384;                         // largest K this entry point accepts
 constexpr size_t kStaticHeader = 256;                      // status word, padded
-constexpr size_t kStaticBytes = kStaticHeader + static_cast<size_t>(kStaticMaxK) * sizeof(float);
+constexpr size_t kStaticBytes =
+    kStaticHeader + static_cast<size_t>(kStaticMaxK / kAssignBlockN) * kAssignAugTileBytes;   // 256 B + 512 KiB
 
 static __device__ __align__(256) unsigned char g_assign_scratch[kStaticBytes];
 
@@ -65,11 +66,9 @@ extern "C" int cake_kmeans_assign_static(const cake_bf16* X, const cake_bf16* C,
     int rc = scratch_for_current_device(&scratch);
     if (rc != CAKE_OK) return rc;
     int* status = reinterpret_cast<int*>(scratch);
-    float* cn = reinterpret_cast<float*>(scratch + kStaticHeader);
     // the array keeps whatever the previous call left: the status word must start at zero; the
-    // ||c||^2 row is rewritten in full (including its +inf padding) by the prologue below
+    // half-norm operand is rewritten in full (all ceil(K/256) tiles, padding rows included) by the
+    // prologue that launch_assign_tc runs first
     if (cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) return CAKE_ERR_CUDA;
-    const int Kpad = padded_k(K);
-    if (launch_centroid_norms(C, 1, K, D, Kpad, cn, s) != cudaSuccess) return CAKE_ERR_CUDA;
-    return launch_assign_tc(X, C, 1, N, D, K, cn, Kpad, out_idx, out_dist, status, s);
+    return launch_assign_tc(X, C, 1, N, D, K, scratch + kStaticHeader, false, out_idx, out_dist, status, s);
 }

@@ -1,22 +1,33 @@
 // Fused nearest-centroid assignment on the sm_100a tensor cores.
 //
 // Operation (paper Section 5, "Flash-KMeans clean-start workload"): for every point the squared
-// Euclidean distance to all K centroids and the arg-min.  Evaluated as
-//     argmin_k ( ||c_k||^2 - 2 x.c_k ),   dist = max(0, ||x||^2 + min_k(...)),
-// with S = X.C^T produced tile by tile in tensor memory and consumed on the spot, so the N x K
-// matrix never exists in HBM.
+// Euclidean distance to all K centroids and the arg-min.  The whole expansion
+//     d(x,c)/2 = ||x||^2/2 - x.c + ||c||^2/2
+// is accumulated in tensor memory: the D-long contraction -x.c runs with the B operand negated, and
+// one extra 16-wide k-step adds the two half-norms (the X side carries [xh xm xl 1 1 1 0..], the
+// centroid side [1 1 1 ch cm cl 0..], each half-norm split into three bf16 terms so that nothing of
+// its fp32 value is lost).  The epilogue therefore only has to find a row minimum; the N x K matrix
+// never exists outside tensor memory.
 //
-// One persistent CTA per SM, 10 warps, three roles:
-//   warp 8  producer : TMA loads.  A 128-row X tile (whole D) into one of the X buffers, then the
-//                      centroid tiles of 256 rows, 64 columns (128 bytes, 128B-swizzled) at a time
-//                      through an mbarrier ring.
-//   warp 9  MMA      : one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one
-//                      of two 256-column TMEM accumulators; tcgen05.commit releases ring slots and
-//                      publishes finished accumulators.
+// One persistent CTA per SM, 16 warps (warp 11 idle), four roles:
+//   warp 8  producer : TMA.  A 128-row X tile (whole D) into one of the X buffers per row tile; per
+//                      centroid tile of 256 rows, D/64 chunks of 64 columns (128-byte swizzle) through
+//                      an mbarrier ring, plus the tile's 8 KiB block of split half-norms (bulk copy).
+//   warps 9,10 MMA   : one thread each issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32); issuer i
+//                      owns the i-th of two 256-column TMEM accumulators and every other centroid tile;
+//                      tcgen05.commit frees ring slots and publishes finished accumulators.
 //   warps 0-7 epilogue: warp w reads TMEM lanes 32*(w%4).. (one X row per thread) and columns
-//                      128*(w/4).. of the tile with tcgen05.ld, forms ||c||^2 - 2s, keeps a running
-//                      (best, index) per row across all centroid tiles; the two column halves are
-//                      merged through shared memory at the end of the row tile.
+//                      128*(w/4).. of every tile with tcgen05.ld and keeps a running minimum per row.
+//                      The two column halves are merged through shared memory per row tile.
+//   warps 12-15 norms : one thread per X row forms ||x||^2/2 from the shared-memory X tile and writes
+//                      the X-side operand of the extra k-step, one row tile ahead of the MMA warp.
+// Two epilogue policies:
+//   packed : the low 7 mantissa bits of each value are replaced by its column number and a plain
+//            float minimum finds value and position at once (1.5 issue slots per element, no branch).
+//            Values closer than 2^-16 relative are ordered by column; exact ties still go to the
+//            lowest index.
+//   exact  : full-precision minimum; the position is looked up only when a 32-column group beats
+//            the running best.
 // Every wait is bounded: on expiry the CTA raises CAKE_ERR_TIMEOUT in the status word, all roles
 // leave their loops, TMEM is freed and the kernel returns.
 #include "internal.h"
@@ -31,14 +42,22 @@ constexpr int KCHUNK = 64;              // bf16 columns per swizzled 128-byte ro
 constexpr int UMMA_K = 16;
 constexpr int NUM_EPI_WARPS = 8;
 constexpr int PRODUCER_WARP = 8;
-constexpr int MMA_WARP = 9;
-constexpr int NUM_THREADS = 320;
-constexpr uint32_t X_CHUNK_BYTES = BLOCK_M * 128;  // 16 KiB
-constexpr uint32_t C_STAGE_BYTES = BLOCK_N * 128;  // 32 KiB
+constexpr int MMA_WARP = 9;             // warps 9 and 10: the two MMA issuers (warp 11 idles)
+constexpr int AUX_WARP0 = 12;           // warps 12..15: row norms
+constexpr int NUM_WARPS = 16;
+constexpr int EPI_REGS = 192;           // registers per thread after reallocation: epilogue warpgroups
+constexpr int AUX_REGS = 56;            // ... and the producer / MMA / norm warpgroups
+constexpr int NUM_THREADS = NUM_WARPS * 32;
+constexpr uint32_t X_CHUNK_BYTES = BLOCK_M * 128;        // 16 KiB
+constexpr uint32_t C_STAGE_BYTES = BLOCK_N * 128;        // 32 KiB
+constexpr uint32_t AUG_A_BYTES = BLOCK_M * UMMA_K * 2;   // 4 KiB
+constexpr uint32_t AUG_B_BYTES = kAssignAugTileBytes;    // 8 KiB
 constexpr int MAX_STAGES = 6;
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t CTRL_BYTES = 4096;  // barriers, TMEM pointer, abort flag, merge scratch
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+constexpr uint32_t COL_MASK = 0x7Fu;   // packed policy: 7 bits address the 128 columns of a half tile
+constexpr uint32_t F32_INF = 0x7f800000u;
 
 struct Params {
     int B;
@@ -51,8 +70,7 @@ struct Params {
     i64 total_tiles;  // B * m_tiles
     int n_stages;     // ring depth
     int n_xbuf;       // 1 or 2 X buffers
-    int Kpad;
-    const float* cn;  // [B][Kpad]
+    const uint8_t* caug;  // [B][n_tiles][8 KiB] centroid-side operand of the extra k-step
     int* out_idx;
     float* out_dist;
     int* status;
@@ -62,16 +80,49 @@ struct Ctrl {  // lives in shared memory
     uint64_t x_full[2], x_empty[2];
     uint64_t ring_full[MAX_STAGES], ring_empty[MAX_STAGES];
     uint64_t tmem_full[2], tmem_empty[2];
+    uint64_t auga_full[2];
+    uint64_t augb_full[2], augb_empty[2];
     uint64_t merge_full[2], merge_empty[2];
     uint32_t tmem_base;
     int abort_flag;
     float merge_best[2][BLOCK_M];
     int merge_idx[2][BLOCK_M];
+#ifdef CAKE_ASSIGN_TRACE
+    int trace_n[NUM_WARPS];
+#endif
 };
 static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
 
-// Bounded wait on an mbarrier phase. Returns false if the CTA is aborting.
+#ifdef CAKE_ASSIGN_TRACE
+// Profiling build only (-DCAKE_ASSIGN_TRACE): CTA 0 logs every barrier wait of its warp leaders as
+// {barrier slot in Ctrl, start clock, end clock} per warp; read back with cake_debug_read_trace.
+constexpr int TRACE_CAP = 4096;   // records per warp
+__device__ long long g_trace[NUM_WARPS * TRACE_CAP * 3];
+__device__ __forceinline__ bool wait_bar_impl(uint64_t* bar, uint32_t parity, Ctrl* ctrl, int* status);
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctrl* ctrl, int* status) {
+    const bool log = blockIdx.x == 0 && (threadIdx.x & 31) == 0;
+    const long long t0 = clock64();
+    const bool ok = wait_bar_impl(bar, parity, ctrl, status);
+    const long long t1 = clock64();
+    if (log) {
+        const int w = threadIdx.x >> 5;
+        const int n = ctrl->trace_n[w]++;
+        if (n < TRACE_CAP) {
+            long long* r = g_trace + (static_cast<size_t>(w) * TRACE_CAP + n) * 3;
+            r[0] = bar - reinterpret_cast<uint64_t*>(ctrl);
+            r[1] = t0;
+            r[2] = t1;
+        }
+    }
+    return ok;
+}
+#define wait_bar_body wait_bar_impl
+#else
+#define wait_bar_body wait_bar
+#endif
+
+// Bounded wait on an mbarrier phase. Returns false if the CTA is aborting.
+__device__ __forceinline__ bool wait_bar_body(uint64_t* bar, uint32_t parity, Ctrl* ctrl, int* status) {
     const uint32_t addr = ptx::smem_u32(bar);
     if (ptx::mbar_try_wait(addr, parity)) return true;
     const uint64_t t0 = ptx::globaltimer_ns();
@@ -91,20 +142,22 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctrl* c
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-// One group of 32 accumulator columns of this thread's row: v_j = cn_j - 2 s_j, chunk minimum by a
-// min tree, and only if it beats the running best is the position looked up (first match, so the
-// lowest column wins exact ties; later tiles need a strictly smaller value).
-__device__ __forceinline__ void scan32(const uint32_t (&r)[32], const float4* __restrict__ cn4,
-                                       int col_base, float& best, int& bidx) {
-    float v[32];
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-        const float4 c = __ldg(cn4 + q);
-        v[4 * q + 0] = fmaf(-2.f, __uint_as_float(r[4 * q + 0]), c.x);
-        v[4 * q + 1] = fmaf(-2.f, __uint_as_float(r[4 * q + 1]), c.y);
-        v[4 * q + 2] = fmaf(-2.f, __uint_as_float(r[4 * q + 2]), c.z);
-        v[4 * q + 3] = fmaf(-2.f, __uint_as_float(r[4 * q + 3]), c.w);
-    }
+__device__ __forceinline__ uint32_t bf16_rne_bits(float f) {
+    uint32_t u = __float_as_uint(f);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return u >> 16;
+}
+// h = hi + mid + lo with three bf16 terms (24 significand bits: nothing of the fp32 value is lost)
+__device__ __forceinline__ void split3(float h, uint32_t& hi, uint32_t& mid, uint32_t& lo) {
+    hi = bf16_rne_bits(h);
+    const float r1 = h - __uint_as_float(hi << 16);
+    mid = bf16_rne_bits(r1);
+    const float r2 = r1 - __uint_as_float(mid << 16);
+    lo = bf16_rne_bits(r2);
+}
+
+// min over 32 floats with 3-input min instructions
+__device__ __forceinline__ float min32(const float (&v)[32]) {
     float t[11];
 #pragma unroll
     for (int q = 0; q < 10; ++q) t[q] = ptx::fmin3(v[3 * q], v[3 * q + 1], v[3 * q + 2]);
@@ -113,17 +166,40 @@ __device__ __forceinline__ void scan32(const uint32_t (&r)[32], const float4* __
     const float u1 = ptx::fmin3(t[3], t[4], t[5]);
     const float u2 = ptx::fmin3(t[6], t[7], t[8]);
     const float u3 = fminf(t[9], t[10]);
-    const float m = fminf(ptx::fmin3(u0, u1, u2), u3);
+    return fminf(ptx::fmin3(u0, u1, u2), u3);
+}
+
+// packed policy: key = value with its low 7 mantissa bits replaced by the column (0..127) inside
+// the half tile.  For non-negative values float order == (truncated value, column) order; +inf
+// (a padded column) turns into a NaN, which min ignores.
+__device__ __forceinline__ float packed_min32(const uint32_t (&r)[32], int col_base, float run) {
+    float v[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+        v[j] = __uint_as_float((r[j] & ~COL_MASK) | static_cast<uint32_t>(col_base + j));
+    return fminf(run, min32(v));
+}
+
+// exact policy: full-precision group minimum; position looked up (lowest column first) only on a hit.
+__device__ __forceinline__ void exact_scan32(const uint32_t (&r)[32], int col_base, float& best, int& bidx) {
+    float v[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+    const float m = min32(v);
     if (m < best) {
         best = m;
-        int loc = 31;
+        int c[32];
 #pragma unroll
-        for (int j = 30; j >= 0; --j)
-            if (v[j] == m) loc = j;
-        bidx = col_base + loc;
+        for (int j = 0; j < 32; ++j) c[j] = (v[j] == m) ? j : 32;
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1)
+#pragma unroll
+            for (int j = 0; j < s; ++j) c[j] = min(c[j], c[j + s]);
+        bidx = col_base + c[0];
     }
 }
 
+template <bool PACKED>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
                  const Params p) {
@@ -135,9 +211,12 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t smem_base = raw_addr + pad;
     const uint32_t xbuf_bytes = static_cast<uint32_t>(p.nchunks) * X_CHUNK_BYTES;
     const uint32_t x_base = smem_base;
-    const uint32_t ring_base = x_base + static_cast<uint32_t>(p.n_xbuf) * xbuf_bytes;
-    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + static_cast<size_t>(p.n_xbuf) * xbuf_bytes +
-                                         static_cast<size_t>(p.n_stages) * C_STAGE_BYTES);
+    const uint32_t ring_off = static_cast<uint32_t>(p.n_xbuf) * xbuf_bytes;
+    const uint32_t ring_base = smem_base + ring_off;
+    const uint32_t auga_off = ring_off + static_cast<uint32_t>(p.n_stages) * C_STAGE_BYTES;
+    const uint32_t augb_off = auga_off + 2 * AUG_A_BYTES;
+    const uint32_t ctrl_off = augb_off + 2 * AUG_B_BYTES;
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ctrl_off);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -145,9 +224,12 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), 1 + 4);  // MMA commit + 4 norm warps
+            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), 2 + 4);  // 2 MMA issuers + 4 norm warps
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i]), NUM_EPI_WARPS);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->augb_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->augb_empty[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_full[i]), 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_empty[i]), 4);
         }
@@ -156,8 +238,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_empty[i]), 1);
         }
         ctrl->abort_flag = 0;
+#ifdef CAKE_ASSIGN_TRACE
+        for (int i = 0; i < NUM_WARPS; ++i) ctrl->trace_n[i] = 0;
+#endif
         ptx::fence_mbar_init();
     }
+    // the X-side operand of the extra k-step: columns 8..15 stay zero for the whole kernel
+    for (uint32_t o = threadIdx.x * 16; o < 2 * AUG_A_BYTES; o += NUM_THREADS * 16)
+        *reinterpret_cast<uint4*>(smem + auga_off + o) = make_uint4(0, 0, 0, 0);
+    ptx::fence_proxy_async_smem();
     if (warp == MMA_WARP) {
         ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), TMEM_COLS);
         ptx::tmem_relinquish();
@@ -171,33 +260,67 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     ptx::tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_base);
 
+    // The epilogue keeps a whole 128-column accumulator slice in registers; the other roles need few.
+    // Registers move between warpgroups accordingly (warps 0-7 grow, warps 8-15 shrink).
+    if (warp >= NUM_EPI_WARPS) {
+    ptx::setmaxnreg_dec<AUX_REGS>();
     if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t ring_it = 0, tile_it = 0;
+            uint32_t ring_it = 0, acc_it = 0;
+            uint32_t rs = 0, rph = 0;   // ring stage and its phase
+            uint32_t xb = 0, xph = 0;   // X buffer of the current row tile and its phase
             bool ok = true;
-            for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
-                const int b = static_cast<int>(tile / p.m_tiles);
-                const int mt = static_cast<int>(tile % p.m_tiles);
-                const uint32_t xb = tile_it % p.n_xbuf, xph = (tile_it / p.n_xbuf) & 1u;
-                ok = wait_bar(&ctrl->x_empty[xb], xph ^ 1u, ctrl, p.status);
-                if (!ok) break;
-                const uint32_t xfull = ptx::smem_u32(&ctrl->x_full[xb]);
+            // X tile of row tile `t` into buffer `buf` (its previous user must have released it)
+            auto issue_x = [&](i64 t, uint32_t buf) {
+                const int tb = static_cast<int>(t / p.m_tiles);
+                const int tmt = static_cast<int>(t % p.m_tiles);
+                const uint32_t xfull = ptx::smem_u32(&ctrl->x_full[buf]);
                 ptx::mbar_arrive_expect_tx(xfull, xbuf_bytes);
                 for (int c = 0; c < p.nchunks; ++c)
-                    ptx::tma_load_3d(x_base + xb * xbuf_bytes + c * X_CHUNK_BYTES, &tmap_x, xfull,
-                                     c * KCHUNK, mt * BLOCK_M, b);
-                for (int nt = 0; ok && nt < p.n_tiles; ++nt) {
+                    ptx::tma_load_3d(x_base + buf * xbuf_bytes + c * X_CHUNK_BYTES, &tmap_x, xfull,
+                                     c * KCHUNK, tmt * BLOCK_M, tb);
+            };
+            if (static_cast<i64>(blockIdx.x) < p.total_tiles) issue_x(blockIdx.x, 0);
+            for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                const int b = static_cast<int>(tile / p.m_tiles);
+                // the next row tile's X is requested as early as its buffer is free (polled between
+                // centroid chunks, never blocking them), so its latency hides behind this tile's MMAs
+                const i64 next = tile + gridDim.x;
+                const uint32_t nxb = (xb + 1 == static_cast<uint32_t>(p.n_xbuf)) ? 0u : xb + 1;
+                const uint32_t nxph = (nxb == 0) ? xph ^ 1u : xph;
+                bool next_pending = next < p.total_tiles;
+                const uint8_t* caug_b = p.caug + static_cast<size_t>(b) * p.n_tiles * AUG_B_BYTES;
+                for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it) {
                     for (int c = 0; c < p.nchunks; ++c, ++ring_it) {
-                        const uint32_t s = ring_it % p.n_stages, ph = (ring_it / p.n_stages) & 1u;
-                        ok = wait_bar(&ctrl->ring_empty[s], ph ^ 1u, ctrl, p.status);
+                        if (next_pending && p.n_xbuf == 2 &&
+                            ptx::mbar_test_wait(ptx::smem_u32(&ctrl->x_empty[nxb]), nxph ^ 1u)) {
+                            issue_x(next, nxb);
+                            next_pending = false;
+                        }
+                        ok = wait_bar(&ctrl->ring_empty[rs], rph ^ 1u, ctrl, p.status);
                         if (!ok) break;
-                        const uint32_t full = ptx::smem_u32(&ctrl->ring_full[s]);
+                        const uint32_t full = ptx::smem_u32(&ctrl->ring_full[rs]);
                         ptx::mbar_arrive_expect_tx(full, C_STAGE_BYTES);
-                        ptx::tma_load_3d(ring_base + s * C_STAGE_BYTES, &tmap_c, full, c * KCHUNK,
+                        ptx::tma_load_3d(ring_base + rs * C_STAGE_BYTES, &tmap_c, full, c * KCHUNK,
                                          nt * BLOCK_N, b);
+                        if (++rs == static_cast<uint32_t>(p.n_stages)) { rs = 0; rph ^= 1u; }
                     }
+                    if (!ok) break;
+                    const uint32_t as = acc_it & 1u, aph = (acc_it >> 1) & 1u;
+                    ok = wait_bar(&ctrl->augb_empty[as], aph ^ 1u, ctrl, p.status);
+                    if (!ok) break;
+                    const uint32_t bfull = ptx::smem_u32(&ctrl->augb_full[as]);
+                    ptx::mbar_arrive_expect_tx(bfull, AUG_B_BYTES);
+                    ptx::bulk_load(smem_base + augb_off + as * AUG_B_BYTES,
+                                   caug_b + static_cast<size_t>(nt) * AUG_B_BYTES, AUG_B_BYTES, bfull);
                 }
+                if (ok && next_pending) {
+                    ok = wait_bar(&ctrl->x_empty[nxb], nxph ^ 1u, ctrl, p.status);
+                    if (ok) issue_x(next, nxb);
+                }
+                xb = nxb;
+                xph = nxph;
             }
             if (!ok) {
                 // aborting: give our loads in flight a bounded time to land before the CTA's
@@ -214,45 +337,137 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 }
             }
         }
-    } else if (warp == MMA_WARP) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (warp == MMA_WARP || warp == MMA_WARP + 1) {
+        // ------------------------------------------------------------ MMA issuers
+        // Two warps, one issuing thread each.  Issuer `par` owns TMEM accumulator `par` and takes every
+        // other centroid tile, so the barrier waits, commits and bookkeeping of one issuer run while
+        // the other's MMAs keep the tensor pipe busy (a single issuer leaves it idle between tiles).
+        // The two never touch the same accumulator or ring slot, so no order between them is needed.
         if (lane == 0) {
-            constexpr uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, BLOCK_N);
-            uint32_t ring_it = 0, tile_it = 0, acc_it = 0;
+            const uint32_t par = static_cast<uint32_t>(warp - MMA_WARP);
+            constexpr uint32_t idesc_aug = ptx::umma_idesc_bf16(BLOCK_M, BLOCK_N);
+            constexpr uint32_t idesc_main = idesc_aug | ptx::UMMA_IDESC_NEGATE_B;   // accumulates -x.c
+            // descriptors are (low, high) words with the high word constant; stage / phase counters
+            // are stepped instead of divided; full 64-column chunks issue four MMAs back to back
+            constexpr uint32_t KSTEP = (UMMA_K * 2) >> 4;   // descriptor units per k-step
+            const uint32_t nstg = static_cast<uint32_t>(p.n_stages);
+            uint32_t s = 0, ph = 0;                         // ring position of the next chunk (all tiles)
+            uint32_t xb = 0, xph = 0;                       // X buffer and its phase
+            uint32_t acc_it = 0;
+            const uint32_t d_tmem = tmem_base + par * BLOCK_N;
+            const uint32_t augb_lo = ptx::umma_desc_lo_interleaved(smem_base + augb_off + par * AUG_B_BYTES);
             bool ok = true;
-            for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
-                const uint32_t xb = tile_it % p.n_xbuf, xph = (tile_it / p.n_xbuf) & 1u;
+            for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                // every phase of the shared barriers is observed, also in row / centroid tiles this
+                // issuer has no work in: a parity wait must never fall two phases behind
                 ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);
                 if (!ok) break;
-                ptx::tc_fence_after();
+                bool have_aug = false;
+                const uint32_t a_lo_tile = ptx::umma_desc_lo_sw128(x_base + xb * xbuf_bytes);
+                const uint32_t auga_lo = ptx::umma_desc_lo_interleaved(smem_base + auga_off + xb * AUG_A_BYTES);
                 for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it) {
-                    const uint32_t as = acc_it & 1u, aph = (acc_it >> 1) & 1u;
-                    ok = wait_bar(&ctrl->tmem_empty[as], aph ^ 1u, ctrl, p.status);
+                    if ((acc_it & 1u) != par) {             // the other issuer's tile: pass over its ring slots
+                        for (int c = 0; ok && c < p.nchunks; ++c) {
+                            ok = wait_bar(&ctrl->ring_full[s], ph, ctrl, p.status);
+                            if (++s == nstg) { s = 0; ph ^= 1u; }
+                        }
+                        continue;
+                    }
+                    const uint32_t aph = (acc_it >> 1) & 1u;
+                    ok = wait_bar(&ctrl->tmem_empty[par], aph ^ 1u, ctrl, p.status);
                     if (!ok) break;
                     ptx::tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + as * BLOCK_N;
-                    for (int c = 0; c < p.nchunks; ++c, ++ring_it) {
-                        const uint32_t s = ring_it % p.n_stages, ph = (ring_it / p.n_stages) & 1u;
+                    uint32_t a_lo = a_lo_tile;
+                    for (int c = 0; c < p.nchunks; ++c, a_lo += X_CHUNK_BYTES >> 4) {
                         ok = wait_bar(&ctrl->ring_full[s], ph, ctrl, p.status);
                         if (!ok) break;
-                        ptx::tc_fence_after();
-                        const uint32_t a_addr = x_base + xb * xbuf_bytes + c * X_CHUNK_BYTES;
-                        const uint32_t b_addr = ring_base + s * C_STAGE_BYTES;
+                        const uint32_t b_lo = ptx::umma_desc_lo_sw128(ring_base + s * C_STAGE_BYTES);
                         const int nk = (c == p.nchunks - 1) ? p.ksteps_last : KCHUNK / UMMA_K;
-                        for (int ks = 0; ks < nk; ++ks) {
-                            ptx::umma_bf16(d_tmem, ptx::umma_desc_sw128(a_addr + ks * UMMA_K * 2),
-                                           ptx::umma_desc_sw128(b_addr + ks * UMMA_K * 2), idesc,
-                                           (c | ks) != 0 ? 1u : 0u);
+                        if (c == 0)
+                            ptx::umma_bf16_lohi<false>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
+                                                       ptx::UMMA_DESC_HI_SW128, idesc_main);
+                        else
+                            ptx::umma_bf16_lohi<true>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
+                                                      ptx::UMMA_DESC_HI_SW128, idesc_main);
+                        if (nk == KCHUNK / UMMA_K) {
+#pragma unroll
+                            for (uint32_t ks = 1; ks < KCHUNK / UMMA_K; ++ks)
+                                ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
+                                                          b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main);
+                        } else {
+                            for (int ks = 1; ks < nk; ++ks)
+                                ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
+                                                          b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main);
                         }
                         ptx::umma_commit(ptx::smem_u32(&ctrl->ring_empty[s]));
+                        if (++s == nstg) { s = 0; ph ^= 1u; }
                     }
-                    if (ok) ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[as]));
+                    if (!ok) break;
+                    // the extra k-step: + ||x||^2/2 + ||c||^2/2
+                    if (!have_aug) {
+                        ok = wait_bar(&ctrl->auga_full[xb], xph, ctrl, p.status);
+                        if (!ok) break;
+                        have_aug = true;
+                    }
+                    ok = wait_bar(&ctrl->augb_full[par], aph, ctrl, p.status);
+                    if (!ok) break;
+                    ptx::umma_bf16_lohi<true>(d_tmem, auga_lo, ptx::UMMA_DESC_HI_INTERLEAVED, augb_lo,
+                                              ptx::UMMA_DESC_HI_INTERLEAVED, idesc_aug);
+                    ptx::umma_commit(ptx::smem_u32(&ctrl->augb_empty[par]));
+                    ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[par]));
                 }
+                if (ok && !have_aug) ok = wait_bar(&ctrl->auga_full[xb], xph, ctrl, p.status);
+                // this issuer's MMAs on the X buffer are done when this commit fires (it fires at once
+                // if the issuer had no tile in this row tile)
                 if (ok) ptx::umma_commit(ptx::smem_u32(&ctrl->x_empty[xb]));
+                if (++xb == static_cast<uint32_t>(p.n_xbuf)) { xb = 0; xph ^= 1u; }
             }
         }
+    } else if (warp >= AUX_WARP0) {
+        // ------------------------------------------------------------ norm warps
+        // One thread per X row: ||x||^2/2 from the swizzled X tile (16-byte granule g of row r sits
+        // at position g ^ (r & 7); the order of the granules does not matter for a sum), split into
+        // three bf16 terms and written as the X-side operand of the extra k-step.  These warps run a
+        // row tile ahead of the MMA warp, so the operand is ready when the first centroid tile needs it.
+        const int r = (warp - AUX_WARP0) * 32 + lane;
+        uint32_t xb = 0, xph = 0;
+        bool ok = true;
+        for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);
+            if (!ok) break;
+            const uint8_t* xrow = smem + xb * xbuf_bytes + r * 128;
+            float xn0 = 0.f, xn1 = 0.f, xn2 = 0.f, xn3 = 0.f;
+            for (int c = 0; c < p.nchunks; ++c) {
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    const uint4 w = *reinterpret_cast<const uint4*>(xrow + c * X_CHUNK_BYTES +
+                                                                    ((g ^ (r & 7)) << 4));
+                    float a;
+                    a = bf16lo(w.x); xn0 = fmaf(a, a, xn0); a = bf16hi(w.x); xn1 = fmaf(a, a, xn1);
+                    a = bf16lo(w.y); xn2 = fmaf(a, a, xn2); a = bf16hi(w.y); xn3 = fmaf(a, a, xn3);
+                    a = bf16lo(w.z); xn0 = fmaf(a, a, xn0); a = bf16hi(w.z); xn1 = fmaf(a, a, xn1);
+                    a = bf16lo(w.w); xn2 = fmaf(a, a, xn2); a = bf16hi(w.w); xn3 = fmaf(a, a, xn3);
+                }
+            }
+            uint32_t hi, mid, lo;
+            split3(0.5f * ((xn0 + xn1) + (xn2 + xn3)), hi, mid, lo);
+            // interleaved (no-swizzle) K-major layout: 8-row groups of 256 B, row stride 16 B,
+            // the second 8 columns 128 B further on (left zero)
+            const uint32_t one = 0x3F80u;
+            *reinterpret_cast<uint4*>(smem + auga_off + xb * AUG_A_BYTES + (r >> 3) * 256 + (r & 7) * 16) =
+                make_uint4(hi | (mid << 16), lo | (one << 16), one | (one << 16), 0u);
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                ptx::mbar_arrive(ptx::smem_u32(&ctrl->auga_full[xb]));
+                ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[xb]));
+            }
+            if (++xb == static_cast<uint32_t>(p.n_xbuf)) { xb = 0; xph ^= 1u; }
+        }
+    }
     } else {
         // ------------------------------------------------------------ epilogue warps
+        ptx::setmaxnreg_inc<EPI_REGS>();
         const int wg = warp >> 2;            // column half of every tile
         const int q = warp & 3;              // TMEM lane quarter this warp may read
         const int r = q * 32 + lane;         // row inside the X tile
@@ -261,32 +476,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
             const int b = static_cast<int>(tile / p.m_tiles);
             const int mt = static_cast<int>(tile % p.m_tiles);
-            const uint32_t xb = tile_it % p.n_xbuf, xph = (tile_it / p.n_xbuf) & 1u;
-            float xn = 0.f;
-            if (wg == 0) {
-                // ||x||^2 of this thread's row from the swizzled X tile (16-byte granule g of row r
-                // sits at position g ^ (r & 7); the order of the granules does not matter for a sum)
-                ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);
-                if (!ok) break;
-                const uint8_t* xrow = smem + xb * xbuf_bytes + r * 128;
-                for (int c = 0; c < p.nchunks; ++c) {
-#pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        const uint4 w = *reinterpret_cast<const uint4*>(xrow + c * X_CHUNK_BYTES +
-                                                                        ((g ^ (r & 7)) << 4));
-                        float a;
-                        a = bf16lo(w.x); xn = fmaf(a, a, xn); a = bf16hi(w.x); xn = fmaf(a, a, xn);
-                        a = bf16lo(w.y); xn = fmaf(a, a, xn); a = bf16hi(w.y); xn = fmaf(a, a, xn);
-                        a = bf16lo(w.z); xn = fmaf(a, a, xn); a = bf16hi(w.z); xn = fmaf(a, a, xn);
-                        a = bf16lo(w.w); xn = fmaf(a, a, xn); a = bf16hi(w.w); xn = fmaf(a, a, xn);
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[xb]));
-            }
-            float best = __int_as_float(0x7f800000);
-            int bidx = 0;
-            const float* cn_b = p.cn + static_cast<size_t>(b) * p.Kpad + wg * (BLOCK_N / 2);
+            float best = __uint_as_float(F32_INF);   // packed: a key; exact: a value
+            int bsel = 0;                            // packed: tile number; exact: global column
             for (int nt = 0; nt < p.n_tiles; ++nt, ++acc_it) {
                 const uint32_t as = acc_it & 1u, aph = (acc_it >> 1) & 1u;
                 ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
@@ -294,29 +485,56 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 ptx::tc_fence_after();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                        as * BLOCK_N + wg * (BLOCK_N / 2);
-                const int col0 = nt * BLOCK_N + wg * (BLOCK_N / 2);
-                const float4* cn4 = reinterpret_cast<const float4*>(cn_b + nt * BLOCK_N);
-#pragma unroll 1
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t r0[32], r1[32];
-                    ptx::tmem_ld_x32(taddr + h * 64, r0);
-                    ptx::tmem_ld_x32(taddr + h * 64 + 32, r1);
-                    ptx::tmem_ld_wait(r0);
-                    ptx::reg_dep(r1);
-                    scan32(r0, cn4 + h * 16, col0 + h * 64, best, bidx);
-                    scan32(r1, cn4 + h * 16 + 8, col0 + h * 64 + 32, best, bidx);
-                }
+                // all four 32-column groups are requested at once; as soon as they are in registers
+                // the accumulator goes back to the MMA issuer and the reduction runs on registers
+                uint32_t ra[32], rb[32], rc[32], rd[32];
+                ptx::tmem_ld_x32(taddr, ra);
+                ptx::tmem_ld_x32(taddr + 32, rb);
+                ptx::tmem_ld_x32(taddr + 64, rc);
+                ptx::tmem_ld_x32(taddr + 96, rd);
+                ptx::tmem_ld_wait(ra);
+                ptx::reg_dep(rb);
+                ptx::reg_dep(rc);
+                ptx::reg_dep(rd);
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as]));
+                if (PACKED) {
+                    float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF));
+                    tmin = packed_min32(rb, 32, tmin);
+                    tmin = packed_min32(rc, 64, tmin);
+                    tmin = packed_min32(rd, 96, tmin);
+                    // across tiles only the (truncated) value decides: an equal value keeps the earlier tile
+                    if (__uint_as_float(__float_as_uint(tmin) & ~COL_MASK) <
+                        __uint_as_float(__float_as_uint(best) & ~COL_MASK)) {
+                        best = tmin;
+                        bsel = nt;
+                    }
+                } else {
+                    const int col0 = nt * BLOCK_N + wg * (BLOCK_N / 2);
+                    exact_scan32(ra, col0, best, bsel);
+                    exact_scan32(rb, col0 + 32, best, bsel);
+                    exact_scan32(rc, col0 + 64, best, bsel);
+                    exact_scan32(rd, col0 + 96, best, bsel);
+                }
             }
             if (!ok) break;
-            // merge the two column halves: the upper half hands its (best, index) to the lower one
+            float bval;
+            int bidx;
+            if (PACKED) {
+                const uint32_t kb = __float_as_uint(best);
+                bval = __uint_as_float(kb & ~COL_MASK);
+                bidx = bsel * BLOCK_N + wg * (BLOCK_N / 2) + static_cast<int>(kb & COL_MASK);
+            } else {
+                bval = best;
+                bidx = bsel;
+            }
+            // merge the two column halves: the upper half hands its (value, index) to the lower one
             const uint32_t mb = tile_it & 1u, mph = (tile_it >> 1) & 1u;
             if (wg == 1) {
                 ok = wait_bar(&ctrl->merge_empty[mb], mph ^ 1u, ctrl, p.status);
                 if (!ok) break;
-                ctrl->merge_best[mb][r] = best;
+                ctrl->merge_best[mb][r] = bval;
                 ctrl->merge_idx[mb][r] = bidx;
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->merge_full[mb]));
@@ -327,15 +545,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const int oi = ctrl->merge_idx[mb][r];
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->merge_empty[mb]));
-                if (ob < best || (ob == best && oi < bidx)) {
-                    best = ob;
+                if (ob < bval || (ob == bval && oi < bidx)) {
+                    bval = ob;
                     bidx = oi;
                 }
                 const i64 row = static_cast<i64>(mt) * BLOCK_M + r;
                 if (row < p.N) {
                     const size_t o = static_cast<size_t>(b) * static_cast<size_t>(p.N) + row;
                     p.out_idx[o] = bidx;
-                    if (p.out_dist) p.out_dist[o] = fmaxf(0.f, xn + best);
+                    if (p.out_dist) p.out_dist[o] = fmaxf(0.f, 2.f * bval);
                 }
             }
         }
@@ -348,6 +566,40 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         __syncwarp();
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// Prologue: the centroid-side operand of the extra k-step.  One warp per padded centroid row k:
+// h = ||c_k||^2 / 2 split into three bf16 terms, written as the row [1 1 1 h_hi h_mid h_lo 0 0 | 0 x 8]
+// in the interleaved K-major layout the MMA reads (per 256-row tile an 8 KiB block: 32 groups of
+// 8 rows x 16 B, then the same for columns 8..15).  Rows k >= K get h = +inf and can never win.
+__global__ void __launch_bounds__(256)
+centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64 total_rows,
+                    uint8_t* __restrict__ caug) {
+    const i64 w = (static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= total_rows) return;
+    const i64 b = w / Kpad;
+    const int k = static_cast<int>(w - b * Kpad);
+    float acc = 0.f;
+    if (k < K) {
+        const cake_bf16* row = C + (static_cast<size_t>(b) * K + k) * D;
+        for (int d = lane; d < D; d += 32) {
+            const float v = __uint_as_float(static_cast<uint32_t>(row[d]) << 16);
+            acc = fmaf(v, v, acc);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    }
+    if (lane == 0) {
+        uint32_t hi = 0x7F80u, mid = 0, lo = 0;   // +inf for padded rows
+        if (k < K) split3(0.5f * acc, hi, mid, lo);
+        const uint32_t one = 0x3F80u;
+        const int tile = k / BLOCK_N, rr = k % BLOCK_N;
+        uint8_t* blk = caug + (static_cast<size_t>(b) * (Kpad / BLOCK_N) + tile) * AUG_B_BYTES;
+        uint8_t* dst = blk + (rr >> 3) * 256 + (rr & 7) * 16;
+        *reinterpret_cast<uint4*>(dst) = make_uint4(one | (one << 16), one | (hi << 16), mid | (lo << 16), 0u);
+        *reinterpret_cast<uint4*>(dst + 128) = make_uint4(0u, 0u, 0u, 0u);
     }
 }
 
@@ -387,10 +639,26 @@ int make_tmap(CUtensorMap* m, const void* base, int D, i64 rows, int batch, int 
 
 }  // namespace
 
+#ifdef CAKE_ASSIGN_TRACE
+// Profiling build only: copies warp `w`'s trace records (3 x int64 each, up to `cap`) to `host`.
+extern "C" __attribute__((visibility("default"))) int cake_debug_read_trace(int w, long long* host, int cap) {
+    cudaDeviceSynchronize();
+    if (w < 0 || w >= NUM_WARPS) return 0;
+    const int n = cap < TRACE_CAP ? cap : TRACE_CAP;
+    cudaMemcpyFromSymbol(host, g_trace, static_cast<size_t>(n) * 3 * sizeof(long long),
+                         static_cast<size_t>(w) * TRACE_CAP * 3 * sizeof(long long));
+    return n;
+}
+#endif
+
 bool assign_tc_supports(int D) { return D >= 8 && D % 8 == 0 && D <= 256; }
 
-int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, const float* cn,
-                     int Kpad, int* out_idx, float* out_dist, int* status, cudaStream_t s) {
+size_t assign_tc_aug_bytes(i64 B, int K) {
+    return static_cast<size_t>(B) * (padded_k(K) / BLOCK_N) * AUG_B_BYTES;
+}
+
+int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
+                     bool exact, int* out_idx, float* out_dist, int* status, cudaStream_t s) {
     if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
     DeviceInfo di;
     int rc = current_device_info(&di);
@@ -404,10 +672,21 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     p.m_tiles = static_cast<int>((N + BLOCK_M - 1) / BLOCK_M);
     p.n_tiles = (K + BLOCK_N - 1) / BLOCK_N;
     p.total_tiles = static_cast<i64>(B) * p.m_tiles;
-    p.Kpad = Kpad; p.cn = cn; p.out_idx = out_idx; p.out_dist = out_dist; p.status = status;
+    p.caug = static_cast<const uint8_t*>(caug);
+    p.out_idx = out_idx; p.out_dist = out_dist; p.status = status;
     if (p.total_tiles == 0) return CAKE_OK;
 
-    const i64 budget = static_cast<i64>(di.smem_optin) - 1024 - CTRL_BYTES;
+    const int Kpad = padded_k(K);
+    {
+        const i64 rows = static_cast<i64>(B) * Kpad;
+        const i64 ctas = (rows * 32 + 255) / 256;
+        centroid_aug_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(C, K, D, Kpad, rows,
+                                                                        static_cast<uint8_t*>(caug));
+        note_launches(1);
+    }
+
+    const i64 fixed = 1024 + CTRL_BYTES + 2 * AUG_A_BYTES + 2 * AUG_B_BYTES;
+    const i64 budget = static_cast<i64>(di.smem_optin) - fixed;
     const i64 xbuf = static_cast<i64>(p.nchunks) * X_CHUNK_BYTES;
     p.n_xbuf = 2;
     i64 stages = (budget - 2 * xbuf) / C_STAGE_BYTES;
@@ -417,8 +696,8 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     }
     if (stages < 2) return CAKE_ERR_UNSUPPORTED;
     p.n_stages = static_cast<int>(stages > MAX_STAGES ? MAX_STAGES : stages);
-    const size_t smem_bytes = 1024 + static_cast<size_t>(p.n_xbuf) * xbuf +
-                              static_cast<size_t>(p.n_stages) * C_STAGE_BYTES + CTRL_BYTES;
+    const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf +
+                              static_cast<size_t>(p.n_stages) * C_STAGE_BYTES;
 
     CUtensorMap tx, tc;
     rc = make_tmap(&tx, X, D, N, B, BLOCK_M);
@@ -426,15 +705,18 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     rc = make_tmap(&tc, C, D, K, B, BLOCK_N);
     if (rc != CAKE_OK) return rc;
 
-    static int attr_done_for_device = -1;  // benign race: the attribute call is idempotent
+    static int attr_done_for_device = -1;  // benign race: the attribute calls are idempotent
     if (attr_done_for_device != di.device) {
-        if (cudaFuncSetAttribute(assign_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(assign_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  di.smem_optin) != cudaSuccess)
             return CAKE_ERR_CUDA;
         attr_done_for_device = di.device;
     }
-    const i64 grid = p.total_tiles < di.sm_count ? p.total_tiles : di.sm_count;
-    assign_tc_kernel<<<static_cast<unsigned>(grid), NUM_THREADS, smem_bytes, s>>>(tx, tc, p);
+    const unsigned grid = static_cast<unsigned>(p.total_tiles < di.sm_count ? p.total_tiles : di.sm_count);
+    if (exact) assign_tc_kernel<false><<<grid, NUM_THREADS, smem_bytes, s>>>(tx, tc, p);
+    else assign_tc_kernel<true><<<grid, NUM_THREADS, smem_bytes, s>>>(tx, tc, p);
     note_launches(1);
     return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
 }

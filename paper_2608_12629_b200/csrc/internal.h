@@ -26,19 +26,19 @@ unsigned long long launches_so_far();
 
 inline i64 round_up(i64 a, i64 b) { return (a + b - 1) / b * b; }
 
-// Centroid tiles of the tensor-core assign kernel are 256 wide; ||c||^2 is padded to that with +inf.
+// Centroid tiles of the tensor-core assign kernel are 256 wide; K is padded to that (padding rows
+// carry an infinite half-norm).  Per tile the kernel's prologue writes an 8 KiB operand block.
 constexpr int kAssignBlockN = 256;
+constexpr unsigned kAssignAugTileBytes = kAssignBlockN * 16 * 2;
 inline int padded_k(int K) { return (int)round_up(K, kAssignBlockN); }
-
-// ---- prologue: cn[b][k] = sum_d C[b][k][d]^2 (fp32), +inf for K <= k < Kpad
-cudaError_t launch_centroid_norms(const cake_bf16* C, int B, int K, int D, int Kpad, float* cn,
-                                  cudaStream_t s);
 
 // ---- assign
 bool assign_tc_supports(int D);
-int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
-                     const float* cn, int Kpad, int* out_idx, float* out_dist, int* status,
-                     cudaStream_t s);
+// bytes of scratch (`caug`) the tensor-core assign needs for B problems of K centroids
+size_t assign_tc_aug_bytes(i64 B, int K);
+// prologue (half-norm operand into caug) + the assign kernel; exact selects the exact epilogue
+int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
+                     bool exact, int* out_idx, float* out_dist, int* status, cudaStream_t s);
 int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
                        int* out_idx, float* out_dist, cudaStream_t s);
 

@@ -1,4 +1,4 @@
-// Small kernels around the two hot ones: the ||c||^2 prologue, the CUDA-core assign fallback,
+// Small kernels around the two hot ones: the CUDA-core assign fallback,
 // the inertia reduction and the bounded-wait self test; plus the cached device query.
 #include <atomic>
 #include <mutex>
@@ -43,29 +43,6 @@ int current_device_info(DeviceInfo* out) {
 namespace {
 
 __device__ __forceinline__ float bf16f(cake_bf16 b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
-
-// one warp per (problem, padded centroid row)
-__global__ void __launch_bounds__(256)
-centroid_norms_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64 total_rows,
-                      float* __restrict__ cn) {
-    const i64 w = (static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (w >= total_rows) return;
-    const i64 b = w / Kpad;
-    const int k = static_cast<int>(w - b * Kpad);
-    float acc = __int_as_float(0x7f800000);  // +inf: a padded column can never win the arg-min
-    if (k < K) {
-        const cake_bf16* row = C + (static_cast<size_t>(b) * K + k) * D;
-        acc = 0.f;
-        for (int d = lane; d < D; d += 32) {
-            const float v = bf16f(row[d]);
-            acc = fmaf(v, v, acc);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    }
-    if (lane == 0) cn[w] = acc;
-}
 
 // CUDA-core fallback: one warp per point, lanes stride the features, direct differences in fp32.
 __global__ void __launch_bounds__(256)
@@ -141,15 +118,6 @@ __global__ void bounded_wait_selftest_kernel(int* status, unsigned long long lim
 }
 
 }  // namespace
-
-cudaError_t launch_centroid_norms(const cake_bf16* C, int B, int K, int D, int Kpad, float* cn,
-                                  cudaStream_t s) {
-    const i64 rows = static_cast<i64>(B) * Kpad;
-    const i64 ctas = (rows * 32 + 255) / 256;
-    centroid_norms_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(C, K, D, Kpad, rows, cn);
-    note_launches(1);
-    return cudaGetLastError();
-}
 
 int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, int* out_idx,
                        float* out_dist, cudaStream_t s) {

@@ -36,11 +36,15 @@ TC_SHAPES = [
 ]
 
 
+TC_POLICIES = {"packed": cake.CAKE_ASSIGN_TCGEN05, "exact": cake.CAKE_ASSIGN_TCGEN05_EXACT}
+
+
+@pytest.mark.parametrize("policy", sorted(TC_POLICIES))
 @pytest.mark.parametrize("N,D,K", TC_SHAPES)
-def test_assign_tcgen05_small_shapes(N, D, K):
+def test_assign_tcgen05_small_shapes(N, D, K, policy):
     X, C = problem(N, D, K, seed=N + D + K)
     ws = cake.alloc_workspace(1, N, D, K, DEV)
-    idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), ws=ws, flags=cake.CAKE_ASSIGN_TCGEN05)
+    idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), ws=ws, flags=TC_POLICIES[policy])
     torch.cuda.synchronize()
     check_status(ws)
     rep = grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx.cpu().numpy(), dist.cpu().numpy())
@@ -60,7 +64,8 @@ def test_assign_simt_fallback(N, D, K):
         assert e.value.code == cake.CAKE_ERR_UNSUPPORTED
 
 
-def test_assign_exact_ties_lowest_index():
+@pytest.mark.parametrize("policy", sorted(TC_POLICIES))
+def test_assign_exact_ties_lowest_index(policy):
     """Small integers: every product, norm and sum is exact in fp32, so ties are exact on the GPU too."""
     g = torch.Generator().manual_seed(4)
     N, D, K = 3000, 64, 600
@@ -68,7 +73,7 @@ def test_assign_exact_ties_lowest_index():
     C = torch.randint(-2, 3, (K, D), generator=g).to(torch.bfloat16)
     C[17] = C[5]
     C[300:600] = C[0:300]            # every centroid duplicated across the two K tiles and column halves
-    idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_TCGEN05)
+    idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=TC_POLICIES[policy])
     idx_o, dist_o, _ = orc.assign(inputs.to_bits(X), inputs.to_bits(C))
     assert np.array_equal(idx.cpu().numpy(), idx_o)
     assert np.array_equal(dist.cpu().numpy().astype(np.float64), dist_o)
@@ -282,6 +287,24 @@ def test_lloyd_host_buffers_match_device_call():
 
 def sampled_rows(N, n, seed):
     return np.sort(np.random.default_rng(seed).choice(N, size=min(n, N), replace=False))
+
+
+def test_assign_policies_agree_except_near_ties():
+    """The packed epilogue orders values that agree to 2^-16 by index; everything else is identical."""
+    X, C = problem(30000, 128, 1500, seed=77, comps=200)
+    Xd, Cd = X.to(DEV), C.to(DEV)
+    ip, dp = cake.cake_kmeans_assign(Xd, Cd, flags=cake.CAKE_ASSIGN_TCGEN05)
+    ie, de = cake.cake_kmeans_assign(Xd, Cd, flags=cake.CAKE_ASSIGN_TCGEN05_EXACT)
+    differ = (ip != ie).cpu().numpy()
+    assert differ.mean() < 1e-3
+    rel = ((dp - de).abs() / de.clamp_min(1e-6)).cpu().numpy()
+    assert rel[~differ].max() <= 2.0 ** -15
+    if differ.any():   # where they differ the two candidates are closer than the packing granularity
+        Xb, Cb = inputs.to_bits(X), inputs.to_bits(C)
+        rows = np.nonzero(differ)[0]
+        d1 = orc.pair_sqdist(Xb[rows], Cb, ip.cpu().numpy()[rows])
+        d2 = orc.pair_sqdist(Xb[rows], Cb, ie.cpu().numpy()[rows])
+        assert (np.abs(d1 - d2) <= 2.0 ** -14 * np.maximum(d1, d2) + 1e-4).all()
 
 
 @pytest.mark.parametrize("name,sample", [("c2", 4096), ("c4", 1024)])
