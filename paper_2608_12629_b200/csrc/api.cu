@@ -14,9 +14,10 @@ struct Workspace {
     int* status;          // [64] header, word 0 = sticky device status
     void* caug;           // [B][Kpad/256][8 KiB] half-norm operand of the tensor-core assign
     float* sums;          // [B][K][D]
-    int* offsets;         // [B][K+1]
+    int* nvalid;          // [B]
     int* cursor;          // [B][K]
-    int* perm;            // [B][N]
+    int2* pairs;          // [B][N] (row, cluster) in cluster order
+    int* part;            // [B][slabs][K] per-slab histograms of the sort route
     cake_bf16* cbuf[2];   // [B][K][D] each
     float* dist;          // [B][N]
     size_t bytes;
@@ -31,9 +32,10 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     w.status = reinterpret_cast<int*>(take(256));
     w.caug = take(assign_tc_aug_bytes(B, K));
     w.sums = reinterpret_cast<float*>(take(kd * 4));
-    w.offsets = reinterpret_cast<int*>(take(static_cast<size_t>(B) * (K + 1) * 4));
+    w.nvalid = reinterpret_cast<int*>(take(static_cast<size_t>(B) * 4));
     w.cursor = reinterpret_cast<int*>(take(static_cast<size_t>(B) * K * 4));
-    w.perm = reinterpret_cast<int*>(take(static_cast<size_t>(B) * N * 4));
+    w.pairs = reinterpret_cast<int2*>(take(static_cast<size_t>(B) * N * 8));
+    w.part = reinterpret_cast<int*>(take(update_sort_part_bytes(B, N, K)));
     w.cbuf[0] = reinterpret_cast<cake_bf16*>(take(kd * 2));
     w.cbuf[1] = reinterpret_cast<cake_bf16*>(take(kd * 2));
     w.dist = reinterpret_cast<float*>(take(static_cast<size_t>(B) * N * 4));
@@ -76,12 +78,16 @@ int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, co
     int rc = current_device_info(&di);
     if (rc != CAKE_OK) return rc;
     unsigned path = flags & CAKE_UPDATE_MASK;
-    if (path == CAKE_UPDATE_AUTO)
-        path = update_smem_supports(D, K, di.smem_optin) ? CAKE_UPDATE_SMEM : CAKE_UPDATE_SORT;
+    if (path == CAKE_UPDATE_AUTO) {
+        // the shared-memory table wins only while the whole problem is launch-bound (measured:
+        // N=32,768 D=64 K=128); the sort route is faster everywhere else
+        const bool tiny = static_cast<double>(B) * N * D <= 4.0e6;
+        path = (tiny && update_smem_supports(D, K, di.smem_optin)) ? CAKE_UPDATE_SMEM : CAKE_UPDATE_SORT;
+    }
     if (path == CAKE_UPDATE_SMEM) {
         rc = launch_update_smem(X, idx, B, N, D, K, w.sums, out_counts, w.status, s);
     } else if (path == CAKE_UPDATE_SORT) {
-        UpdateScratch scr{w.sums, w.offsets, w.cursor, w.perm};
+        UpdateScratch scr{w.sums, w.nvalid, w.cursor, w.pairs, w.part};
         rc = launch_update_sort(X, idx, B, N, D, K, scr, out_counts, w.status, s);
     } else {
         rc = CAKE_ERR_UNSUPPORTED;

@@ -7,7 +7,8 @@
 //                global one at the end.  For K*D*4 bytes that fit in one SM's shared memory.
 //   sort route : counting sort by cluster (histogram, exclusive scan, scatter of row numbers) and a
 //                segmented reduction in which each warp sums a fixed-size run of the sorted order
-//                in registers and adds one partial per cluster it touches.  Any K.
+//                in registers and adds one partial per cluster it touches.  Any K; for K <= 8192 the
+//                sort works on per-slab shared-memory histograms and needs no global atomics.
 // Both stream X exactly once with 16-byte (smem route: 4-byte) loads; HBM bandwidth is the bound.
 #include "internal.h"
 
@@ -90,18 +91,18 @@ update_smem_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
 }
 
 // ======================================================================= sort route
+// Counting sort of the row numbers by cluster, then a segmented reduction over the sorted order.
+//   sorted array : pairs[pos] = (row number, its cluster), pos in [0, n_valid)
+// K <= BLK_MAX_K ("blocked"): per-slab shared-memory histograms, no global atomics, no zero-fill
+// launches (hist_blocked zeroes `sums`, colscan writes `counts`).
+// Larger K: global atomics (few rows per cluster, little contention).
+
+// ---- large-K pieces
 constexpr int HIST_THREADS = 512;
-constexpr int HIST_SMEM_MAX_K = 8192;
 
 __global__ void __launch_bounds__(HIST_THREADS)
 hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts, int* status) {
-    extern __shared__ int h[];
     const int b = blockIdx.y;
-    const bool use_smem = K <= HIST_SMEM_MAX_K;
-    if (use_smem) {
-        for (int e = threadIdx.x; e < K; e += blockDim.x) h[e] = 0;
-        __syncthreads();
-    }
     const int* idx_b = idx + static_cast<size_t>(b) * N;
     int* counts_b = counts + static_cast<size_t>(b) * K;
     bool bad = false;
@@ -109,30 +110,45 @@ hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts,
          i += static_cast<i64>(gridDim.x) * blockDim.x) {
         const int k = idx_b[i];
         if (k < 0 || k >= K) { bad = true; continue; }
-        if (use_smem) atomicAdd(&h[k], 1);
-        else atomicAdd(counts_b + k, 1);
+        atomicAdd(counts_b + k, 1);
     }
     if (bad) atomicCAS(status, CAKE_OK, CAKE_ERR_BAD_INDEX);
-    if (use_smem) {
-        __syncthreads();
-        for (int e = threadIdx.x; e < K; e += blockDim.x)
-            if (h[e]) atomicAdd(counts_b + e, h[e]);
-    }
 }
 
-// offsets[b][k] = sum_{j<k} counts[b][j], offsets[b][K] = total; cursor = offsets[0..K)
+// cursor[b][k] = sum_{j<k} counts[b][j]; nvalid[b] = total.  CTA (tile, problem) owns SCAN_TILE
+// consecutive clusters; it first re-sums everything before its tile (coalesced, a few hundred KB at
+// most), so the tiles need no communication and one launch does the whole scan.
+constexpr int SCAN_TILE = 4096;
+
 __global__ void __launch_bounds__(1024)
-scan_kernel(const int* __restrict__ counts, int K, int* __restrict__ offsets, int* __restrict__ cursor) {
+scan_kernel(const int* __restrict__ counts, int K, int* __restrict__ cursor, int* __restrict__ nvalid) {
     __shared__ int warp_tot[32];
-    const int b = blockIdx.x;
+    __shared__ int pre_s;
+    const int b = blockIdx.y, tile = blockIdx.x;
     const int* c = counts + static_cast<size_t>(b) * K;
-    int* off = offsets + static_cast<size_t>(b) * (K + 1);
     int* cur = cursor + static_cast<size_t>(b) * K;
-    const int per = (K + blockDim.x - 1) / blockDim.x;
-    const int k0 = threadIdx.x * per, k1 = (k0 + per < K) ? k0 + per : K;
-    int local = 0;
-    for (int k = k0; k < k1; ++k) local += c[k];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // 1. everything before the tile
+    int pre = 0;
+    for (int i = threadIdx.x; i < tile * SCAN_TILE; i += 1024) pre += c[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) pre += __shfl_xor_sync(0xffffffffu, pre, o);
+    if (lane == 0) warp_tot[warp] = pre;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int w = 0; w < 32; ++w) t += warp_tot[w];
+        pre_s = t;
+    }
+    __syncthreads();
+    pre = pre_s;
+    __syncthreads();
+    // 2. the tile: four consecutive clusters per thread
+    const int k0 = tile * SCAN_TILE + threadIdx.x * 4;
+    int v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = (k0 + j < K) ? c[k0 + j] : 0;
+    const int local = v[0] + v[1] + v[2] + v[3];
     int incl = local;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -151,23 +167,23 @@ scan_kernel(const int* __restrict__ counts, int K, int* __restrict__ offsets, in
         warp_tot[lane] = t;  // inclusive over warps
     }
     __syncthreads();
-    int run = incl - local + (warp ? warp_tot[warp - 1] : 0);
-    for (int k = k0; k < k1; ++k) {
-        off[k] = run;
-        cur[k] = run;
-        run += c[k];
+    int run = pre + incl - local + (warp ? warp_tot[warp - 1] : 0);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (k0 + j < K) cur[k0 + j] = run;
+        run += v[j];
     }
-    if (threadIdx.x == blockDim.x - 1) off[K] = warp_tot[31];
+    if (tile == static_cast<int>(gridDim.x) - 1 && threadIdx.x == 0) nvalid[b] = pre + warp_tot[31];
 }
 
-// perm[b][pos] = i, pos taken from the cluster's cursor; lanes of a warp that hit the same cluster
-// take their slots with a single atomic.
+// pos taken from the cluster's cursor; lanes of a warp that hit the same cluster take their slots
+// with a single atomic.
 __global__ void __launch_bounds__(256)
-scatter_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ cursor, int* __restrict__ perm) {
+scatter_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ cursor, int2* __restrict__ pairs) {
     const int b = blockIdx.y;
     const int* idx_b = idx + static_cast<size_t>(b) * N;
     int* cur = cursor + static_cast<size_t>(b) * K;
-    int* perm_b = perm + static_cast<size_t>(b) * N;
+    int2* pairs_b = pairs + static_cast<size_t>(b) * N;
     const int lane = threadIdx.x & 31;
     const i64 span = static_cast<i64>(gridDim.x) * blockDim.x;
     const i64 n_round = (N + 31) / 32 * 32;  // keep whole warps in the loop for the match
@@ -184,50 +200,191 @@ scatter_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ curs
             int base = 0;
             if (lane == leader) base = atomicAdd(cur + k, __popc(peers));
             base = __shfl_sync(peers, base, leader);
-            perm_b[base + rank] = static_cast<int>(i);
+            pairs_b[base + rank] = make_int2(static_cast<int>(i), k);
         }
     }
 }
 
-// Segmented reduction over the sorted order. Each warp owns SEG_ROWS consecutive sorted positions.
-// A row is read as 16-byte granules (8 bf16); LPR lanes share a row, 32/LPR rows are read at once.
+// ---- blocked pieces (K <= BLK_MAX_K)
+//   hist_blocked : CTA (slab, problem) histograms its slab of idx in shared memory and writes the
+//                  K counters to part[problem][slab][*]; it also zeroes its share of `sums`.
+//   colscan      : per cluster, exclusive prefix over the slabs (in place) and the total -> counts.
+//   scatter_blocked : CTA (slab, problem) scans counts (redundantly per CTA) into cluster offsets,
+//                  forms base[k] = offset[k] + part[slab][k] in shared memory and hands every row of
+//                  its slab the next free position of its cluster.
+constexpr int BLK_THREADS = 256;
+constexpr int BLK_MAX_K = 8192;
+constexpr int BLK_MAX_BLOCKS = 128;
+constexpr int BLK_MIN_SLAB = 8192;
+constexpr int BLK_VEC = 4;            // idx values per load; slabs are multiples of it
+
+__global__ void __launch_bounds__(BLK_THREADS)
+hist_blocked_kernel(const int* __restrict__ idx, i64 N, int K, i64 slab, int* __restrict__ part,
+                    float* __restrict__ sums, i64 sums_per_problem, int* status) {
+    extern __shared__ int h[];
+    const int b = blockIdx.y, blk = blockIdx.x, nblk = gridDim.x;
+    for (int e = threadIdx.x; e < K; e += blockDim.x) h[e] = 0;
+    __syncthreads();
+    const int* idx_b = idx + static_cast<size_t>(b) * N;
+    const i64 r0 = slab * blk, r1 = (r0 + slab < N) ? r0 + slab : N;
+    bool bad = false;
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(idx_b + r0) & 15) == 0;
+    i64 i = r0 + static_cast<i64>(threadIdx.x) * BLK_VEC;
+    if (vec_ok) {
+        for (; i + BLK_VEC <= r1; i += static_cast<i64>(blockDim.x) * BLK_VEC) {
+            const int4 k4 = *reinterpret_cast<const int4*>(idx_b + i);
+            const int ks[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (ks[u] < 0 || ks[u] >= K) bad = true;
+                else atomicAdd(&h[ks[u]], 1);
+            }
+        }
+    }
+    // ragged tail (or everything, if the slab start is not 16-byte aligned)
+    for (i64 j = vec_ok ? i : r0 + threadIdx.x; j < r1; j += vec_ok ? 1 : blockDim.x) {
+        if (vec_ok && j >= i + BLK_VEC) break;
+        const int k = idx_b[j];
+        if (k < 0 || k >= K) bad = true;
+        else atomicAdd(&h[k], 1);
+    }
+    if (bad) atomicCAS(status, CAKE_OK, CAKE_ERR_BAD_INDEX);
+    // this CTA's share of the fp32 sums starts at zero
+    const i64 z0 = sums_per_problem * blk / nblk, z1 = sums_per_problem * (blk + 1) / nblk;
+    float* sums_b = sums + static_cast<size_t>(b) * sums_per_problem;
+    for (i64 e = z0 + threadIdx.x; e < z1; e += blockDim.x) sums_b[e] = 0.f;
+    __syncthreads();
+    int* out = part + (static_cast<size_t>(b) * nblk + blk) * K;
+    for (int e = threadIdx.x; e < K; e += blockDim.x) out[e] = h[e];
+}
+
+// CTA = 32 clusters (lanes) x 8 warps; warp w owns a contiguous range of slabs.
+__global__ void __launch_bounds__(256)
+colscan_kernel(int* __restrict__ part, int nblk, int K, int* __restrict__ counts, int* __restrict__ nvalid) {
+    __shared__ int tot[8][32];
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int k = blockIdx.x * 32 + lane;
+    const int per = (nblk + 7) / 8;
+    const int j0 = warp * per, j1 = (j0 + per < nblk) ? j0 + per : nblk;
+    int* p = part + static_cast<size_t>(b) * nblk * K + k;
+    int v[16];                                     // nblk <= 128 -> per <= 16
+#pragma unroll
+    for (int u = 0; u < 16; ++u) v[u] = (k < K && j0 + u < j1) ? p[static_cast<size_t>(j0 + u) * K] : 0;
+    int sum = 0;
+#pragma unroll
+    for (int u = 0; u < 16; ++u) sum += v[u];
+    tot[warp][lane] = sum;
+    __syncthreads();
+    int run = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        if (w < warp) run += tot[w][lane];
+        total += tot[w][lane];
+    }
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
+        if (k < K && j0 + u < j1) p[static_cast<size_t>(j0 + u) * K] = run;
+        run += v[u];
+    }
+    if (warp == 0 && k < K) counts[static_cast<size_t>(b) * K + k] = total;
+    (void)nvalid;
+}
+
+__global__ void __launch_bounds__(BLK_THREADS)
+scatter_blocked_kernel(const int* __restrict__ idx, i64 N, int K, i64 slab, const int* __restrict__ part,
+                       const int* __restrict__ counts, int* __restrict__ nvalid, int2* __restrict__ pairs) {
+    extern __shared__ int base[];                 // [K]
+    __shared__ int warp_tot[BLK_THREADS / 32];
+    const int b = blockIdx.y, blk = blockIdx.x, nblk = gridDim.x;
+    const int* c = counts + static_cast<size_t>(b) * K;
+    const int* pre = part + (static_cast<size_t>(b) * nblk + blk) * K;
+    // exclusive scan of counts: each thread owns `per` consecutive clusters
+    const int per = (K + BLK_THREADS - 1) / BLK_THREADS;
+    const int k0 = threadIdx.x * per, k1 = (k0 + per < K) ? k0 + per : K;
+    int local = 0;
+    for (int k = k0; k < k1; ++k) local += c[k];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < BLK_THREADS / 32; ++w) {
+        if (w < warp) before += warp_tot[w];
+        total += warp_tot[w];
+    }
+    int run = before + incl - local;
+    for (int k = k0; k < k1; ++k) {
+        base[k] = run + pre[k];
+        run += c[k];
+    }
+    if (blk == 0 && threadIdx.x == 0) nvalid[b] = total;
+    __syncthreads();
+    const int* idx_b = idx + static_cast<size_t>(b) * N;
+    int2* pairs_b = pairs + static_cast<size_t>(b) * N;
+    const i64 r0 = slab * blk, r1 = (r0 + slab < N) ? r0 + slab : N;
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(idx_b + r0) & 15) == 0;
+    i64 i = r0 + static_cast<i64>(threadIdx.x) * BLK_VEC;
+    if (vec_ok) {
+        for (; i + BLK_VEC <= r1; i += static_cast<i64>(blockDim.x) * BLK_VEC) {
+            const int4 k4 = *reinterpret_cast<const int4*>(idx_b + i);
+            const int ks[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (ks[u] >= 0 && ks[u] < K)
+                    pairs_b[atomicAdd(&base[ks[u]], 1)] = make_int2(static_cast<int>(i + u), ks[u]);
+            }
+        }
+    }
+    for (i64 j = vec_ok ? i : r0 + threadIdx.x; j < r1; j += vec_ok ? 1 : blockDim.x) {
+        if (vec_ok && j >= i + BLK_VEC) break;
+        const int k = idx_b[j];
+        if (k >= 0 && k < K) pairs_b[atomicAdd(&base[k], 1)] = make_int2(static_cast<int>(j), k);
+    }
+}
+
+// ---- segmented reduction over the sorted order.  Each warp owns SEG_ROWS consecutive sorted
+// positions; it loads their row numbers and cluster ids once (two per lane) and hands them out by
+// shuffles.  A row is read as 16-byte granules (8 bf16); LPR lanes share a row, 32/LPR rows are read
+// per pass and several passes are in flight.  One vector atomic pair per granule per cluster touched.
 constexpr int SEG_ROWS = 64;
 constexpr int SEG_WARPS = 8;
-constexpr int SEG_UNROLL = 4;
 
 template <int GPL>  // granules per lane (D <= 256*GPL)
 __global__ void __launch_bounds__(SEG_WARPS * 32)
-segreduce_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ perm,
-                 const int* __restrict__ offsets, i64 N, int D, int K, int lpr,
-                 float* __restrict__ sums) {
+segreduce_kernel(const cake_bf16* __restrict__ X, const int2* __restrict__ pairs,
+                 const int* __restrict__ nvalid, i64 N, int D, int K, int lpr, float* __restrict__ sums) {
+    constexpr int SEG_UNROLL = GPL == 1 ? 8 : 4;   // passes in flight
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const i64 w = static_cast<i64>(blockIdx.x) * SEG_WARPS + (threadIdx.x >> 5);
-    const int* off = offsets + static_cast<size_t>(b) * (K + 1);
-    const int n_valid = off[K];
+    const int n_valid = nvalid[b];
     const i64 p0 = w * SEG_ROWS;
     if (p0 >= n_valid) return;
     const int p1 = static_cast<int>((p0 + SEG_ROWS < n_valid) ? p0 + SEG_ROWS : n_valid);
-    const int* perm_b = perm + static_cast<size_t>(b) * N;
+    const int2* pairs_b = pairs + static_cast<size_t>(b) * N;
     const uint4* Xg = reinterpret_cast<const uint4*>(X) + static_cast<size_t>(b) * N * (D >> 3);
     float* sums_b = sums + static_cast<size_t>(b) * K * D;
     const int G = D >> 3;           // granules per row
     const int rpp = 32 / lpr;       // rows per pass
     const int sl = lane % lpr;      // granule slot inside the row
     const int rs = lane / lpr;      // row slot
+    const bool in0 = p0 + lane < p1, in1 = p0 + 32 + lane < p1;
+    const int2 pk0 = in0 ? __ldg(pairs_b + p0 + lane) : make_int2(0, -1);
+    const int2 pk1 = in1 ? __ldg(pairs_b + p0 + 32 + lane) : make_int2(0, -1);
+    const int pr0 = pk0.x, pr1 = pk1.x, ky0 = pk0.y, ky1 = pk1.y;
 
-    // cluster containing position p0: largest k with off[k] <= p0
-    int lo = 0, hi = K;             // invariant: off[lo] <= p0 < off[hi]
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (off[mid] <= static_cast<int>(p0)) lo = mid; else hi = mid;
-    }
-    int k = lo;
     int p = static_cast<int>(p0);
     while (p < p1) {
-        const int kend = off[k + 1];
-        if (kend <= p) { ++k; continue; }
-        const int e = kend < p1 ? kend : p1;
+        // the run of equal keys that starts at p (the order is sorted, so it is contiguous)
+        const int o0 = p - static_cast<int>(p0);
+        const int k = o0 < 32 ? __shfl_sync(0xffffffffu, ky0, o0) : __shfl_sync(0xffffffffu, ky1, o0 - 32);
+        const int e = p + __popc(__ballot_sync(0xffffffffu, ky0 == k)) + __popc(__ballot_sync(0xffffffffu, ky1 == k));
         float acc[GPL][8];
 #pragma unroll
         for (int g = 0; g < GPL; ++g)
@@ -239,7 +396,10 @@ segreduce_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ perm,
             for (int u = 0; u < SEG_UNROLL; ++u) {
                 const int pos = q + u * rpp + rs;
                 const bool on = pos < e;
-                const int row = on ? __ldg(perm_b + pos) : 0;
+                const int o = pos - static_cast<int>(p0);
+                const int ra = __shfl_sync(0xffffffffu, pr0, o & 31);
+                const int rb = __shfl_sync(0xffffffffu, pr1, o & 31);
+                const int row = o < 32 ? ra : rb;
 #pragma unroll
                 for (int g = 0; g < GPL; ++g) {
                     const int gi = sl + g * lpr;
@@ -280,33 +440,27 @@ segreduce_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ perm,
 
 // Scalar variant for D not a multiple of 8 (or very large D): one warp per run, lanes stride columns.
 __global__ void __launch_bounds__(SEG_WARPS * 32)
-segreduce_scalar_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ perm,
-                        const int* __restrict__ offsets, i64 N, int D, int K, float* __restrict__ sums) {
+segreduce_scalar_kernel(const cake_bf16* __restrict__ X, const int2* __restrict__ pairs,
+                        const int* __restrict__ nvalid, i64 N, int D, int K, float* __restrict__ sums) {
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const i64 w = static_cast<i64>(blockIdx.x) * SEG_WARPS + (threadIdx.x >> 5);
-    const int* off = offsets + static_cast<size_t>(b) * (K + 1);
-    const int n_valid = off[K];
+    const int n_valid = nvalid[b];
     const i64 p0 = w * SEG_ROWS;
     if (p0 >= n_valid) return;
     const int p1 = static_cast<int>((p0 + SEG_ROWS < n_valid) ? p0 + SEG_ROWS : n_valid);
-    const int* perm_b = perm + static_cast<size_t>(b) * N;
+    const int2* pairs_b = pairs + static_cast<size_t>(b) * N;
     const cake_bf16* Xb = X + static_cast<size_t>(b) * N * D;
     float* sums_b = sums + static_cast<size_t>(b) * K * D;
-    int lo = 0, hi = K;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (off[mid] <= static_cast<int>(p0)) lo = mid; else hi = mid;
-    }
-    int k = lo, p = static_cast<int>(p0);
+    int p = static_cast<int>(p0);
     while (p < p1) {
-        const int kend = off[k + 1];
-        if (kend <= p) { ++k; continue; }
-        const int e = kend < p1 ? kend : p1;
+        const int k = pairs_b[p].y;
+        int e = p + 1;
+        while (e < p1 && pairs_b[e].y == k) ++e;
         for (int c = lane; c < D; c += 32) {
             float a = 0.f;
             for (int q = p; q < e; ++q)
-                a += __uint_as_float(static_cast<uint32_t>(Xb[static_cast<size_t>(perm_b[q]) * D + c]) << 16);
+                a += __uint_as_float(static_cast<uint32_t>(Xb[static_cast<size_t>(pairs_b[q].x) * D + c]) << 16);
             atomicAdd(sums_b + static_cast<size_t>(k) * D + c, a);
         }
         p = e;
@@ -334,6 +488,35 @@ finalize_kernel(const float* __restrict__ sums, const int* __restrict__ counts,
         else v = C_prev ? __uint_as_float(static_cast<uint32_t>(C_prev[e]) << 16) : 0.f;
         out_C[e] = v;
         if (out_C_bf16) out_C_bf16[e] = f32_to_bf16_rne(v);
+    }
+}
+
+// D % 4 == 0: four columns per thread, 16-byte loads and stores
+__global__ void __launch_bounds__(256)
+finalize4_kernel(const float4* __restrict__ sums, const int* __restrict__ counts,
+                 const uint2* __restrict__ C_prev, i64 total4, int D4, float4* __restrict__ out_C,
+                 uint2* __restrict__ out_C_bf16) {
+    for (i64 e = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; e < total4;
+         e += static_cast<i64>(gridDim.x) * blockDim.x) {
+        const int n = counts[e / D4];
+        float4 v;
+        if (n > 0) {
+            const float4 sv = sums[e];
+            const float fn = static_cast<float>(n);
+            v = make_float4(sv.x / fn, sv.y / fn, sv.z / fn, sv.w / fn);
+        } else if (C_prev) {
+            const uint2 pv = C_prev[e];
+            v = make_float4(bf16lo(pv.x), bf16hi(pv.x), bf16lo(pv.y), bf16hi(pv.y));
+        } else {
+            v = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        out_C[e] = v;
+        if (out_C_bf16) {
+            uint2 o;
+            o.x = static_cast<uint32_t>(f32_to_bf16_rne(v.x)) | (static_cast<uint32_t>(f32_to_bf16_rne(v.y)) << 16);
+            o.y = static_cast<uint32_t>(f32_to_bf16_rne(v.z)) | (static_cast<uint32_t>(f32_to_bf16_rne(v.w)) << 16);
+            out_C_bf16[e] = o;
+        }
     }
 }
 
@@ -379,31 +562,66 @@ int launch_update_smem(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
     return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
 }
 
+namespace {
+struct SortPlan {
+    bool blocked;
+    int nblk;
+    i64 slab;
+};
+SortPlan sort_plan(i64 N, int K) {
+    SortPlan pl;
+    pl.blocked = K <= BLK_MAX_K;
+    i64 nblk = (N + BLK_MIN_SLAB - 1) / BLK_MIN_SLAB;
+    if (nblk > BLK_MAX_BLOCKS) nblk = BLK_MAX_BLOCKS;
+    if (nblk < 1) nblk = 1;
+    pl.nblk = static_cast<int>(nblk);
+    pl.slab = ((N + nblk - 1) / nblk + BLK_VEC - 1) / BLK_VEC * BLK_VEC;
+    return pl;
+}
+}  // namespace
+
+size_t update_sort_part_bytes(i64 B, i64 N, int K) {
+    const SortPlan pl = sort_plan(N, K);
+    return pl.blocked ? static_cast<size_t>(B) * pl.nblk * K * sizeof(int) : 0;
+}
+
 int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K,
                        const UpdateScratch& scr, int* counts, int* status, cudaStream_t s) {
     DeviceInfo di;
     int rc = current_device_info(&di);
     if (rc != CAKE_OK) return rc;
     const size_t kd = static_cast<size_t>(B) * K * D;
-    if (cudaMemsetAsync(scr.sums, 0, kd * sizeof(float), s) != cudaSuccess) return CAKE_ERR_CUDA;
-    if (cudaMemsetAsync(counts, 0, static_cast<size_t>(B) * K * sizeof(int), s) != cudaSuccess)
-        return CAKE_ERR_CUDA;
-    if (N == 0) return CAKE_OK;
-    {
-        i64 ctas = (N + HIST_THREADS * 8 - 1) / (HIST_THREADS * 8);
-        const i64 cap = (static_cast<i64>(di.sm_count) * 4 + B - 1) / B;
-        if (ctas > cap) ctas = cap;
-        if (ctas < 1) ctas = 1;
-        const size_t smem = K <= HIST_SMEM_MAX_K ? static_cast<size_t>(K) * 4 : 0;
-        hist_kernel<<<dim3(static_cast<unsigned>(ctas), B), HIST_THREADS, smem, s>>>(idx, N, K, counts, status);
+    const SortPlan pl = sort_plan(N, K);
+    if (N == 0 || !pl.blocked) {
+        if (cudaMemsetAsync(scr.sums, 0, kd * sizeof(float), s) != cudaSuccess) return CAKE_ERR_CUDA;
+        if (cudaMemsetAsync(counts, 0, static_cast<size_t>(B) * K * sizeof(int), s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
     }
-    scan_kernel<<<B, 1024, 0, s>>>(counts, K, scr.offsets, scr.cursor);
-    {
-        i64 ctas = (N + 256 * 4 - 1) / (256 * 4);
-        const i64 cap = (static_cast<i64>(di.sm_count) * 8 + B - 1) / B;
-        if (ctas > cap) ctas = cap;
-        if (ctas < 1) ctas = 1;
-        scatter_kernel<<<dim3(static_cast<unsigned>(ctas), B), 256, 0, s>>>(idx, N, K, scr.cursor, scr.perm);
+    if (N == 0) return CAKE_OK;
+    if (pl.blocked) {
+        const dim3 grid(static_cast<unsigned>(pl.nblk), static_cast<unsigned>(B));
+        const size_t smem = static_cast<size_t>(K) * sizeof(int);
+        hist_blocked_kernel<<<grid, BLK_THREADS, smem, s>>>(idx, N, K, pl.slab, scr.part, scr.sums,
+                                                            static_cast<i64>(K) * D, status);
+        colscan_kernel<<<dim3((K + 31) / 32, B), 256, 0, s>>>(scr.part, pl.nblk, K, counts, scr.nvalid);
+        scatter_blocked_kernel<<<grid, BLK_THREADS, smem, s>>>(idx, N, K, pl.slab, scr.part, counts, scr.nvalid,
+                                                               scr.pairs);
+    } else {
+        {
+            i64 ctas = (N + HIST_THREADS * 8 - 1) / (HIST_THREADS * 8);
+            const i64 cap = (static_cast<i64>(di.sm_count) * 4 + B - 1) / B;
+            if (ctas > cap) ctas = cap;
+            if (ctas < 1) ctas = 1;
+            hist_kernel<<<dim3(static_cast<unsigned>(ctas), B), HIST_THREADS, 0, s>>>(idx, N, K, counts, status);
+        }
+        scan_kernel<<<dim3((K + SCAN_TILE - 1) / SCAN_TILE, B), 1024, 0, s>>>(counts, K, scr.cursor, scr.nvalid);
+        {
+            i64 ctas = (N + 256 * 4 - 1) / (256 * 4);
+            const i64 cap = (static_cast<i64>(di.sm_count) * 8 + B - 1) / B;
+            if (ctas > cap) ctas = cap;
+            if (ctas < 1) ctas = 1;
+            scatter_kernel<<<dim3(static_cast<unsigned>(ctas), B), 256, 0, s>>>(idx, N, K, scr.cursor, scr.pairs);
+        }
     }
     {
         const i64 warps = (N + SEG_ROWS - 1) / SEG_ROWS;
@@ -415,13 +633,13 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
             while (lpr < G && lpr < 32) lpr <<= 1;
             const int gpl = (G + lpr - 1) / lpr;
             if (gpl == 1)
-                segreduce_kernel<1><<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.perm, scr.offsets, N, D, K, lpr, scr.sums);
+                segreduce_kernel<1><<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.pairs, scr.nvalid, N, D, K, lpr, scr.sums);
             else if (gpl == 2)
-                segreduce_kernel<2><<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.perm, scr.offsets, N, D, K, lpr, scr.sums);
+                segreduce_kernel<2><<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.pairs, scr.nvalid, N, D, K, lpr, scr.sums);
             else
-                segreduce_kernel<4><<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.perm, scr.offsets, N, D, K, lpr, scr.sums);
+                segreduce_kernel<4><<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.pairs, scr.nvalid, N, D, K, lpr, scr.sums);
         } else {
-            segreduce_scalar_kernel<<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.perm, scr.offsets, N, D, K, scr.sums);
+            segreduce_scalar_kernel<<<grid, SEG_WARPS * 32, 0, s>>>(X, scr.pairs, scr.nvalid, N, D, K, scr.sums);
         }
     }
     note_launches(4);  // histogram, scan, scatter, segmented reduction
@@ -431,6 +649,16 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
 cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B, int K,
                             int D, float* out_C, cake_bf16* out_C_bf16, cudaStream_t s) {
     const i64 total = static_cast<i64>(B) * K * D;
+    if (D % 4 == 0) {
+        i64 ctas = (total / 4 + 255) / 256;
+        if (ctas > 148 * 16) ctas = 148 * 16;
+        if (ctas < 1) ctas = 1;
+        finalize4_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(
+            reinterpret_cast<const float4*>(sums), counts, reinterpret_cast<const uint2*>(C_prev), total / 4, D / 4,
+            reinterpret_cast<float4*>(out_C), reinterpret_cast<uint2*>(out_C_bf16));
+        note_launches(1);
+        return cudaGetLastError();
+    }
     i64 ctas = (total + 256 * 4 - 1) / (256 * 4);
     if (ctas > 148 * 16) ctas = 148 * 16;
     if (ctas < 1) ctas = 1;
