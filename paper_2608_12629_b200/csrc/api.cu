@@ -67,8 +67,10 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
     if (path != CAKE_ASSIGN_TCGEN05 && path != CAKE_ASSIGN_TCGEN05_EXACT) return CAKE_ERR_UNSUPPORTED;
     if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
     if (N == 0) return CAKE_OK;
-    return launch_assign_tc(X, C, B, N, D, K, w.caug, path == CAKE_ASSIGN_TCGEN05_EXACT, out_idx, out_dist,
-                            w.status, s);
+    // automatic choice of the epilogue: with many centroid tiles per row a 32-column group rarely
+    // beats the running best, and the exact epilogue is then as fast as the packed one or faster
+    const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT || ((flags & CAKE_ASSIGN_MASK) == CAKE_ASSIGN_AUTO && K >= 4096);
+    return launch_assign_tc(X, C, B, N, D, K, w.caug, exact, out_idx, out_dist, w.status, s);
 }
 
 int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, const cake_bf16* C_prev,

@@ -10,7 +10,8 @@
 // never exists outside tensor memory.
 //
 // One persistent CTA per SM, 16 warps (warp 11 idle), four roles:
-//   warp 8  producer : TMA.  A 128-row X tile (whole D) into one of the X buffers per row tile; per
+//   warp 8  producer : TMA.  A 128-row X tile (whole D) into one of the X buffers per row tile (up to
+//                      four row tiles ahead); per
 //                      centroid tile of 256 rows, D/64 chunks of 64 columns (128-byte swizzle) through
 //                      an mbarrier ring, plus the tile's 8 KiB block of split half-norms (bulk copy).
 //   warps 9,10 MMA   : one thread each issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32); issuer i
@@ -53,9 +54,11 @@ constexpr uint32_t C_STAGE_BYTES = BLOCK_N * 128;        // 32 KiB
 constexpr uint32_t AUG_A_BYTES = BLOCK_M * UMMA_K * 2;   // 4 KiB
 constexpr uint32_t AUG_B_BYTES = kAssignAugTileBytes;    // 8 KiB
 constexpr int MAX_STAGES = 6;
+constexpr int MAX_XBUF = 4;
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t CTRL_BYTES = 4096;  // barriers, TMEM pointer, abort flag, merge scratch
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+constexpr uint32_t WAIT_SLICE_NS = 20000;   // longest single sleep inside a wait
 constexpr uint32_t COL_MASK = 0x7Fu;   // packed policy: 7 bits address the 128 columns of a half tile
 constexpr uint32_t F32_INF = 0x7f800000u;
 
@@ -77,10 +80,10 @@ struct Params {
 };
 
 struct Ctrl {  // lives in shared memory
-    uint64_t x_full[2], x_empty[2];
+    uint64_t x_full[MAX_XBUF], x_empty[MAX_XBUF];
     uint64_t ring_full[MAX_STAGES], ring_empty[MAX_STAGES];
     uint64_t tmem_full[2], tmem_empty[2];
-    uint64_t auga_full[2];
+    uint64_t auga_full[MAX_XBUF];
     uint64_t augb_full[2], augb_empty[2];
     uint64_t merge_full[2], merge_empty[2];
     uint32_t tmem_base;
@@ -121,20 +124,21 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctrl* c
 #define wait_bar_body wait_bar
 #endif
 
-// Bounded wait on an mbarrier phase. Returns false if the CTA is aborting.
+// Bounded wait on an mbarrier phase. Returns false if the CTA is aborting.  After a first quick
+// poll the thread sleeps in the barrier unit (it wakes when the phase completes or after
+// WAIT_SLICE_NS), so a waiting warp issues next to nothing and leaves the issue slots and the ALU
+// pipe to the warps that have work.
 __device__ __forceinline__ bool wait_bar_body(uint64_t* bar, uint32_t parity, Ctrl* ctrl, int* status) {
     const uint32_t addr = ptx::smem_u32(bar);
     if (ptx::mbar_try_wait(addr, parity)) return true;
     const uint64_t t0 = ptx::globaltimer_ns();
-    for (uint32_t it = 1;; ++it) {
-        if (ptx::mbar_try_wait(addr, parity)) return true;
-        if ((it & 63u) == 0) {
-            if (*reinterpret_cast<volatile int*>(&ctrl->abort_flag)) return false;
-            if (ptx::globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
-                *reinterpret_cast<volatile int*>(&ctrl->abort_flag) = 1;
-                atomicCAS(status, CAKE_OK, CAKE_ERR_TIMEOUT);
-                return false;
-            }
+    for (;;) {
+        if (ptx::mbar_try_wait_hint(addr, parity, WAIT_SLICE_NS)) return true;
+        if (*reinterpret_cast<volatile int*>(&ctrl->abort_flag)) return false;
+        if (ptx::globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+            *reinterpret_cast<volatile int*>(&ctrl->abort_flag) = 1;
+            atomicCAS(status, CAKE_OK, CAKE_ERR_TIMEOUT);
+            return false;
         }
     }
 }
@@ -214,7 +218,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t ring_off = static_cast<uint32_t>(p.n_xbuf) * xbuf_bytes;
     const uint32_t ring_base = smem_base + ring_off;
     const uint32_t auga_off = ring_off + static_cast<uint32_t>(p.n_stages) * C_STAGE_BYTES;
-    const uint32_t augb_off = auga_off + 2 * AUG_A_BYTES;
+    const uint32_t augb_off = auga_off + static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES;
     const uint32_t ctrl_off = augb_off + 2 * AUG_B_BYTES;
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ctrl_off);
 
@@ -222,12 +226,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < MAX_XBUF; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), 2 + 4);  // 2 MMA issuers + 4 norm warps
+            ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
+        }
+        for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i]), NUM_EPI_WARPS);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->augb_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->augb_empty[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_full[i]), 4);
@@ -244,7 +250,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         ptx::fence_mbar_init();
     }
     // the X-side operand of the extra k-step: columns 8..15 stay zero for the whole kernel
-    for (uint32_t o = threadIdx.x * 16; o < 2 * AUG_A_BYTES; o += NUM_THREADS * 16)
+    for (uint32_t o = threadIdx.x * 16; o < static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES; o += NUM_THREADS * 16)
         *reinterpret_cast<uint4*>(smem + auga_off + o) = make_uint4(0, 0, 0, 0);
     ptx::fence_proxy_async_smem();
     if (warp == MMA_WARP) {
@@ -269,35 +275,40 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (lane == 0) {
             uint32_t ring_it = 0, acc_it = 0;
             uint32_t rs = 0, rph = 0;   // ring stage and its phase
-            uint32_t xb = 0, xph = 0;   // X buffer of the current row tile and its phase
             bool ok = true;
-            // X tile of row tile `t` into buffer `buf` (its previous user must have released it)
-            auto issue_x = [&](i64 t, uint32_t buf) {
-                const int tb = static_cast<int>(t / p.m_tiles);
-                const int tmt = static_cast<int>(t % p.m_tiles);
-                const uint32_t xfull = ptx::smem_u32(&ctrl->x_full[buf]);
+            // X tiles run ahead of the MMAs by up to n_xbuf row tiles: `x_next` is the next row tile
+            // whose X has not been requested yet, (ixb, ixph) the buffer and phase it will use
+            i64 x_next = blockIdx.x;
+            uint32_t ixb = 0, ixph = 0;
+            auto issue_x = [&]() {
+                const int tb = static_cast<int>(x_next / p.m_tiles);
+                const int tmt = static_cast<int>(x_next % p.m_tiles);
+                const uint32_t xfull = ptx::smem_u32(&ctrl->x_full[ixb]);
                 ptx::mbar_arrive_expect_tx(xfull, xbuf_bytes);
                 for (int c = 0; c < p.nchunks; ++c)
-                    ptx::tma_load_3d(x_base + buf * xbuf_bytes + c * X_CHUNK_BYTES, &tmap_x, xfull,
+                    ptx::tma_load_3d(x_base + ixb * xbuf_bytes + c * X_CHUNK_BYTES, &tmap_x, xfull,
                                      c * KCHUNK, tmt * BLOCK_M, tb);
+                x_next += gridDim.x;
+                if (++ixb == static_cast<uint32_t>(p.n_xbuf)) { ixb = 0; ixph ^= 1u; }
             };
-            if (static_cast<i64>(blockIdx.x) < p.total_tiles) issue_x(blockIdx.x, 0);
+            // request X tiles for as long as a buffer is free, without ever blocking
+            auto prefetch_x = [&]() {
+                while (x_next < p.total_tiles &&
+                       ptx::mbar_test_wait(ptx::smem_u32(&ctrl->x_empty[ixb]), ixph ^ 1u))
+                    issue_x();
+            };
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 const int b = static_cast<int>(tile / p.m_tiles);
-                // the next row tile's X is requested as early as its buffer is free (polled between
-                // centroid chunks, never blocking them), so its latency hides behind this tile's MMAs
-                const i64 next = tile + gridDim.x;
-                const uint32_t nxb = (xb + 1 == static_cast<uint32_t>(p.n_xbuf)) ? 0u : xb + 1;
-                const uint32_t nxph = (nxb == 0) ? xph ^ 1u : xph;
-                bool next_pending = next < p.total_tiles;
+                prefetch_x();
+                if (x_next <= tile) {   // this tile's own X is still outstanding: its buffer must free up
+                    ok = wait_bar(&ctrl->x_empty[ixb], ixph ^ 1u, ctrl, p.status);
+                    if (!ok) break;
+                    issue_x();
+                }
                 const uint8_t* caug_b = p.caug + static_cast<size_t>(b) * p.n_tiles * AUG_B_BYTES;
                 for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it) {
                     for (int c = 0; c < p.nchunks; ++c, ++ring_it) {
-                        if (next_pending && p.n_xbuf == 2 &&
-                            ptx::mbar_test_wait(ptx::smem_u32(&ctrl->x_empty[nxb]), nxph ^ 1u)) {
-                            issue_x(next, nxb);
-                            next_pending = false;
-                        }
+                        prefetch_x();
                         ok = wait_bar(&ctrl->ring_empty[rs], rph ^ 1u, ctrl, p.status);
                         if (!ok) break;
                         const uint32_t full = ptx::smem_u32(&ctrl->ring_full[rs]);
@@ -315,12 +326,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     ptx::bulk_load(smem_base + augb_off + as * AUG_B_BYTES,
                                    caug_b + static_cast<size_t>(nt) * AUG_B_BYTES, AUG_B_BYTES, bfull);
                 }
-                if (ok && next_pending) {
-                    ok = wait_bar(&ctrl->x_empty[nxb], nxph ^ 1u, ctrl, p.status);
-                    if (ok) issue_x(next, nxb);
-                }
-                xb = nxb;
-                xph = nxph;
             }
             if (!ok) {
                 // aborting: give our loads in flight a bounded time to land before the CTA's
@@ -685,14 +690,19 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         note_launches(1);
     }
 
-    const i64 fixed = 1024 + CTRL_BYTES + 2 * AUG_A_BYTES + 2 * AUG_B_BYTES;
+    // Shared memory: X buffers (each with its 4 KiB norm operand), the centroid ring, fixed parts.
+    // Few centroid tiles per row tile make row tiles short, so X has to run further ahead: up to four
+    // X buffers then, two otherwise; a single one only if the ring would drop below three stages.
+    const i64 fixed = 1024 + CTRL_BYTES + 2 * AUG_B_BYTES;
     const i64 budget = static_cast<i64>(di.smem_optin) - fixed;
-    const i64 xbuf = static_cast<i64>(p.nchunks) * X_CHUNK_BYTES;
-    p.n_xbuf = 2;
-    i64 stages = (budget - 2 * xbuf) / C_STAGE_BYTES;
-    if (stages < 3 || (p.nchunks >= 4 && p.n_tiles >= 8)) {
-        p.n_xbuf = 1;
-        stages = (budget - xbuf) / C_STAGE_BYTES;
+    const i64 xbuf = static_cast<i64>(p.nchunks) * X_CHUNK_BYTES + AUG_A_BYTES;
+    int want_xbuf = p.n_tiles <= 2 ? MAX_XBUF : 2;
+    if (p.nchunks >= 4 && p.n_tiles >= 8) want_xbuf = 1;
+    const i64 min_stages = p.n_tiles <= 2 ? 2 : 3;
+    i64 stages = 0;
+    for (p.n_xbuf = want_xbuf; p.n_xbuf >= 1; --p.n_xbuf) {
+        stages = (budget - p.n_xbuf * xbuf) / C_STAGE_BYTES;
+        if (stages >= min_stages || p.n_xbuf == 1) break;
     }
     if (stages < 2) return CAKE_ERR_UNSUPPORTED;
     p.n_stages = static_cast<int>(stages > MAX_STAGES ? MAX_STAGES : stages);
