@@ -1,0 +1,67 @@
+"""Host-side logic of bench.py that needs no GPU: the reference arm, and the multi-rank reduction
+(world_size 2 over gloo on CPU)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+import bench  # noqa: E402
+
+
+def test_algorithmic_bytes_and_peaks():
+    from paper_2608_12629_b200 import inputs
+    w = inputs.WORKLOADS["c2"]
+    assert bench.algorithmic_update_bytes(w) == 2 * w.N * w.D + 4 * w.N + 8 * w.K * w.D + 4 * w.K
+    p = bench.measured_peaks()
+    assert p["hbm_gbs"] > 1000 and p["bf16_tflops"] > 100 and p["source"] in ("measured", "fallback")
+
+
+def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():
+    env = dict(os.environ, OMP_NUM_THREADS="4")
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c1", "--steps", "2",
+           "--warmup", "1"]
+    out = subprocess.run(cmd, env=dict(env, RANK="0", WORLD_SIZE="2"), capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr
+    lines = [ln for ln in out.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["metric"] == bench.METRIC and line["unit"] == bench.UNIT
+    assert line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["gpu_launches"] == 0
+    other = subprocess.run(cmd, env=dict(env, RANK="1", WORLD_SIZE="2"), capture_output=True, text=True, timeout=300)
+    assert other.returncode == 0 and other.stdout.strip() == ""
+
+
+def _rank_main(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    times = [10.0 + rank, 3.0 - rank, 1.0, 7.0 * (rank + 1)]       # ms per quantity, different on each rank
+    red = bench.max_over_ranks(times, torch.device("cpu"), world)
+    line = bench.assemble_value(world, steps=4, ms_total=red[0])
+    dist.barrier()
+    if rank == 0:
+        q.put((red, line))
+    dist.destroy_process_group()
+
+
+def test_max_over_ranks_and_whole_job_value_with_gloo_world_size_2():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_rank_main, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    red, line = q.get(timeout=120)
+    for p in procs:
+        p.join(60)
+        assert p.exitcode == 0
+    assert red == [11.0, 3.0, 1.0, 14.0]                            # the slowest rank decides every time
+    assert line["ms_per_step"] == pytest.approx(11.0 / 4)
+    assert line["value"] == pytest.approx(2 * 1000.0 / (11.0 / 4))   # units of ALL ranks / max time

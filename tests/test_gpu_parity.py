@@ -22,6 +22,10 @@ def problem(N, D, K, seed, comps=None, mean_std=1.0, sigma=0.5):
     return X, C
 
 
+def sampled_rows(N, n, seed):
+    return np.sort(np.random.default_rng(seed).choice(N, size=min(n, N), replace=False))
+
+
 def check_status(ws, want=cake.CAKE_OK):
     assert cake.cake_kmeans_device_status(ws) == want
 
@@ -94,6 +98,18 @@ def test_assign_batched_matches_per_problem_and_oracle():
         assert torch.equal(i1, idx[b]) and torch.equal(d1, dist[b])
 
 
+def test_assign_many_row_tiles_few_centroids_and_single_buffer_shapes():
+    """Row tiles far beyond the SM count with 1-2 centroid tiles (deep X prefetch), and D=256 with
+    many centroid tiles (single X buffer)."""
+    for N, D, K, sample in [(148 * 128 * 3 + 77, 128, 300, 3000), (40000, 256, 2304, 600), (33333, 64, 64, 3000)]:
+        X, C = problem(N, D, K, seed=N % 1000 + K)
+        ws = cake.alloc_workspace(1, N, D, K, DEV)
+        idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), ws=ws)
+        check_status(ws)
+        rows = sampled_rows(N, sample, K)
+        grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx.cpu().numpy(), dist.cpu().numpy(), rows=rows)
+
+
 def test_assign_edge_cases():
     X, C = problem(64, 64, 4, seed=1)
     # N = 0
@@ -144,6 +160,33 @@ def test_update_paths(path, N, D, K):
     check_status(ws)
     grading.grade_update(inputs.to_bits(X), idx.numpy(), K, inputs.to_bits(C), Cf.cpu().numpy(),
                          inputs.to_bits(Cb), counts.cpu().numpy())
+
+
+@pytest.mark.parametrize("N,D,K", [(70001, 64, 100), (9000, 128, 9000), (40000, 32, 20000), (8193, 16, 8193)])
+def test_update_sort_route_slab_tails_and_large_k(N, D, K):
+    """Ragged slabs (N not a multiple of 4 or of the slab), and K above the shared-memory histogram limit."""
+    X, C = problem(N, D, K, seed=N + D)
+    g = torch.Generator().manual_seed(K)
+    idx = torch.randint(0, K, (N,), generator=g, dtype=torch.int32)
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=C.to(DEV), ws=ws,
+                                             flags=cake.CAKE_UPDATE_SORT)
+    check_status(ws)
+    grading.grade_update(inputs.to_bits(X), idx.numpy(), K, inputs.to_bits(C), Cf.cpu().numpy(),
+                         inputs.to_bits(Cb), counts.cpu().numpy())
+
+
+def test_update_batched_unaligned_problem_size():
+    """B > 1 with N % 4 != 0: the per-problem idx slices are not 16-byte aligned."""
+    B, N, D, K = 3, 10001, 64, 37
+    Xs, Cs = zip(*(problem(N, D, K, seed=20 + b) for b in range(B)))
+    X, C = torch.stack(Xs), torch.stack(Cs)
+    g = torch.Generator().manual_seed(1)
+    idx = torch.randint(0, K, (B, N), generator=g, dtype=torch.int32)
+    Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=C.to(DEV), flags=cake.CAKE_UPDATE_SORT)
+    for b in range(B):
+        grading.grade_update(inputs.to_bits(Xs[b]), idx[b].numpy(), K, inputs.to_bits(Cs[b]), Cf[b].cpu().numpy(),
+                             inputs.to_bits(Cb[b]), counts[b].cpu().numpy())
 
 
 def test_update_odd_feature_count_and_null_prev():
@@ -284,10 +327,6 @@ def test_lloyd_host_buffers_match_device_call():
 
 
 # ------------------------------------------------------------------------------------ full-size workloads
-
-def sampled_rows(N, n, seed):
-    return np.sort(np.random.default_rng(seed).choice(N, size=min(n, N), replace=False))
-
 
 def test_assign_policies_agree_except_near_ties():
     """The packed epilogue orders values that agree to 2^-16 by index; everything else is identical."""
