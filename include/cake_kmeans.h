@@ -111,7 +111,7 @@ CAKE_API int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, 
  * inside another framework's allocator callback, or in a process whose device memory is already
  * fully carved up, has no cudaMalloc to give this library a scratch buffer).  The paper has no
  * counterpart: this is the un-batched cake_kmeans_assign with its scratch (the centroid half-norm
- * operand and the status word) held in a fixed 524,544-byte array inside the library image, which every GPU that
+ * operand and the status word) held in a fixed 262,400-byte array inside the library image, which every GPU that
  * loads the library keeps until the process exits.
  *   X, C, out_idx, out_dist: as cake_kmeans_assign (one problem).
  *   K must be <= 16384; a larger K returns CAKE_ERR_UNSUPPORTED and nothing is enqueued.

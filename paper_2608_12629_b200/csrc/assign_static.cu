@@ -6,7 +6,7 @@
 // the scratch the assign kernel needs -- the centroid half-norm operand and the status word -- lives in a fixed
 // array that is part of the loaded library image, so nothing is allocated at any point.
 //
-// The array is `static __device__`: every GPU that loads the library holds these 524,544 bytes until
+// The array is `static __device__`: every GPU that loads the library holds these 262,400 bytes until
 // the process exits.  In host code the array's name is only a host-side handle, not a device
 // address, so the address is obtained once per device with cudaGetSymbolAddress (with that device
 // current) and that pointer is what the kernels receive.
@@ -20,7 +20,7 @@ namespace {
 constexpr int kStaticMaxK = 16384;                         // largest K this entry point accepts
 constexpr size_t kStaticHeader = 256;                      // status word, padded
 constexpr size_t kStaticBytes =
-    kStaticHeader + static_cast<size_t>(kStaticMaxK / kAssignBlockN) * kAssignAugTileBytes;   // 256 B + 512 KiB
+    kStaticHeader + static_cast<size_t>(kStaticMaxK / kAssignBlockN) * kAssignAugTileBytes;   // 256 B + 256 KiB
 
 static __device__ __align__(256) unsigned char g_assign_scratch[kStaticBytes];
 

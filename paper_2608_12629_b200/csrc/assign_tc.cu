@@ -13,7 +13,7 @@
 //   warp 8  producer : TMA.  A 128-row X tile (whole D) into one of the X buffers per row tile (up to
 //                      four row tiles ahead); per
 //                      centroid tile of 256 rows, D/64 chunks of 64 columns (128-byte swizzle) through
-//                      an mbarrier ring, plus the tile's 8 KiB block of split half-norms (bulk copy).
+//                      an mbarrier ring, plus the tile's 4 KiB block of split half-norms (bulk copy).
 //   warps 9,10 MMA   : one thread each issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32); issuer i
 //                      owns the i-th of two 256-column TMEM accumulators and every other centroid tile;
 //                      tcgen05.commit frees ring slots and publishes finished accumulators.
@@ -51,8 +51,13 @@ constexpr int AUX_REGS = 56;            // ... and the producer / MMA / norm war
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr uint32_t X_CHUNK_BYTES = BLOCK_M * 128;        // 16 KiB
 constexpr uint32_t C_STAGE_BYTES = BLOCK_N * 128;        // 32 KiB
-constexpr uint32_t AUG_A_BYTES = BLOCK_M * UMMA_K * 2;   // 4 KiB
-constexpr uint32_t AUG_B_BYTES = kAssignAugTileBytes;    // 8 KiB
+// Operands of the extra k-step: only columns 0..7 are non-zero, so each buffer holds just those
+// (one 16-byte row per X row / centroid) and every descriptor points its second 8-column core
+// matrices at one shared block of zeros.
+constexpr uint32_t AUG_A_BYTES = BLOCK_M * 16;           // 2 KiB
+constexpr uint32_t AUG_B_BYTES = kAssignAugTileBytes;    // 4 KiB
+constexpr uint32_t AUG_ZERO_BYTES = BLOCK_N * 16;        // 4 KiB of zeros
+constexpr int N_AUGB = 4;                                // centroid-side buffers in flight
 constexpr int MAX_STAGES = 6;
 constexpr int MAX_XBUF = 4;
 constexpr int TMEM_COLS = 512;
@@ -84,7 +89,7 @@ struct Ctrl {  // lives in shared memory
     uint64_t ring_full[MAX_STAGES], ring_empty[MAX_STAGES];
     uint64_t tmem_full[2], tmem_empty[2];
     uint64_t auga_full[MAX_XBUF];
-    uint64_t augb_full[2], augb_empty[2];
+    uint64_t augb_full[N_AUGB], augb_empty[N_AUGB];
     uint64_t merge_full[2], merge_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -119,9 +124,22 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctrl* c
     }
     return ok;
 }
+// a bare time stamp with a caller-chosen tag (>= 100)
+__device__ __forceinline__ void trace_mark(Ctrl* ctrl, int tag) {
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) {
+        const int w = threadIdx.x >> 5;
+        const int n = ctrl->trace_n[w]++;
+        if (n < TRACE_CAP) {
+            long long* r = g_trace + (static_cast<size_t>(w) * TRACE_CAP + n) * 3;
+            r[0] = tag;
+            r[1] = r[2] = clock64();
+        }
+    }
+}
 #define wait_bar_body wait_bar_impl
 #else
 #define wait_bar_body wait_bar
+#define trace_mark(ctrl, tag) ((void)0)
 #endif
 
 // Bounded wait on an mbarrier phase. Returns false if the CTA is aborting.  After a first quick
@@ -219,7 +237,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t ring_base = smem_base + ring_off;
     const uint32_t auga_off = ring_off + static_cast<uint32_t>(p.n_stages) * C_STAGE_BYTES;
     const uint32_t augb_off = auga_off + static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES;
-    const uint32_t ctrl_off = augb_off + 2 * AUG_B_BYTES;
+    const uint32_t zero_off = augb_off + N_AUGB * AUG_B_BYTES;
+    const uint32_t ctrl_off = zero_off + AUG_ZERO_BYTES;
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ctrl_off);
 
     const int warp = threadIdx.x >> 5;
@@ -234,10 +253,12 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i]), NUM_EPI_WARPS);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->augb_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->augb_empty[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_full[i]), 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_empty[i]), 4);
+        }
+        for (int i = 0; i < N_AUGB; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&ctrl->augb_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->augb_empty[i]), 1);
         }
         for (int i = 0; i < MAX_STAGES; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_full[i]), 1);
@@ -249,9 +270,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 #endif
         ptx::fence_mbar_init();
     }
-    // the X-side operand of the extra k-step: columns 8..15 stay zero for the whole kernel
-    for (uint32_t o = threadIdx.x * 16; o < static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES; o += NUM_THREADS * 16)
-        *reinterpret_cast<uint4*>(smem + auga_off + o) = make_uint4(0, 0, 0, 0);
+    // columns 8..15 of both operands of the extra k-step: one block of zeros for the whole kernel
+    for (uint32_t o = threadIdx.x * 16; o < AUG_ZERO_BYTES; o += NUM_THREADS * 16)
+        *reinterpret_cast<uint4*>(smem + zero_off + o) = make_uint4(0, 0, 0, 0);
     ptx::fence_proxy_async_smem();
     if (warp == MMA_WARP) {
         ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), TMEM_COLS);
@@ -318,12 +339,12 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         if (++rs == static_cast<uint32_t>(p.n_stages)) { rs = 0; rph ^= 1u; }
                     }
                     if (!ok) break;
-                    const uint32_t as = acc_it & 1u, aph = (acc_it >> 1) & 1u;
-                    ok = wait_bar(&ctrl->augb_empty[as], aph ^ 1u, ctrl, p.status);
+                    const uint32_t ab = acc_it % N_AUGB, abph = (acc_it / N_AUGB) & 1u;
+                    ok = wait_bar(&ctrl->augb_empty[ab], abph ^ 1u, ctrl, p.status);
                     if (!ok) break;
-                    const uint32_t bfull = ptx::smem_u32(&ctrl->augb_full[as]);
+                    const uint32_t bfull = ptx::smem_u32(&ctrl->augb_full[ab]);
                     ptx::mbar_arrive_expect_tx(bfull, AUG_B_BYTES);
-                    ptx::bulk_load(smem_base + augb_off + as * AUG_B_BYTES,
+                    ptx::bulk_load(smem_base + augb_off + ab * AUG_B_BYTES,
                                    caug_b + static_cast<size_t>(nt) * AUG_B_BYTES, AUG_B_BYTES, bfull);
                 }
             }
@@ -360,7 +381,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             uint32_t xb = 0, xph = 0;                       // X buffer and its phase
             uint32_t acc_it = 0;
             const uint32_t d_tmem = tmem_base + par * BLOCK_N;
-            const uint32_t augb_lo = ptx::umma_desc_lo_interleaved(smem_base + augb_off + par * AUG_B_BYTES);
             bool ok = true;
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 // every phase of the shared barriers is observed, also in row / centroid tiles this
@@ -369,7 +389,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 if (!ok) break;
                 bool have_aug = false;
                 const uint32_t a_lo_tile = ptx::umma_desc_lo_sw128(x_base + xb * xbuf_bytes);
-                const uint32_t auga_lo = ptx::umma_desc_lo_interleaved(smem_base + auga_off + xb * AUG_A_BYTES);
+                const uint32_t auga_lo = ptx::umma_desc_lo_aug(smem_base + auga_off + xb * AUG_A_BYTES,
+                                                               smem_base + zero_off);
                 for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it) {
                     if ((acc_it & 1u) != par) {             // the other issuer's tile: pass over its ring slots
                         for (int c = 0; ok && c < p.nchunks; ++c) {
@@ -414,11 +435,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         if (!ok) break;
                         have_aug = true;
                     }
-                    ok = wait_bar(&ctrl->augb_full[par], aph, ctrl, p.status);
+                    const uint32_t ab = acc_it % N_AUGB, abph = (acc_it / N_AUGB) & 1u;
+                    ok = wait_bar(&ctrl->augb_full[ab], abph, ctrl, p.status);
                     if (!ok) break;
-                    ptx::umma_bf16_lohi<true>(d_tmem, auga_lo, ptx::UMMA_DESC_HI_INTERLEAVED, augb_lo,
-                                              ptx::UMMA_DESC_HI_INTERLEAVED, idesc_aug);
-                    ptx::umma_commit(ptx::smem_u32(&ctrl->augb_empty[par]));
+                    ptx::umma_bf16_lohi<true>(d_tmem, auga_lo, ptx::UMMA_DESC_HI_AUG,
+                                              ptx::umma_desc_lo_aug(smem_base + augb_off + ab * AUG_B_BYTES,
+                                                                    smem_base + zero_off),
+                                              ptx::UMMA_DESC_HI_AUG, idesc_aug);
+                    ptx::umma_commit(ptx::smem_u32(&ctrl->augb_empty[ab]));
                     ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[par]));
                 }
                 if (ok && !have_aug) ok = wait_bar(&ctrl->auga_full[xb], xph, ctrl, p.status);
@@ -456,10 +480,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             }
             uint32_t hi, mid, lo;
             split3(0.5f * ((xn0 + xn1) + (xn2 + xn3)), hi, mid, lo);
-            // interleaved (no-swizzle) K-major layout: 8-row groups of 256 B, row stride 16 B,
-            // the second 8 columns 128 B further on (left zero)
+            // interleaved (no-swizzle) K-major layout, columns 0..7 only: one 16-byte row per X row
             const uint32_t one = 0x3F80u;
-            *reinterpret_cast<uint4*>(smem + auga_off + xb * AUG_A_BYTES + (r >> 3) * 256 + (r & 7) * 16) =
+            *reinterpret_cast<uint4*>(smem + auga_off + xb * AUG_A_BYTES + r * 16) =
                 make_uint4(hi | (mid << 16), lo | (one << 16), one | (one << 16), 0u);
             ptx::fence_proxy_async_smem();
             __syncwarp();
@@ -504,6 +527,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as]));
+                trace_mark(ctrl, 100);
                 if (PACKED) {
                     float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF));
                     tmin = packed_min32(rb, 32, tmin);
@@ -524,6 +548,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 }
             }
             if (!ok) break;
+            trace_mark(ctrl, 102);
             float bval;
             int bidx;
             if (PACKED) {
@@ -561,6 +586,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     if (p.out_dist) p.out_dist[o] = fmaxf(0.f, 2.f * bval);
                 }
             }
+            trace_mark(ctrl, 103);
         }
     }
 
@@ -575,9 +601,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 }
 
 // Prologue: the centroid-side operand of the extra k-step.  One warp per padded centroid row k:
-// h = ||c_k||^2 / 2 split into three bf16 terms, written as the row [1 1 1 h_hi h_mid h_lo 0 0 | 0 x 8]
-// in the interleaved K-major layout the MMA reads (per 256-row tile an 8 KiB block: 32 groups of
-// 8 rows x 16 B, then the same for columns 8..15).  Rows k >= K get h = +inf and can never win.
+// h = ||c_k||^2 / 2 split into three bf16 terms, written as the 16-byte row [1 1 1 h_hi h_mid h_lo 0 0]
+// (columns 0..7 of the operand in the interleaved K-major layout the MMA reads: 256 rows x 16 B = 4 KiB
+// per tile; columns 8..15 are zeros the kernel supplies itself).  Rows k >= K get h = +inf and can never win.
 __global__ void __launch_bounds__(256)
 centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64 total_rows,
                     uint8_t* __restrict__ caug) {
@@ -602,9 +628,7 @@ centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64
         const uint32_t one = 0x3F80u;
         const int tile = k / BLOCK_N, rr = k % BLOCK_N;
         uint8_t* blk = caug + (static_cast<size_t>(b) * (Kpad / BLOCK_N) + tile) * AUG_B_BYTES;
-        uint8_t* dst = blk + (rr >> 3) * 256 + (rr & 7) * 16;
-        *reinterpret_cast<uint4*>(dst) = make_uint4(one | (one << 16), one | (hi << 16), mid | (lo << 16), 0u);
-        *reinterpret_cast<uint4*>(dst + 128) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(blk + rr * 16) = make_uint4(one | (one << 16), one | (hi << 16), mid | (lo << 16), 0u);
     }
 }
 
@@ -693,7 +717,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     // Shared memory: X buffers (each with its 4 KiB norm operand), the centroid ring, fixed parts.
     // Few centroid tiles per row tile make row tiles short, so X has to run further ahead: up to four
     // X buffers then, two otherwise; a single one only if the ring would drop below three stages.
-    const i64 fixed = 1024 + CTRL_BYTES + 2 * AUG_B_BYTES;
+    const i64 fixed = 1024 + CTRL_BYTES + N_AUGB * AUG_B_BYTES + AUG_ZERO_BYTES;
     const i64 budget = static_cast<i64>(di.smem_optin) - fixed;
     const i64 xbuf = static_cast<i64>(p.nchunks) * X_CHUNK_BYTES + AUG_A_BYTES;
     int want_xbuf = p.n_tiles <= 2 ? MAX_XBUF : 2;

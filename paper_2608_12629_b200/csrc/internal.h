@@ -27,9 +27,9 @@ unsigned long long launches_so_far();
 inline i64 round_up(i64 a, i64 b) { return (a + b - 1) / b * b; }
 
 // Centroid tiles of the tensor-core assign kernel are 256 wide; K is padded to that (padding rows
-// carry an infinite half-norm).  Per tile the kernel's prologue writes an 8 KiB operand block.
+// carry an infinite half-norm).  Per tile the kernel's prologue writes a 4 KiB operand block.
 constexpr int kAssignBlockN = 256;
-constexpr unsigned kAssignAugTileBytes = kAssignBlockN * 16 * 2;
+constexpr unsigned kAssignAugTileBytes = kAssignBlockN * 16;
 inline int padded_k(int K) { return (int)round_up(K, kAssignBlockN); }
 
 // ---- assign

@@ -228,6 +228,13 @@ __device__ __forceinline__ uint64_t umma_desc_interleaved(uint32_t smem_addr) {
 // instruction count per MMA small (it is the issue rate of that one thread that feeds the tensor core).
 constexpr uint32_t UMMA_DESC_HI_SW128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 constexpr uint32_t UMMA_DESC_HI_INTERLEAVED = (256u >> 4) | (1u << 14);
+// Interleaved layout whose columns 0..7 are stored as plain 16-byte rows (8-row groups 128 B apart)
+// and whose columns 8..15 live elsewhere (a block of zeros shared by many operands): the leading byte
+// offset is simply the distance from the operand to that block (which lies at a higher address).
+constexpr uint32_t UMMA_DESC_HI_AUG = (128u >> 4) | (1u << 14);
+__device__ __forceinline__ uint32_t umma_desc_lo_aug(uint32_t smem_addr, uint32_t zeros_addr) {
+    return ((smem_addr & 0x3FFFFu) >> 4) | ((((zeros_addr - smem_addr) >> 4) & 0x3FFFu) << 16);
+}
 __device__ __forceinline__ uint32_t umma_desc_lo_sw128(uint32_t smem_addr) {
     return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);
 }
