@@ -59,18 +59,27 @@ int check_ws(void* ws, size_t ws_bytes, i64 B, i64 N, int D, int K, Workspace* o
     return CAKE_OK;
 }
 
+// inertia (nullable): inertia[b * inertia_stride] += sum of problem b's distances.  The tensor-core
+// kernel adds it up itself; the fallback needs `dist` (out_dist or scratch) and a reduction kernel.
 int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, int* out_idx,
-              float* out_dist, const Workspace& w, cudaStream_t s, unsigned flags) {
+              float* out_dist, double* inertia, int inertia_stride, const Workspace& w, cudaStream_t s,
+              unsigned flags) {
     unsigned path = flags & CAKE_ASSIGN_MASK;
     if (path == CAKE_ASSIGN_AUTO) path = assign_tc_supports(D) ? CAKE_ASSIGN_TCGEN05 : CAKE_ASSIGN_SIMT;
-    if (path == CAKE_ASSIGN_SIMT) return launch_assign_simt(X, C, B, N, D, K, out_idx, out_dist, s);
+    if (path == CAKE_ASSIGN_SIMT) {
+        float* dist = out_dist ? out_dist : (inertia ? w.dist : nullptr);
+        int rc = launch_assign_simt(X, C, B, N, D, K, out_idx, dist, s);
+        if (rc == CAKE_OK && inertia && launch_inertia(dist, B, N, inertia, inertia_stride, s) != cudaSuccess)
+            rc = CAKE_ERR_CUDA;
+        return rc;
+    }
     if (path != CAKE_ASSIGN_TCGEN05 && path != CAKE_ASSIGN_TCGEN05_EXACT) return CAKE_ERR_UNSUPPORTED;
     if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
     if (N == 0) return CAKE_OK;
     // automatic choice of the epilogue: with many centroid tiles per row a 32-column group rarely
     // beats the running best, and the exact epilogue is then as fast as the packed one or faster
     const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT || ((flags & CAKE_ASSIGN_MASK) == CAKE_ASSIGN_AUTO && K >= 4096);
-    return launch_assign_tc(X, C, B, N, D, K, w.caug, exact, out_idx, out_dist, w.status, s);
+    return launch_assign_tc(X, C, B, N, D, K, w.caug, exact, out_idx, out_dist, inertia, inertia_stride, w.status, s);
 }
 
 int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, const cake_bf16* C_prev,
@@ -146,7 +155,7 @@ int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, long long
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;
-    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, w,
+    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, w,
                      reinterpret_cast<cudaStream_t>(stream), flags);
 }
 
@@ -210,12 +219,10 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
         if (launch_finalize(w.sums, w.cursor, w.cbuf[0], Bi, K, D, out_C, nullptr, s) != cudaSuccess)
             return CAKE_ERR_CUDA;
     }
-    float* dist = out_dist ? out_dist : (out_inertia ? w.dist : nullptr);
     for (int t = 0; t < iters; ++t) {
-        rc = do_assign(X, w.cbuf[cur], Bi, N, D, K, out_idx, dist, w, s, flags);
+        rc = do_assign(X, w.cbuf[cur], Bi, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr,
+                       iters, w, s, flags);
         if (rc != CAKE_OK) return rc;
-        if (out_inertia && launch_inertia(dist, Bi, N, out_inertia + t, iters, s) != cudaSuccess)
-            return CAKE_ERR_CUDA;
         rc = do_update(X, out_idx, Bi, N, D, K, w.cbuf[cur], out_C, w.cbuf[cur ^ 1], out_counts, w, s, flags);
         if (rc != CAKE_OK) return rc;
         cur ^= 1;

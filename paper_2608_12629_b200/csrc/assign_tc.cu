@@ -81,6 +81,8 @@ struct Params {
     const uint8_t* caug;  // [B][n_tiles][8 KiB] centroid-side operand of the extra k-step
     int* out_idx;
     float* out_dist;
+    double* inertia;      // optional: inertia[b * inertia_stride] += sum of the problem's distances
+    int inertia_stride;
     int* status;
 };
 
@@ -501,9 +503,25 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int r = q * 32 + lane;         // row inside the X tile
         uint32_t tile_it = 0, acc_it = 0;
         bool ok = true;
+        double dsum = 0.0;                   // this thread's share of the current problem's inertia
+        int dsum_b = -1;
+        // one fp64 atomic per warp and problem
+        auto flush_inertia = [&]() {
+            if (wg == 0 && p.inertia && dsum_b >= 0) {
+                double t = dsum;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+                if (lane == 0) atomicAdd(p.inertia + static_cast<size_t>(dsum_b) * p.inertia_stride, t);
+            }
+            dsum = 0.0;
+        };
         for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
             const int b = static_cast<int>(tile / p.m_tiles);
             const int mt = static_cast<int>(tile % p.m_tiles);
+            if (b != dsum_b) {
+                flush_inertia();
+                dsum_b = b;
+            }
             float best = __uint_as_float(F32_INF);   // packed: a key; exact: a value
             int bsel = 0;                            // packed: tile number; exact: global column
             for (int nt = 0; nt < p.n_tiles; ++nt, ++acc_it) {
@@ -582,12 +600,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const i64 row = static_cast<i64>(mt) * BLOCK_M + r;
                 if (row < p.N) {
                     const size_t o = static_cast<size_t>(b) * static_cast<size_t>(p.N) + row;
+                    const float dist = fmaxf(0.f, 2.f * bval);
                     p.out_idx[o] = bidx;
-                    if (p.out_dist) p.out_dist[o] = fmaxf(0.f, 2.f * bval);
+                    if (p.out_dist) p.out_dist[o] = dist;
+                    dsum += static_cast<double>(dist);
                 }
             }
             trace_mark(ctrl, 103);
         }
+        if (ok) flush_inertia();
     }
 
     // ---------------------------------------------------------------- teardown
@@ -687,7 +708,8 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
 }
 
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
-                     bool exact, int* out_idx, float* out_dist, int* status, cudaStream_t s) {
+                     bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride,
+                     int* status, cudaStream_t s) {
     if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
     DeviceInfo di;
     int rc = current_device_info(&di);
@@ -703,6 +725,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     p.total_tiles = static_cast<i64>(B) * p.m_tiles;
     p.caug = static_cast<const uint8_t*>(caug);
     p.out_idx = out_idx; p.out_dist = out_dist; p.status = status;
+    p.inertia = inertia; p.inertia_stride = inertia_stride;
     if (p.total_tiles == 0) return CAKE_OK;
 
     const int Kpad = padded_k(K);
