@@ -180,6 +180,57 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Shape sweep (3 Lloyd iterations per shape): one markdown table row per shape with the fraction of
+    the roofline (the slower of 2NKD at the tensor peak and the bytes moved at HBM bandwidth)."""
+    import paper_2608_12629_b200 as cake
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = measured_peaks()
+    Ns = [1 << 16, 1 << 20, 1 << 24] if not args.sweep_full else [1 << e for e in range(16, 25)]
+    Ds = [64, 96, 128, 256]
+    Ks = [64, 256, 1000, 1024, 4096, 65536] if not args.sweep_full else [64, 128, 256, 512, 1000, 1024, 2048, 4096,
+                                                                          8192, 16384, 32768, 65536]
+    print("| N | D | K | lloyd it/s | assign ms | TFLOP/s | update ms | GB/s | roofline it/s | fraction |")
+    print("|---|---|---|---|---|---|---|---|---|---|", flush=True)
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    for D in Ds:
+        for N in Ns:
+            w0 = inputs.sweep_workload(N, D, 64)
+            X, _ = inputs.gaussian_mixture(N, D, 16384, w0.mean_std, w0.sigma, w0.seed, device=dev)
+            for K in Ks:
+                if K > N:
+                    continue
+                w = inputs.sweep_workload(N, D, K)
+                C0 = inputs.sample_init(X, K, w.seed)
+                ws = cake.alloc_workspace(1, N, D, K, dev)
+                out = cake.alloc_lloyd_outputs(X, C0, w.iters)
+                cake.cake_kmeans_lloyd(X, C0, 1, out=cake.alloc_lloyd_outputs(X, C0, 1), ws=ws)      # warm-up
+                e[0].record()
+                cake.cake_kmeans_lloyd(X, C0, w.iters, out=out, ws=ws)
+                e[1].record()
+                cake.cake_kmeans_assign(X, out.C_bf16, out_idx=out.idx, out_dist=out.dist, ws=ws)
+                e[2].record()
+                cake.cake_kmeans_update(X, out.idx, K, C_prev=out.C_bf16, out_C=out.C, out_C_bf16=out.C_bf16,
+                                        out_counts=out.counts, ws=ws)
+                e[3].record()
+                torch.cuda.synchronize()
+                if cake.cake_kmeans_device_status(ws) != cake.CAKE_OK:
+                    raise SystemExit("device status raised during the sweep")
+                it_ms = e[0].elapsed_time(e[1]) / w.iters
+                a_ms, u_ms = e[1].elapsed_time(e[2]), e[2].elapsed_time(e[3])
+                flop = 2.0 * N * K * D
+                a_bytes = 2 * N * D + 2 * K * D + 8 * N
+                u_bytes = algorithmic_update_bytes(w)
+                floor_ms = max(flop / (peaks["bf16_tflops"] * 1e12), a_bytes / (peaks["hbm_gbs"] * 1e9)) * 1e3 + \
+                    u_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+                print(f"| {N} | {D} | {K} | {1000.0 / it_ms:.1f} | {a_ms:.4f} | {flop / a_ms / 1e9:.1f} | {u_ms:.4f} | "
+                      f"{u_bytes / u_ms / 1e6:.0f} | {1000.0 / floor_ms:.1f} | {floor_ms / it_ms:.3f} |", flush=True)
+                del ws, out
+            del X
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -189,7 +240,12 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="print the shape-sweep table instead of the JSON line")
+    ap.add_argument("--sweep-full", action="store_true", help="with --sweep: every power of two in N and K")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     rank = int(os.environ.get("RANK", "0"))

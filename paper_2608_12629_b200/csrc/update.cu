@@ -214,7 +214,7 @@ scatter_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ curs
 //                  its slab the next free position of its cluster.
 constexpr int BLK_THREADS = 256;
 constexpr int BLK_MAX_K = 8192;
-constexpr int BLK_MAX_BLOCKS = 128;
+constexpr int BLK_MAX_BLOCKS = 1024;
 constexpr int BLK_MIN_SLAB = 8192;
 constexpr int BLK_VEC = 4;            // idx values per load; slabs are multiples of it
 
@@ -258,9 +258,9 @@ hist_blocked_kernel(const int* __restrict__ idx, i64 N, int K, i64 slab, int* __
     for (int e = threadIdx.x; e < K; e += blockDim.x) out[e] = h[e];
 }
 
-// CTA = 32 clusters (lanes) x 8 warps; warp w owns a contiguous range of slabs.
+// CTA = 32 clusters (lanes) x 8 warps; warp w owns a contiguous range of slabs, walked 16 at a time.
 __global__ void __launch_bounds__(256)
-colscan_kernel(int* __restrict__ part, int nblk, int K, int* __restrict__ counts, int* __restrict__ nvalid) {
+colscan_kernel(int* __restrict__ part, int nblk, int K, int* __restrict__ counts) {
     __shared__ int tot[8][32];
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -268,12 +268,15 @@ colscan_kernel(int* __restrict__ part, int nblk, int K, int* __restrict__ counts
     const int per = (nblk + 7) / 8;
     const int j0 = warp * per, j1 = (j0 + per < nblk) ? j0 + per : nblk;
     int* p = part + static_cast<size_t>(b) * nblk * K + k;
-    int v[16];                                     // nblk <= 128 -> per <= 16
-#pragma unroll
-    for (int u = 0; u < 16; ++u) v[u] = (k < K && j0 + u < j1) ? p[static_cast<size_t>(j0 + u) * K] : 0;
+    // pass 1: this warp's total per cluster
     int sum = 0;
+    for (int j = j0; j < j1; j += 16) {
+        int v[16];
 #pragma unroll
-    for (int u = 0; u < 16; ++u) sum += v[u];
+        for (int u = 0; u < 16; ++u) v[u] = (k < K && j + u < j1) ? p[static_cast<size_t>(j + u) * K] : 0;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) sum += v[u];
+    }
     tot[warp][lane] = sum;
     __syncthreads();
     int run = 0, total = 0;
@@ -282,13 +285,18 @@ colscan_kernel(int* __restrict__ part, int nblk, int K, int* __restrict__ counts
         if (w < warp) run += tot[w][lane];
         total += tot[w][lane];
     }
+    // pass 2: exclusive prefix in place
+    for (int j = j0; j < j1; j += 16) {
+        int v[16];
 #pragma unroll
-    for (int u = 0; u < 16; ++u) {
-        if (k < K && j0 + u < j1) p[static_cast<size_t>(j0 + u) * K] = run;
-        run += v[u];
+        for (int u = 0; u < 16; ++u) v[u] = (k < K && j + u < j1) ? p[static_cast<size_t>(j + u) * K] : 0;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+            if (k < K && j + u < j1) p[static_cast<size_t>(j + u) * K] = run;
+            run += v[u];
+        }
     }
     if (warp == 0 && k < K) counts[static_cast<size_t>(b) * K + k] = total;
-    (void)nvalid;
 }
 
 __global__ void __launch_bounds__(BLK_THREADS)
@@ -603,7 +611,7 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
         const size_t smem = static_cast<size_t>(K) * sizeof(int);
         hist_blocked_kernel<<<grid, BLK_THREADS, smem, s>>>(idx, N, K, pl.slab, scr.part, scr.sums,
                                                             static_cast<i64>(K) * D, status);
-        colscan_kernel<<<dim3((K + 31) / 32, B), 256, 0, s>>>(scr.part, pl.nblk, K, counts, scr.nvalid);
+        colscan_kernel<<<dim3((K + 31) / 32, B), 256, 0, s>>>(scr.part, pl.nblk, K, counts);
         scatter_blocked_kernel<<<grid, BLK_THREADS, smem, s>>>(idx, N, K, pl.slab, scr.part, counts, scr.nvalid,
                                                                scr.pairs);
     } else {
