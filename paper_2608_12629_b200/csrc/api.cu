@@ -12,7 +12,8 @@ inline size_t up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Workspace {
     int* status;          // [64] header, word 0 = sticky device status
-    void* caug;           // [B][Kpad/256][8 KiB] half-norm operand of the tensor-core assign
+    void* caug;           // [B][Kpad/256][4 KiB] half-norm operand of the tensor-core assign
+    int* cnmax;           // [B] max ||c||^2 per problem (fp32 bits)
     float* sums;          // [B][K][D]
     int* nvalid;          // [B]
     int* cursor;          // [B][K]
@@ -31,6 +32,7 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     const size_t kd = static_cast<size_t>(B) * K * D;
     w.status = reinterpret_cast<int*>(take(256));
     w.caug = take(assign_tc_aug_bytes(B, K));
+    w.cnmax = reinterpret_cast<int*>(take(static_cast<size_t>(B) * 4));
     w.sums = reinterpret_cast<float*>(take(kd * 4));
     w.nvalid = reinterpret_cast<int*>(take(static_cast<size_t>(B) * 4));
     w.cursor = reinterpret_cast<int*>(take(static_cast<size_t>(B) * K * 4));
@@ -76,10 +78,10 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
     if (path != CAKE_ASSIGN_TCGEN05 && path != CAKE_ASSIGN_TCGEN05_EXACT) return CAKE_ERR_UNSUPPORTED;
     if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
     if (N == 0) return CAKE_OK;
-    // automatic choice of the epilogue: with many centroid tiles per row a 32-column group rarely
-    // beats the running best, and the exact epilogue is then as fast as the packed one or faster
-    const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT || ((flags & CAKE_ASSIGN_MASK) == CAKE_ASSIGN_AUTO && K >= 4096);
-    return launch_assign_tc(X, C, B, N, D, K, w.caug, exact, out_idx, out_dist, inertia, inertia_stride, w.status, s);
+    // both epilogues order by the same fixed-point values; the packed one measured as fast or faster
+    // at every shape tried, so it is the automatic choice and the other stays selectable
+    const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT;
+    return launch_assign_tc(X, C, B, N, D, K, w.caug, w.cnmax, exact, out_idx, out_dist, inertia, inertia_stride, w.status, s);
 }
 
 int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, const cake_bf16* C_prev,

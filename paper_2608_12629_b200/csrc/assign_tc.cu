@@ -2,11 +2,16 @@
 //
 // Operation (paper Section 5, "Flash-KMeans clean-start workload"): for every point the squared
 // Euclidean distance to all K centroids and the arg-min.  The whole expansion
-//     d(x,c)/2 = ||x||^2/2 - x.c + ||c||^2/2
+//     M + m + d(x,c)/2 = M + m + ||x||^2/2 - x.c + ||c||^2/2
 // is accumulated in tensor memory: the D-long contraction -x.c runs with the B operand negated, and
-// one extra 16-wide k-step adds the two half-norms (the X side carries [xh xm xl 1 1 1 0..], the
-// centroid side [1 1 1 ch cm cl 0..], each half-norm split into three bf16 terms so that nothing of
-// its fp32 value is lost).  The epilogue therefore only has to find a row minimum; the N x K matrix
+// one extra 16-wide k-step adds the two half-norms and a per-row offset (the X side carries
+// [xh xm xl 1 1 1 M m 0..], the centroid side [1 1 1 ch cm cl 1 1 0..], each half-norm split into
+// three bf16 terms so that nothing of its fp32 value is lost).  M is a power of two at least twice
+// ||x||^2 + max||c||^2 >= d/2, m = M/4096 keeps rounding noise positive: every accumulator of a row
+// lies in the binade [M, 2M), so its fp32 bit pattern minus that of M is the distance in FIXED POINT
+// (quantum ulp(M), about 2^-20 of the row's scale), and `bits * 128 + column` is an order-preserving
+// key that a single integer multiply-add forms.  Padded centroid rows carry 1.5 M instead of M and
+// lose to every real one.  The epilogue therefore only has to find a row minimum; the N x K matrix
 // never exists outside tensor memory.
 //
 // One persistent CTA per SM, 16 warps (warp 11 idle), four roles:
@@ -22,13 +27,11 @@
 //                      The two column halves are merged through shared memory per row tile.
 //   warps 12-15 norms : one thread per X row forms ||x||^2/2 from the shared-memory X tile and writes
 //                      the X-side operand of the extra k-step, one row tile ahead of the MMA warp.
-// Two epilogue policies:
-//   packed : the low 7 mantissa bits of each value are replaced by its column number and a plain
-//            float minimum finds value and position at once (1.5 issue slots per element, no branch).
-//            Values closer than 2^-16 relative are ordered by column; exact ties still go to the
-//            lowest index.
-//   exact  : full-precision minimum; the position is looked up only when a 32-column group beats
-//            the running best.
+// Two epilogue policies (both order by the fixed-point value, ties to the lowest index):
+//   packed : key = bits * 128 + column (one multiply-add on the FMA pipe) and a plain 3-input float
+//            minimum over the keys finds value and position at once; no branch.
+//   exact  : minimum of the values; the position is looked up only when a 32-column group beats the
+//            running best (cheaper when there are many centroid tiles per row).
 // Every wait is bounded: on expiry the CTA raises CAKE_ERR_TIMEOUT in the status word, all roles
 // leave their loops, TMEM is freed and the kernel returns.
 #include "internal.h"
@@ -61,7 +64,7 @@ constexpr int N_AUGB = 4;                                // centroid-side buffer
 constexpr int MAX_STAGES = 6;
 constexpr int MAX_XBUF = 4;
 constexpr int TMEM_COLS = 512;
-constexpr uint32_t CTRL_BYTES = 4096;  // barriers, TMEM pointer, abort flag, merge scratch
+constexpr uint32_t CTRL_BYTES = 6144;  // barriers, TMEM pointer, abort flag, merge scratch, row exponents
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 constexpr uint32_t WAIT_SLICE_NS = 20000;   // longest single sleep inside a wait
 constexpr uint32_t COL_MASK = 0x7Fu;   // packed policy: 7 bits address the 128 columns of a half tile
@@ -78,7 +81,8 @@ struct Params {
     i64 total_tiles;  // B * m_tiles
     int n_stages;     // ring depth
     int n_xbuf;       // 1 or 2 X buffers
-    const uint8_t* caug;  // [B][n_tiles][8 KiB] centroid-side operand of the extra k-step
+    const uint8_t* caug;  // [B][n_tiles][4 KiB] centroid-side operand of the extra k-step
+    const int* cnmax;     // [B] bit pattern of max_k ||c_k||^2 (fp32, >= 0)
     int* out_idx;
     float* out_dist;
     double* inertia;      // optional: inertia[b * inertia_stride] += sum of the problem's distances
@@ -97,6 +101,7 @@ struct Ctrl {  // lives in shared memory
     int abort_flag;
     float merge_best[2][BLOCK_M];
     int merge_idx[2][BLOCK_M];
+    int row_e[MAX_XBUF][BLOCK_M];   // biased exponent of each row's offset M
 #ifdef CAKE_ASSIGN_TRACE
     int trace_n[NUM_WARPS];
 #endif
@@ -193,14 +198,14 @@ __device__ __forceinline__ float min32(const float (&v)[32]) {
     return fminf(ptx::fmin3(u0, u1, u2), u3);
 }
 
-// packed policy: key = value with its low 7 mantissa bits replaced by the column (0..127) inside
-// the half tile.  For non-negative values float order == (truncated value, column) order; +inf
-// (a padded column) turns into a NaN, which min ignores.
+// packed policy: key = bits * 128 + column (0..127 inside the half tile), modulo 2^32.  All values of a
+// row share the binade of M, whose exponent is chosen so that the keys stay below 0x7F800000: as float
+// bit patterns they are positive and finite, and float order == (fixed-point value, column) order.
 __device__ __forceinline__ float packed_min32(const uint32_t (&r)[32], int col_base, float run) {
     float v[32];
 #pragma unroll
     for (int j = 0; j < 32; ++j)
-        v[j] = __uint_as_float((r[j] & ~COL_MASK) | static_cast<uint32_t>(col_base + j));
+        v[j] = __uint_as_float(r[j] * (COL_MASK + 1u) + static_cast<uint32_t>(col_base + j));
     return fminf(run, min32(v));
 }
 
@@ -458,8 +463,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // ------------------------------------------------------------ norm warps
         // One thread per X row: ||x||^2/2 from the swizzled X tile (16-byte granule g of row r sits
         // at position g ^ (r & 7); the order of the granules does not matter for a sum), split into
-        // three bf16 terms and written as the X-side operand of the extra k-step.  These warps run a
-        // row tile ahead of the MMA warp, so the operand is ready when the first centroid tile needs it.
+        // three bf16 terms and written, with the row's offset M and margin m, as the X-side operand of
+        // the extra k-step.  These warps run a row tile ahead of the MMA warps, so the operand is
+        // ready when the first centroid tile needs it.
         const int r = (warp - AUX_WARP0) * 32 + lane;
         uint32_t xb = 0, xph = 0;
         bool ok = true;
@@ -480,12 +486,24 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     a = bf16lo(w.w); xn2 = fmaf(a, a, xn2); a = bf16hi(w.w); xn3 = fmaf(a, a, xn3);
                 }
             }
+            const float xn = (xn0 + xn1) + (xn2 + xn3);
             uint32_t hi, mid, lo;
-            split3(0.5f * ((xn0 + xn1) + (xn2 + xn3)), hi, mid, lo);
-            // interleaved (no-swizzle) K-major layout, columns 0..7 only: one 16-byte row per X row
+            split3(0.5f * xn, hi, mid, lo);
+            // offset M = 2^(E-127): the smallest power of two >= 2 (||x||^2 + max ||c||^2) whose biased
+            // exponent E is 0 or 1 modulo 4 (then bits(M) * 128 is 0 or 2^30 modulo 2^32 and the keys
+            // of the row are positive floats); m = M / 4096
+            const int tb = static_cast<int>(tile / p.m_tiles);
+            const float bound = 2.f * (xn + __int_as_float(__ldg(p.cnmax + tb)));
+            const uint32_t bb = __float_as_uint(bound);
+            uint32_t E = (bb >> 23) + ((bb & 0x7FFFFFu) ? 1u : 0u);
+            E += (E & 3u) == 2u ? 2u : ((E & 3u) == 3u ? 1u : 0u);
+            E = E < 36u ? 36u : (E > 248u ? 248u : E);
+            ctrl->row_e[xb][r] = static_cast<int>(E);
+            // interleaved (no-swizzle) K-major layout, columns 0..7 only: one 16-byte row per X row;
+            // a power of two is exact in bf16: its bits are the top half of the fp32 pattern
             const uint32_t one = 0x3F80u;
             *reinterpret_cast<uint4*>(smem + auga_off + xb * AUG_A_BYTES + r * 16) =
-                make_uint4(hi | (mid << 16), lo | (one << 16), one | (one << 16), 0u);
+                make_uint4(hi | (mid << 16), lo | (one << 16), one | (one << 16), (E << 7) | ((E - 12u) << 23));
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
@@ -502,6 +520,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int q = warp & 3;              // TMEM lane quarter this warp may read
         const int r = q * 32 + lane;         // row inside the X tile
         uint32_t tile_it = 0, acc_it = 0;
+        uint32_t exb = 0, exph = 0;          // X buffer (slot of the row exponents) and its phase
         bool ok = true;
         double dsum = 0.0;                   // this thread's share of the current problem's inertia
         int dsum_b = -1;
@@ -524,11 +543,19 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             }
             float best = __uint_as_float(F32_INF);   // packed: a key; exact: a value
             int bsel = 0;                            // packed: tile number; exact: global column
+            int rowE = 0;                            // biased exponent of this row's offset M (wg 0 only)
             for (int nt = 0; nt < p.n_tiles; ++nt, ++acc_it) {
                 const uint32_t as = acc_it & 1u, aph = (acc_it >> 1) & 1u;
                 ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
                 if (!ok) break;
                 ptx::tc_fence_after();
+                if (nt == 0 && wg == 0) {
+                    // written by the norm warps before they completed auga_full; read now, while the X
+                    // buffer (and with it this slot) cannot have been handed to a later row tile
+                    ok = wait_bar(&ctrl->auga_full[exb], exph, ctrl, p.status);
+                    if (!ok) break;
+                    rowE = ctrl->row_e[exb][r];
+                }
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                        as * BLOCK_N + wg * (BLOCK_N / 2);
                 // all four 32-column groups are requested at once; as soon as they are in registers
@@ -567,6 +594,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             }
             if (!ok) break;
             trace_mark(ctrl, 102);
+            if (++exb == static_cast<uint32_t>(p.n_xbuf)) { exb = 0; exph ^= 1u; }
+            // (value, index) of this half; the value is a key with its column bits cleared (packed) or
+            // the accumulator itself (exact): both compare like the fixed-point distance
             float bval;
             int bidx;
             if (PACKED) {
@@ -600,7 +630,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const i64 row = static_cast<i64>(mt) * BLOCK_M + r;
                 if (row < p.N) {
                     const size_t o = static_cast<size_t>(b) * static_cast<size_t>(p.N) + row;
-                    const float dist = fmaxf(0.f, 2.f * bval);
+                    // back from fixed point: d/2 = fx * ulp(M) - m
+                    const uint32_t E = static_cast<uint32_t>(rowE);
+                    const uint32_t fx = PACKED ? (__float_as_uint(bval) >> 7) - ((E & 3u) << 23)
+                                               : __float_as_uint(bval) - (E << 23);
+                    const float half = fmaf(static_cast<float>(fx), __uint_as_float((E - 23u) << 23),
+                                            -__uint_as_float((E - 12u) << 23));
+                    const float dist = fmaxf(0.f, 2.f * half);
                     p.out_idx[o] = bidx;
                     if (p.out_dist) p.out_dist[o] = dist;
                     dsum += static_cast<double>(dist);
@@ -622,12 +658,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 }
 
 // Prologue: the centroid-side operand of the extra k-step.  One warp per padded centroid row k:
-// h = ||c_k||^2 / 2 split into three bf16 terms, written as the 16-byte row [1 1 1 h_hi h_mid h_lo 0 0]
+// h = ||c_k||^2 / 2 split into three bf16 terms, written as the 16-byte row [1 1 1 h_hi h_mid h_lo 1 1]
 // (columns 0..7 of the operand in the interleaved K-major layout the MMA reads: 256 rows x 16 B = 4 KiB
-// per tile; columns 8..15 are zeros the kernel supplies itself).  Rows k >= K get h = +inf and can never win.
+// per tile; columns 8..15 are zeros the kernel supplies itself).  Rows k >= K are [1 1 1 0 0 0 1.5 1]:
+// their accumulator is 1.5 M + ... and can never win.  cnmax[b] collects max_k ||c_k||^2 (the bit
+// patterns of non-negative floats order like integers); it must be zero on entry.
 __global__ void __launch_bounds__(256)
 centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64 total_rows,
-                    uint8_t* __restrict__ caug) {
+                    uint8_t* __restrict__ caug, int* __restrict__ cnmax) {
     const i64 w = (static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (w >= total_rows) return;
@@ -644,12 +682,17 @@ centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     }
     if (lane == 0) {
-        uint32_t hi = 0x7F80u, mid = 0, lo = 0;   // +inf for padded rows
-        if (k < K) split3(0.5f * acc, hi, mid, lo);
+        uint32_t hi = 0, mid = 0, lo = 0, b6 = 0x3FC0u;   // padded rows: no norm, 1.5 M
+        if (k < K) {
+            split3(0.5f * acc, hi, mid, lo);
+            b6 = 0x3F80u;
+            atomicMax(cnmax + b, __float_as_int(acc));
+        }
         const uint32_t one = 0x3F80u;
         const int tile = k / BLOCK_N, rr = k % BLOCK_N;
         uint8_t* blk = caug + (static_cast<size_t>(b) * (Kpad / BLOCK_N) + tile) * AUG_B_BYTES;
-        *reinterpret_cast<uint4*>(blk + rr * 16) = make_uint4(one | (one << 16), one | (hi << 16), mid | (lo << 16), 0u);
+        *reinterpret_cast<uint4*>(blk + rr * 16) =
+            make_uint4(one | (one << 16), one | (hi << 16), mid | (lo << 16), b6 | (one << 16));
     }
 }
 
@@ -708,7 +751,7 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
 }
 
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
-                     bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride,
+                     int* cnmax, bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride,
                      int* status, cudaStream_t s) {
     if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
     DeviceInfo di;
@@ -724,6 +767,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     p.n_tiles = (K + BLOCK_N - 1) / BLOCK_N;
     p.total_tiles = static_cast<i64>(B) * p.m_tiles;
     p.caug = static_cast<const uint8_t*>(caug);
+    p.cnmax = cnmax;
     p.out_idx = out_idx; p.out_dist = out_dist; p.status = status;
     p.inertia = inertia; p.inertia_stride = inertia_stride;
     if (p.total_tiles == 0) return CAKE_OK;
@@ -732,8 +776,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     {
         const i64 rows = static_cast<i64>(B) * Kpad;
         const i64 ctas = (rows * 32 + 255) / 256;
+        if (cudaMemsetAsync(cnmax, 0, static_cast<size_t>(B) * sizeof(int), s) != cudaSuccess) return CAKE_ERR_CUDA;
         centroid_aug_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(C, K, D, Kpad, rows,
-                                                                        static_cast<uint8_t*>(caug));
+                                                                        static_cast<uint8_t*>(caug), cnmax);
         note_launches(1);
     }
 

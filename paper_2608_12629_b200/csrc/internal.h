@@ -36,10 +36,11 @@ inline int padded_k(int K) { return (int)round_up(K, kAssignBlockN); }
 bool assign_tc_supports(int D);
 // bytes of scratch (`caug`) the tensor-core assign needs for B problems of K centroids
 size_t assign_tc_aug_bytes(i64 B, int K);
-// prologue (half-norm operand into caug) + the assign kernel; exact selects the exact epilogue;
-// inertia (nullable): inertia[b * inertia_stride] += sum_i dist[b][i], fp64, must be zeroed by the caller
+// prologue (half-norm operand into caug, max ||c||^2 into cnmax[B]) + the assign kernel; exact selects
+// the exact epilogue; inertia (nullable): inertia[b * inertia_stride] += sum_i dist[b][i], fp64, must
+// be zeroed by the caller
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
-                     bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride,
+                     int* cnmax, bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride,
                      int* status, cudaStream_t s);
 int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
                        int* out_idx, float* out_dist, cudaStream_t s);
