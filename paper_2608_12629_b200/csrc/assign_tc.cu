@@ -534,9 +534,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             }
             dsum = 0.0;
         };
-        for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
-            const int b = static_cast<int>(tile / p.m_tiles);
-            const int mt = static_cast<int>(tile % p.m_tiles);
+        // (problem, row tile) of the current tile, stepped instead of divided
+        int b = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
+        int mt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
+        auto next_tile = [&]() {
+            mt += static_cast<int>(gridDim.x);
+            while (mt >= p.m_tiles) { mt -= p.m_tiles; ++b; }
+        };
+        for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
             if (b != dsum_b) {
                 flush_inertia();
                 dsum_b = b;
