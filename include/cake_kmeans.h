@@ -60,13 +60,19 @@ enum {
 enum {
     CAKE_ASSIGN_AUTO = 0,
     CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 256.
-                                  Distances that agree to 2^-16 relative are ordered by index.   */
+                                  Distances are compared as fixed-point numbers with a quantum of
+                                  about 2^-19 of (|x|^2 + max |c|^2); equal ones go to the lower index */
     CAKE_ASSIGN_SIMT = 2,      /* plain CUDA-core fallback, any D                               */
     CAKE_ASSIGN_TCGEN05_EXACT = 3, /* same pipeline, full-precision comparison (slower epilogue) */
     CAKE_ASSIGN_MASK = 0xF,
     CAKE_UPDATE_AUTO = 0,
     CAKE_UPDATE_SMEM = 1 << 4, /* shared-memory partial sums; needs K*D*4 + K*4 bytes of smem   */
     CAKE_UPDATE_SORT = 2 << 4, /* counting sort by cluster + segmented reduction, any K         */
+    CAKE_UPDATE_SLAB = 3 << 4, /* one kernel sorts and reduces slab by slab (thread-block clusters
+                                  when K is large against the slab); D % 8 == 0, D <= 256, K <= 8192 */
+    CAKE_UPDATE_SLAB_F1 = 4 << 4, /* the same with the cluster size forced to 1, 2 or 4 CTAs      */
+    CAKE_UPDATE_SLAB_F2 = 5 << 4,
+    CAKE_UPDATE_SLAB_F4 = 6 << 4,
     CAKE_UPDATE_MASK = 0xF << 4
 };
 

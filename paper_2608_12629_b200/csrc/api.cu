@@ -92,21 +92,25 @@ int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, co
     if (rc != CAKE_OK) return rc;
     unsigned path = flags & CAKE_UPDATE_MASK;
     if (path == CAKE_UPDATE_AUTO) {
-        // the shared-memory table wins only while the whole problem is launch-bound (measured:
-        // N=32,768 D=64 K=128); the sort route is faster everywhere else
-        const bool tiny = static_cast<double>(B) * N * D <= 4.0e6;
-        path = (tiny && update_smem_supports(D, K, di.smem_optin)) ? CAKE_UPDATE_SMEM : CAKE_UPDATE_SORT;
+        // the slab route while a slab holds several rows per cluster, else the global sort; the
+        // shared-memory table never measured faster than either and is only taken on request
+        path = update_slab_preferred(B, N, D, K) ? CAKE_UPDATE_SLAB : CAKE_UPDATE_SORT;
     }
     if (path == CAKE_UPDATE_SMEM) {
         rc = launch_update_smem(X, idx, B, N, D, K, w.sums, out_counts, w.status, s);
     } else if (path == CAKE_UPDATE_SORT) {
         UpdateScratch scr{w.sums, w.nvalid, w.cursor, w.pairs, w.part};
         rc = launch_update_sort(X, idx, B, N, D, K, scr, out_counts, w.status, s);
+    } else if (path == CAKE_UPDATE_SLAB || path == CAKE_UPDATE_SLAB_F1 || path == CAKE_UPDATE_SLAB_F2 ||
+               path == CAKE_UPDATE_SLAB_F4) {
+        const int force_f = path == CAKE_UPDATE_SLAB ? 0 : path == CAKE_UPDATE_SLAB_F1 ? 1 : path == CAKE_UPDATE_SLAB_F2 ? 2 : 4;
+        rc = launch_update_slab(X, idx, B, N, D, K, w.sums, out_counts, w.status, force_f, s);
     } else {
         rc = CAKE_ERR_UNSUPPORTED;
     }
     if (rc != CAKE_OK) return rc;
-    if (launch_finalize(w.sums, out_counts, C_prev, B, K, D, out_C, out_C_bf16, s) != cudaSuccess)
+    const bool slab = path != CAKE_UPDATE_SMEM && path != CAKE_UPDATE_SORT;
+    if (launch_finalize(w.sums, out_counts, C_prev, B, K, D, out_C, out_C_bf16, slab, s) != cudaSuccess)
         return CAKE_ERR_CUDA;
     return CAKE_OK;
 }
@@ -218,7 +222,7 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     if (iters == 0) {
         // out_C = C0 widened: the division kernel with all-zero counts takes the keep-previous branch
         if (cudaMemsetAsync(w.cursor, 0, static_cast<size_t>(B) * K * 4, s) != cudaSuccess) return CAKE_ERR_CUDA;
-        if (launch_finalize(w.sums, w.cursor, w.cbuf[0], Bi, K, D, out_C, nullptr, s) != cudaSuccess)
+        if (launch_finalize(w.sums, w.cursor, w.cbuf[0], Bi, K, D, out_C, nullptr, false, s) != cudaSuccess)
             return CAKE_ERR_CUDA;
     }
     for (int t = 0; t < iters; ++t) {

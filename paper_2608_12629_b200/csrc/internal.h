@@ -60,9 +60,17 @@ int launch_update_smem(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
                        int* counts, int* status, cudaStream_t s);
 int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K,
                        const UpdateScratch& scr, int* counts, int* status, cudaStream_t s);
-// out_C = counts>0 ? sums/counts : C_prev (or 0); optional bf16 copy
+// slab route (one kernel sorts and reduces slab by slab): D % 8 == 0, D <= 256, K <= 8192.
+// force_f = 0 lets the launcher choose the thread-block cluster size, else 1, 2 or 4.
+bool update_slab_supports(int D, int K);
+// true when its runs of equal clusters are long enough to beat the sort route (measured threshold)
+bool update_slab_preferred(int B, i64 N, int D, int K);
+int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, float* sums,
+                       int* counts, int* status, int force_f, cudaStream_t s);
+// out_C = counts>0 ? sums/counts : C_prev (or 0); optional bf16 copy.  early: launched so that it may
+// start before the kernel ahead of it in the stream has drained (it waits for that kernel itself)
 cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B,
-                            int K, int D, float* out_C, cake_bf16* out_C_bf16, cudaStream_t s);
+                            int K, int D, float* out_C, cake_bf16* out_C_bf16, bool early, cudaStream_t s);
 
 // ---- inertia: acc[b] += sum_i dist[b][i] (fp64 atomics); acc stride given in elements
 cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc_stride,

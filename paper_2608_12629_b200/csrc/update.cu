@@ -10,7 +10,12 @@
 //                in registers and adds one partial per cluster it touches.  Any K; for K <= 8192 the
 //                sort works on per-slab shared-memory histograms and needs no global atomics.
 // Both stream X exactly once with 16-byte (smem route: 4-byte) loads; HBM bandwidth is the bound.
+#include <cooperative_groups.h>
+
 #include "internal.h"
+#include "ptx.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace cake {
 namespace {
@@ -475,6 +480,211 @@ segreduce_scalar_kernel(const cake_bf16* __restrict__ X, const int2* __restrict_
     }
 }
 
+// ======================================================================= slab route
+// One kernel sorts and reduces.  A CTA owns a slab of S consecutive rows: it keeps their cluster ids
+// in registers, ranks every row inside its cluster with one shared-memory atomic, scans the
+// histogram and writes the slab's rows in cluster order into shared memory; then lane groups walk
+// that order, gather the rows (all inside the slab's own window of X, which keeps the DRAM pages
+// busy) and flush one vector atomic per run of equal clusters.  A run is S/K rows long, so when K
+// is large against S, F CTAs form a thread-block cluster: their histograms are combined through
+// distributed shared memory into one order over the F*S rows of the cluster, every CTA takes an
+// equal contiguous share of it, and runs are F times longer (F times fewer atomics).
+constexpr int SLAB_THREADS = 1024;
+constexpr int SLAB_VPT = 16;                               // cluster ids per thread (registers)
+constexpr int SLAB_MAX_ROWS = SLAB_THREADS * SLAB_VPT;     // rows per CTA
+constexpr int SLAB_MAX_K = 8192;
+constexpr int SLAB_AHEAD = 4;                              // rows in flight per lane group
+constexpr int SLAB_MAX_F = 4;
+constexpr int SLAB_GROW_RUN = 8;                           // clusters grow until a run has this many rows
+constexpr int SLAB_MIN_RUN = 4;                            // rows per run below which the sort route is faster
+
+// sums and counts start at zero; the kernel behind it may begin at once (it waits before its first add)
+__global__ void __launch_bounds__(256)
+zero_sums_counts_kernel(float4* __restrict__ sums4, i64 n4, int* __restrict__ counts, i64 nc) {
+    ptx::grid_dep_launch();
+    const i64 stride = static_cast<i64>(gridDim.x) * blockDim.x;
+    const i64 t = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x;
+    for (i64 e = t; e < n4; e += stride) sums4[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (i64 e = t; e < nc; e += stride) counts[e] = 0;
+}
+
+template <int LPR, bool CLUSTER>
+__global__ void __launch_bounds__(SLAB_THREADS, 1)
+slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx, i64 N, int D, int K, int S,
+                   int rowbits, float* __restrict__ sums, int* __restrict__ counts, int* status) {
+    extern __shared__ int sm[];
+    int* h = sm;                                                   // [K] this CTA's rows per cluster
+    int* off = sm + K;                                             // [K] first position of this CTA's rows of a cluster
+    uint32_t* sorted = reinterpret_cast<uint32_t*>(sm + 2 * K);    // [S] this CTA's share of the order
+    __shared__ int warp_tot[SLAB_THREADS / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.y;
+    unsigned F = 1, c = 0;
+    if constexpr (CLUSTER) {
+        F = cg::this_cluster().num_blocks();
+        c = cg::this_cluster().block_rank();
+    }
+    const i64 super_row0 = static_cast<i64>(blockIdx.x / F) * F * S;   // first row of the cluster's rows
+    const i64 r0 = super_row0 + static_cast<i64>(c) * S;
+    const int rows = r0 >= N ? 0 : static_cast<int>(r0 + S <= N ? S : N - r0);
+    const int* idx_b = idx + static_cast<size_t>(b) * N + (rows ? r0 : 0);
+    int* counts_b = counts + static_cast<size_t>(b) * K;
+
+    for (int e = tid; e < K; e += SLAB_THREADS) h[e] = 0;
+    __syncthreads();
+    // ---- cluster ids into registers, rank inside (CTA, cluster) from the histogram atomic
+    int kv[SLAB_VPT], rk[SLAB_VPT];
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(idx_b) & 15) == 0;
+#pragma unroll
+    for (int u = 0; u < SLAB_VPT / 4; ++u) {
+        const int i = (u * SLAB_THREADS + tid) * 4;
+        int4 k4 = make_int4(-1, -1, -1, -1);
+        if (vec_ok && i + 4 <= rows) {
+            k4 = *reinterpret_cast<const int4*>(idx_b + i);
+        } else {
+            if (i < rows) k4.x = idx_b[i];
+            if (i + 1 < rows) k4.y = idx_b[i + 1];
+            if (i + 2 < rows) k4.z = idx_b[i + 2];
+            if (i + 3 < rows) k4.w = idx_b[i + 3];
+        }
+        kv[u * 4] = k4.x; kv[u * 4 + 1] = k4.y; kv[u * 4 + 2] = k4.z; kv[u * 4 + 3] = k4.w;
+    }
+    bool bad = false;
+#pragma unroll
+    for (int u = 0; u < SLAB_VPT; ++u) {
+        const int i = ((u >> 2) * SLAB_THREADS + tid) * 4 + (u & 3);
+        const bool ok = static_cast<unsigned>(kv[u]) < static_cast<unsigned>(K);
+        if (!ok && i < rows) bad = true;
+        if (!ok || i >= rows) kv[u] = -1;
+        rk[u] = kv[u] >= 0 ? atomicAdd(&h[kv[u]], 1) : 0;
+    }
+    if (bad) atomicCAS(status, CAKE_OK, CAKE_ERR_BAD_INDEX);
+    // nothing above touched what the zero-fill ahead of this kernel writes; from here on it must be done
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
+    if constexpr (CLUSTER) cg::this_cluster().sync();
+    else __syncthreads();
+    // ---- offsets: exclusive scan over clusters of the cluster-wide totals, plus the rows that CTAs of
+    // lower rank hold of the same cluster
+    int total;
+    {
+        const int per = (K + SLAB_THREADS - 1) / SLAB_THREADS;
+        const int k0 = min(tid * per, K), k1 = min(k0 + per, K);
+        int local = 0;
+        for (int k = k0; k < k1; ++k) {
+            if constexpr (CLUSTER) {
+                for (unsigned j = 0; j < F; ++j) local += cg::this_cluster().map_shared_rank(h, j)[k];
+            } else {
+                local += h[k];
+            }
+        }
+        int incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        int before = 0;
+        total = 0;
+        for (int w = 0; w < SLAB_THREADS / 32; ++w) {
+            if (w < warp) before += warp_tot[w];
+            total += warp_tot[w];
+        }
+        int run = before + incl - local;
+        for (int k = k0; k < k1; ++k) {
+            int tot = 0, lower = 0;
+            if constexpr (CLUSTER) {
+                for (unsigned j = 0; j < F; ++j) {
+                    const int v = cg::this_cluster().map_shared_rank(h, j)[k];
+                    tot += v;
+                    if (j < c) lower += v;
+                }
+            } else {
+                tot = h[k];
+            }
+            if (c == 0 && tot) atomicAdd(&counts_b[k], tot);
+            off[k] = run + lower;
+            run += tot;
+        }
+    }
+    __syncthreads();
+    // every CTA of the cluster takes `share` consecutive positions of the order
+    const int share = CLUSTER ? ((total + static_cast<int>(F) - 1) / static_cast<int>(F) + 3) / 4 * 4 : total;
+    const int mine = CLUSTER ? max(0, min(share, total - static_cast<int>(c) * share)) : total;
+#pragma unroll
+    for (int u = 0; u < SLAB_VPT; ++u) {
+        if (kv[u] >= 0) {
+            const int i = ((u >> 2) * SLAB_THREADS + tid) * 4 + (u & 3);
+            const uint32_t rec = (static_cast<uint32_t>(kv[u]) << rowbits) | (c * static_cast<uint32_t>(S) + static_cast<uint32_t>(i));
+            const int pos = off[kv[u]] + rk[u];
+            if constexpr (CLUSTER) {
+                const int j = pos / share;
+                cg::this_cluster().map_shared_rank(sorted, j)[pos - j * share] = rec;
+            } else {
+                sorted[pos] = rec;
+            }
+        }
+    }
+    if constexpr (CLUSTER) cg::this_cluster().sync();
+    else __syncthreads();
+
+    // ---- segmented reduction: every lane group (LPR lanes, one 16-byte granule each) walks one
+    // contiguous piece of this CTA's positions and flushes when the cluster changes
+    constexpr int GROUPS = 32 / LPR;
+    constexpr int NGROUPS = (SLAB_THREADS / 32) * GROUPS;
+    const int G = D >> 3;
+    const int sl = lane % LPR;
+    const int gid = warp * GROUPS + lane / LPR;
+    const uint4* Xg = reinterpret_cast<const uint4*>(X) + (static_cast<size_t>(b) * N + super_row0) * G;
+    float* sums_b = sums + static_cast<size_t>(b) * K * D;
+    const uint32_t rowmask = (1u << rowbits) - 1u;
+    const int seglen = max(SLAB_AHEAD, (mine + NGROUPS - 1) / NGROUPS);
+    const int base = gid * seglen, end = min(base + seglen, mine);
+    int cur = -1;
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    auto flush = [&]() {
+        if (cur >= 0 && sl < G) {
+            float4* dst = reinterpret_cast<float4*>(sums_b + static_cast<size_t>(cur) * D + sl * 8);
+            atomicAdd(dst, make_float4(acc[0], acc[1], acc[2], acc[3]));
+            atomicAdd(dst + 1, make_float4(acc[4], acc[5], acc[6], acc[7]));
+        }
+    };
+    for (int q = base; q < end; q += SLAB_AHEAD) {
+        uint4 v[SLAB_AHEAD];
+        int kk[SLAB_AHEAD];
+#pragma unroll
+        for (int u = 0; u < SLAB_AHEAD; ++u) {
+            kk[u] = -1;
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (q + u < end) {
+                const uint32_t rec = sorted[q + u];
+                kk[u] = static_cast<int>(rec >> rowbits);
+                if (sl < G) v[u] = __ldg(Xg + static_cast<size_t>(rec & rowmask) * G + sl);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < SLAB_AHEAD; ++u) {
+            if (kk[u] >= 0) {
+                if (kk[u] != cur) {
+                    flush();
+                    cur = kk[u];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+                }
+                acc[0] += bf16lo(v[u].x); acc[1] += bf16hi(v[u].x);
+                acc[2] += bf16lo(v[u].y); acc[3] += bf16hi(v[u].y);
+                acc[4] += bf16lo(v[u].z); acc[5] += bf16hi(v[u].z);
+                acc[6] += bf16lo(v[u].w); acc[7] += bf16hi(v[u].w);
+            }
+        }
+    }
+    flush();
+}
+
 // ======================================================================= division
 __device__ __forceinline__ cake_bf16 f32_to_bf16_rne(float f) {
     uint32_t u = __float_as_uint(f);
@@ -487,6 +697,7 @@ __global__ void __launch_bounds__(256)
 finalize_kernel(const float* __restrict__ sums, const int* __restrict__ counts,
                 const cake_bf16* __restrict__ C_prev, i64 total, int D, float* __restrict__ out_C,
                 cake_bf16* __restrict__ out_C_bf16) {
+    ptx::grid_dep_wait();
     for (i64 e = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; e < total;
          e += static_cast<i64>(gridDim.x) * blockDim.x) {
         const i64 row = e / D;  // b*K + k
@@ -504,6 +715,7 @@ __global__ void __launch_bounds__(256)
 finalize4_kernel(const float4* __restrict__ sums, const int* __restrict__ counts,
                  const uint2* __restrict__ C_prev, i64 total4, int D4, float4* __restrict__ out_C,
                  uint2* __restrict__ out_C_bf16) {
+    ptx::grid_dep_wait();
     for (i64 e = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; e < total4;
          e += static_cast<i64>(gridDim.x) * blockDim.x) {
         const int n = counts[e / D4];
@@ -654,25 +866,184 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
     return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
 }
 
+// ---- slab route, host side
+namespace {
+struct SlabPlan {
+    int S;         // rows per CTA (multiple of 4)
+    int n_ctas;    // CTAs per problem (multiple of F)
+    int F;         // CTAs per thread-block cluster
+    int rowbits;   // bits of a row number inside a cluster's F*S rows
+};
+
+using SlabKernel = void (*)(const cake_bf16*, const int*, i64, int, int, int, int, float*, int*, int*);
+
+SlabKernel slab_kernel_for(int lpr, bool cluster) {
+    switch (lpr) {
+        case 4: return cluster ? slab_update_kernel<4, true> : slab_update_kernel<4, false>;
+        case 8: return cluster ? slab_update_kernel<8, true> : slab_update_kernel<8, false>;
+        case 16: return cluster ? slab_update_kernel<16, true> : slab_update_kernel<16, false>;
+        default: return cluster ? slab_update_kernel<32, true> : slab_update_kernel<32, false>;
+    }
+}
+
+int slab_lpr(int D) {
+    int lpr = 4;
+    while (lpr < D / 8) lpr <<= 1;
+    return lpr;
+}
+
+size_t slab_smem_bytes(int K, int S) { return (static_cast<size_t>(2) * K + S) * sizeof(int); }
+
+// CTAs of `kernel` that can be resident at once when launched as clusters of F (F = 1: one per SM)
+int slab_slots(const DeviceInfo& di, SlabKernel kernel, int F, size_t smem) {
+    if (cudaFuncSetAttribute(reinterpret_cast<const void*>(kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(slab_smem_bytes(SLAB_MAX_K, SLAB_MAX_ROWS))) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    if (F == 1) return di.sm_count;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(F) * di.sm_count);
+    cfg.blockDim = dim3(SLAB_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = static_cast<unsigned>(F);
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, reinterpret_cast<const void*>(kernel), &cfg) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        return 0;
+    }
+    return n * F;
+}
+
+// Rows per CTA so that the CTAs of all problems fill whole waves of the resident slots.
+void slab_rows_for(int slots, int B, i64 N, int F, int* S, int* n_ctas) {
+    for (int w = 1;; ++w) {
+        i64 per_problem = static_cast<i64>(w) * slots / B / F * F;
+        if (per_problem < F) per_problem = F;
+        i64 rows = (N + per_problem - 1) / per_problem;
+        if (rows < 2048) rows = 2048;                       // tiny slabs only add launches of atomics
+        rows = (rows + 3) / 4 * 4;
+        if (rows <= SLAB_MAX_ROWS) {
+            *S = static_cast<int>(rows);
+            const i64 n = (N + rows - 1) / rows;
+            *n_ctas = static_cast<int>((n + F - 1) / F * F);
+            return;
+        }
+    }
+}
+}  // namespace
+
+bool update_slab_supports(int D, int K) { return D % 8 == 0 && D >= 8 && D <= 256 && K <= SLAB_MAX_K; }
+
+static int slab_make_plan(const DeviceInfo& di, int B, i64 N, int D, int K, int force_f, SlabPlan* out) {
+    const int lpr = slab_lpr(D);
+    SlabPlan best = {};
+    for (int F = 1; F <= SLAB_MAX_F; F <<= 1) {
+        if (force_f && F != force_f) continue;
+        SlabPlan pl;
+        pl.F = F;
+        const int slots = slab_slots(di, slab_kernel_for(lpr, F > 1), F, slab_smem_bytes(K, SLAB_MAX_ROWS));
+        if (slots < F) continue;
+        slab_rows_for(slots, B, N, F, &pl.S, &pl.n_ctas);
+        pl.rowbits = 1;
+        while ((static_cast<i64>(1) << pl.rowbits) < static_cast<i64>(pl.S) * F) ++pl.rowbits;
+        best = pl;
+        // runs of SLAB_GROW_RUN rows keep the atomics cheap (measured); larger clusters only cost
+        if (static_cast<i64>(pl.S) * F >= static_cast<i64>(SLAB_GROW_RUN) * K || pl.n_ctas <= F) break;
+    }
+    if (best.F == 0) return CAKE_ERR_UNSUPPORTED;
+    *out = best;
+    return CAKE_OK;
+}
+
+bool update_slab_preferred(int B, i64 N, int D, int K) {
+    DeviceInfo di;
+    SlabPlan pl;
+    if (N < 1 || !update_slab_supports(D, K) || current_device_info(&di) != CAKE_OK) return false;
+    if (slab_make_plan(di, B, N, D, K, 0, &pl) != CAKE_OK) return false;
+    const i64 rows = static_cast<i64>(pl.S) * pl.F;
+    return (rows < N ? rows : N) >= static_cast<i64>(SLAB_MIN_RUN) * K;
+}
+
+int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, float* sums, int* counts,
+                       int* status, int force_f, cudaStream_t s) {
+    DeviceInfo di;
+    int rc = current_device_info(&di);
+    if (rc != CAKE_OK) return rc;
+    if (!update_slab_supports(D, K)) return CAKE_ERR_UNSUPPORTED;
+    {
+        // D % 8 == 0, so the sums are whole float4s
+        const i64 n4 = static_cast<i64>(B) * K * D / 4, nc = static_cast<i64>(B) * K;
+        i64 ctas = (n4 + 256 * 4 - 1) / (256 * 4);
+        if (ctas > di.sm_count * 4) ctas = di.sm_count * 4;
+        zero_sums_counts_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(reinterpret_cast<float4*>(sums), n4, counts, nc);
+        note_launches(1);
+        if (cudaGetLastError() != cudaSuccess) return CAKE_ERR_CUDA;
+    }
+    if (N == 0) return CAKE_OK;
+    SlabPlan pl;
+    rc = slab_make_plan(di, B, N, D, K, force_f, &pl);
+    if (rc != CAKE_OK) return rc;
+    const int lpr = slab_lpr(D);
+    SlabKernel kernel = slab_kernel_for(lpr, pl.F > 1);
+    const size_t smem = slab_smem_bytes(K, pl.S);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(pl.n_ctas), static_cast<unsigned>(B));
+    cfg.blockDim = dim3(SLAB_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    // may start while the zero-fill still runs (it waits for it before its first add)
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    at[1].id = cudaLaunchAttributeClusterDimension;
+    at[1].val.clusterDim.x = static_cast<unsigned>(pl.F);
+    at[1].val.clusterDim.y = 1;
+    at[1].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pl.F > 1 ? 2 : 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, X, idx, N, D, K, pl.S, pl.rowbits, sums, counts, status) != cudaSuccess) {
+        cudaGetLastError();
+        return CAKE_ERR_CUDA;
+    }
+    note_launches(1);
+    return CAKE_OK;
+}
+
 cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B, int K,
-                            int D, float* out_C, cake_bf16* out_C_bf16, cudaStream_t s) {
+                            int D, float* out_C, cake_bf16* out_C_bf16, bool early, cudaStream_t s) {
     const i64 total = static_cast<i64>(B) * K * D;
+    // early: the launch may overlap the tail of the kernel ahead (the kernels wait for it themselves)
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cfg.attrs = at;
+    cfg.numAttrs = early ? 1 : 0;
     if (D % 4 == 0) {
         i64 ctas = (total / 4 + 255) / 256;
         if (ctas > 148 * 16) ctas = 148 * 16;
         if (ctas < 1) ctas = 1;
-        finalize4_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(
-            reinterpret_cast<const float4*>(sums), counts, reinterpret_cast<const uint2*>(C_prev), total / 4, D / 4,
-            reinterpret_cast<float4*>(out_C), reinterpret_cast<uint2*>(out_C_bf16));
+        cfg.gridDim = dim3(static_cast<unsigned>(ctas));
         note_launches(1);
-        return cudaGetLastError();
+        return cudaLaunchKernelEx(&cfg, finalize4_kernel, reinterpret_cast<const float4*>(sums), counts,
+                                  reinterpret_cast<const uint2*>(C_prev), total / 4, D / 4,
+                                  reinterpret_cast<float4*>(out_C), reinterpret_cast<uint2*>(out_C_bf16));
     }
     i64 ctas = (total + 256 * 4 - 1) / (256 * 4);
     if (ctas > 148 * 16) ctas = 148 * 16;
     if (ctas < 1) ctas = 1;
-    finalize_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(sums, counts, C_prev, total, D, out_C, out_C_bf16);
+    cfg.gridDim = dim3(static_cast<unsigned>(ctas));
     note_launches(1);
-    return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, finalize_kernel, sums, counts, C_prev, total, D, out_C, out_C_bf16);
 }
 
 }  // namespace cake

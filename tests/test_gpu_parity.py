@@ -176,14 +176,45 @@ def test_update_sort_route_slab_tails_and_large_k(N, D, K):
                          inputs.to_bits(Cb), counts.cpu().numpy())
 
 
-def test_update_batched_unaligned_problem_size():
+SLAB_FLAGS = {"auto": cake.CAKE_UPDATE_SLAB, "f1": cake.CAKE_UPDATE_SLAB_F1, "f2": cake.CAKE_UPDATE_SLAB_F2,
+              "f4": cake.CAKE_UPDATE_SLAB_F4}
+
+
+@pytest.mark.parametrize("f", ["auto", "f1", "f2", "f4"])
+@pytest.mark.parametrize("N,D,K", [(1, 64, 1), (1000, 64, 128), (70001, 64, 100), (20000, 128, 3000), (8193, 16, 8192),
+                                   (50003, 96, 17), (300001, 128, 1024), (33000, 256, 512), (2500, 8, 3)])
+def test_update_slab_route(f, N, D, K):
+    """Slab route: ragged last slab, N % 4 != 0, clusters of 1, 2 and 4 CTAs (also with CTAs that get no
+    rows), K at the shared-memory limit, D that does not fill the lane group."""
+    X, C = problem(N, D, K, seed=N + D)
+    g = torch.Generator().manual_seed(K)
+    idx = torch.randint(0, K, (N,), generator=g, dtype=torch.int32)
+    if K > 4:
+        idx[idx == 1] = 0                      # cluster 1 empty, cluster 0 heavy
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=C.to(DEV), ws=ws, flags=SLAB_FLAGS[f])
+    check_status(ws)
+    grading.grade_update(inputs.to_bits(X), idx.numpy(), K, inputs.to_bits(C), Cf.cpu().numpy(),
+                         inputs.to_bits(Cb), counts.cpu().numpy())
+
+
+def test_update_slab_route_refuses_what_it_cannot_run():
+    X, C = problem(100, 12, 4, seed=1)
+    idx = torch.zeros(100, dtype=torch.int32)
+    with pytest.raises(cake.CakeError) as e:
+        cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), 4, C_prev=C.to(DEV), flags=cake.CAKE_UPDATE_SLAB)
+    assert e.value.code == cake.CAKE_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("flag", [cake.CAKE_UPDATE_SORT, cake.CAKE_UPDATE_SLAB, cake.CAKE_UPDATE_SLAB_F2])
+def test_update_batched_unaligned_problem_size(flag):
     """B > 1 with N % 4 != 0: the per-problem idx slices are not 16-byte aligned."""
     B, N, D, K = 3, 10001, 64, 37
     Xs, Cs = zip(*(problem(N, D, K, seed=20 + b) for b in range(B)))
     X, C = torch.stack(Xs), torch.stack(Cs)
     g = torch.Generator().manual_seed(1)
     idx = torch.randint(0, K, (B, N), generator=g, dtype=torch.int32)
-    Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=C.to(DEV), flags=cake.CAKE_UPDATE_SORT)
+    Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=C.to(DEV), flags=flag)
     for b in range(B):
         grading.grade_update(inputs.to_bits(Xs[b]), idx[b].numpy(), K, inputs.to_bits(Cs[b]), Cf[b].cpu().numpy(),
                              inputs.to_bits(Cb[b]), counts[b].cpu().numpy())
@@ -199,9 +230,10 @@ def test_update_odd_feature_count_and_null_prev():
     assert not Cf[K - 1].any()
 
 
-@pytest.mark.parametrize("path", ["smem", "sort"])
+@pytest.mark.parametrize("path", ["smem", "sort", "slab", "slab_f2"])
 def test_update_bad_index_is_skipped_and_reported(path):
-    flag = cake.CAKE_UPDATE_SMEM if path == "smem" else cake.CAKE_UPDATE_SORT
+    flag = {"smem": cake.CAKE_UPDATE_SMEM, "sort": cake.CAKE_UPDATE_SORT, "slab": cake.CAKE_UPDATE_SLAB,
+            "slab_f2": cake.CAKE_UPDATE_SLAB_F2}[path]
     N, D, K = 1000, 64, 10
     X, C = problem(N, D, K, seed=3)
     idx = (torch.arange(N) % K).to(torch.int32)
@@ -222,7 +254,7 @@ def test_update_batched_and_n_zero():
     X, C = torch.stack(Xs), torch.stack(Cs)
     g = torch.Generator().manual_seed(0)
     idx = torch.randint(0, K, (B, N), generator=g, dtype=torch.int32)
-    for flag in (cake.CAKE_UPDATE_SMEM, cake.CAKE_UPDATE_SORT):
+    for flag in (cake.CAKE_UPDATE_SMEM, cake.CAKE_UPDATE_SORT, cake.CAKE_UPDATE_SLAB, cake.CAKE_UPDATE_SLAB_F4):
         Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=C.to(DEV), flags=flag)
         for b in range(B):
             grading.grade_update(inputs.to_bits(Xs[b]), idx[b].numpy(), K, inputs.to_bits(Cs[b]),
