@@ -269,7 +269,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
         for (int i = 0; i < MAX_STAGES; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->ring_empty[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->ring_empty[i]), 2);   // the consuming issuer and the one passing over
         }
         ctrl->abort_flag = 0;
 #ifdef CAKE_ASSIGN_TRACE
@@ -399,9 +399,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const uint32_t auga_lo = ptx::umma_desc_lo_aug(smem_base + auga_off + xb * AUG_A_BYTES,
                                                                smem_base + zero_off);
                 for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it) {
-                    if ((acc_it & 1u) != par) {             // the other issuer's tile: pass over its ring slots
+                    if ((acc_it & 1u) != par) {
+                        // The other issuer's tile: pass over its ring slots, but see each of them filled
+                        // and only then let the slot be refilled.  That keeps the two issuers in tile
+                        // order and this one at most one phase behind any slot (a parity wait that
+                        // falls two phases behind waits for ever).
                         for (int c = 0; ok && c < p.nchunks; ++c) {
                             ok = wait_bar(&ctrl->ring_full[s], ph, ctrl, p.status);
+                            if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->ring_empty[s]));
                             if (++s == nstg) { s = 0; ph ^= 1u; }
                         }
                         continue;
