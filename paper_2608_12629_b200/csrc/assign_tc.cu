@@ -46,7 +46,8 @@ constexpr int KCHUNK = 64;              // bf16 columns per swizzled 128-byte ro
 constexpr int UMMA_K = 16;
 constexpr int NUM_EPI_WARPS = 8;
 constexpr int PRODUCER_WARP = 8;
-constexpr int MMA_WARP = 9;             // warps 9 and 10: the two MMA issuers (warp 11 idles)
+constexpr int MMA_WARP = 9;             // warps 9, 10 and 11: the MMA issuers
+constexpr int NUM_ISSUERS = 3;
 constexpr int AUX_WARP0 = 12;           // warps 12..15: row norms
 constexpr int NUM_WARPS = 16;
 constexpr int EPI_REGS = 192;           // registers per thread after reallocation: epilogue warpgroups
@@ -93,7 +94,10 @@ struct Params {
 struct Ctrl {  // lives in shared memory
     uint64_t x_full[MAX_XBUF], x_empty[MAX_XBUF];
     uint64_t ring_full[MAX_STAGES], ring_empty[MAX_STAGES];
-    uint64_t tmem_full[2], tmem_empty[2];
+    uint64_t tmem_full[2];
+    // release of accumulator a, one barrier per issuer that may take it next: each barrier has a
+    // single waiter that sees every one of its phases
+    uint64_t tmem_empty[2][NUM_ISSUERS];
     uint64_t auga_full[MAX_XBUF];
     uint64_t augb_full[N_AUGB], augb_empty[N_AUGB];
     uint64_t merge_full[2], merge_empty[2];
@@ -254,12 +258,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAX_XBUF; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), 2 + 4);  // 2 MMA issuers + 4 norm warps
+            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), NUM_ISSUERS + 4);  // MMA issuers + 4 norm warps
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i]), NUM_EPI_WARPS);
+            for (int j = 0; j < NUM_ISSUERS; ++j)
+                ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i][j]), NUM_EPI_WARPS);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_full[i]), 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_empty[i]), 4);
         }
@@ -269,7 +274,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
         for (int i = 0; i < MAX_STAGES; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->ring_empty[i]), 2);   // the consuming issuer and the one passing over
+            ptx::mbar_init(ptx::smem_u32(&ctrl->ring_empty[i]), NUM_ISSUERS);   // the consuming issuer and those passing over
         }
         ctrl->abort_flag = 0;
 #ifdef CAKE_ASSIGN_TRACE
@@ -370,14 +375,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 }
             }
         }
-    } else if (warp == MMA_WARP || warp == MMA_WARP + 1) {
+    } else if (warp >= MMA_WARP && warp < MMA_WARP + NUM_ISSUERS) {
         // ------------------------------------------------------------ MMA issuers
-        // Two warps, one issuing thread each.  Issuer `par` owns TMEM accumulator `par` and takes every
-        // other centroid tile, so the barrier waits, commits and bookkeeping of one issuer run while
-        // the other's MMAs keep the tensor pipe busy (a single issuer leaves it idle between tiles).
-        // The two never touch the same accumulator or ring slot, so no order between them is needed.
+        // Three warps, one issuing thread each; centroid tiles go round robin over them (tile t to
+        // issuer t mod 3, into accumulator t mod 2).  One thread cannot keep the tensor pipe fed: per
+        // tile it spends about three times the pipe's 9 x 128 clocks on its own instruction stream
+        // (waits, descriptor arithmetic, commits, and MMA issue that blocks at the pipe's pace), so
+        // three of them take turns.  No two ever hold the same accumulator or ring slot at a time.
         if (lane == 0) {
-            const uint32_t par = static_cast<uint32_t>(warp - MMA_WARP);
+            const uint32_t iss = static_cast<uint32_t>(warp - MMA_WARP);
             constexpr uint32_t idesc_aug = ptx::umma_idesc_bf16(BLOCK_M, BLOCK_N);
             constexpr uint32_t idesc_main = idesc_aug | ptx::UMMA_IDESC_NEGATE_B;   // accumulates -x.c
             // descriptors are (low, high) words with the high word constant; stage / phase counters
@@ -387,7 +393,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             uint32_t s = 0, ph = 0;                         // ring position of the next chunk (all tiles)
             uint32_t xb = 0, xph = 0;                       // X buffer and its phase
             uint32_t acc_it = 0;
-            const uint32_t d_tmem = tmem_base + par * BLOCK_N;
+            uint32_t turn = 0;                              // acc_it mod NUM_ISSUERS
+            uint32_t rel0 = 0, rel1 = 0;                    // releases of accumulator 0 / 1 this issuer has consumed
             bool ok = true;
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 // every phase of the shared barriers is observed, also in row / centroid tiles this
@@ -398,12 +405,12 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const uint32_t a_lo_tile = ptx::umma_desc_lo_sw128(x_base + xb * xbuf_bytes);
                 const uint32_t auga_lo = ptx::umma_desc_lo_aug(smem_base + auga_off + xb * AUG_A_BYTES,
                                                                smem_base + zero_off);
-                for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it) {
-                    if ((acc_it & 1u) != par) {
-                        // The other issuer's tile: pass over its ring slots, but see each of them filled
-                        // and only then let the slot be refilled.  That keeps the two issuers in tile
-                        // order and this one at most one phase behind any slot (a parity wait that
-                        // falls two phases behind waits for ever).
+                for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it, turn = (turn + 1 == NUM_ISSUERS) ? 0 : turn + 1) {
+                    if (turn != iss) {
+                        // Another issuer's tile: pass over its ring slots, but see each of them filled
+                        // and only then let the slot be refilled.  That keeps the issuers in tile order
+                        // and this one at most one phase behind any slot (a parity wait that falls two
+                        // phases behind waits for ever).
                         for (int c = 0; ok && c < p.nchunks; ++c) {
                             ok = wait_bar(&ctrl->ring_full[s], ph, ctrl, p.status);
                             if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->ring_empty[s]));
@@ -411,9 +418,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         }
                         continue;
                     }
-                    const uint32_t aph = (acc_it >> 1) & 1u;
-                    ok = wait_bar(&ctrl->tmem_empty[par], aph ^ 1u, ctrl, p.status);
-                    if (!ok) break;
+                    const uint32_t acc = acc_it & 1u;
+                    const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
+                    // the accumulator was last used by tile acc_it - 2, whose release is addressed to
+                    // this issuer (the first two tiles find their accumulators free)
+                    if (acc_it >= 2u) {
+                        const uint32_t rel = acc ? rel1 : rel0;
+                        ok = wait_bar(&ctrl->tmem_empty[acc][iss], rel & 1u, ctrl, p.status);
+                        if (!ok) break;
+                        if (acc) ++rel1; else ++rel0;
+                    }
                     ptx::tc_fence_after();
                     uint32_t a_lo = a_lo_tile;
                     for (int c = 0; c < p.nchunks; ++c, a_lo += X_CHUNK_BYTES >> 4) {
@@ -455,7 +469,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                                                     smem_base + zero_off),
                                               ptx::UMMA_DESC_HI_AUG, idesc_aug);
                     ptx::umma_commit(ptx::smem_u32(&ctrl->augb_empty[ab]));
-                    ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[par]));
+                    ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[acc]));
                 }
                 if (ok && !have_aug) ok = wait_bar(&ctrl->auga_full[xb], xph, ctrl, p.status);
                 // this issuer's MMAs on the X buffer are done when this commit fires (it fires at once
@@ -525,6 +539,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int q = warp & 3;              // TMEM lane quarter this warp may read
         const int r = q * 32 + lane;         // row inside the X tile
         uint32_t tile_it = 0, acc_it = 0;
+        uint32_t next_iss = 2 % NUM_ISSUERS;   // (acc_it + 2) mod NUM_ISSUERS
         uint32_t exb = 0, exph = 0;          // X buffer (slot of the row exponents) and its phase
         bool ok = true;
         double dsum = 0.0;                   // this thread's share of the current problem's inertia
@@ -581,7 +596,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 ptx::reg_dep(rd);
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as]));
+                // to the issuer of tile acc_it + 2, which takes this accumulator next
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
+                next_iss = (next_iss + 1 == NUM_ISSUERS) ? 0 : next_iss + 1;
                 trace_mark(ctrl, 100);
                 if (PACKED) {
                     float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF));
