@@ -258,7 +258,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAX_XBUF; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), NUM_ISSUERS + 4);  // MMA issuers + 4 norm warps
+            // MMA issuers + 4 norm warps + the 4 epilogue warps that read the row exponents
+            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), NUM_ISSUERS + 4 + 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
         }
         for (int i = 0; i < 2; ++i) {
@@ -575,11 +576,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 if (!ok) break;
                 ptx::tc_fence_after();
                 if (nt == 0 && wg == 0) {
-                    // written by the norm warps before they completed auga_full; read now, while the X
-                    // buffer (and with it this slot) cannot have been handed to a later row tile
+                    // Written by the norm warps before they completed auga_full.  The X buffer -- and with
+                    // it this slot and the next phase of this barrier -- is handed to a later row tile
+                    // only after these warps have arrived on x_empty: without that, with one centroid
+                    // tile per row tile, the norm warps can get two row tiles of this buffer ahead,
+                    // overwrite the exponents and leave this parity wait behind for good.
                     ok = wait_bar(&ctrl->auga_full[exb], exph, ctrl, p.status);
                     if (!ok) break;
                     rowE = ctrl->row_e[exb][r];
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[exb]));
                 }
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                        as * BLOCK_N + wg * (BLOCK_N / 2);

@@ -414,6 +414,29 @@ def test_full_size_batched_workload_sampled():
                              out.counts[b].cpu().numpy())
 
 
+@pytest.mark.parametrize("N,D,K", [(1 << 24, 64, 64), (1 << 23, 64, 300)])
+def test_assign_many_row_tiles_few_centroid_tiles(N, D, K):
+    """Hundreds of row tiles per CTA with one or two centroid tiles each: the X buffers, the norm warps'
+    row exponents and the accumulators turn over as fast as they can, which is where a barrier protocol
+    that lets any role run a whole buffer cycle ahead of another shows up (as a time-out in the status
+    word, or as distances decoded with another row's exponent)."""
+    w = inputs.sweep_workload(N, D, K)
+    X, _ = inputs.gaussian_mixture(N, D, 4096, w.mean_std, w.sigma, w.seed, device=DEV)
+    C0 = inputs.sample_init(X, K, w.seed)
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    for _ in range(2):
+        idx, dist = cake.cake_kmeans_assign(X, C0, ws=ws)
+        torch.cuda.synchronize()
+        check_status(ws)
+    rows = sampled_rows(N, 2048, K)
+    rows_t = torch.from_numpy(rows).to(DEV)
+    Xs = inputs.to_bits(X[rows_t].cpu())
+    rep = grading.grade_assign(Xs, inputs.to_bits(C0.cpu()), idx[rows_t].cpu().numpy(), dist[rows_t].cpu().numpy())
+    assert rep["mismatch"] <= 4, rep
+    # every row was written: a valid index and a finite distance
+    assert int(idx.min()) >= 0 and int(idx.max()) < K and bool(torch.isfinite(dist).all())
+
+
 # ------------------------------------------------------------------------------------ bounded waits
 
 def test_bounded_wait_expires_and_context_survives():
