@@ -33,7 +33,9 @@ from paper_2608_12629_b200 import inputs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel (assign_tc_kernel),
 # from the ncu capture summarised in profiles/assign_tc_kernel_c2.md (same workload, same launch shape)
-NCU_DRAM_BYTES_PER_ASSIGN_LAUNCH = {"c2": 268780032 + 9104384}
+NCU_DRAM_BYTES_PER_ASSIGN_LAUNCH = {"c2": 268772352 + 8958464}
+# the same for the dominant update kernel (slab_update_kernel), profiles/update_slab_route_c2.md
+NCU_DRAM_BYTES_PER_UPDATE_LAUNCH = {"c2": 273207040 + 4733952}
 
 METRIC = "lloyd_iters_per_sec"
 UNIT = "iter/s"
@@ -372,7 +374,8 @@ def main():
             "assign": {"ms": assign_ms, "tflops": a_tflops, "frac_of_measured_bf16_peak": a_tflops / peaks["bf16_tflops"],
                        "frac_of_nominal_2250": a_tflops / 2250.0},
             "update": {"ms": update_ms, "gbs": u_gbs, "frac_of_measured_hbm": u_gbs / peaks["hbm_gbs"],
-                       "frac_of_nominal_8000": u_gbs / 8000.0, "algorithmic_bytes": algorithmic_update_bytes(w)},
+                       "frac_of_nominal_8000": u_gbs / 8000.0, "algorithmic_bytes": algorithmic_update_bytes(w),
+                       "traffic": NCU_DRAM_BYTES_PER_UPDATE_LAUNCH.get(w.name)},
             "roofline": {"bound": "tensor", "kernel": "assign_tc_kernel (+ half-norm prologue)", "achieved": a_tflops,
                          "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst", "unit": "TFLOP/s",
                          "frac": a_tflops / peaks["bf16_tflops"], "traffic": None},

@@ -14,21 +14,24 @@
 // lose to every real one.  The epilogue therefore only has to find a row minimum; the N x K matrix
 // never exists outside tensor memory.
 //
-// One persistent CTA per SM, 16 warps (warp 11 idle), four roles:
+// One persistent CTA per SM, 16 warps, four roles:
 //   warp 8  producer : TMA.  A 128-row X tile (whole D) into one of the X buffers per row tile (up to
-//                      four row tiles ahead); per
-//                      centroid tile of 256 rows, D/64 chunks of 64 columns (128-byte swizzle) through
-//                      an mbarrier ring, plus the tile's 4 KiB block of split half-norms (bulk copy).
-//   warps 9,10 MMA   : one thread each issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32); issuer i
-//                      owns the i-th of two 256-column TMEM accumulators and every other centroid tile;
-//                      tcgen05.commit frees ring slots and publishes finished accumulators.
+//                      four row tiles ahead); per centroid tile of 256 rows, D/64 chunks of 64 columns
+//                      (128-byte swizzle) through an mbarrier ring, plus the tile's 4 KiB block of
+//                      split half-norms (bulk copy).
+//   warps 9-11 MMA   : one thread each issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32); centroid
+//                      tiles go round robin over the three (tile t: issuer t mod 3, accumulator t mod 2
+//                      of two 256-column TMEM accumulators); tcgen05.commit frees ring slots and
+//                      publishes finished accumulators.
 //   warps 0-7 epilogue: warp w reads TMEM lanes 32*(w%4).. (one X row per thread) and columns
 //                      128*(w/4).. of every tile with tcgen05.ld and keeps a running minimum per row.
 //                      The two column halves are merged through shared memory per row tile.
 //   warps 12-15 norms : one thread per X row forms ||x||^2/2 from the shared-memory X tile and writes
-//                      the X-side operand of the extra k-step, one row tile ahead of the MMA warp.
+//                      the X-side operand of the extra k-step, one row tile ahead of the MMA warps.
+// Barrier discipline: every mbarrier has waiters that see each of its phases, and whoever refills a
+// buffer waits for every reader of it (a parity wait that falls two phases behind never returns).
 // Two epilogue policies (both order by the fixed-point value, ties to the lowest index):
-//   packed : key = bits * 128 + column (one multiply-add on the FMA pipe) and a plain 3-input float
+//   packed : key = bits * 128 + column (one shift-and-add) and a plain 3-input float
 //            minimum over the keys finds value and position at once; no branch.
 //   exact  : minimum of the values; the position is looked up only when a 32-column group beats the
 //            running best (cheaper when there are many centroid tiles per row).

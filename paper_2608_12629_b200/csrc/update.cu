@@ -1,15 +1,20 @@
 // Centroid update: per-cluster sums and counts of the assigned points (paper Section 5,
 // "Flash-KMeans clean-start workload": centroid_update), then the division into means.
 //
-// Two routes produce sums[B][K][D] (fp32) and counts[B][K]:
+// Three routes produce sums[B][K][D] (fp32) and counts[B][K]:
+//   slab route : one kernel; every CTA counting-sorts its slab of rows by cluster in shared memory
+//                and reduces the slab in that order (thread-block clusters combine the histograms of
+//                2 or 4 CTAs over distributed shared memory when K is large against a slab).  The
+//                automatic choice while a slab holds several rows per cluster.
+//   sort route : global counting sort by cluster (histogram, exclusive scan, scatter of row numbers)
+//                and a segmented reduction in which each warp sums a fixed-size run of the sorted
+//                order in registers and adds one partial per cluster it touches.  Any K; for K <= 8192
+//                the sort works on per-slab shared-memory histograms and needs no global atomics.
 //   smem route : every CTA keeps a private K x D table of partial sums in shared memory, streams a
 //                slab of rows through it with shared-memory atomics and adds its table to the
-//                global one at the end.  For K*D*4 bytes that fit in one SM's shared memory.
-//   sort route : counting sort by cluster (histogram, exclusive scan, scatter of row numbers) and a
-//                segmented reduction in which each warp sums a fixed-size run of the sorted order
-//                in registers and adds one partial per cluster it touches.  Any K; for K <= 8192 the
-//                sort works on per-slab shared-memory histograms and needs no global atomics.
-// Both stream X exactly once with 16-byte (smem route: 4-byte) loads; HBM bandwidth is the bound.
+//                global one at the end.  For K*D*4 bytes that fit in one SM's shared memory; slow
+//                (shared-memory float atomics), on request only.
+// All stream X exactly once with 16-byte (smem route: 4-byte) loads; HBM bandwidth is the bound.
 #include <cooperative_groups.h>
 
 #include "internal.h"
