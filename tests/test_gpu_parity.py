@@ -220,6 +220,22 @@ def test_update_batched_unaligned_problem_size(flag):
                              inputs.to_bits(Cb[b]), counts[b].cpu().numpy())
 
 
+@pytest.mark.parametrize("D", [8, 64, 256])
+def test_update_many_clusters_few_rows_with_and_without_prev(D):
+    """K > 8192 with a few rows per cluster: the sort route hands every cluster to one warp, which writes
+    the centroid itself; most clusters are empty here and keep the previous centroid (or zeros)."""
+    N, K = 12000, 20000
+    X, C = problem(N, D, 64, seed=D)
+    g = torch.Generator().manual_seed(D)
+    idx = torch.randint(0, K, (N,), generator=g, dtype=torch.int32)
+    Cprev = inputs.from_bits(np.random.default_rng(D).integers(0x3C00, 0x4100, size=(K, D), dtype=np.uint16))
+    for prev in (Cprev, None):
+        Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=None if prev is None else prev.to(DEV),
+                                                 flags=cake.CAKE_UPDATE_SORT)
+        grading.grade_update(inputs.to_bits(X), idx.numpy(), K, None if prev is None else inputs.to_bits(prev),
+                             Cf.cpu().numpy(), inputs.to_bits(Cb), counts.cpu().numpy())
+
+
 def test_update_odd_feature_count_and_null_prev():
     N, D, K = 500, 7, 9
     X, _ = problem(N, D, K, seed=2)
