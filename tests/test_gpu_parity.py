@@ -453,6 +453,29 @@ def test_assign_many_row_tiles_few_centroid_tiles(N, D, K):
     assert int(idx.min()) >= 0 and int(idx.max()) < K and bool(torch.isfinite(dist).all())
 
 
+@pytest.mark.parametrize("N,D,K", [(1 << 21, 64, 64), (1 << 21, 128, 300), (1 << 20, 256, 600), (1 << 21, 96, 1000),
+                                   (1 << 20, 128, 1300)])
+def test_assign_repeatable_over_many_launches(N, D, K):
+    """The assign kernel has no data-dependent order (no atomics on its outputs): repeated launches must
+    return identical bits.  A role that gets ahead of a buffer it must not yet reuse (X tile, row
+    exponents, half-norm block, accumulator) shows up here as a difference or as a time-out."""
+    w = inputs.sweep_workload(N, D, K)
+    X, _ = inputs.gaussian_mixture(N, D, 1024, w.mean_std, w.sigma, w.seed, device=DEV)
+    C0 = inputs.sample_init(X, K, w.seed)
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    idx0, dist0 = cake.cake_kmeans_assign(X, C0, ws=ws)
+    idx0, dist0 = idx0.clone(), dist0.clone()
+    for _ in range(6):
+        idx, dist = cake.cake_kmeans_assign(X, C0, ws=ws)
+        torch.cuda.synchronize()
+        check_status(ws)
+        assert torch.equal(idx, idx0) and torch.equal(dist, dist0)
+    rows = sampled_rows(N, 1024, D)
+    rows_t = torch.from_numpy(rows).to(DEV)
+    grading.grade_assign(inputs.to_bits(X[rows_t].cpu()), inputs.to_bits(C0.cpu()), idx0[rows_t].cpu().numpy(),
+                         dist0[rows_t].cpu().numpy())
+
+
 # ------------------------------------------------------------------------------------ bounded waits
 
 def test_bounded_wait_expires_and_context_survives():
