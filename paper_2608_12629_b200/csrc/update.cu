@@ -105,14 +105,21 @@ update_smem_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
 //   sorted array : pairs[pos] = (row number, its cluster), pos in [0, n_valid)
 // K <= BLK_MAX_K ("blocked"): per-slab shared-memory histograms, no global atomics, no zero-fill
 // launches (hist_blocked zeroes `sums`, colscan writes `counts`).
-// Larger K: global atomics (few rows per cluster, little contention).
+// Larger K: global atomics (few rows per cluster, little contention); the histogram kernel zeroes `sums`.
 
 // ---- large-K pieces
 constexpr int HIST_THREADS = 512;
 
 __global__ void __launch_bounds__(HIST_THREADS)
-hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts, int* status) {
+hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts, float4* __restrict__ sums4,
+            i64 sums4_per_problem, int* status) {
     const int b = blockIdx.y;
+    // this CTA's share of the fp32 sums starts at zero (the loads below are in flight meanwhile)
+    {
+        const i64 z0 = sums4_per_problem * blockIdx.x / gridDim.x, z1 = sums4_per_problem * (blockIdx.x + 1) / gridDim.x;
+        float4* sb = sums4 + static_cast<size_t>(b) * sums4_per_problem;
+        for (i64 e = z0 + threadIdx.x; e < z1; e += blockDim.x) sb[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     const int* idx_b = idx + static_cast<size_t>(b) * N;
     int* counts_b = counts + static_cast<size_t>(b) * K;
     bool bad = false;
@@ -817,8 +824,9 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
     if (rc != CAKE_OK) return rc;
     const size_t kd = static_cast<size_t>(B) * K * D;
     const SortPlan pl = sort_plan(N, K);
+    const bool zero_in_hist = N > 0 && !pl.blocked && (static_cast<i64>(K) * D) % 4 == 0;
     if (N == 0 || !pl.blocked) {
-        if (cudaMemsetAsync(scr.sums, 0, kd * sizeof(float), s) != cudaSuccess) return CAKE_ERR_CUDA;
+        if (!zero_in_hist && cudaMemsetAsync(scr.sums, 0, kd * sizeof(float), s) != cudaSuccess) return CAKE_ERR_CUDA;
         if (cudaMemsetAsync(counts, 0, static_cast<size_t>(B) * K * sizeof(int), s) != cudaSuccess)
             return CAKE_ERR_CUDA;
     }
@@ -837,7 +845,9 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
             const i64 cap = (static_cast<i64>(di.sm_count) * 4 + B - 1) / B;
             if (ctas > cap) ctas = cap;
             if (ctas < 1) ctas = 1;
-            hist_kernel<<<dim3(static_cast<unsigned>(ctas), B), HIST_THREADS, 0, s>>>(idx, N, K, counts, status);
+            hist_kernel<<<dim3(static_cast<unsigned>(ctas), B), HIST_THREADS, 0, s>>>(
+                idx, N, K, counts, reinterpret_cast<float4*>(scr.sums),
+                zero_in_hist ? static_cast<i64>(K) * D / 4 : 0, status);
         }
         scan_kernel<<<dim3((K + SCAN_TILE - 1) / SCAN_TILE, B), 1024, 0, s>>>(counts, K, scr.cursor, scr.nvalid);
         {
