@@ -372,6 +372,7 @@ def main():
                        "step": "one Lloyd iteration = cake_kmeans_lloyd(iters=1)",
                        "x_checksum": inputs.checksum(X.view(-1)[: 1 << 20])},
             "assign": {"ms": assign_ms, "tflops": a_tflops, "frac_of_measured_bf16_peak": a_tflops / peaks["bf16_tflops"],
+                       "frac_of_measured_bf16_sustained": a_tflops / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
                        "frac_of_nominal_2250": a_tflops / 2250.0},
             "update": {"ms": update_ms, "gbs": u_gbs, "frac_of_measured_hbm": u_gbs / peaks["hbm_gbs"],
                        "frac_of_nominal_8000": u_gbs / 8000.0, "algorithmic_bytes": algorithmic_update_bytes(w),

@@ -11,7 +11,8 @@ constexpr size_t kAlign = 256;
 inline size_t up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Workspace {
-    int* status;          // [64] header, word 0 = sticky device status
+    int* status;          // [64] header, zeroed by the caller once: word 0 = sticky device status, word 1 =
+                          // ticket of the assign kernel, words 16..47 = max ||c||^2 of up to 32 problems
     void* caug;           // [B][Kpad/256][4 KiB] half-norm operand of the tensor-core assign
     int* cnmax;           // [B] max ||c||^2 per problem (fp32 bits)
     float* sums;          // [B][K][D]
@@ -63,11 +64,17 @@ int check_ws(void* ws, size_t ws_bytes, i64 B, i64 N, int D, int K, Workspace* o
 
 // inertia (nullable): inertia[b * inertia_stride] += sum of problem b's distances.  The tensor-core
 // kernel adds it up itself; the fallback needs `dist` (out_dist or scratch) and a reduction kernel.
+// zero_inertia: the entries still have to be cleared (the tensor-core prologue does it on the way).
 int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, int* out_idx,
-              float* out_dist, double* inertia, int inertia_stride, const Workspace& w, cudaStream_t s,
-              unsigned flags) {
+              float* out_dist, double* inertia, int inertia_stride, bool zero_inertia, const Workspace& w,
+              cudaStream_t s, unsigned flags) {
     unsigned path = flags & CAKE_ASSIGN_MASK;
     if (path == CAKE_ASSIGN_AUTO) path = assign_tc_supports(D) ? CAKE_ASSIGN_TCGEN05 : CAKE_ASSIGN_SIMT;
+    if (zero_inertia && inertia && (path == CAKE_ASSIGN_SIMT || N == 0)) {
+        if (cudaMemset2DAsync(inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
+                              static_cast<size_t>(B), s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
+    }
     if (path == CAKE_ASSIGN_SIMT) {
         float* dist = out_dist ? out_dist : (inertia ? w.dist : nullptr);
         int rc = launch_assign_simt(X, C, B, N, D, K, out_idx, dist, s);
@@ -81,7 +88,10 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
     // both epilogues order by the same fixed-point values; the packed one measured as fast or faster
     // at every shape tried, so it is the automatic choice and the other stays selectable
     const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT;
-    return launch_assign_tc(X, C, B, N, D, K, w.caug, w.cnmax, exact, out_idx, out_dist, inertia, inertia_stride, w.status, s);
+    // up to 32 problems keep max ||c||^2 in the header, which the kernel leaves zeroed: no memset per call
+    const bool in_header = B <= 32;
+    return launch_assign_tc(X, C, B, N, D, K, w.caug, in_header ? w.status + 16 : w.cnmax, in_header ? w.status + 1 : nullptr,
+                            exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia, w.status, s);
 }
 
 int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, const cake_bf16* C_prev,
@@ -161,7 +171,7 @@ int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, long long
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;
-    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, w,
+    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, false, w,
                      reinterpret_cast<cudaStream_t>(stream), flags);
 }
 
@@ -214,28 +224,30 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     const int Bi = static_cast<int>(B);
     const size_t kd = static_cast<size_t>(B) * K * D;
 
-    if (cudaMemcpyAsync(w.cbuf[0], C0, kd * 2, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return CAKE_ERR_CUDA;
-    if (out_inertia && iters > 0 &&
-        cudaMemsetAsync(out_inertia, 0, static_cast<size_t>(B) * iters * sizeof(double), s) != cudaSuccess)
-        return CAKE_ERR_CUDA;
-    int cur = 0;
     if (iters == 0) {
         // out_C = C0 widened: the division kernel with all-zero counts takes the keep-previous branch
         if (cudaMemsetAsync(w.cursor, 0, static_cast<size_t>(B) * K * 4, s) != cudaSuccess) return CAKE_ERR_CUDA;
-        if (launch_finalize(w.sums, w.cursor, w.cbuf[0], Bi, K, D, out_C, nullptr, false, s) != cudaSuccess)
+        if (launch_finalize(w.sums, w.cursor, C0, Bi, K, D, out_C, nullptr, false, s) != cudaSuccess)
             return CAKE_ERR_CUDA;
+        if (out_C_bf16 && cudaMemcpyAsync(out_C_bf16, C0, kd * 2, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
+        return CAKE_OK;
     }
+    // No copies: the first iteration reads C0 itself, the bf16 centroids ping-pong between the two
+    // workspace buffers and the last iteration writes the caller's buffer directly.  Each iteration's
+    // inertia entries are cleared by its own assign step.
+    const cake_bf16* cur = C0;
+    int nxt = 0;
     for (int t = 0; t < iters; ++t) {
-        rc = do_assign(X, w.cbuf[cur], Bi, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr,
-                       iters, w, s, flags);
+        rc = do_assign(X, cur, Bi, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr, iters,
+                       true, w, s, flags);
         if (rc != CAKE_OK) return rc;
-        rc = do_update(X, out_idx, Bi, N, D, K, w.cbuf[cur], out_C, w.cbuf[cur ^ 1], out_counts, w, s, flags);
+        cake_bf16* dst = (t == iters - 1 && out_C_bf16) ? out_C_bf16 : w.cbuf[nxt];
+        rc = do_update(X, out_idx, Bi, N, D, K, cur, out_C, dst, out_counts, w, s, flags);
         if (rc != CAKE_OK) return rc;
-        cur ^= 1;
+        cur = dst;
+        nxt ^= 1;
     }
-    if (out_C_bf16 &&
-        cudaMemcpyAsync(out_C_bf16, w.cbuf[cur], kd * 2, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
-        return CAKE_ERR_CUDA;
     return CAKE_OK;
 }
 

@@ -86,7 +86,8 @@ struct Params {
     int n_stages;     // ring depth
     int n_xbuf;       // 1 or 2 X buffers
     const uint8_t* caug;  // [B][n_tiles][4 KiB] centroid-side operand of the extra k-step
-    const int* cnmax;     // [B] bit pattern of max_k ||c_k||^2 (fp32, >= 0)
+    int* cnmax;           // [B] bit pattern of max_k ||c_k||^2 (fp32, >= 0)
+    int* ticket;          // optional: CTAs that have finished; the last one clears cnmax and the ticket
     int* out_idx;
     float* out_dist;
     double* inertia;      // optional: inertia[b * inertia_stride] += sum of the problem's distances
@@ -302,6 +303,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_base);
+    // everything above touched no global memory: it may overlap the prologue kernel's tail
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
 
     // The epilogue keeps a whole 128-column accumulator slice in registers; the other roles need few.
     // Registers move between warpgroups accordingly (warps 0-7 grow, warps 8-15 shrink).
@@ -691,6 +695,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, TMEM_COLS);
     }
+    // cnmax lives in memory that is zero between calls: the last CTA to get here (none reads cnmax any
+    // more) clears it for the next call
+    if (p.ticket && threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(p.ticket, 1) == static_cast<int>(gridDim.x) - 1) {
+            for (int b = 0; b < p.B; ++b) p.cnmax[b] = 0;
+            __threadfence();
+            *p.ticket = 0;
+        }
+    }
 }
 
 // Prologue: the centroid-side operand of the extra k-step.  One warp per padded centroid row k:
@@ -698,10 +712,17 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 // (columns 0..7 of the operand in the interleaved K-major layout the MMA reads: 256 rows x 16 B = 4 KiB
 // per tile; columns 8..15 are zeros the kernel supplies itself).  Rows k >= K are [1 1 1 0 0 0 1.5 1]:
 // their accumulator is 1.5 M + ... and can never win.  cnmax[b] collects max_k ||c_k||^2 (the bit
-// patterns of non-negative floats order like integers); it must be zero on entry.
+// patterns of non-negative floats order like integers); it must be zero on entry.  With `inertia` the
+// kernel also zeroes inertia[b * inertia_stride] for the B <= 256 problems (what the assign kernel adds to).
 __global__ void __launch_bounds__(256)
 centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64 total_rows,
-                    uint8_t* __restrict__ caug, int* __restrict__ cnmax) {
+                    uint8_t* __restrict__ caug, int* __restrict__ cnmax, double* __restrict__ inertia,
+                    int inertia_stride, int B) {
+    ptx::grid_dep_wait();      // C may come from the kernel ahead (the previous iteration's division)
+    ptx::grid_dep_launch();
+    // the assign kernel adds the distances up here: start from zero
+    if (inertia && blockIdx.x == 0 && static_cast<int>(threadIdx.x) < B)
+        inertia[static_cast<size_t>(threadIdx.x) * inertia_stride] = 0.0;
     const i64 w = (static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (w >= total_rows) return;
@@ -787,8 +808,8 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
 }
 
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
-                     int* cnmax, bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride,
-                     int* status, cudaStream_t s) {
+                     int* cnmax, int* ticket, bool exact, int* out_idx, float* out_dist, double* inertia,
+                     int inertia_stride, bool zero_inertia, int* status, cudaStream_t s) {
     if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
     DeviceInfo di;
     int rc = current_device_info(&di);
@@ -804,17 +825,41 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     p.total_tiles = static_cast<i64>(B) * p.m_tiles;
     p.caug = static_cast<const uint8_t*>(caug);
     p.cnmax = cnmax;
+    p.ticket = ticket;
     p.out_idx = out_idx; p.out_dist = out_dist; p.status = status;
     p.inertia = inertia; p.inertia_stride = inertia_stride;
     if (p.total_tiles == 0) return CAKE_OK;
 
     const int Kpad = padded_k(K);
+    // Every launch of a step may start while its predecessor drains (each kernel waits for the
+    // predecessor itself before it touches global memory).
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
     {
         const i64 rows = static_cast<i64>(B) * Kpad;
         const i64 ctas = (rows * 32 + 255) / 256;
-        if (cudaMemsetAsync(cnmax, 0, static_cast<size_t>(B) * sizeof(int), s) != cudaSuccess) return CAKE_ERR_CUDA;
-        centroid_aug_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(C, K, D, Kpad, rows,
-                                                                        static_cast<uint8_t*>(caug), cnmax);
+        // cnmax must start at zero: either it lives where the last CTA of the previous call cleared it
+        // (ticket), or it is cleared here
+        if (!ticket && cudaMemsetAsync(cnmax, 0, static_cast<size_t>(B) * sizeof(int), s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
+        if (zero_inertia && inertia && B > 256) {   // more problems than the prologue's first CTA has threads
+            if (cudaMemset2DAsync(inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
+                                  static_cast<size_t>(B), s) != cudaSuccess)
+                return CAKE_ERR_CUDA;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(ctas));
+        cfg.blockDim = dim3(256);
+        cfg.stream = s;
+        cfg.attrs = pdl;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, centroid_aug_kernel, C, K, D, Kpad, rows, static_cast<uint8_t*>(caug), cnmax,
+                               (zero_inertia && B <= 256) ? inertia : static_cast<double*>(nullptr), inertia_stride,
+                               B) != cudaSuccess) {
+            cudaGetLastError();
+            return CAKE_ERR_CUDA;
+        }
         note_launches(1);
     }
 
@@ -853,10 +898,21 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         attr_done_for_device = di.device;
     }
     const unsigned grid = static_cast<unsigned>(p.total_tiles < di.sm_count ? p.total_tiles : di.sm_count);
-    if (exact) assign_tc_kernel<false><<<grid, NUM_THREADS, smem_bytes, s>>>(tx, tc, p);
-    else assign_tc_kernel<true><<<grid, NUM_THREADS, smem_bytes, s>>>(tx, tc, p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = s;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    const cudaError_t e = exact ? cudaLaunchKernelEx(&cfg, assign_tc_kernel<false>, tx, tc, p)
+                                : cudaLaunchKernelEx(&cfg, assign_tc_kernel<true>, tx, tc, p);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return CAKE_ERR_CUDA;
+    }
     note_launches(1);
-    return cudaGetLastError() == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
+    return CAKE_OK;
 }
 
 }  // namespace cake

@@ -39,9 +39,12 @@ size_t assign_tc_aug_bytes(i64 B, int K);
 // prologue (half-norm operand into caug, max ||c||^2 into cnmax[B]) + the assign kernel; exact selects
 // the exact epilogue; inertia (nullable): inertia[b * inertia_stride] += sum_i dist[b][i], fp64, must
 // be zeroed by the caller
+// ticket (nullable): cnmax and *ticket lie in memory that is zero between calls (the kernel's last CTA
+// clears them again); without it cnmax is cleared by a memset.  zero_inertia: the prologue starts the
+// inertia entries from zero (otherwise the caller has).
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
-                     int* cnmax, bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride,
-                     int* status, cudaStream_t s);
+                     int* cnmax, int* ticket, bool exact, int* out_idx, float* out_dist, double* inertia,
+                     int inertia_stride, bool zero_inertia, int* status, cudaStream_t s);
 int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
                        int* out_idx, float* out_dist, cudaStream_t s);
 

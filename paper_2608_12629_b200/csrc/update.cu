@@ -513,6 +513,9 @@ constexpr int SLAB_MIN_RUN = 4;                            // rows per run below
 // sums and counts start at zero; the kernel behind it may begin at once (it waits before its first add)
 __global__ void __launch_bounds__(256)
 zero_sums_counts_kernel(float4* __restrict__ sums4, i64 n4, int* __restrict__ counts, i64 nc) {
+    // the kernel ahead (assign) may still read or write what this one clears, and the kernel behind (the
+    // slab sort) reads what the one ahead wrote: it may start only once this wait has returned
+    ptx::grid_dep_wait();
     ptx::grid_dep_launch();
     const i64 stride = static_cast<i64>(gridDim.x) * blockDim.x;
     const i64 t = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -710,6 +713,7 @@ finalize_kernel(const float* __restrict__ sums, const int* __restrict__ counts,
                 const cake_bf16* __restrict__ C_prev, i64 total, int D, float* __restrict__ out_C,
                 cake_bf16* __restrict__ out_C_bf16) {
     ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
     for (i64 e = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; e < total;
          e += static_cast<i64>(gridDim.x) * blockDim.x) {
         const i64 row = e / D;  // b*K + k
@@ -728,6 +732,7 @@ finalize4_kernel(const float4* __restrict__ sums, const int* __restrict__ counts
                  const uint2* __restrict__ C_prev, i64 total4, int D4, float4* __restrict__ out_C,
                  uint2* __restrict__ out_C_bf16) {
     ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
     for (i64 e = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; e < total4;
          e += static_cast<i64>(gridDim.x) * blockDim.x) {
         const int n = counts[e / D4];
@@ -997,9 +1002,20 @@ int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
         const i64 n4 = static_cast<i64>(B) * K * D / 4, nc = static_cast<i64>(B) * K;
         i64 ctas = (n4 + 256 * 4 - 1) / (256 * 4);
         if (ctas > di.sm_count * 4) ctas = di.sm_count * 4;
-        zero_sums_counts_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(reinterpret_cast<float4*>(sums), n4, counts, nc);
+        cudaLaunchAttribute zat[1];
+        zat[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        zat[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t zcfg = {};
+        zcfg.gridDim = dim3(static_cast<unsigned>(ctas));
+        zcfg.blockDim = dim3(256);
+        zcfg.stream = s;
+        zcfg.attrs = zat;
+        zcfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&zcfg, zero_sums_counts_kernel, reinterpret_cast<float4*>(sums), n4, counts, nc) != cudaSuccess) {
+            cudaGetLastError();
+            return CAKE_ERR_CUDA;
+        }
         note_launches(1);
-        if (cudaGetLastError() != cudaSuccess) return CAKE_ERR_CUDA;
     }
     if (N == 0) return CAKE_OK;
     SlabPlan pl;
