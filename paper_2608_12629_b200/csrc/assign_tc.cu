@@ -49,8 +49,9 @@ constexpr int KCHUNK = 64;              // bf16 columns per swizzled 128-byte ro
 constexpr int UMMA_K = 16;
 constexpr int NUM_EPI_WARPS = 8;
 constexpr int PRODUCER_WARP = 8;
-constexpr int MMA_WARP = 9;             // warps 9, 10 and 11: the MMA issuers
-constexpr int NUM_ISSUERS = 3;
+constexpr int MMA_WARP = 9;             // warps 9, 10 (and 11): the MMA issuers
+constexpr int MAX_ISSUERS = 3;
+constexpr int XLOAD_WARP = 11;          // or warp 11 loads the X tiles (then two issuers)
 constexpr int AUX_WARP0 = 12;           // warps 12..15: row norms
 constexpr int NUM_WARPS = 16;
 constexpr int EPI_REGS = 192;           // registers per thread after reallocation: epilogue warpgroups
@@ -101,7 +102,7 @@ struct Ctrl {  // lives in shared memory
     uint64_t tmem_full[2];
     // release of accumulator a, one barrier per issuer that may take it next: each barrier has a
     // single waiter that sees every one of its phases
-    uint64_t tmem_empty[2][NUM_ISSUERS];
+    uint64_t tmem_empty[2][MAX_ISSUERS];
     uint64_t auga_full[MAX_XBUF];
     uint64_t augb_full[N_AUGB], augb_empty[N_AUGB];
     uint64_t merge_full[2], merge_empty[2];
@@ -236,7 +237,9 @@ __device__ __forceinline__ void exact_scan32(const uint32_t (&r)[32], int col_ba
     }
 }
 
-template <bool PACKED>
+// XLOAD: warp 11 loads the X tiles and two warps issue MMAs (few centroid tiles per row tile);
+// otherwise the centroid producer also loads X and three warps issue MMAs.
+template <bool PACKED, bool XLOAD>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
                  const Params p) {
@@ -258,6 +261,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    constexpr int NUM_ISSUERS = XLOAD ? 2 : MAX_ISSUERS;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAX_XBUF; ++i) {
@@ -268,7 +272,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1);
-            for (int j = 0; j < NUM_ISSUERS; ++j)
+            for (int j = 0; j < MAX_ISSUERS; ++j)
                 ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i][j]), NUM_EPI_WARPS);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_full[i]), 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_empty[i]), 4);
@@ -340,8 +344,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             };
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 const int b = static_cast<int>(tile / p.m_tiles);
-                prefetch_x();
-                if (x_next <= tile) {   // this tile's own X is still outstanding: its buffer must free up
+                if (!XLOAD) prefetch_x();
+                if (!XLOAD && x_next <= tile) {   // this tile's own X is still outstanding: its buffer must free up
                     ok = wait_bar(&ctrl->x_empty[ixb], ixph ^ 1u, ctrl, p.status);
                     if (!ok) break;
                     issue_x();
@@ -349,7 +353,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const uint8_t* caug_b = p.caug + static_cast<size_t>(b) * p.n_tiles * AUG_B_BYTES;
                 for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it) {
                     for (int c = 0; c < p.nchunks; ++c, ++ring_it) {
-                        prefetch_x();
+                        if (!XLOAD) prefetch_x();
                         ok = wait_bar(&ctrl->ring_empty[rs], rph ^ 1u, ctrl, p.status);
                         if (!ok) break;
                         const uint32_t full = ptx::smem_u32(&ctrl->ring_full[rs]);
@@ -383,10 +387,39 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 }
             }
         }
+    } else if (XLOAD && warp == XLOAD_WARP) {
+        // ------------------------------------------------------------ X producer (few centroid tiles per row tile)
+        // A 128-row X tile per row tile, into the next X buffer the moment that buffer is free (up to
+        // n_xbuf row tiles ahead of the MMAs).  With one or two centroid tiles per row tile the kernel
+        // is as fast as X arrives, and behind the centroid stream's barriers in one thread it arrives
+        // late: here the X loads have a thread of their own, at the price of the third MMA issuer.
+        if (lane == 0) {
+            uint32_t ixb = 0, ixph = 0;
+            int tb = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
+            int tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
+            bool ok = true;
+            for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                ok = wait_bar(&ctrl->x_empty[ixb], ixph ^ 1u, ctrl, p.status);
+                if (!ok) break;
+                const uint32_t xfull = ptx::smem_u32(&ctrl->x_full[ixb]);
+                ptx::mbar_arrive_expect_tx(xfull, xbuf_bytes);
+                for (int c = 0; c < p.nchunks; ++c)
+                    ptx::tma_load_3d(x_base + ixb * xbuf_bytes + c * X_CHUNK_BYTES, &tmap_x, xfull,
+                                     c * KCHUNK, tmt * BLOCK_M, tb);
+                if (++ixb == static_cast<uint32_t>(p.n_xbuf)) { ixb = 0; ixph ^= 1u; }
+                tmt += static_cast<int>(gridDim.x);
+                while (tmt >= p.m_tiles) { tmt -= p.m_tiles; ++tb; }
+            }
+            if (!ok) {   // aborting: a bounded time for the X loads in flight to land
+                const uint64_t t0 = ptx::globaltimer_ns();
+                while (ptx::globaltimer_ns() - t0 < 20000ull) {
+                }
+            }
+        }
     } else if (warp >= MMA_WARP && warp < MMA_WARP + NUM_ISSUERS) {
         // ------------------------------------------------------------ MMA issuers
-        // Three warps, one issuing thread each; centroid tiles go round robin over them (tile t to
-        // issuer t mod 3, into accumulator t mod 2).  One thread cannot keep the tensor pipe fed: per
+        // Three warps (two when warp 11 loads X), one issuing thread each; centroid tiles go round robin
+        // over them (tile t to issuer t mod 3, into accumulator t mod 2).  One thread cannot keep the tensor pipe fed: per
         // tile it spends about three times the pipe's 9 x 128 clocks on its own instruction stream
         // (waits, descriptor arithmetic, commits, and MMA issue that blocks at the pipe's pace), so
         // three of them take turns.  No two ever hold the same accumulator or ring slot at a time.
@@ -401,7 +434,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             uint32_t s = 0, ph = 0;                         // ring position of the next chunk (all tiles)
             uint32_t xb = 0, xph = 0;                       // X buffer and its phase
             uint32_t acc_it = 0;
-            uint32_t turn = 0;                              // acc_it mod NUM_ISSUERS
+            constexpr uint32_t n_iss = NUM_ISSUERS;
+            uint32_t turn = 0;                              // acc_it mod n_iss
             uint32_t rel0 = 0, rel1 = 0;                    // releases of accumulator 0 / 1 this issuer has consumed
             bool ok = true;
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
@@ -413,7 +447,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const uint32_t a_lo_tile = ptx::umma_desc_lo_sw128(x_base + xb * xbuf_bytes);
                 const uint32_t auga_lo = ptx::umma_desc_lo_aug(smem_base + auga_off + xb * AUG_A_BYTES,
                                                                smem_base + zero_off);
-                for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it, turn = (turn + 1 == NUM_ISSUERS) ? 0 : turn + 1) {
+                for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it, turn = (turn + 1 == n_iss) ? 0 : turn + 1) {
                     if (turn != iss) {
                         // Another issuer's tile: pass over its ring slots, but see each of them filled
                         // and only then let the slot be refilled.  That keeps the issuers in tile order
@@ -547,7 +581,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int q = warp & 3;              // TMEM lane quarter this warp may read
         const int r = q * 32 + lane;         // row inside the X tile
         uint32_t tile_it = 0, acc_it = 0;
-        uint32_t next_iss = 2 % NUM_ISSUERS;   // (acc_it + 2) mod NUM_ISSUERS
+        constexpr uint32_t n_iss = NUM_ISSUERS;
+        uint32_t next_iss = 2 % n_iss;         // (acc_it + 2) mod n_iss
         uint32_t exb = 0, exph = 0;          // X buffer (slot of the row exponents) and its phase
         bool ok = true;
         double dsum = 0.0;                   // this thread's share of the current problem's inertia
@@ -611,7 +646,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 __syncwarp();
                 // to the issuer of tile acc_it + 2, which takes this accumulator next
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
-                next_iss = (next_iss + 1 == NUM_ISSUERS) ? 0 : next_iss + 1;
+                next_iss = (next_iss + 1 == n_iss) ? 0 : next_iss + 1;
                 trace_mark(ctrl, 100);
                 if (PACKED) {
                     float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF));
@@ -888,12 +923,17 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     rc = make_tmap(&tc, C, D, K, B, BLOCK_N);
     if (rc != CAKE_OK) return rc;
 
+    // one or two centroid tiles per row tile: the kernel is as fast as X arrives, X gets its own producer
+    const bool xload = p.n_tiles <= 2;
+    using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const Params);
+    Kernel kernel = exact ? (xload ? assign_tc_kernel<false, true> : assign_tc_kernel<false, false>)
+                          : (xload ? assign_tc_kernel<true, true> : assign_tc_kernel<true, false>);
     static int attr_done_for_device = -1;  // benign race: the attribute calls are idempotent
     if (attr_done_for_device != di.device) {
-        if (cudaFuncSetAttribute(assign_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 di.smem_optin) != cudaSuccess ||
-            cudaFuncSetAttribute(assign_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 di.smem_optin) != cudaSuccess)
+        if (cudaFuncSetAttribute(assign_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
             return CAKE_ERR_CUDA;
         attr_done_for_device = di.device;
     }
@@ -905,9 +945,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     cfg.stream = s;
     cfg.attrs = pdl;
     cfg.numAttrs = 1;
-    const cudaError_t e = exact ? cudaLaunchKernelEx(&cfg, assign_tc_kernel<false>, tx, tc, p)
-                                : cudaLaunchKernelEx(&cfg, assign_tc_kernel<true>, tx, tc, p);
-    if (e != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kernel, tx, tc, p) != cudaSuccess) {
         cudaGetLastError();
         return CAKE_ERR_CUDA;
     }
