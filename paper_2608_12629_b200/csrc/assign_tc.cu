@@ -23,6 +23,8 @@
 //                      tiles go round robin over the three (tile t: issuer t mod 3, accumulator t mod 2
 //                      of two 256-column TMEM accumulators); tcgen05.commit frees ring slots and
 //                      publishes finished accumulators.
+//                      With one or two centroid tiles per row tile a second instantiation makes
+//                      warp 11 a producer for the X tiles alone and keeps two issuers.
 //   warps 0-7 epilogue: warp w reads TMEM lanes 32*(w%4).. (one X row per thread) and columns
 //                      128*(w/4).. of every tile with tcgen05.ld and keeps a running minimum per row.
 //                      The two column halves are merged through shared memory per row tile.
