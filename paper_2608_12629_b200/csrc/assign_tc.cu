@@ -60,14 +60,15 @@ constexpr int EPI_REGS = 192;           // registers per thread after reallocati
 constexpr int AUX_REGS = 56;            // ... and the producer / MMA / norm warpgroups
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr uint32_t X_CHUNK_BYTES = BLOCK_M * 128;        // 16 KiB
-constexpr uint32_t C_STAGE_BYTES = BLOCK_N * 128;        // 32 KiB
+constexpr uint32_t C_CHUNK_BYTES = BLOCK_N * 128;        // 32 KiB: 256 centroid rows x 64 columns
 // Operands of the extra k-step: only columns 0..7 are non-zero, so each buffer holds just those
 // (one 16-byte row per X row / centroid) and every descriptor points its second 8-column core
 // matrices at one shared block of zeros.
 constexpr uint32_t AUG_A_BYTES = BLOCK_M * 16;           // 2 KiB
 constexpr uint32_t AUG_B_BYTES = kAssignAugTileBytes;    // 4 KiB
+// a ring stage: a centroid chunk plus room for the tile's half-norm block, which rides with the last chunk
+constexpr uint32_t C_STAGE_BYTES = C_CHUNK_BYTES + AUG_B_BYTES;
 constexpr uint32_t AUG_ZERO_BYTES = BLOCK_N * 16;        // 4 KiB of zeros
-constexpr int N_AUGB = 4;                                // centroid-side buffers in flight
 constexpr int MAX_STAGES = 6;
 constexpr int MAX_XBUF = 4;
 constexpr int TMEM_COLS = 512;
@@ -106,7 +107,6 @@ struct Ctrl {  // lives in shared memory
     // single waiter that sees every one of its phases
     uint64_t tmem_empty[2][MAX_ISSUERS];
     uint64_t auga_full[MAX_XBUF];
-    uint64_t augb_full[N_AUGB], augb_empty[N_AUGB];
     uint64_t merge_full[2], merge_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -256,8 +256,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t ring_off = static_cast<uint32_t>(p.n_xbuf) * xbuf_bytes;
     const uint32_t ring_base = smem_base + ring_off;
     const uint32_t auga_off = ring_off + static_cast<uint32_t>(p.n_stages) * C_STAGE_BYTES;
-    const uint32_t augb_off = auga_off + static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES;
-    const uint32_t zero_off = augb_off + N_AUGB * AUG_B_BYTES;
+    const uint32_t zero_off = auga_off + static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES;
     const uint32_t ctrl_off = zero_off + AUG_ZERO_BYTES;
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ctrl_off);
 
@@ -278,10 +277,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i][j]), NUM_EPI_WARPS);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_full[i]), 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_empty[i]), 4);
-        }
-        for (int i = 0; i < N_AUGB; ++i) {
-            ptx::mbar_init(ptx::smem_u32(&ctrl->augb_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->augb_empty[i]), 1);
         }
         for (int i = 0; i < MAX_STAGES; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_full[i]), 1);
@@ -359,19 +354,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         ok = wait_bar(&ctrl->ring_empty[rs], rph ^ 1u, ctrl, p.status);
                         if (!ok) break;
                         const uint32_t full = ptx::smem_u32(&ctrl->ring_full[rs]);
-                        ptx::mbar_arrive_expect_tx(full, C_STAGE_BYTES);
+                        const bool last = c == p.nchunks - 1;
+                        ptx::mbar_arrive_expect_tx(full, last ? C_STAGE_BYTES : C_CHUNK_BYTES);
                         ptx::tma_load_3d(ring_base + rs * C_STAGE_BYTES, &tmap_c, full, c * KCHUNK,
                                          nt * BLOCK_N, b);
+                        if (last)   // the tile's half-norm block rides with its last chunk
+                            ptx::bulk_load(ring_base + rs * C_STAGE_BYTES + C_CHUNK_BYTES,
+                                           caug_b + static_cast<size_t>(nt) * AUG_B_BYTES, AUG_B_BYTES, full);
                         if (++rs == static_cast<uint32_t>(p.n_stages)) { rs = 0; rph ^= 1u; }
                     }
                     if (!ok) break;
-                    const uint32_t ab = acc_it % N_AUGB, abph = (acc_it / N_AUGB) & 1u;
-                    ok = wait_bar(&ctrl->augb_empty[ab], abph ^ 1u, ctrl, p.status);
-                    if (!ok) break;
-                    const uint32_t bfull = ptx::smem_u32(&ctrl->augb_full[ab]);
-                    ptx::mbar_arrive_expect_tx(bfull, AUG_B_BYTES);
-                    ptx::bulk_load(smem_base + augb_off + ab * AUG_B_BYTES,
-                                   caug_b + static_cast<size_t>(nt) * AUG_B_BYTES, AUG_B_BYTES, bfull);
                 }
             }
             if (!ok) {
@@ -495,24 +487,22 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                 ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
                                                           b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main);
                         }
+                        if (c == p.nchunks - 1) {
+                            // the extra k-step: + ||x||^2/2 + ||c||^2/2 + M + m; its centroid side came with this chunk
+                            if (!have_aug) {
+                                ok = wait_bar(&ctrl->auga_full[xb], xph, ctrl, p.status);
+                                if (!ok) break;
+                                have_aug = true;
+                            }
+                            ptx::umma_bf16_lohi<true>(d_tmem, auga_lo, ptx::UMMA_DESC_HI_AUG,
+                                                      ptx::umma_desc_lo_aug(ring_base + s * C_STAGE_BYTES + C_CHUNK_BYTES,
+                                                                            smem_base + zero_off),
+                                                      ptx::UMMA_DESC_HI_AUG, idesc_aug);
+                        }
                         ptx::umma_commit(ptx::smem_u32(&ctrl->ring_empty[s]));
                         if (++s == nstg) { s = 0; ph ^= 1u; }
                     }
                     if (!ok) break;
-                    // the extra k-step: + ||x||^2/2 + ||c||^2/2
-                    if (!have_aug) {
-                        ok = wait_bar(&ctrl->auga_full[xb], xph, ctrl, p.status);
-                        if (!ok) break;
-                        have_aug = true;
-                    }
-                    const uint32_t ab = acc_it % N_AUGB, abph = (acc_it / N_AUGB) & 1u;
-                    ok = wait_bar(&ctrl->augb_full[ab], abph, ctrl, p.status);
-                    if (!ok) break;
-                    ptx::umma_bf16_lohi<true>(d_tmem, auga_lo, ptx::UMMA_DESC_HI_AUG,
-                                              ptx::umma_desc_lo_aug(smem_base + augb_off + ab * AUG_B_BYTES,
-                                                                    smem_base + zero_off),
-                                              ptx::UMMA_DESC_HI_AUG, idesc_aug);
-                    ptx::umma_commit(ptx::smem_u32(&ctrl->augb_empty[ab]));
                     ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[acc]));
                 }
                 if (ok && !have_aug) ok = wait_bar(&ctrl->auga_full[xb], xph, ctrl, p.status);
@@ -903,7 +893,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     // Shared memory: X buffers (each with its 4 KiB norm operand), the centroid ring, fixed parts.
     // Few centroid tiles per row tile make row tiles short, so X has to run further ahead: up to four
     // X buffers then, two otherwise; a single one only if the ring would drop below three stages.
-    const i64 fixed = 1024 + CTRL_BYTES + N_AUGB * AUG_B_BYTES + AUG_ZERO_BYTES;
+    const i64 fixed = 1024 + CTRL_BYTES + AUG_ZERO_BYTES;
     const i64 budget = static_cast<i64>(di.smem_optin) - fixed;
     const i64 xbuf = static_cast<i64>(p.nchunks) * X_CHUNK_BYTES + AUG_A_BYTES;
     int want_xbuf = p.n_tiles <= 2 ? MAX_XBUF : 2;
