@@ -20,6 +20,7 @@ struct Workspace {
     int* cursor;          // [B][K]
     int2* pairs;          // [B][N] (row, cluster) in cluster order
     int* part;            // [B][slabs][K] per-slab histograms of the sort route
+    int* done;            // [B][K] arrival counters of heavy clusters (sort route, K > 8192)
     cake_bf16* cbuf[2];   // [B][K][D] each
     float* dist;          // [B][N]
     size_t bytes;
@@ -39,6 +40,7 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     w.cursor = reinterpret_cast<int*>(take(static_cast<size_t>(B) * K * 4));
     w.pairs = reinterpret_cast<int2*>(take(static_cast<size_t>(B) * N * 8));
     w.part = reinterpret_cast<int*>(take(update_sort_part_bytes(B, N, K)));
+    w.done = reinterpret_cast<int*>(take(static_cast<size_t>(B) * K * 4));
     w.cbuf[0] = reinterpret_cast<cake_bf16*>(take(kd * 2));
     w.cbuf[1] = reinterpret_cast<cake_bf16*>(take(kd * 2));
     w.dist = reinterpret_cast<float*>(take(static_cast<size_t>(B) * N * 4));
@@ -101,6 +103,7 @@ int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, co
     int rc = current_device_info(&di);
     if (rc != CAKE_OK) return rc;
     unsigned path = flags & CAKE_UPDATE_MASK;
+    bool divided = false;
     if (path == CAKE_UPDATE_AUTO) {
         // the slab route while a slab holds several rows per cluster, else the global sort; the
         // shared-memory table never measured faster than either and is only taken on request
@@ -109,8 +112,8 @@ int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, co
     if (path == CAKE_UPDATE_SMEM) {
         rc = launch_update_smem(X, idx, B, N, D, K, w.sums, out_counts, w.status, s);
     } else if (path == CAKE_UPDATE_SORT) {
-        UpdateScratch scr{w.sums, w.nvalid, w.cursor, w.pairs, w.part};
-        rc = launch_update_sort(X, idx, B, N, D, K, scr, out_counts, w.status, s);
+        UpdateScratch scr{w.sums, w.nvalid, w.cursor, w.pairs, w.part, w.done};
+        rc = launch_update_sort(X, idx, B, N, D, K, scr, out_counts, C_prev, out_C, out_C_bf16, &divided, w.status, s);
     } else if (path == CAKE_UPDATE_SLAB || path == CAKE_UPDATE_SLAB_F1 || path == CAKE_UPDATE_SLAB_F2 ||
                path == CAKE_UPDATE_SLAB_F4) {
         const int force_f = path == CAKE_UPDATE_SLAB ? 0 : path == CAKE_UPDATE_SLAB_F1 ? 1 : path == CAKE_UPDATE_SLAB_F2 ? 2 : 4;
@@ -119,6 +122,7 @@ int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, co
         rc = CAKE_ERR_UNSUPPORTED;
     }
     if (rc != CAKE_OK) return rc;
+    if (divided) return CAKE_OK;
     const bool slab = path != CAKE_UPDATE_SMEM && path != CAKE_UPDATE_SORT;
     if (launch_finalize(w.sums, out_counts, C_prev, B, K, D, out_C, out_C_bf16, slab, s) != cudaSuccess)
         return CAKE_ERR_CUDA;

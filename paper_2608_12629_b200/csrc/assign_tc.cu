@@ -66,8 +66,8 @@ constexpr uint32_t C_CHUNK_BYTES = BLOCK_N * 128;        // 32 KiB: 256 centroid
 // matrices at one shared block of zeros.
 constexpr uint32_t AUG_A_BYTES = BLOCK_M * 16;           // 2 KiB
 constexpr uint32_t AUG_B_BYTES = kAssignAugTileBytes;    // 4 KiB
-// a ring stage: a centroid chunk plus room for the tile's half-norm block, which rides with the last chunk
-constexpr uint32_t C_STAGE_BYTES = C_CHUNK_BYTES + AUG_B_BYTES;
+// a ring stage: one or two centroid chunks plus room for the tile's half-norm block, which rides with the
+// last chunk (Params::cps, Params::stage_bytes)
 constexpr uint32_t AUG_ZERO_BYTES = BLOCK_N * 16;        // 4 KiB of zeros
 constexpr int MAX_STAGES = 6;
 constexpr int MAX_XBUF = 4;
@@ -87,7 +87,9 @@ struct Params {
     int m_tiles;      // ceil(N / 128)
     int n_tiles;      // ceil(K / 256)
     i64 total_tiles;  // B * m_tiles
-    int n_stages;     // ring depth
+    int n_stages;     // ring depth (stages)
+    int cps;          // centroid chunks per ring stage: 2 when nchunks is even (half the barrier traffic), else 1
+    uint32_t stage_bytes;   // cps * 32 KiB + 4 KiB
     int n_xbuf;       // 1 or 2 X buffers
     const uint8_t* caug;  // [B][n_tiles][4 KiB] centroid-side operand of the extra k-step
     int* cnmax;           // [B] bit pattern of max_k ||c_k||^2 (fp32, >= 0)
@@ -255,7 +257,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t x_base = smem_base;
     const uint32_t ring_off = static_cast<uint32_t>(p.n_xbuf) * xbuf_bytes;
     const uint32_t ring_base = smem_base + ring_off;
-    const uint32_t auga_off = ring_off + static_cast<uint32_t>(p.n_stages) * C_STAGE_BYTES;
+    const uint32_t auga_off = ring_off + static_cast<uint32_t>(p.n_stages) * p.stage_bytes;
     const uint32_t zero_off = auga_off + static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES;
     const uint32_t ctrl_off = zero_off + AUG_ZERO_BYTES;
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ctrl_off);
@@ -349,17 +351,18 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 }
                 const uint8_t* caug_b = p.caug + static_cast<size_t>(b) * p.n_tiles * AUG_B_BYTES;
                 for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it) {
-                    for (int c = 0; c < p.nchunks; ++c, ++ring_it) {
+                    for (int c = 0; c < p.nchunks; c += p.cps, ++ring_it) {
                         if (!XLOAD) prefetch_x();
                         ok = wait_bar(&ctrl->ring_empty[rs], rph ^ 1u, ctrl, p.status);
                         if (!ok) break;
                         const uint32_t full = ptx::smem_u32(&ctrl->ring_full[rs]);
-                        const bool last = c == p.nchunks - 1;
-                        ptx::mbar_arrive_expect_tx(full, last ? C_STAGE_BYTES : C_CHUNK_BYTES);
-                        ptx::tma_load_3d(ring_base + rs * C_STAGE_BYTES, &tmap_c, full, c * KCHUNK,
-                                         nt * BLOCK_N, b);
+                        const uint32_t stage = ring_base + rs * p.stage_bytes;
+                        const bool last = c + p.cps == p.nchunks;
+                        ptx::mbar_arrive_expect_tx(full, static_cast<uint32_t>(p.cps) * C_CHUNK_BYTES + (last ? AUG_B_BYTES : 0u));
+                        for (int j = 0; j < p.cps; ++j)
+                            ptx::tma_load_3d(stage + j * C_CHUNK_BYTES, &tmap_c, full, (c + j) * KCHUNK, nt * BLOCK_N, b);
                         if (last)   // the tile's half-norm block rides with its last chunk
-                            ptx::bulk_load(ring_base + rs * C_STAGE_BYTES + C_CHUNK_BYTES,
+                            ptx::bulk_load(stage + static_cast<uint32_t>(p.cps) * C_CHUNK_BYTES,
                                            caug_b + static_cast<size_t>(nt) * AUG_B_BYTES, AUG_B_BYTES, full);
                         if (++rs == static_cast<uint32_t>(p.n_stages)) { rs = 0; rph ^= 1u; }
                     }
@@ -447,7 +450,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         // and only then let the slot be refilled.  That keeps the issuers in tile order
                         // and this one at most one phase behind any slot (a parity wait that falls two
                         // phases behind waits for ever).
-                        for (int c = 0; ok && c < p.nchunks; ++c) {
+                        for (int c = 0; ok && c < p.nchunks; c += p.cps) {
                             ok = wait_bar(&ctrl->ring_full[s], ph, ctrl, p.status);
                             if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->ring_empty[s]));
                             if (++s == nstg) { s = 0; ph ^= 1u; }
@@ -466,36 +469,40 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     }
                     ptx::tc_fence_after();
                     uint32_t a_lo = a_lo_tile;
-                    for (int c = 0; c < p.nchunks; ++c, a_lo += X_CHUNK_BYTES >> 4) {
+                    for (int c0 = 0; c0 < p.nchunks; c0 += p.cps) {
                         ok = wait_bar(&ctrl->ring_full[s], ph, ctrl, p.status);
                         if (!ok) break;
-                        const uint32_t b_lo = ptx::umma_desc_lo_sw128(ring_base + s * C_STAGE_BYTES);
-                        const int nk = (c == p.nchunks - 1) ? p.ksteps_last : KCHUNK / UMMA_K;
-                        if (c == 0)
-                            ptx::umma_bf16_lohi<false>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
-                                                       ptx::UMMA_DESC_HI_SW128, idesc_main);
-                        else
-                            ptx::umma_bf16_lohi<true>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
-                                                      ptx::UMMA_DESC_HI_SW128, idesc_main);
-                        if (nk == KCHUNK / UMMA_K) {
+                        const uint32_t stage = ring_base + s * p.stage_bytes;
+                        for (int j = 0; j < p.cps; ++j, a_lo += X_CHUNK_BYTES >> 4) {
+                            const int c = c0 + j;
+                            const uint32_t b_lo = ptx::umma_desc_lo_sw128(stage + j * C_CHUNK_BYTES);
+                            const int nk = (c == p.nchunks - 1) ? p.ksteps_last : KCHUNK / UMMA_K;
+                            if (c == 0)
+                                ptx::umma_bf16_lohi<false>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
+                                                           ptx::UMMA_DESC_HI_SW128, idesc_main);
+                            else
+                                ptx::umma_bf16_lohi<true>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
+                                                          ptx::UMMA_DESC_HI_SW128, idesc_main);
+                            if (nk == KCHUNK / UMMA_K) {
 #pragma unroll
-                            for (uint32_t ks = 1; ks < KCHUNK / UMMA_K; ++ks)
-                                ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
-                                                          b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main);
-                        } else {
-                            for (int ks = 1; ks < nk; ++ks)
-                                ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
-                                                          b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main);
+                                for (uint32_t ks = 1; ks < KCHUNK / UMMA_K; ++ks)
+                                    ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
+                                                              b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main);
+                            } else {
+                                for (int ks = 1; ks < nk; ++ks)
+                                    ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
+                                                              b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main);
+                            }
                         }
-                        if (c == p.nchunks - 1) {
-                            // the extra k-step: + ||x||^2/2 + ||c||^2/2 + M + m; its centroid side came with this chunk
+                        if (c0 + p.cps == p.nchunks) {
+                            // the extra k-step: + ||x||^2/2 + ||c||^2/2 + M + m; its centroid side came with this stage
                             if (!have_aug) {
                                 ok = wait_bar(&ctrl->auga_full[xb], xph, ctrl, p.status);
                                 if (!ok) break;
                                 have_aug = true;
                             }
                             ptx::umma_bf16_lohi<true>(d_tmem, auga_lo, ptx::UMMA_DESC_HI_AUG,
-                                                      ptx::umma_desc_lo_aug(ring_base + s * C_STAGE_BYTES + C_CHUNK_BYTES,
+                                                      ptx::umma_desc_lo_aug(stage + static_cast<uint32_t>(p.cps) * C_CHUNK_BYTES,
                                                                             smem_base + zero_off),
                                                       ptx::UMMA_DESC_HI_AUG, idesc_aug);
                         }
@@ -898,16 +905,23 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     const i64 xbuf = static_cast<i64>(p.nchunks) * X_CHUNK_BYTES + AUG_A_BYTES;
     int want_xbuf = p.n_tiles <= 2 ? MAX_XBUF : 2;
     if (p.nchunks >= 4 && p.n_tiles >= 8) want_xbuf = 1;
-    const i64 min_stages = p.n_tiles <= 2 ? 2 : 3;
+    // two chunks per ring stage when the chunk count is even (one wait and one commit per stage), unless the
+    // ring would then hold a single stage or X is the bound (few centroid tiles: X buffers matter more)
     i64 stages = 0;
-    for (p.n_xbuf = want_xbuf; p.n_xbuf >= 1; --p.n_xbuf) {
-        stages = (budget - p.n_xbuf * xbuf) / C_STAGE_BYTES;
-        if (stages >= min_stages || p.n_xbuf == 1) break;
+    for (p.cps = (p.nchunks % 2 == 0 && p.n_tiles > 2) ? 2 : 1; p.cps >= 1; --p.cps) {
+        p.stage_bytes = static_cast<uint32_t>(p.cps) * C_CHUNK_BYTES + AUG_B_BYTES;
+        const int spt = p.nchunks / p.cps;                       // stages per centroid tile
+        const i64 min_stages = p.cps == 1 ? (p.n_tiles <= 2 ? 2 : 3) : (p.n_tiles <= 2 ? 2 : 2 * spt);
+        for (p.n_xbuf = want_xbuf; p.n_xbuf >= 1; --p.n_xbuf) {
+            stages = (budget - p.n_xbuf * xbuf) / p.stage_bytes;
+            if (stages >= min_stages || p.n_xbuf == 1) break;
+        }
+        if (stages >= 2) break;
     }
     if (stages < 2) return CAKE_ERR_UNSUPPORTED;
     p.n_stages = static_cast<int>(stages > MAX_STAGES ? MAX_STAGES : stages);
     const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf +
-                              static_cast<size_t>(p.n_stages) * C_STAGE_BYTES;
+                              static_cast<size_t>(p.n_stages) * p.stage_bytes;
 
     CUtensorMap tx, tc;
     rc = make_tmap(&tx, X, D, N, B, BLOCK_M);

@@ -55,14 +55,18 @@ struct UpdateScratch {
     int* cursor;      // [B][K]     next free position per cluster (sort path, K > 8192)
     int2* pairs;      // [B][N]     (row number, cluster) in cluster order (sort path)
     int* part;        // [B][slabs][K] per-slab histograms (sort path, K <= 8192)
+    int* done;        // [B][K]     rows of a heavy cluster already added to sums (sort path, K > 8192)
 };
 // bytes of the per-slab histogram scratch of the sort route (0 when it uses global atomics instead)
 size_t update_sort_part_bytes(i64 B, i64 N, int K);
 bool update_smem_supports(int D, int K, int smem_optin);
 int launch_update_smem(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, float* sums,
                        int* counts, int* status, cudaStream_t s);
+// *divided = true when the route wrote out_C / out_C_bf16 itself (means, keep-previous rule and all);
+// otherwise sums and counts are ready for launch_finalize.
 int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K,
-                       const UpdateScratch& scr, int* counts, int* status, cudaStream_t s);
+                       const UpdateScratch& scr, int* counts, const cake_bf16* C_prev, float* out_C,
+                       cake_bf16* out_C_bf16, bool* divided, int* status, cudaStream_t s);
 // slab route (one kernel sorts and reduces slab by slab): D % 8 == 0, D <= 256, K <= 8192.
 // force_f = 0 lets the launcher choose the thread-block cluster size, else 1, 2 or 4.
 bool update_slab_supports(int D, int K);

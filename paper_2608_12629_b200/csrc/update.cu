@@ -27,6 +27,12 @@ namespace {
 
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ cake_bf16 f32_to_bf16_rne(float f) {
+    uint32_t u = __float_as_uint(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<cake_bf16>((u >> 16) | 0x40u);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return static_cast<cake_bf16>(u >> 16);
+}
 
 // ======================================================================= smem route
 // Table layout per cluster: the D/2 even columns first, then the D/2 odd ones, so that the 32 lanes
@@ -136,11 +142,20 @@ hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts,
 // consecutive clusters; it first re-sums everything before its tile (coalesced, a few hundred KB at
 // most), so the tiles need no communication and one launch does the whole scan.
 constexpr int SCAN_TILE = 4096;
+// A cluster with more rows than this is "heavy": the per-cluster mean kernel splits it over every warp
+// whose window of the sorted order touches it (partials added into `sums`, the last one to arrive
+// divides); lighter clusters are summed by the single warp in whose window they start.
+constexpr int MEAN_HEAVY = 1024;
 
+// heavy_sums (nullable): the scan also clears the sums row and the arrival counter of every heavy cluster.
 __global__ void __launch_bounds__(1024)
-scan_kernel(const int* __restrict__ counts, int K, int* __restrict__ cursor, int* __restrict__ nvalid) {
+scan_kernel(const int* __restrict__ counts, int K, int* __restrict__ cursor, int* __restrict__ nvalid,
+            float* __restrict__ heavy_sums, int* __restrict__ heavy_done, int D) {
     __shared__ int warp_tot[32];
     __shared__ int pre_s;
+    __shared__ int heavy_n;
+    __shared__ int heavy_list[SCAN_TILE];
+    if (threadIdx.x == 0) heavy_n = 0;
     const int b = blockIdx.y, tile = blockIdx.x;
     const int* c = counts + static_cast<size_t>(b) * K;
     int* cur = cursor + static_cast<size_t>(b) * K;
@@ -191,6 +206,18 @@ scan_kernel(const int* __restrict__ counts, int K, int* __restrict__ cursor, int
         run += v[j];
     }
     if (tile == static_cast<int>(gridDim.x) - 1 && threadIdx.x == 0) nvalid[b] = pre + warp_tot[31];
+    if (heavy_sums) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (v[j] > MEAN_HEAVY) heavy_list[atomicAdd(&heavy_n, 1)] = k0 + j;
+        __syncthreads();
+        const int nh = heavy_n;
+        for (int h = 0; h < nh; ++h) {
+            const size_t bk = static_cast<size_t>(b) * K + heavy_list[h];
+            for (int d = threadIdx.x; d < D; d += 1024) heavy_sums[bk * D + d] = 0.f;
+            if (threadIdx.x == 0) heavy_done[bk] = 0;
+        }
+    }
 }
 
 // pos taken from the cluster's cursor; lanes of a warp that hit the same cluster take their slots
@@ -492,6 +519,313 @@ segreduce_scalar_kernel(const cake_bf16* __restrict__ X, const int2* __restrict_
     }
 }
 
+// ---- per-cluster means straight from the sorted order (K > 8192, D % 8 == 0): no partial sums in
+// memory, no separate division pass.  The sorted positions are cut into windows of SEG_ROWS, one per
+// warp (equal work whatever the cluster sizes).  A cluster belongs to the warp in whose window it
+// starts: that warp follows it to its end (counts[k] rows, past the window if need be), sums it in
+// registers, divides and writes the centroid.  Only a heavy cluster (more than MEAN_HEAVY rows) is
+// shared: every warp adds the part inside its own window to `sums` (cleared by the scan) and counts its
+// rows into `done`; the warp that completes the count divides.  Clusters without rows are dealt out
+// evenly over all warps by cluster number and keep their previous centroid.
+//
+// The rows a warp has to read form one stream of sorted positions, cut into passes (one warp-wide
+// load of 32/LPR rows) that never cross a run of equal clusters.  They are fetched with 16-byte
+// asynchronous copies into a ring of the warp's own in shared memory (every lane later reads back the
+// bytes it copied itself, so the copy groups of the thread are all the synchronisation there is; a
+// lane without a row gets zeros): the loads run MEAN_AHEAD-1 batches ahead of the additions whatever
+// the cluster boundaries, which keeps enough bytes in flight for random 2D-byte rows to arrive at the
+// full HBM rate with few registers.  Few warps per CTA: streams differ in length, and a CTA holds its
+// slots until its longest one ends.
+constexpr int MEAN_WARPS = 2;
+constexpr int MEAN_AHEAD = 3;          // batches in the ring (two in flight while one is added)
+constexpr int MEAN_BATCH_GRANULES = 4; // 16-byte granules per lane and batch
+// per warp: the ring (MEAN_AHEAD batches) and 128 row numbers
+constexpr int MEAN_WARP_UINT4 = MEAN_AHEAD * MEAN_BATCH_GRANULES * 32 + 32;
+
+// 16 bytes global -> shared, or 16 zero bytes when src_bytes == 0
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// two floats rounded to nearest-even bf16: lo in the low half, hi in the high half
+__device__ __forceinline__ uint32_t bf16x2_rn(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// two fp32 sums per instruction: acc.{lo,hi} += {bf16 in the low half, bf16 in the high half} of w
+__device__ __forceinline__ void add_bf16x2(unsigned long long& acc, uint32_t w) {
+    unsigned long long p;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "r"(w << 16), "r"(w & 0xFFFF0000u));
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(acc) : "l"(p));
+}
+
+template <int GPL, int LPR>   // granules per lane and row, lanes per row: D <= 8 * GPL * LPR
+__global__ void __launch_bounds__(MEAN_WARPS * 32)
+segmean_kernel(const cake_bf16* __restrict__ X, const int2* __restrict__ pairs, const int* __restrict__ nvalid,
+               const int* __restrict__ counts, i64 N, int D, int K, const cake_bf16* __restrict__ C_prev,
+               float* __restrict__ out_C, cake_bf16* __restrict__ out_C_bf16, float* sums, int* done) {
+    constexpr int RPP = 32 / LPR;                  // rows per pass
+    constexpr int U = MEAN_BATCH_GRANULES / GPL;   // passes per batch
+    constexpr int R = U * MEAN_AHEAD;              // passes in the ring
+    static_assert(U * RPP <= 32, "a batch must fit two blocks of the row table");
+    extern __shared__ uint4 mean_ring[];           // [warp]{[R][GPL][32] ring, 128 row numbers}
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const i64 w = static_cast<i64>(blockIdx.x) * MEAN_WARPS + warp;
+    const i64 n_warps = static_cast<i64>(gridDim.x) * MEAN_WARPS;
+    const int G = D >> 3;           // granules per row
+    const int sl = lane % LPR;      // granule slot inside the row
+    const int rs = lane / LPR;      // row slot
+    const int* counts_b = counts + static_cast<size_t>(b) * K;
+    const size_t row0 = static_cast<size_t>(b) * K;     // first centroid row of this problem
+    float4* out4 = reinterpret_cast<float4*>(out_C);
+    uint4* outb = reinterpret_cast<uint4*>(out_C_bf16);
+    bool gran_on[GPL];
+#pragma unroll
+    for (int g = 0; g < GPL; ++g) gran_on[g] = sl + g * LPR < G;
+
+    // lanes (rs == 0) hold eight consecutive columns of granule sl + g*LPR: the centroid row k
+    auto write_row = [&](int k, const float (&val)[GPL][8]) {
+        if (rs != 0) return;
+#pragma unroll
+        for (int g = 0; g < GPL; ++g) {
+            if (!gran_on[g]) continue;
+            const size_t e = (row0 + k) * G + sl + g * LPR;
+            out4[2 * e] = make_float4(val[g][0], val[g][1], val[g][2], val[g][3]);
+            out4[2 * e + 1] = make_float4(val[g][4], val[g][5], val[g][6], val[g][7]);
+            if (outb)
+                outb[e] = make_uint4(bf16x2_rn(val[g][0], val[g][1]), bf16x2_rn(val[g][2], val[g][3]),
+                                     bf16x2_rn(val[g][4], val[g][5]), bf16x2_rn(val[g][6], val[g][7]));
+        }
+    };
+
+    // 1. clusters without rows: the previous centroid (or zero)
+    for (i64 k = w; k < K; k += n_warps) {
+        if (__ldg(counts_b + k) != 0) continue;
+        float val[GPL][8];
+#pragma unroll
+        for (int g = 0; g < GPL; ++g) {
+            uint4 pv = make_uint4(0, 0, 0, 0);
+            if (C_prev && rs == 0 && gran_on[g])
+                pv = __ldg(reinterpret_cast<const uint4*>(C_prev) + (row0 + k) * G + sl + g * LPR);
+            val[g][0] = bf16lo(pv.x); val[g][1] = bf16hi(pv.x); val[g][2] = bf16lo(pv.y); val[g][3] = bf16hi(pv.y);
+            val[g][4] = bf16lo(pv.z); val[g][5] = bf16hi(pv.z); val[g][6] = bf16lo(pv.w); val[g][7] = bf16hi(pv.w);
+        }
+        write_row(static_cast<int>(k), val);
+    }
+
+    // 2. this warp's window of the sorted order
+    const int n_valid = nvalid[b];
+    const i64 p0 = w * SEG_ROWS;
+    if (p0 >= n_valid) return;
+    const int nwin = static_cast<int>((p0 + SEG_ROWS < n_valid) ? SEG_ROWS : n_valid - p0);
+    const int2* pairs_b = pairs + static_cast<size_t>(b) * N;
+    const uint4* Xg = reinterpret_cast<const uint4*>(X) + static_cast<size_t>(b) * N * G;
+    const bool in0 = lane < nwin, in1 = 32 + lane < nwin;
+    const int2 pk0 = in0 ? __ldg(pairs_b + p0 + lane) : make_int2(0, -1);
+    const int2 pk1 = in1 ? __ldg(pairs_b + p0 + 32 + lane) : make_int2(0, -1);
+    const int k_before = p0 > 0 ? __ldg(&pairs_b[p0 - 1].y) : -1;   // cluster of the position ahead of the window
+    const int ky0 = pk0.y, ky1 = pk1.y;
+    const int cn0 = in0 ? __ldg(counts_b + ky0) : 0, cn1 = in1 ? __ldg(counts_b + ky1) : 0;
+    auto key_at = [&](int o) { const int a = __shfl_sync(0xffffffffu, ky0, o & 31), c = __shfl_sync(0xffffffffu, ky1, o & 31); return o < 32 ? a : c; };
+    auto cnt_at = [&](int o) { const int a = __shfl_sync(0xffffffffu, cn0, o & 31), c = __shfl_sync(0xffffffffu, cn1, o & 31); return o < 32 ? a : c; };
+
+    // last[o]: position o closes a run of equal clusters inside the window (invalid positions carry -1)
+    uint64_t last;
+    {
+        int nx0 = __shfl_down_sync(0xffffffffu, ky0, 1);
+        const int first1 = __shfl_sync(0xffffffffu, ky1, 0);
+        if (lane == 31) nx0 = first1;
+        int nx1 = __shfl_down_sync(0xffffffffu, ky1, 1);
+        if (lane == 31) nx1 = -2;
+        const uint32_t l0 = __ballot_sync(0xffffffffu, in0 && nx0 != ky0), l1 = __ballot_sync(0xffffffffu, in1 && nx1 != ky1);
+        last = (static_cast<uint64_t>(l1) << 32) | l0;
+    }
+    // the stream: everything in the window but a leading piece of a light cluster that started earlier,
+    // plus what the last cluster (if light and started here) has beyond the window
+    const int k_first = key_at(0), n_first = cnt_at(0);
+    int ps = 0;
+    if (k_first == k_before && n_first <= MEAN_HEAVY) ps = __ffsll(static_cast<long long>(last));   // end of the first run
+    if (ps >= nwin) return;
+    const int k_last = key_at(nwin - 1), n_last = cnt_at(nwin - 1);
+    int ext = 0;
+    {
+        const uint64_t inner = last & ~(1ull << (nwin - 1));
+        const int so = inner ? 64 - __clzll(static_cast<long long>(inner)) : 0;   // where the last run starts
+        if (n_last <= MEAN_HEAVY && n_last > nwin - so) {
+            ext = n_last - (nwin - so);      // then nwin == SEG_ROWS: the order goes on past the window
+            last &= ~(1ull << (nwin - 1));
+        }
+    }
+    const int S = nwin - ps + ext;                  // stream length
+    // end (exclusive, as a stream index) of the run that holds stream index i
+    auto run_end = [&](int i) {
+        const int o = ps + i;
+        if (o < SEG_ROWS) {
+            const uint64_t m = last >> o;
+            if (m) return i + __ffsll(static_cast<long long>(m));
+        }
+        return S;
+    };
+
+    // per warp: the ring, then a table of 128 row numbers indexed by position modulo 128 (the window's 64
+    // first; blocks of 32 past the window replace entries the issuing side has long passed)
+    uint4* ring = mean_ring + static_cast<size_t>(warp) * MEAN_WARP_UINT4;
+    int* tab = reinterpret_cast<int*>(ring + R * GPL * 32);
+    const uint32_t ring_a = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + lane * 16;
+    tab[lane] = pk0.x;
+    tab[32 + lane] = pk1.x;
+    int ext_loaded = 0;    // blocks of 32 positions past the window already in the table
+    int ext_next = -1;     // this lane's row number of the block after those (fetched one block early)
+    if (ext > 0) ext_next = lane < ext ? __ldg(&pairs_b[p0 + SEG_ROWS + lane].x) : 0;
+    __syncwarp();
+
+    const char* Xlane[GPL];     // this lane's granules of row 0
+#pragma unroll
+    for (int g = 0; g < GPL; ++g) Xlane[g] = reinterpret_cast<const char*>(Xg + (gran_on[g] ? sl + g * LPR : 0));
+    const uint32_t row_bytes = static_cast<uint32_t>(D) * 2u;
+
+    int iq = 0, ie = run_end(0);          // issuing side: next position, end of its run
+    uint32_t wr = ring_a;                 // where the next pass lands
+    auto issue_batch = [&]() {
+        // make sure the table covers the batch
+        while (ps + iq + U * RPP > SEG_ROWS + 32 * ext_loaded && 32 * ext_loaded < ext) {
+            tab[((2 + ext_loaded) & 3) * 32 + lane] = ext_next;
+            ++ext_loaded;
+            const int e = 32 * ext_loaded + lane;
+            ext_next = e < ext ? __ldg(&pairs_b[p0 + SEG_ROWS + e].x) : 0;
+            __syncwarp();
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            // a lane without a row (past the run, past the stream, past the row's granules) gets zeros
+            const int pos = iq + rs;
+            const bool on = pos < ie;
+            const uint32_t row = static_cast<uint32_t>(tab[(ps + pos) & 127]);
+            const uint64_t off = static_cast<uint64_t>(row) * row_bytes;
+#pragma unroll
+            for (int g = 0; g < GPL; ++g)
+                cp_async16(wr + (u * GPL + g) * 512, Xlane[g] + off, on && gran_on[g] ? 16u : 0u);
+            iq += RPP;
+            if (iq >= ie) { iq = ie; ie = run_end(iq); }
+        }
+        wr += U * GPL * 512;
+        if (wr == ring_a + R * GPL * 512) wr = ring_a;
+    };
+
+#pragma unroll
+    for (int bt = 0; bt < MEAN_AHEAD - 1; ++bt) {
+        issue_batch();
+        cp_async_commit();
+    }
+
+    unsigned long long acc[GPL][4];   // four pairs of fp32 sums per granule
+#pragma unroll
+    for (int g = 0; g < GPL; ++g)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[g][j] = 0ull;
+
+    // the run that ends at stream index i_close is complete (`piece` of its rows were read here): divide
+    // and write, or (heavy) add the partial and count it
+    auto flush = [&](int i_close, int piece) {
+        const int o = ps + i_close;
+        int k = key_at(o < nwin ? o : 0), n = cnt_at(o < nwin ? o : 0);
+        if (o >= nwin) { k = k_last; n = n_last; }
+        float val[GPL][8];
+#pragma unroll
+        for (int g = 0; g < GPL; ++g)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                asm("mov.b64 {%0, %1}, %2;" : "=f"(val[g][2 * j]), "=f"(val[g][2 * j + 1]) : "l"(acc[g][j]));
+                acc[g][j] = 0ull;
+            }
+#pragma unroll
+        for (int g = 0; g < GPL; ++g)
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int x = LPR; x < 32; x <<= 1) val[g][j] += __shfl_xor_sync(0xffffffffu, val[g][j], x);
+        const float fn = static_cast<float>(n);
+        if (n <= MEAN_HEAVY) {
+            const float inv = 1.0f / fn;     // one division per cluster; the products are within 1 ulp of sum / n
+#pragma unroll
+            for (int g = 0; g < GPL; ++g)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) val[g][j] *= inv;
+            write_row(k, val);
+        } else {
+            float* srow = sums + (row0 + k) * static_cast<size_t>(D);
+            if (rs == 0) {
+#pragma unroll
+                for (int g = 0; g < GPL; ++g) {
+                    if (!gran_on[g]) continue;
+                    float4* dst = reinterpret_cast<float4*>(srow + (sl + g * LPR) * 8);
+                    atomicAdd(dst, make_float4(val[g][0], val[g][1], val[g][2], val[g][3]));
+                    atomicAdd(dst + 1, make_float4(val[g][4], val[g][5], val[g][6], val[g][7]));
+                }
+            }
+            __threadfence();
+            __syncwarp();
+            int arrived = 0;
+            if (lane == 0) arrived = atomicAdd(done + row0 + k, piece) + piece;
+            arrived = __shfl_sync(0xffffffffu, arrived, 0);
+            if (arrived == n) {   // every part is in: divide
+                __threadfence();
+#pragma unroll
+                for (int g = 0; g < GPL; ++g) {
+                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), c = a;
+                    if (rs == 0 && gran_on[g]) {
+                        a = __ldcg(reinterpret_cast<const float4*>(srow + (sl + g * LPR) * 8));
+                        c = __ldcg(reinterpret_cast<const float4*>(srow + (sl + g * LPR) * 8) + 1);
+                    }
+                    val[g][0] = a.x / fn; val[g][1] = a.y / fn; val[g][2] = a.z / fn; val[g][3] = a.w / fn;
+                    val[g][4] = c.x / fn; val[g][5] = c.y / fn; val[g][6] = c.z / fn; val[g][7] = c.w / fn;
+                }
+                write_row(k, val);
+            }
+        }
+    };
+
+    int cq = 0, ce = run_end(0), run_start = 0;   // adding side: next position, end and start of its run
+    const uint4* rd = ring + lane;
+    int left = 0;                                 // passes of the current batch not yet added
+    while (cq < S) {
+        if (left == 0) {
+            // keep the ring full, then wait for the next batch (all but the newest MEAN_AHEAD-1 groups)
+            issue_batch();
+            cp_async_commit();
+            cp_async_wait<MEAN_AHEAD - 1>();
+            left = U;
+            if (rd == ring + lane + R * GPL * 32) rd = ring + lane;
+        }
+        // passes until the run or the batch ends
+        int np = (ce - cq + RPP - 1) / RPP;
+        if (np > left) np = left;
+        left -= np;
+        cq += np * RPP;
+        for (; np > 0; --np) {
+#pragma unroll
+            for (int g = 0; g < GPL; ++g) {
+                const uint4 v = rd[g * 32];
+                add_bf16x2(acc[g][0], v.x); add_bf16x2(acc[g][1], v.y);
+                add_bf16x2(acc[g][2], v.z); add_bf16x2(acc[g][3], v.w);
+            }
+            rd += GPL * 32;
+        }
+        if (cq >= ce) {
+            flush(ce - 1, ce - run_start);
+            cq = ce;
+            run_start = ce;
+            ce = run_end(cq);
+        }
+    }
+    cp_async_wait<0>();
+}
+
 // ======================================================================= slab route
 // One kernel sorts and reduces.  A CTA owns a slab of S consecutive rows: it keeps their cluster ids
 // in registers, ranks every row inside its cluster with one shared-memory atomic, scans the
@@ -701,12 +1035,6 @@ slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
 }
 
 // ======================================================================= division
-__device__ __forceinline__ cake_bf16 f32_to_bf16_rne(float f) {
-    uint32_t u = __float_as_uint(f);
-    if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<cake_bf16>((u >> 16) | 0x40u);
-    u += 0x7fffu + ((u >> 16) & 1u);
-    return static_cast<cake_bf16>(u >> 16);
-}
 
 __global__ void __launch_bounds__(256)
 finalize_kernel(const float* __restrict__ sums, const int* __restrict__ counts,
@@ -823,15 +1151,20 @@ size_t update_sort_part_bytes(i64 B, i64 N, int K) {
 }
 
 int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K,
-                       const UpdateScratch& scr, int* counts, int* status, cudaStream_t s) {
+                       const UpdateScratch& scr, int* counts, const cake_bf16* C_prev, float* out_C,
+                       cake_bf16* out_C_bf16, bool* divided, int* status, cudaStream_t s) {
     DeviceInfo di;
     int rc = current_device_info(&di);
     if (rc != CAKE_OK) return rc;
+    *divided = false;
     const size_t kd = static_cast<size_t>(B) * K * D;
     const SortPlan pl = sort_plan(N, K);
-    const bool zero_in_hist = N > 0 && !pl.blocked && (static_cast<i64>(K) * D) % 4 == 0;
+    // large K, rows of whole 16-byte granules: the last kernel writes the means itself (no partial sums)
+    const bool means = N > 0 && !pl.blocked && D % 8 == 0 && D >= 24 && D <= 1024;
+    const bool zero_in_hist = N > 0 && !pl.blocked && !means && (static_cast<i64>(K) * D) % 4 == 0;
     if (N == 0 || !pl.blocked) {
-        if (!zero_in_hist && cudaMemsetAsync(scr.sums, 0, kd * sizeof(float), s) != cudaSuccess) return CAKE_ERR_CUDA;
+        if (!means && !zero_in_hist && cudaMemsetAsync(scr.sums, 0, kd * sizeof(float), s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
         if (cudaMemsetAsync(counts, 0, static_cast<size_t>(B) * K * sizeof(int), s) != cudaSuccess)
             return CAKE_ERR_CUDA;
     }
@@ -854,7 +1187,8 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
                 idx, N, K, counts, reinterpret_cast<float4*>(scr.sums),
                 zero_in_hist ? static_cast<i64>(K) * D / 4 : 0, status);
         }
-        scan_kernel<<<dim3((K + SCAN_TILE - 1) / SCAN_TILE, B), 1024, 0, s>>>(counts, K, scr.cursor, scr.nvalid);
+        scan_kernel<<<dim3((K + SCAN_TILE - 1) / SCAN_TILE, B), 1024, 0, s>>>(
+            counts, K, scr.cursor, scr.nvalid, means ? scr.sums : nullptr, scr.done, D);
         {
             i64 ctas = (N + 256 * 4 - 1) / (256 * 4);
             const i64 cap = (static_cast<i64>(di.sm_count) * 8 + B - 1) / B;
@@ -863,7 +1197,26 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
             scatter_kernel<<<dim3(static_cast<unsigned>(ctas), B), 256, 0, s>>>(idx, N, K, scr.cursor, scr.pairs);
         }
     }
-    {
+    if (means) {
+        // one warp per window of the sorted order, and enough warps to deal out the empty clusters
+        i64 warps = (N + SEG_ROWS - 1) / SEG_ROWS;
+        if (warps < K / 4) warps = K / 4;
+        dim3 grid(static_cast<unsigned>((warps + MEAN_WARPS - 1) / MEAN_WARPS), B);
+        const int G = D / 8;
+        int lpr = 4;
+        while (lpr < G && lpr < 32) lpr <<= 1;
+        const int gpl = (G + lpr - 1) / lpr;
+        // per warp: MEAN_AHEAD batches of MEAN_BATCH_GRANULES granules per lane (6 KiB) and the row table
+        const size_t mean_smem = static_cast<size_t>(MEAN_WARPS) * MEAN_WARP_UINT4 * sizeof(uint4);
+        using MeanKernel = void (*)(const cake_bf16*, const int2*, const int*, const int*, i64, int, int,
+                                    const cake_bf16*, float*, cake_bf16*, float*, int*);
+        MeanKernel kernel = gpl == 4 ? segmean_kernel<4, 32> : gpl == 2 ? segmean_kernel<2, 32>
+                          : lpr == 32 ? segmean_kernel<1, 32> : lpr == 16 ? segmean_kernel<1, 16>
+                          : lpr == 8 ? segmean_kernel<1, 8> : segmean_kernel<1, 4>;
+        kernel<<<grid, MEAN_WARPS * 32, mean_smem, s>>>(X, scr.pairs, scr.nvalid, counts, N, D, K, C_prev, out_C,
+                                                       out_C_bf16, scr.sums, scr.done);
+        *divided = true;
+    } else {
         const i64 warps = (N + SEG_ROWS - 1) / SEG_ROWS;
         const unsigned ctas = static_cast<unsigned>((warps + SEG_WARPS - 1) / SEG_WARPS);
         dim3 grid(ctas, B);

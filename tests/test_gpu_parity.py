@@ -236,6 +236,36 @@ def test_update_many_clusters_few_rows_with_and_without_prev(D):
                              Cf.cpu().numpy(), inputs.to_bits(Cb), counts.cpu().numpy())
 
 
+@pytest.mark.parametrize("D", [8, 24, 128, 256, 512, 1024])
+def test_update_many_clusters_skewed_sizes(D):
+    """K > 8192 with cluster sizes from 0 to several thousand rows: clusters that cross the 64-row windows
+    of the sorted order, heavy clusters shared by many warps (partials + arrival count), runs of empty
+    clusters at both ends, a few invalid indices, two problems."""
+    B, N, K = 2, 40000, 9000 + D
+    g = torch.Generator().manual_seed(100 + D)
+    X = inputs.from_bits(np.random.default_rng(D).integers(0x3C00, 0x4100, size=(B, N, D), dtype=np.uint16))
+    idx = torch.randint(500, K - 700, (B, N), generator=g, dtype=torch.int32)
+    idx[0, :6000] = 777                  # heavy
+    idx[0, 6000:7500] = K - 701          # heavy, the last cluster with rows
+    idx[0, 7500:7700] = 778              # crosses windows, light
+    idx[1, 1000:3100] = 500              # heavy, the first cluster with rows
+    idx[1, 5000:5065] = 6000
+    idx[1, 7] = -1
+    idx[1, 9] = K
+    perm = torch.randperm(N, generator=g)
+    idx = idx[:, perm].contiguous()
+    Cprev = inputs.from_bits(np.random.default_rng(D + 1).integers(0x3C00, 0x4100, size=(B, K, D), dtype=np.uint16))
+    ws = cake.alloc_workspace(B, N, D, K, DEV)
+    for _ in range(2):                  # twice: the arrival counters must start from zero every time
+        Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=Cprev.to(DEV), ws=ws,
+                                                 flags=cake.CAKE_UPDATE_SORT)
+        check_status(ws, cake.CAKE_ERR_BAD_INDEX)
+        for b in range(B):
+            keep = ((idx[b] >= 0) & (idx[b] < K)).numpy()
+            grading.grade_update(inputs.to_bits(X[b])[keep], idx[b].numpy()[keep], K, inputs.to_bits(Cprev[b]),
+                                 Cf[b].cpu().numpy(), inputs.to_bits(Cb[b]), counts[b].cpu().numpy())
+
+
 def test_update_odd_feature_count_and_null_prev():
     N, D, K = 500, 7, 9
     X, _ = problem(N, D, K, seed=2)
