@@ -21,6 +21,7 @@ struct Workspace {
     int2* pairs;          // [B][N] (row, cluster) in cluster order
     int* part;            // [B][slabs][K] per-slab histograms of the sort route
     int* done;            // [B][K] arrival counters of heavy clusters (sort route, K > 8192)
+    int* rank;            // [B][N] rank of every row inside its cluster (sort route, K > 8192)
     cake_bf16* cbuf[2];   // [B][K][D] each
     float* dist;          // [B][N]
     size_t bytes;
@@ -41,6 +42,7 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     w.pairs = reinterpret_cast<int2*>(take(static_cast<size_t>(B) * N * 8));
     w.part = reinterpret_cast<int*>(take(update_sort_part_bytes(B, N, K)));
     w.done = reinterpret_cast<int*>(take(static_cast<size_t>(B) * K * 4));
+    w.rank = reinterpret_cast<int*>(take(update_sort_rank_bytes(B, N, K)));
     w.cbuf[0] = reinterpret_cast<cake_bf16*>(take(kd * 2));
     w.cbuf[1] = reinterpret_cast<cake_bf16*>(take(kd * 2));
     w.dist = reinterpret_cast<float*>(take(static_cast<size_t>(B) * N * 4));
@@ -112,7 +114,7 @@ int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, co
     if (path == CAKE_UPDATE_SMEM) {
         rc = launch_update_smem(X, idx, B, N, D, K, w.sums, out_counts, w.status, s);
     } else if (path == CAKE_UPDATE_SORT) {
-        UpdateScratch scr{w.sums, w.nvalid, w.cursor, w.pairs, w.part, w.done};
+        UpdateScratch scr{w.sums, w.nvalid, w.cursor, w.pairs, w.part, w.done, w.rank};
         rc = launch_update_sort(X, idx, B, N, D, K, scr, out_counts, C_prev, out_C, out_C_bf16, &divided, w.status, s);
     } else if (path == CAKE_UPDATE_SLAB || path == CAKE_UPDATE_SLAB_F1 || path == CAKE_UPDATE_SLAB_F2 ||
                path == CAKE_UPDATE_SLAB_F4) {

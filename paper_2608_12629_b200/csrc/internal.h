@@ -52,13 +52,16 @@ int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int
 struct UpdateScratch {
     float* sums;      // [B][K][D]
     int* nvalid;      // [B]        rows with a valid index (sort path)
-    int* cursor;      // [B][K]     next free position per cluster (sort path, K > 8192)
+    int* cursor;      // [B][K]     first sorted position of every cluster (sort path, K > 8192)
     int2* pairs;      // [B][N]     (row number, cluster) in cluster order (sort path)
     int* part;        // [B][slabs][K] per-slab histograms (sort path, K <= 8192)
     int* done;        // [B][K]     rows of a heavy cluster already added to sums (sort path, K > 8192)
+    int* rank;        // [B][N]     rank of every row inside its cluster (sort path, K > 8192)
 };
 // bytes of the per-slab histogram scratch of the sort route (0 when it uses global atomics instead)
 size_t update_sort_part_bytes(i64 B, i64 N, int K);
+// bytes of the per-row rank scratch of the sort route (0 when it sorts slab by slab in shared memory)
+size_t update_sort_rank_bytes(i64 B, i64 N, int K);
 bool update_smem_supports(int D, int K, int smem_optin);
 int launch_update_smem(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, float* sums,
                        int* counts, int* status, cudaStream_t s);

@@ -116,9 +116,14 @@ update_smem_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
 // ---- large-K pieces
 constexpr int HIST_THREADS = 512;
 
+// counts[b][k] += 1 per row, and rank[b][i] = how many rows of the same cluster were counted before
+// row i (-1 for an index outside [0, K)): the scatter then needs no second round of atomics.  Lanes of
+// a warp that hit the same cluster take their ranks with a single atomic.
+constexpr int HIST_PER_THREAD = 4;
+
 __global__ void __launch_bounds__(HIST_THREADS)
-hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts, float4* __restrict__ sums4,
-            i64 sums4_per_problem, int* status) {
+hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts, int* __restrict__ rank,
+            float4* __restrict__ sums4, i64 sums4_per_problem, int* status) {
     const int b = blockIdx.y;
     // this CTA's share of the fp32 sums starts at zero (the loads below are in flight meanwhile)
     {
@@ -127,13 +132,36 @@ hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts,
         for (i64 e = z0 + threadIdx.x; e < z1; e += blockDim.x) sb[e] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     const int* idx_b = idx + static_cast<size_t>(b) * N;
+    int* rank_b = rank + static_cast<size_t>(b) * N;
     int* counts_b = counts + static_cast<size_t>(b) * K;
+    const int lane = threadIdx.x & 31;
     bool bad = false;
-    for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < N;
-         i += static_cast<i64>(gridDim.x) * blockDim.x) {
-        const int k = idx_b[i];
-        if (k < 0 || k >= K) { bad = true; continue; }
-        atomicAdd(counts_b + k, 1);
+    const i64 span = static_cast<i64>(gridDim.x) * HIST_THREADS * HIST_PER_THREAD;
+    const i64 n_round = (N + span - 1) / span * span;   // whole warps stay in the loop for the match
+    for (i64 base = static_cast<i64>(blockIdx.x) * HIST_THREADS * HIST_PER_THREAD + threadIdx.x; base < n_round; base += span) {
+        int k[HIST_PER_THREAD], r[HIST_PER_THREAD];
+#pragma unroll
+        for (int j = 0; j < HIST_PER_THREAD; ++j) {
+            const i64 i = base + static_cast<i64>(j) * HIST_THREADS;
+            k[j] = -1;
+            if (i < N) {
+                k[j] = idx_b[i];
+                if (k[j] < 0 || k[j] >= K) { bad = true; k[j] = -1; }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < HIST_PER_THREAD; ++j) {
+            const unsigned peers = __match_any_sync(0xffffffffu, k[j]);
+            const int leader = __ffs(peers) - 1;
+            r[j] = 0;
+            if (k[j] >= 0 && lane == leader) r[j] = atomicAdd(counts_b + k[j], __popc(peers));
+            r[j] = __shfl_sync(0xffffffffu, r[j], leader) + __popc(peers & ((1u << lane) - 1u));
+        }
+#pragma unroll
+        for (int j = 0; j < HIST_PER_THREAD; ++j) {
+            const i64 i = base + static_cast<i64>(j) * HIST_THREADS;
+            if (i < N) rank_b[i] = k[j] >= 0 ? r[j] : -1;
+        }
     }
     if (bad) atomicCAS(status, CAKE_OK, CAKE_ERR_BAD_INDEX);
 }
@@ -220,32 +248,21 @@ scan_kernel(const int* __restrict__ counts, int K, int* __restrict__ cursor, int
     }
 }
 
-// pos taken from the cluster's cursor; lanes of a warp that hit the same cluster take their slots
-// with a single atomic.
+// row i goes to position offset[its cluster] + rank[i] of the sorted order
 __global__ void __launch_bounds__(256)
-scatter_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ cursor, int2* __restrict__ pairs) {
+scatter_kernel(const int* __restrict__ idx, const int* __restrict__ rank, i64 N, int K,
+               const int* __restrict__ offset, int2* __restrict__ pairs) {
     const int b = blockIdx.y;
     const int* idx_b = idx + static_cast<size_t>(b) * N;
-    int* cur = cursor + static_cast<size_t>(b) * K;
+    const int* rank_b = rank + static_cast<size_t>(b) * N;
+    const int* off = offset + static_cast<size_t>(b) * K;
     int2* pairs_b = pairs + static_cast<size_t>(b) * N;
-    const int lane = threadIdx.x & 31;
     const i64 span = static_cast<i64>(gridDim.x) * blockDim.x;
-    const i64 n_round = (N + 31) / 32 * 32;  // keep whole warps in the loop for the match
-    for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_round; i += span) {
-        int k = -1;
-        if (i < N) {
-            k = idx_b[i];
-            if (k < 0 || k >= K) k = -1;
-        }
-        const unsigned peers = __match_any_sync(0xffffffffu, k);
-        if (k >= 0) {
-            const int leader = __ffs(peers) - 1;
-            const int rank = __popc(peers & ((1u << lane) - 1u));
-            int base = 0;
-            if (lane == leader) base = atomicAdd(cur + k, __popc(peers));
-            base = __shfl_sync(peers, base, leader);
-            pairs_b[base + rank] = make_int2(static_cast<int>(i), k);
-        }
+    for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < N; i += span) {
+        const int r = rank_b[i];
+        if (r < 0) continue;
+        const int k = idx_b[i];
+        pairs_b[__ldg(off + k) + r] = make_int2(static_cast<int>(i), k);
     }
 }
 
@@ -1150,6 +1167,10 @@ size_t update_sort_part_bytes(i64 B, i64 N, int K) {
     return pl.blocked ? static_cast<size_t>(B) * pl.nblk * K * sizeof(int) : 0;
 }
 
+size_t update_sort_rank_bytes(i64 B, i64 N, int K) {
+    return sort_plan(N, K).blocked ? 0 : static_cast<size_t>(B) * N * sizeof(int);
+}
+
 int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K,
                        const UpdateScratch& scr, int* counts, const cake_bf16* C_prev, float* out_C,
                        cake_bf16* out_C_bf16, bool* divided, int* status, cudaStream_t s) {
@@ -1179,12 +1200,12 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
                                                                scr.pairs);
     } else {
         {
-            i64 ctas = (N + HIST_THREADS * 8 - 1) / (HIST_THREADS * 8);
+            i64 ctas = (N + HIST_THREADS * HIST_PER_THREAD - 1) / (HIST_THREADS * HIST_PER_THREAD);
             const i64 cap = (static_cast<i64>(di.sm_count) * 4 + B - 1) / B;
             if (ctas > cap) ctas = cap;
             if (ctas < 1) ctas = 1;
             hist_kernel<<<dim3(static_cast<unsigned>(ctas), B), HIST_THREADS, 0, s>>>(
-                idx, N, K, counts, reinterpret_cast<float4*>(scr.sums),
+                idx, N, K, counts, scr.rank, reinterpret_cast<float4*>(scr.sums),
                 zero_in_hist ? static_cast<i64>(K) * D / 4 : 0, status);
         }
         scan_kernel<<<dim3((K + SCAN_TILE - 1) / SCAN_TILE, B), 1024, 0, s>>>(
@@ -1194,7 +1215,7 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
             const i64 cap = (static_cast<i64>(di.sm_count) * 8 + B - 1) / B;
             if (ctas > cap) ctas = cap;
             if (ctas < 1) ctas = 1;
-            scatter_kernel<<<dim3(static_cast<unsigned>(ctas), B), 256, 0, s>>>(idx, N, K, scr.cursor, scr.pairs);
+            scatter_kernel<<<dim3(static_cast<unsigned>(ctas), B), 256, 0, s>>>(idx, scr.rank, N, K, scr.cursor, scr.pairs);
         }
     }
     if (means) {
