@@ -906,9 +906,10 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     int want_xbuf = p.n_tiles <= 2 ? MAX_XBUF : 2;
     if (p.nchunks >= 4 && p.n_tiles >= 8) want_xbuf = 1;
     // two chunks per ring stage when the chunk count is even (one wait and one commit per stage), unless the
-    // ring would then hold a single stage or X is the bound (few centroid tiles: X buffers matter more)
+    // ring would then hold a single stage, X is the bound (few centroid tiles: X buffers matter more) or the
+    // last chunk is a partial one (short tiles: waiting for both chunks costs more than the barriers saved)
     i64 stages = 0;
-    for (p.cps = (p.nchunks % 2 == 0 && p.n_tiles > 2) ? 2 : 1; p.cps >= 1; --p.cps) {
+    for (p.cps = (p.nchunks % 2 == 0 && D % KCHUNK == 0 && p.n_tiles > 2) ? 2 : 1; p.cps >= 1; --p.cps) {
         p.stage_bytes = static_cast<uint32_t>(p.cps) * C_CHUNK_BYTES + AUG_B_BYTES;
         const int spt = p.nchunks / p.cps;                       // stages per centroid tile
         const i64 min_stages = p.cps == 1 ? (p.n_tiles <= 2 ? 2 : 3) : (p.n_tiles <= 2 ? 2 : 2 * spt);
