@@ -17,8 +17,10 @@
 // One persistent CTA per SM, 16 warps, four roles:
 //   warp 8  producer : TMA.  A 128-row X tile (whole D) into one of the X buffers per row tile (up to
 //                      four row tiles ahead); per centroid tile of 256 rows, D/64 chunks of 64 columns
-//                      (128-byte swizzle) through an mbarrier ring, plus the tile's 4 KiB block of
-//                      split half-norms (bulk copy).
+//                      (128-byte swizzle) through an mbarrier ring.  A ring stage holds one chunk, or two
+//                      when the chunk count is even (one wait and one commit for both), and has room
+//                      for the tile's 4 KiB block of split half-norms, which arrives (bulk copy) on the
+//                      barrier of the tile's last stage.
 //   warps 9-11 MMA   : one thread each issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32); centroid
 //                      tiles go round robin over the three (tile t: issuer t mod 3, accumulator t mod 2
 //                      of two 256-column TMEM accumulators); tcgen05.commit frees ring slots and

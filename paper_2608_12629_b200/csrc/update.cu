@@ -6,10 +6,13 @@
 //                and reduces the slab in that order (thread-block clusters combine the histograms of
 //                2 or 4 CTAs over distributed shared memory when K is large against a slab).  The
 //                automatic choice while a slab holds several rows per cluster.
-//   sort route : global counting sort by cluster (histogram, exclusive scan, scatter of row numbers)
-//                and a segmented reduction in which each warp sums a fixed-size run of the sorted
-//                order in registers and adds one partial per cluster it touches.  Any K; for K <= 8192
-//                the sort works on per-slab shared-memory histograms and needs no global atomics.
+//   sort route : global counting sort by cluster (histogram, exclusive scan, scatter of row numbers),
+//                then one pass over X in that order.  K <= 8192: the sort works on per-slab
+//                shared-memory histograms (no global atomics) and a segmented reduction follows in
+//                which each warp sums a fixed-size run of the sorted order in registers and adds one
+//                partial per cluster it touches.  Larger K (rows a multiple of 16 bytes): every
+//                cluster is summed by one warp, which divides and writes the centroid itself; this
+//                variant produces the means directly and needs no division pass.
 //   smem route : every CTA keeps a private K x D table of partial sums in shared memory, streams a
 //                slab of rows through it with shared-memory atomics and adds its table to the
 //                global one at the end.  For K*D*4 bytes that fit in one SM's shared memory; slow
@@ -847,8 +850,7 @@ segmean_kernel(const cake_bf16* __restrict__ X, const int2* __restrict__ pairs, 
 // One kernel sorts and reduces.  A CTA owns a slab of S consecutive rows: it keeps their cluster ids
 // in registers, ranks every row inside its cluster with one shared-memory atomic, scans the
 // histogram and writes the slab's rows in cluster order into shared memory; then lane groups walk
-// that order, gather the rows (all inside the slab's own window of X, which keeps the DRAM pages
-// busy) and flush one vector atomic per run of equal clusters.  A run is S/K rows long, so when K
+// that order, gather the rows and flush one vector atomic per run of equal clusters.  A run is S/K rows long, so when K
 // is large against S, F CTAs form a thread-block cluster: their histograms are combined through
 // distributed shared memory into one order over the F*S rows of the cluster, every CTA takes an
 // equal contiguous share of it, and runs are F times longer (F times fewer atomics).
