@@ -128,6 +128,7 @@ __global__ void __launch_bounds__(HIST_THREADS)
 hist_kernel(const int* __restrict__ idx, i64 N, int K, int* __restrict__ counts, int* __restrict__ rank,
             float4* __restrict__ sums4, i64 sums4_per_problem, int* status) {
     const int b = blockIdx.y;
+    ptx::grid_dep_launch();    // the scan behind this kernel waits for its end by itself
     // this CTA's share of the fp32 sums starts at zero (the loads below are in flight meanwhile)
     {
         const i64 z0 = sums4_per_problem * blockIdx.x / gridDim.x, z1 = sums4_per_problem * (blockIdx.x + 1) / gridDim.x;
@@ -186,6 +187,8 @@ scan_kernel(const int* __restrict__ counts, int K, int* __restrict__ cursor, int
     __shared__ int pre_s;
     __shared__ int heavy_n;
     __shared__ int heavy_list[SCAN_TILE];
+    ptx::grid_dep_wait();      // the histogram ahead of this kernel is complete
+    ptx::grid_dep_launch();
     if (threadIdx.x == 0) heavy_n = 0;
     const int b = blockIdx.y, tile = blockIdx.x;
     const int* c = counts + static_cast<size_t>(b) * K;
@@ -256,6 +259,8 @@ __global__ void __launch_bounds__(256)
 scatter_kernel(const int* __restrict__ idx, const int* __restrict__ rank, i64 N, int K,
                const int* __restrict__ offset, int2* __restrict__ pairs) {
     const int b = blockIdx.y;
+    ptx::grid_dep_wait();      // the scan (and with it the histogram) is complete
+    ptx::grid_dep_launch();
     const int* idx_b = idx + static_cast<size_t>(b) * N;
     const int* rank_b = rank + static_cast<size_t>(b) * N;
     const int* off = offset + static_cast<size_t>(b) * K;
@@ -592,6 +597,7 @@ segmean_kernel(const cake_bf16* __restrict__ X, const int2* __restrict__ pairs, 
     constexpr int R = U * MEAN_AHEAD;              // passes in the ring
     static_assert(U * RPP <= 32, "a batch must fit two blocks of the row table");
     extern __shared__ uint4 mean_ring[];           // [warp]{[R][GPL][32] ring, 128 row numbers}
+    ptx::grid_dep_wait();      // the scatter (and with it scan and histogram) is complete
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -1107,6 +1113,22 @@ finalize4_kernel(const float4* __restrict__ sums, const int* __restrict__ counts
 }  // namespace
 
 // ======================================================================= host side
+// Launch that may start while the kernel ahead of it in the stream drains (programmatic dependent
+// launch): the kernel itself waits (griddepcontrol.wait) before it touches what that kernel wrote.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_early(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 bool update_smem_supports(int D, int K, int smem_optin) {
     if (D % 2 != 0) return false;
     const i64 need = static_cast<i64>(K) * D * 4 + static_cast<i64>(K) * 4;
@@ -1210,14 +1232,17 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
                 idx, N, K, counts, scr.rank, reinterpret_cast<float4*>(scr.sums),
                 zero_in_hist ? static_cast<i64>(K) * D / 4 : 0, status);
         }
-        scan_kernel<<<dim3((K + SCAN_TILE - 1) / SCAN_TILE, B), 1024, 0, s>>>(
-            counts, K, scr.cursor, scr.nvalid, means ? scr.sums : nullptr, scr.done, D);
+        if (launch_early(scan_kernel, dim3((K + SCAN_TILE - 1) / SCAN_TILE, B), dim3(1024), 0, s, counts, K, scr.cursor,
+                         scr.nvalid, means ? scr.sums : nullptr, scr.done, D) != cudaSuccess)
+            return CAKE_ERR_CUDA;
         {
             i64 ctas = (N + 256 * 4 - 1) / (256 * 4);
             const i64 cap = (static_cast<i64>(di.sm_count) * 8 + B - 1) / B;
             if (ctas > cap) ctas = cap;
             if (ctas < 1) ctas = 1;
-            scatter_kernel<<<dim3(static_cast<unsigned>(ctas), B), 256, 0, s>>>(idx, scr.rank, N, K, scr.cursor, scr.pairs);
+            if (launch_early(scatter_kernel, dim3(static_cast<unsigned>(ctas), B), dim3(256), 0, s, idx, scr.rank, N, K,
+                             scr.cursor, scr.pairs) != cudaSuccess)
+                return CAKE_ERR_CUDA;
         }
     }
     if (means) {
@@ -1236,8 +1261,9 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
         MeanKernel kernel = gpl == 4 ? segmean_kernel<4, 32> : gpl == 2 ? segmean_kernel<2, 32>
                           : lpr == 32 ? segmean_kernel<1, 32> : lpr == 16 ? segmean_kernel<1, 16>
                           : lpr == 8 ? segmean_kernel<1, 8> : segmean_kernel<1, 4>;
-        kernel<<<grid, MEAN_WARPS * 32, mean_smem, s>>>(X, scr.pairs, scr.nvalid, counts, N, D, K, C_prev, out_C,
-                                                       out_C_bf16, scr.sums, scr.done);
+        if (launch_early(kernel, grid, dim3(MEAN_WARPS * 32), mean_smem, s, X, scr.pairs, scr.nvalid, counts, N, D, K, C_prev,
+                         out_C, out_C_bf16, scr.sums, scr.done) != cudaSuccess)
+            return CAKE_ERR_CUDA;
         *divided = true;
     } else {
         const i64 warps = (N + SEG_ROWS - 1) / SEG_ROWS;
