@@ -67,7 +67,9 @@ enum {
     CAKE_ASSIGN_MASK = 0xF,
     CAKE_UPDATE_AUTO = 0,
     CAKE_UPDATE_SMEM = 1 << 4, /* shared-memory partial sums; needs K*D*4 + K*4 bytes of smem   */
-    CAKE_UPDATE_SORT = 2 << 4, /* counting sort by cluster + segmented reduction, any K         */
+    CAKE_UPDATE_SORT = 2 << 4, /* counting sort by cluster, then one pass over X in that order (a
+                                  segmented reduction; for K > 8192 and D % 8 == 0 every cluster is
+                                  summed and divided by one warp), any K                         */
     CAKE_UPDATE_SLAB = 3 << 4, /* one kernel sorts and reduces slab by slab (thread-block clusters
                                   when K is large against the slab); D % 8 == 0, D <= 256, K <= 8192 */
     CAKE_UPDATE_SLAB_F1 = 4 << 4, /* the same with the cluster size forced to 1, 2 or 4 CTAs      */
