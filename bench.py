@@ -1,8 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the Flash-KMeans Lloyd hot path on B200.
 
-A "step" is one Lloyd iteration (assign + centroid update, through cake_kmeans_lloyd with iters=1,
-the centroids of each step feeding the next) over the workload's seeded synthetic Gaussian mixture.
+A "step" is one Lloyd iteration (assign + centroid update) over the workload's seeded synthetic Gaussian
+mixture; the K timed steps are ONE cake_kmeans_lloyd(iters=K) call (the library's own loop, centroids fed
+forward on the device) after one warm-up call of W iterations.
 Prints ONE JSON line (rank 0):
   value      Lloyd iterations/s with X resident in HBM (whole job, all ranks)
   e2e        the same through cake_kmeans_lloyd_host: pinned HOST buffers, H2D + D2H inside the timing
@@ -287,21 +288,25 @@ def main():
         torch.cuda.synchronize(dev)
 
     # ---------------- timed region 1: whole steps through cake_kmeans_lloyd (value)
+    # W warm-up iterations in one call, then the K timed iterations in one call that starts from the
+    # warm-up's centroids: the library's own Lloyd loop, no host work between the steps
     cur = C0.clone()
-    for _ in range(args.warmup):
-        cake.cake_kmeans_lloyd(X, cur, 1, out=out, ws=ws)
-        cur.copy_(out.C_bf16)
+    if args.warmup > 0:
+        out_w = cake.alloc_lloyd_outputs(X, C0, args.warmup)
+        cake.cake_kmeans_lloyd(X, cur, args.warmup, out=out_w, ws=ws)
+        cur.copy_(out_w.C_bf16)
+        del out_w
+    out_k = cake.alloc_lloyd_outputs(X, C0, args.steps)
     barrier()
     launches0 = cake.cake_kmeans_kernel_launches()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(physical_gpu_index(local)) as clocks:
         barrier()
         e0.record(stream)
-        for _ in range(args.steps):
-            cake.cake_kmeans_lloyd(X, cur, 1, out=out, ws=ws)
-            cur.copy_(out.C_bf16)
+        cake.cake_kmeans_lloyd(X, cur, args.steps, out=out_k, ws=ws)
         e1.record(stream)
         barrier()
+    del out_k
     launches = cake.cake_kmeans_kernel_launches() - launches0
     ms_total = e0.elapsed_time(e1)
     status = cake.cake_kmeans_device_status(ws)
@@ -369,7 +374,7 @@ def main():
             "config": {"workload": f"{w.name}: N={N} D={D} K={K} B={B}, {w.components}-component Gaussian mixture, "
                                    f"sigma={w.sigma}, random-sample init, seed {w.seed}+rank",
                        "l2": f"X is {B * N * D * 2 / 2**20:.0f} MiB per step, larger than the 126 MB L2; no flush",
-                       "step": "one Lloyd iteration = cake_kmeans_lloyd(iters=1)",
+                       "step": "one Lloyd iteration; the K timed steps are one cake_kmeans_lloyd(iters=K) call that starts from the warm-up call's centroids",
                        "x_checksum": inputs.checksum(X.view(-1)[: 1 << 20])},
             "assign": {"ms": assign_ms, "tflops": a_tflops, "frac_of_measured_bf16_peak": a_tflops / peaks["bf16_tflops"],
                        "frac_of_measured_bf16_sustained": a_tflops / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),

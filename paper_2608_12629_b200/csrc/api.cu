@@ -69,9 +69,10 @@ int check_ws(void* ws, size_t ws_bytes, i64 B, i64 N, int D, int K, Workspace* o
 // inertia (nullable): inertia[b * inertia_stride] += sum of problem b's distances.  The tensor-core
 // kernel adds it up itself; the fallback needs `dist` (out_dist or scratch) and a reduction kernel.
 // zero_inertia: the entries still have to be cleared (the tensor-core prologue does it on the way).
+// aug_ready: the update ahead prepared this assign (see NextAssign): the tensor-core route skips its prologue
 int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, int* out_idx,
-              float* out_dist, double* inertia, int inertia_stride, bool zero_inertia, const Workspace& w,
-              cudaStream_t s, unsigned flags) {
+              float* out_dist, double* inertia, int inertia_stride, bool zero_inertia, bool aug_ready,
+              const Workspace& w, cudaStream_t s, unsigned flags) {
     unsigned path = flags & CAKE_ASSIGN_MASK;
     if (path == CAKE_ASSIGN_AUTO) path = assign_tc_supports(D) ? CAKE_ASSIGN_TCGEN05 : CAKE_ASSIGN_SIMT;
     if (zero_inertia && inertia && (path == CAKE_ASSIGN_SIMT || N == 0)) {
@@ -95,12 +96,14 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
     // up to 32 problems keep max ||c||^2 in the header, which the kernel leaves zeroed: no memset per call
     const bool in_header = B <= 32;
     return launch_assign_tc(X, C, B, N, D, K, w.caug, in_header ? w.status + 16 : w.cnmax, in_header ? w.status + 1 : nullptr,
-                            exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia, w.status, s);
+                            exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia, aug_ready, w.status, s);
 }
 
+// next / prepared: see launch_finalize
 int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, const cake_bf16* C_prev,
               float* out_C, cake_bf16* out_C_bf16, int* out_counts, const Workspace& w, cudaStream_t s,
-              unsigned flags) {
+              unsigned flags, const NextAssign* next = nullptr, bool* prepared = nullptr) {
+    if (prepared) *prepared = false;
     DeviceInfo di;
     int rc = current_device_info(&di);
     if (rc != CAKE_OK) return rc;
@@ -126,7 +129,7 @@ int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, co
     if (rc != CAKE_OK) return rc;
     if (divided) return CAKE_OK;
     const bool slab = path != CAKE_UPDATE_SMEM && path != CAKE_UPDATE_SORT;
-    if (launch_finalize(w.sums, out_counts, C_prev, B, K, D, out_C, out_C_bf16, slab, s) != cudaSuccess)
+    if (launch_finalize(w.sums, out_counts, C_prev, B, K, D, out_C, out_C_bf16, slab, next, prepared, s) != cudaSuccess)
         return CAKE_ERR_CUDA;
     return CAKE_OK;
 }
@@ -177,7 +180,7 @@ int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, long long
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;
-    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, false, w,
+    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, false, false, w,
                      reinterpret_cast<cudaStream_t>(stream), flags);
 }
 
@@ -233,7 +236,7 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     if (iters == 0) {
         // out_C = C0 widened: the division kernel with all-zero counts takes the keep-previous branch
         if (cudaMemsetAsync(w.cursor, 0, static_cast<size_t>(B) * K * 4, s) != cudaSuccess) return CAKE_ERR_CUDA;
-        if (launch_finalize(w.sums, w.cursor, C0, Bi, K, D, out_C, nullptr, false, s) != cudaSuccess)
+        if (launch_finalize(w.sums, w.cursor, C0, Bi, K, D, out_C, nullptr, false, nullptr, nullptr, s) != cudaSuccess)
             return CAKE_ERR_CUDA;
         if (out_C_bf16 && cudaMemcpyAsync(out_C_bf16, C0, kd * 2, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
             return CAKE_ERR_CUDA;
@@ -242,14 +245,22 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     // No copies: the first iteration reads C0 itself, the bf16 centroids ping-pong between the two
     // workspace buffers and the last iteration writes the caller's buffer directly.  Each iteration's
     // inertia entries are cleared by its own assign step.
+    // The division kernel of iteration t also writes what the tensor-core assign of iteration t + 1 would
+    // otherwise compute in a prologue launch of its own (while max ||c||^2 lives in the header, B <= 32).
+    const unsigned apath = flags & CAKE_ASSIGN_MASK;
+    const bool tc_assign = N > 0 && assign_tc_supports(D) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
+                                                              apath == CAKE_ASSIGN_TCGEN05_EXACT);
     const cake_bf16* cur = C0;
     int nxt = 0;
+    bool prepared = false;
     for (int t = 0; t < iters; ++t) {
         rc = do_assign(X, cur, Bi, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr, iters,
-                       true, w, s, flags);
+                       true, prepared, w, s, flags);
         if (rc != CAKE_OK) return rc;
         cake_bf16* dst = (t == iters - 1 && out_C_bf16) ? out_C_bf16 : w.cbuf[nxt];
-        rc = do_update(X, out_idx, Bi, N, D, K, cur, out_C, dst, out_counts, w, s, flags);
+        NextAssign next{w.caug, w.status + 16, out_inertia ? out_inertia + t + 1 : nullptr, iters};
+        const bool want = tc_assign && Bi <= 32 && t + 1 < iters;
+        rc = do_update(X, out_idx, Bi, N, D, K, cur, out_C, dst, out_counts, w, s, flags, want ? &next : nullptr, &prepared);
         if (rc != CAKE_OK) return rc;
         cur = dst;
         nxt ^= 1;

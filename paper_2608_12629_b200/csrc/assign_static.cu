@@ -72,5 +72,5 @@ extern "C" int cake_kmeans_assign_static(const cake_bf16* X, const cake_bf16* C,
     if (cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) return CAKE_ERR_CUDA;
     // header: word 0 = status, word 16 = max ||c||^2 (cleared by the prologue launch)
     return launch_assign_tc(X, C, 1, N, D, K, scratch + kStaticHeader, status + 16, nullptr, false, out_idx, out_dist, nullptr, 0,
-                            false, status, s);
+                            false, false, status, s);
 }

@@ -41,6 +41,7 @@
 //            running best (cheaper when there are many centroid tiles per row).
 // Every wait is bounded: on expiry the CTA raises CAKE_ERR_TIMEOUT in the status word, all roles
 // leave their loops, TMEM is freed and the kernel returns.
+#include "aug.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -186,19 +187,7 @@ __device__ __forceinline__ bool wait_bar_body(uint64_t* bar, uint32_t parity, Ct
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-__device__ __forceinline__ uint32_t bf16_rne_bits(float f) {
-    uint32_t u = __float_as_uint(f);
-    u += 0x7fffu + ((u >> 16) & 1u);
-    return u >> 16;
-}
-// h = hi + mid + lo with three bf16 terms (24 significand bits: nothing of the fp32 value is lost)
-__device__ __forceinline__ void split3(float h, uint32_t& hi, uint32_t& mid, uint32_t& lo) {
-    hi = bf16_rne_bits(h);
-    const float r1 = h - __uint_as_float(hi << 16);
-    mid = bf16_rne_bits(r1);
-    const float r2 = r1 - __uint_as_float(mid << 16);
-    lo = bf16_rne_bits(r2);
-}
+using aug::split3;
 
 // min over 32 floats with 3-input min instructions
 __device__ __forceinline__ float min32(const float (&v)[32]) {
@@ -767,26 +756,21 @@ centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64
     float acc = 0.f;
     if (k < K) {
         const cake_bf16* row = C + (static_cast<size_t>(b) * K + k) * D;
-        for (int d = lane; d < D; d += 32) {
-            const float v = __uint_as_float(static_cast<uint32_t>(row[d]) << 16);
-            acc = fmaf(v, v, acc);
+        if (D % 4 == 0) {   // rows are 8-byte aligned: four columns per load
+            const uint2* row4 = reinterpret_cast<const uint2*>(row);
+            for (int j = lane; j < D / 4; j += 32) {
+                const uint2 q = __ldg(row4 + j);
+                acc = aug::add_squares(acc, q.x, q.y);
+            }
+        } else {
+            for (int d = lane; d < D; d += 32) {
+                const float v = __uint_as_float(static_cast<uint32_t>(row[d]) << 16);
+                acc = fmaf(v, v, acc);
+            }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        acc = aug::fold_lanes(acc);
     }
-    if (lane == 0) {
-        uint32_t hi = 0, mid = 0, lo = 0, b6 = 0x3FC0u;   // padded rows: no norm, 1.5 M
-        if (k < K) {
-            split3(0.5f * acc, hi, mid, lo);
-            b6 = 0x3F80u;
-            atomicMax(cnmax + b, __float_as_int(acc));
-        }
-        const uint32_t one = 0x3F80u;
-        const int tile = k / BLOCK_N, rr = k % BLOCK_N;
-        uint8_t* blk = caug + (static_cast<size_t>(b) * (Kpad / BLOCK_N) + tile) * AUG_B_BYTES;
-        *reinterpret_cast<uint4*>(blk + rr * 16) =
-            make_uint4(one | (one << 16), one | (hi << 16), mid | (lo << 16), b6 | (one << 16));
-    }
+    if (lane == 0) aug::write_row(caug, cnmax, b, k, K, Kpad, acc);
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time libcuda dependency)
@@ -845,7 +829,7 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
 
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      int* cnmax, int* ticket, bool exact, int* out_idx, float* out_dist, double* inertia,
-                     int inertia_stride, bool zero_inertia, int* status, cudaStream_t s) {
+                     int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s) {
     if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
     DeviceInfo di;
     int rc = current_device_info(&di);
@@ -872,7 +856,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     cudaLaunchAttribute pdl[1];
     pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl[0].val.programmaticStreamSerializationAllowed = 1;
-    {
+    if (!aug_ready) {
         const i64 rows = static_cast<i64>(B) * Kpad;
         const i64 ctas = (rows * 32 + 255) / 256;
         // cnmax must start at zero: either it lives where the last CTA of the previous call cleared it

@@ -42,9 +42,11 @@ size_t assign_tc_aug_bytes(i64 B, int K);
 // ticket (nullable): cnmax and *ticket lie in memory that is zero between calls (the kernel's last CTA
 // clears them again); without it cnmax is cleared by a memset.  zero_inertia: the prologue starts the
 // inertia entries from zero (otherwise the caller has).
+// aug_ready: caug, cnmax and (if asked for) the cleared inertia entries are already what the prologue
+// would write for these centroids (the division kernel of the update ahead wrote them): no prologue.
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      int* cnmax, int* ticket, bool exact, int* out_idx, float* out_dist, double* inertia,
-                     int inertia_stride, bool zero_inertia, int* status, cudaStream_t s);
+                     int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s);
 int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
                        int* out_idx, float* out_dist, cudaStream_t s);
 
@@ -79,8 +81,18 @@ int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
                        int* counts, int* status, int force_f, cudaStream_t s);
 // out_C = counts>0 ? sums/counts : C_prev (or 0); optional bf16 copy.  early: launched so that it may
 // start before the kernel ahead of it in the stream has drained (it waits for that kernel itself)
+// next (nullable): also prepare the tensor-core assign of the centroids being written (its half-norm
+// operand, max ||c||^2, cleared inertia entries), so that that assign needs no prologue.  Needs
+// D % 4 == 0 and out_C_bf16; *prepared tells whether it was done.
+struct NextAssign {
+    void* caug;             // as for launch_assign_tc
+    int* cnmax;             // zero on entry (the assign kernel ahead left it so)
+    double* inertia;        // nullable: inertia[b * inertia_stride] = 0 for b < B (B <= 256)
+    int inertia_stride;
+};
 cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B,
-                            int K, int D, float* out_C, cake_bf16* out_C_bf16, bool early, cudaStream_t s);
+                            int K, int D, float* out_C, cake_bf16* out_C_bf16, bool early,
+                            const NextAssign* next, bool* prepared, cudaStream_t s);
 
 // ---- inertia: acc[b] += sum_i dist[b][i] (fp64 atomics); acc stride given in elements
 cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc_stride,

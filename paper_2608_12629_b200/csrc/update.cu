@@ -20,6 +20,7 @@
 // All stream X exactly once with 16-byte (smem route: 4-byte) loads; HBM bandwidth is the bound.
 #include <cooperative_groups.h>
 
+#include "aug.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -1110,6 +1111,49 @@ finalize4_kernel(const float4* __restrict__ sums, const int* __restrict__ counts
     }
 }
 
+// D % 4 == 0, one warp per centroid row (lanes stride the row in quads of columns): the division as in
+// finalize4_kernel and, on the way, what the tensor-core assign of these centroids needs as its
+// prologue: ||c||^2 of the bf16-rounded row (summed as the assign prologue sums it), split into the
+// k-step operand row, the problem's max ||c||^2 and cleared inertia entries.
+__global__ void __launch_bounds__(256)
+finalize_rows_kernel(const float4* __restrict__ sums, const int* __restrict__ counts,
+                     const uint2* __restrict__ C_prev, i64 rows, int K, int D4, float4* __restrict__ out_C,
+                     uint2* __restrict__ out_C_bf16, uint8_t* __restrict__ caug, int* __restrict__ cnmax, int Kpad,
+                     double* __restrict__ inertia, int inertia_stride, int B) {
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
+    if (inertia && blockIdx.x == 0 && static_cast<int>(threadIdx.x) < B)
+        inertia[static_cast<size_t>(threadIdx.x) * inertia_stride] = 0.0;
+    const int lane = threadIdx.x & 31;
+    const i64 n_warps = static_cast<i64>(gridDim.x) * (blockDim.x >> 5);
+    for (i64 row = static_cast<i64>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); row < rows; row += n_warps) {
+        const int n = counts[row];
+        const float fn = static_cast<float>(n);
+        float acc = 0.f;
+        for (int j = lane; j < D4; j += 32) {
+            const i64 e = row * D4 + j;
+            float4 v;
+            if (n > 0) {
+                const float4 sv = sums[e];
+                v = make_float4(sv.x / fn, sv.y / fn, sv.z / fn, sv.w / fn);
+            } else if (C_prev) {
+                const uint2 pv = C_prev[e];
+                v = make_float4(bf16lo(pv.x), bf16hi(pv.x), bf16lo(pv.y), bf16hi(pv.y));
+            } else {
+                v = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            out_C[e] = v;
+            uint2 o;
+            o.x = static_cast<uint32_t>(f32_to_bf16_rne(v.x)) | (static_cast<uint32_t>(f32_to_bf16_rne(v.y)) << 16);
+            o.y = static_cast<uint32_t>(f32_to_bf16_rne(v.z)) | (static_cast<uint32_t>(f32_to_bf16_rne(v.w)) << 16);
+            out_C_bf16[e] = o;
+            acc = aug::add_squares(acc, o.x, o.y);
+        }
+        acc = aug::fold_lanes(acc);
+        if (lane == 0) aug::write_row(caug, cnmax, row / K, static_cast<int>(row % K), K, Kpad, acc);
+    }
+}
+
 }  // namespace
 
 // ======================================================================= host side
@@ -1450,8 +1494,24 @@ int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
 }
 
 cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B, int K,
-                            int D, float* out_C, cake_bf16* out_C_bf16, bool early, cudaStream_t s) {
+                            int D, float* out_C, cake_bf16* out_C_bf16, bool early, const NextAssign* next,
+                            bool* prepared, cudaStream_t s) {
     const i64 total = static_cast<i64>(B) * K * D;
+    if (prepared) *prepared = false;
+    if (next && out_C_bf16 && D % 4 == 0 && B <= 256) {
+        const i64 rows = static_cast<i64>(B) * K;
+        i64 ctas = (rows + 7) / 8;
+        if (ctas > 148 * 8) ctas = 148 * 8;
+        if (ctas < 1) ctas = 1;
+        cudaError_t e = launch_early(finalize_rows_kernel, dim3(static_cast<unsigned>(ctas)), dim3(256), 0, s,
+                                     reinterpret_cast<const float4*>(sums), counts, reinterpret_cast<const uint2*>(C_prev), rows,
+                                     K, D / 4, reinterpret_cast<float4*>(out_C), reinterpret_cast<uint2*>(out_C_bf16),
+                                     static_cast<uint8_t*>(next->caug), next->cnmax, padded_k(K), next->inertia,
+                                     next->inertia_stride, B);
+        note_launches(1);
+        if (e == cudaSuccess && prepared) *prepared = true;
+        return e;
+    }
     // early: the launch may overlap the tail of the kernel ahead (the kernels wait for it themselves)
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -374,6 +374,33 @@ def test_lloyd_handworked_example_on_gpu():
     assert out.C_bf16.float().cpu()[:, :2].tolist() == [[171 / 256, 171 / 256], [171 / 16, 171 / 16]]
 
 
+@pytest.mark.parametrize("B,N,D,K", [(1, 5000, 64, 37), (2, 3000, 128, 300), (1, 2000, 24, 9)])
+def test_lloyd_call_equals_stepwise_calls(B, N, D, K):
+    """Inside a Lloyd call the division kernel prepares the next assign (half-norm operand, max ||c||^2,
+    cleared inertia): the result must be bit-identical to assign and update called one by one, where the
+    assign computes all that in its own prologue.  Small integer data: the sums are exact in fp32
+    whatever their order, so bit-identity is well defined."""
+    g = torch.Generator().manual_seed(B * 1000 + D)
+    X = torch.randint(-4, 5, (B, N, D), generator=g).to(torch.bfloat16)
+    C0 = X[:, :K].contiguous().clone()
+    C0[:, :, 0] += torch.arange(K).to(torch.bfloat16)          # distinct centroids
+    Xd, C0d = X.to(DEV), C0.to(DEV)
+    if B == 1:
+        Xd, C0d = Xd[0], C0d[0]
+    iters = 4
+    out = cake.cake_kmeans_lloyd(Xd, C0d, iters)
+    C = C0d
+    inertia = []
+    for _ in range(iters):
+        idx, dist = cake.cake_kmeans_assign(Xd, C)
+        inertia.append(dist.double().sum(-1))
+        Cf, Cb, counts = cake.cake_kmeans_update(Xd, idx, K, C_prev=C)
+        C = Cb
+    assert torch.equal(out.idx, idx) and torch.equal(out.dist, dist)
+    assert torch.equal(out.C, Cf) and torch.equal(out.C_bf16, Cb) and torch.equal(out.counts, counts)
+    np.testing.assert_allclose(out.inertia.cpu().numpy(), torch.stack(inertia, -1).cpu().numpy(), rtol=1e-12)
+
+
 def test_lloyd_iters_zero_and_batched():
     B, N, D, K = 3, 1500, 64, 24
     Xs, Cs = zip(*(problem(N, D, K, seed=90 + b, comps=24, mean_std=2.0, sigma=1.0) for b in range(B)))
