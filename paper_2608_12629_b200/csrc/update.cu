@@ -1302,7 +1302,7 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
         const size_t mean_smem = static_cast<size_t>(MEAN_WARPS) * MEAN_WARP_UINT4 * sizeof(uint4);
         using MeanKernel = void (*)(const cake_bf16*, const int2*, const int*, const int*, i64, int, int,
                                     const cake_bf16*, float*, cake_bf16*, float*, int*);
-        MeanKernel kernel = gpl == 4 ? segmean_kernel<4, 32> : gpl == 2 ? segmean_kernel<2, 32>
+        MeanKernel kernel = gpl > 2 ? segmean_kernel<4, 32> : gpl == 2 ? segmean_kernel<2, 32>
                           : lpr == 32 ? segmean_kernel<1, 32> : lpr == 16 ? segmean_kernel<1, 16>
                           : lpr == 8 ? segmean_kernel<1, 8> : segmean_kernel<1, 4>;
         if (launch_early(kernel, grid, dim3(MEAN_WARPS * 32), mean_smem, s, X, scr.pairs, scr.nvalid, counts, N, D, K, C_prev,

@@ -266,6 +266,35 @@ def test_update_many_clusters_skewed_sizes(D):
                                  Cf[b].cpu().numpy(), inputs.to_bits(Cb[b]), counts[b].cpu().numpy())
 
 
+@pytest.mark.parametrize("case", ["one_row", "few_rows", "all_invalid", "one_cluster", "two_clusters_alternating"])
+@pytest.mark.parametrize("D", [24, 40, 256, 520])
+def test_update_many_clusters_degenerate(case, D):
+    """K > 8192, degenerate index sets: a single row, fewer rows than a window, no valid index at all (every
+    centroid keeps its previous value and the status word says so), every row in one heavy cluster, rows
+    alternating between the first and the last cluster; granule counts that do not fill the lanes."""
+    K = 9001
+    N = {"one_row": 1, "few_rows": 50, "all_invalid": 300, "one_cluster": 5000, "two_clusters_alternating": 4100}[case]
+    X = inputs.from_bits(np.random.default_rng(D + N).integers(0x3C00, 0x4100, size=(N, D), dtype=np.uint16))
+    g = torch.Generator().manual_seed(N)
+    if case == "all_invalid":
+        idx = torch.full((N,), K + 5, dtype=torch.int32)
+        idx[::2] = -1
+    elif case == "one_cluster":
+        idx = torch.full((N,), 4242, dtype=torch.int32)
+    elif case == "two_clusters_alternating":
+        idx = torch.where(torch.arange(N) % 2 == 0, 0, K - 1).to(torch.int32)
+    else:
+        idx = torch.randint(0, K, (N,), generator=g, dtype=torch.int32)
+    Cprev = inputs.from_bits(np.random.default_rng(D).integers(0x3C00, 0x4100, size=(K, D), dtype=np.uint16))
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    Cf, Cb, counts = cake.cake_kmeans_update(X.to(DEV), idx.to(DEV), K, C_prev=Cprev.to(DEV), ws=ws,
+                                             flags=cake.CAKE_UPDATE_SORT)
+    check_status(ws, cake.CAKE_ERR_BAD_INDEX if case == "all_invalid" else cake.CAKE_OK)
+    keep = ((idx >= 0) & (idx < K)).numpy()
+    grading.grade_update(inputs.to_bits(X)[keep], idx.numpy()[keep], K, inputs.to_bits(Cprev), Cf.cpu().numpy(),
+                         inputs.to_bits(Cb), counts.cpu().numpy())
+
+
 def test_update_odd_feature_count_and_null_prev():
     N, D, K = 500, 7, 9
     X, _ = problem(N, D, K, seed=2)
