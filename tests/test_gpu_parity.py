@@ -403,7 +403,7 @@ def test_lloyd_handworked_example_on_gpu():
     assert out.C_bf16.float().cpu()[:, :2].tolist() == [[171 / 256, 171 / 256], [171 / 16, 171 / 16]]
 
 
-@pytest.mark.parametrize("B,N,D,K", [(1, 5000, 64, 37), (2, 3000, 128, 300), (1, 2000, 24, 9)])
+@pytest.mark.parametrize("B,N,D,K", [(1, 5000, 64, 37), (2, 3000, 128, 300), (1, 2000, 24, 9), (33, 300, 64, 5), (1, 700, 12, 6)])
 def test_lloyd_call_equals_stepwise_calls(B, N, D, K):
     """Inside a Lloyd call the division kernel prepares the next assign (half-norm operand, max ||c||^2,
     cleared inertia): the result must be bit-identical to assign and update called one by one, where the
