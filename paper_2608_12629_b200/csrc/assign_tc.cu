@@ -93,7 +93,10 @@ struct Params {
     int n_stages;     // ring depth (stages)
     int cps;          // centroid chunks per ring stage: 2 when nchunks is even (half the barrier traffic), else 1
     uint32_t stage_bytes;   // cps * 32 KiB + 4 KiB
-    int n_xbuf;       // 1 or 2 X buffers
+    int n_xbuf;       // X buffers (1..4)
+    int alt_epi;      // one centroid tile per row tile: the two epilogue warpgroups take whole row tiles in turn
+    int res_c;        // ... and the centroid tile stays in shared memory (loaded once per problem): the two
+                      // issuers share no ring and each works on its own row tiles only (implies alt_epi)
     const uint8_t* caug;  // [B][n_tiles][4 KiB] centroid-side operand of the extra k-step
     int* cnmax;           // [B] bit pattern of max_k ||c_k||^2 (fp32, >= 0)
     int* ticket;          // optional: CTAs that have finished; the last one clears cnmax and the ticket
@@ -113,6 +116,7 @@ struct Ctrl {  // lives in shared memory
     uint64_t tmem_empty[2][MAX_ISSUERS];
     uint64_t auga_full[MAX_XBUF];
     uint64_t merge_full[2], merge_empty[2];
+    uint64_t turn[2];   // resident-centroid mode: issuer i may issue its next tile's MMAs (the other one has issued its own)
     uint32_t tmem_base;
     int abort_flag;
     float merge_best[2][BLOCK_M];
@@ -261,15 +265,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         for (int i = 0; i < MAX_XBUF; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
             // MMA issuers + 4 norm warps + the 4 epilogue warps that read the row exponents
-            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), NUM_ISSUERS + 4 + 4);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), (p.res_c ? 1 : NUM_ISSUERS) + 4 + 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1);
             for (int j = 0; j < MAX_ISSUERS; ++j)
-                ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i][j]), NUM_EPI_WARPS);
+                ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i][j]), p.alt_epi ? NUM_EPI_WARPS / 2 : NUM_EPI_WARPS);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_full[i]), 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_empty[i]), 4);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->turn[i]), 1);
         }
         for (int i = 0; i < MAX_STAGES; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_full[i]), 1);
@@ -332,6 +337,38 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                        ptx::mbar_test_wait(ptx::smem_u32(&ctrl->x_empty[ixb]), ixph ^ 1u))
                     issue_x();
             };
+            if (XLOAD && p.res_c) {
+                // resident centroids: the whole tile (all chunks and the half-norm block) once per problem
+                // this CTA meets; "stage 0" of the ring stands for the whole buffer
+                int cur_b = -1;
+                uint32_t pc = 0;
+                int tb = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
+                int tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
+                for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                    if (tb != cur_b) {
+                        ok = wait_bar(&ctrl->ring_empty[0], (pc & 1u) ^ 1u, ctrl, p.status);
+                        if (!ok) break;
+                        const uint32_t full = ptx::smem_u32(&ctrl->ring_full[0]);
+                        ptx::mbar_arrive_expect_tx(full, static_cast<uint32_t>(p.nchunks) * C_CHUNK_BYTES + AUG_B_BYTES);
+                        for (int c = 0; c < p.nchunks; ++c)
+                            ptx::tma_load_3d(ring_base + c * p.stage_bytes, &tmap_c, full, c * KCHUNK, 0, tb);
+                        ptx::bulk_load(ring_base + (p.nchunks - 1) * p.stage_bytes + C_CHUNK_BYTES,
+                                       p.caug + static_cast<size_t>(tb) * AUG_B_BYTES, AUG_B_BYTES, full);
+                        cur_b = tb;
+                        ++pc;
+                    }
+                    tmt += static_cast<int>(gridDim.x);
+                    while (tmt >= p.m_tiles) { tmt -= p.m_tiles; ++tb; }
+                }
+                if (!ok || pc == 0) {
+                } else {
+                    // leave only when the last load has landed (bounded)
+                    const uint64_t t0 = ptx::globaltimer_ns();
+                    while (!ptx::mbar_try_wait(ptx::smem_u32(&ctrl->ring_full[0]), (pc - 1u) & 1u) &&
+                           ptx::globaltimer_ns() - t0 < 100000000ull) {
+                    }
+                }
+            } else {
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 const int b = static_cast<int>(tile / p.m_tiles);
                 if (!XLOAD) prefetch_x();
@@ -373,6 +410,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                            ptx::globaltimer_ns() - t0 < 100000000ull) {
                     }
                 }
+            }
             }
         }
     } else if (XLOAD && warp == XLOAD_WARP) {
@@ -426,6 +464,74 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             uint32_t turn = 0;                              // acc_it mod n_iss
             uint32_t rel0 = 0, rel1 = 0;                    // releases of accumulator 0 / 1 this issuer has consumed
             bool ok = true;
+            if (XLOAD && p.res_c) {
+                // Resident centroids, one tile per row tile: issuer i takes the row tiles with
+                // tile_it % 2 == i, and with them accumulator i and the X buffers of its parity (their
+                // number is even): every barrier it waits on has phases only it consumes.  The two meet
+                // only when the problem changes: each hands the centroid buffer back once its own MMAs
+                // on it are done, and waits for the next problem's centroids.
+                int cur_b = -1;
+                uint32_t pc = 0, tile_it = 0;
+                int tb = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
+                int tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
+                const uint32_t nxb = static_cast<uint32_t>(p.n_xbuf);
+                for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
+                    const int b_now = tb;
+                    tmt += static_cast<int>(gridDim.x);
+                    while (tmt >= p.m_tiles) { tmt -= p.m_tiles; ++tb; }
+                    if (b_now != cur_b) {
+                        if (cur_b >= 0) ptx::umma_commit(ptx::smem_u32(&ctrl->ring_empty[0]));
+                        ok = wait_bar(&ctrl->ring_full[0], pc & 1u, ctrl, p.status);
+                        if (!ok) break;
+                        cur_b = b_now;
+                        ++pc;
+                    }
+                    if ((tile_it & 1u) != iss) continue;
+                    const uint32_t rxb = tile_it % nxb, rxph = (tile_it / nxb) & 1u;
+                    ok = wait_bar(&ctrl->x_full[rxb], rxph, ctrl, p.status);
+                    if (!ok) break;
+                    const uint32_t use = tile_it >> 1;          // how often this accumulator has been used before
+                    if (use > 0u) {
+                        ok = wait_bar(&ctrl->tmem_empty[iss][iss], (use - 1u) & 1u, ctrl, p.status);
+                        if (!ok) break;
+                    }
+                    // The two issuers hand the tensor pipe to each other tile by tile.  Left alone they fall
+                    // into step (X tiles arrive in pairs), their MMAs interleave instruction by instruction,
+                    // both accumulators complete together and both epilogue warpgroups then work while
+                    // the pipe idles.  In turns, one tile's MMAs run while the other tile is being reduced.
+                    if (tile_it > 0u) {
+                        ok = wait_bar(&ctrl->turn[iss], ((tile_it - 1u) >> 1) & 1u, ctrl, p.status);
+                        if (!ok) break;
+                    }
+                    ptx::tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + iss * BLOCK_N;
+                    uint32_t a_lo = ptx::umma_desc_lo_sw128(x_base + rxb * xbuf_bytes);
+                    for (int c = 0; c < p.nchunks; ++c, a_lo += X_CHUNK_BYTES >> 4) {
+                        const uint32_t b_lo = ptx::umma_desc_lo_sw128(ring_base + c * p.stage_bytes);
+                        const int nk = (c == p.nchunks - 1) ? p.ksteps_last : KCHUNK / UMMA_K;
+                        if (c == 0)
+                            ptx::umma_bf16_lohi<false>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
+                                                       ptx::UMMA_DESC_HI_SW128, idesc_main);
+                        else
+                            ptx::umma_bf16_lohi<true>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
+                                                      ptx::UMMA_DESC_HI_SW128, idesc_main);
+                        for (int ks = 1; ks < nk; ++ks)
+                            ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
+                                                      b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main);
+                    }
+                    ptx::mbar_arrive(ptx::smem_u32(&ctrl->turn[iss ^ 1u]));
+                    ok = wait_bar(&ctrl->auga_full[rxb], rxph, ctrl, p.status);
+                    if (!ok) break;
+                    ptx::umma_bf16_lohi<true>(d_tmem,
+                                              ptx::umma_desc_lo_aug(smem_base + auga_off + rxb * AUG_A_BYTES, smem_base + zero_off),
+                                              ptx::UMMA_DESC_HI_AUG,
+                                              ptx::umma_desc_lo_aug(ring_base + (p.nchunks - 1) * p.stage_bytes + C_CHUNK_BYTES,
+                                                                    smem_base + zero_off),
+                                              ptx::UMMA_DESC_HI_AUG, idesc_aug);
+                    ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[iss]));
+                    ptx::umma_commit(ptx::smem_u32(&ctrl->x_empty[rxb]));
+                }
+            } else
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 // every phase of the shared barriers is observed, also in row / centroid tiles this
                 // issuer has no work in: a parity wait must never fall two phases behind
@@ -579,7 +685,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         int dsum_b = -1;
         // one fp64 atomic per warp and problem
         auto flush_inertia = [&]() {
-            if (wg == 0 && p.inertia && dsum_b >= 0) {
+            if ((wg == 0 || p.alt_epi) && p.inertia && dsum_b >= 0) {
                 double t = dsum;
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
@@ -594,7 +700,117 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             mt += static_cast<int>(gridDim.x);
             while (mt >= p.m_tiles) { mt -= p.m_tiles; ++b; }
         };
-        for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
+        // One centroid tile per row tile: accumulator, X buffer and warpgroup all alternate with the row
+        // tile.  Warpgroup g takes the row tiles with tile_it % 2 == g and reads all 256 columns of their
+        // accumulator (two passes of 128), so nothing is merged through shared memory and neither
+        // warpgroup ever waits for the other; with an even number of X buffers each warpgroup sees every
+        // phase of the barriers of "its" buffers.
+        for (i64 tile = blockIdx.x; p.alt_epi && ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
+            if ((tile_it & 1u) != static_cast<uint32_t>(wg)) continue;
+            if (b != dsum_b) {
+                flush_inertia();
+                dsum_b = b;
+            }
+            const uint32_t as = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+            ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            const uint32_t axb = tile_it % static_cast<uint32_t>(p.n_xbuf);
+            const uint32_t axph = (tile_it / static_cast<uint32_t>(p.n_xbuf)) & 1u;
+            ok = wait_bar(&ctrl->auga_full[axb], axph, ctrl, p.status);
+            if (!ok) break;
+            const int rowE = ctrl->row_e[axb][r];
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
+            float best = __uint_as_float(F32_INF);
+            int bsel = 0;
+            {
+                // lower 128 columns into registers; then every 32-column group is reduced and its
+                // registers take the matching group of the upper half at once: the accumulator goes
+                // back to its issuer after one and a half passes instead of two
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + as * BLOCK_N;
+                uint32_t ra[32], rb[32], rc[32], rd[32];
+                ptx::tmem_ld_x32(taddr, ra);
+                ptx::tmem_ld_x32(taddr + 32, rb);
+                ptx::tmem_ld_x32(taddr + 64, rc);
+                ptx::tmem_ld_x32(taddr + 96, rd);
+                ptx::tmem_ld_wait(ra);
+                ptx::reg_dep(rb);
+                ptx::reg_dep(rc);
+                ptx::reg_dep(rd);
+                float lo_min = 0.f;
+                if (PACKED) {
+                    lo_min = packed_min32(ra, 0, __uint_as_float(F32_INF));
+                    ptx::tmem_ld_x32(taddr + 128, ra);
+                    lo_min = packed_min32(rb, 32, lo_min);
+                    ptx::tmem_ld_x32(taddr + 160, rb);
+                    lo_min = packed_min32(rc, 64, lo_min);
+                    ptx::tmem_ld_x32(taddr + 192, rc);
+                    lo_min = packed_min32(rd, 96, lo_min);
+                    ptx::tmem_ld_x32(taddr + 224, rd);
+                } else {
+                    exact_scan32(ra, 0, best, bsel);
+                    ptx::tmem_ld_x32(taddr + 128, ra);
+                    exact_scan32(rb, 32, best, bsel);
+                    ptx::tmem_ld_x32(taddr + 160, rb);
+                    exact_scan32(rc, 64, best, bsel);
+                    ptx::tmem_ld_x32(taddr + 192, rc);
+                    exact_scan32(rd, 96, best, bsel);
+                    ptx::tmem_ld_x32(taddr + 224, rd);
+                }
+                ptx::tmem_ld_wait(ra);
+                ptx::reg_dep(rb);
+                ptx::reg_dep(rc);
+                ptx::reg_dep(rd);
+                ptx::tc_fence_before();
+                __syncwarp();
+                // to the issuer of row tile tile_it + 2, which takes this accumulator next
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][(tile_it + 2u) % n_iss]));
+                if (PACKED) {
+                    float hi_min = packed_min32(ra, 0, __uint_as_float(F32_INF));
+                    hi_min = packed_min32(rb, 32, hi_min);
+                    hi_min = packed_min32(rc, 64, hi_min);
+                    hi_min = packed_min32(rd, 96, hi_min);
+                    // across the halves only the (truncated) value decides: an equal value keeps the lower half
+                    best = lo_min;
+                    bsel = 0;
+                    if (__uint_as_float(__float_as_uint(hi_min) & ~COL_MASK) <
+                        __uint_as_float(__float_as_uint(lo_min) & ~COL_MASK)) {
+                        best = hi_min;
+                        bsel = 1;
+                    }
+                } else {
+                    exact_scan32(ra, 128, best, bsel);
+                    exact_scan32(rb, 160, best, bsel);
+                    exact_scan32(rc, 192, best, bsel);
+                    exact_scan32(rd, 224, best, bsel);
+                }
+            }
+            float bval;
+            int bidx;
+            if (PACKED) {
+                const uint32_t kb = __float_as_uint(best);
+                bval = __uint_as_float(kb & ~COL_MASK);
+                bidx = bsel * (BLOCK_N / 2) + static_cast<int>(kb & COL_MASK);
+            } else {
+                bval = best;
+                bidx = bsel;
+            }
+            const i64 row = static_cast<i64>(mt) * BLOCK_M + r;
+            if (row < p.N) {
+                const size_t o = static_cast<size_t>(b) * static_cast<size_t>(p.N) + row;
+                const uint32_t E = static_cast<uint32_t>(rowE);
+                const uint32_t fx = PACKED ? (__float_as_uint(bval) >> 7) - ((E & 3u) << 23)
+                                           : __float_as_uint(bval) - (E << 23);
+                const float half = fmaf(static_cast<float>(fx), __uint_as_float((E - 23u) << 23),
+                                        -__uint_as_float((E - 12u) << 23));
+                const float dist = fmaxf(0.f, 2.f * half);
+                p.out_idx[o] = bidx;
+                if (p.out_dist) p.out_dist[o] = dist;
+                dsum += static_cast<double>(dist);
+            }
+        }
+        for (i64 tile = blockIdx.x; !p.alt_epi && ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
             if (b != dsum_b) {
                 flush_inertia();
                 dsum_b = b;
@@ -907,8 +1123,6 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     }
     if (stages < 2) return CAKE_ERR_UNSUPPORTED;
     p.n_stages = static_cast<int>(stages > MAX_STAGES ? MAX_STAGES : stages);
-    const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf +
-                              static_cast<size_t>(p.n_stages) * p.stage_bytes;
 
     CUtensorMap tx, tc;
     rc = make_tmap(&tx, X, D, N, B, BLOCK_M);
@@ -918,6 +1132,25 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
 
     // one or two centroid tiles per row tile: the kernel is as fast as X arrives, X gets its own producer
     const bool xload = p.n_tiles <= 2;
+    p.alt_epi = 0;   // without resident centroids (D = 256) the shared epilogue measured faster
+    p.res_c = 0;
+    if (p.n_tiles == 1) {
+        // a single centroid tile: keep it in shared memory if an even number of X buffers fits beside it
+        const i64 c_bytes = static_cast<i64>(p.nchunks) * (C_CHUNK_BYTES + AUG_B_BYTES);
+        for (int nx = MAX_XBUF; nx >= 2; nx -= 2) {
+            if (c_bytes + nx * xbuf <= budget) {
+                p.res_c = 1;
+                p.alt_epi = 1;
+                p.cps = 1;
+                p.stage_bytes = C_CHUNK_BYTES + AUG_B_BYTES;
+                p.n_stages = p.nchunks;
+                p.n_xbuf = nx;
+                break;
+            }
+        }
+    }
+    const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf +
+                              static_cast<size_t>(p.n_stages) * p.stage_bytes;
     using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const Params);
     Kernel kernel = exact ? (xload ? assign_tc_kernel<false, true> : assign_tc_kernel<false, false>)
                           : (xload ? assign_tc_kernel<true, true> : assign_tc_kernel<true, false>);
