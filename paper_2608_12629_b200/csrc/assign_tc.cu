@@ -81,8 +81,11 @@ constexpr uint32_t WAIT_SLICE_NS = 20000;   // longest single sleep inside a wai
 constexpr uint32_t COL_MASK = 0x7Fu;   // packed policy: 7 bits address the 128 columns of a half tile
 constexpr uint32_t F32_INF = 0x7f800000u;
 
+// (The two flags sit in what would be padding: a larger Params measurably slowed the many-tile kernel down,
+// 3-6 %, whatever the order of the members.)
 struct Params {
     int B;
+    int alt_epi;      // one centroid tile per row tile: the two epilogue warpgroups take whole row tiles in turn
     i64 N;
     int D, K;
     int nchunks;      // ceil(D / 64)
@@ -94,9 +97,6 @@ struct Params {
     int cps;          // centroid chunks per ring stage: 2 when nchunks is even (half the barrier traffic), else 1
     uint32_t stage_bytes;   // cps * 32 KiB + 4 KiB
     int n_xbuf;       // X buffers (1..4)
-    int alt_epi;      // one centroid tile per row tile: the two epilogue warpgroups take whole row tiles in turn
-    int res_c;        // ... and the centroid tile stays in shared memory (loaded once per problem): the two
-                      // issuers share no ring and each works on its own row tiles only (implies alt_epi)
     const uint8_t* caug;  // [B][n_tiles][4 KiB] centroid-side operand of the extra k-step
     int* cnmax;           // [B] bit pattern of max_k ||c_k||^2 (fp32, >= 0)
     int* ticket;          // optional: CTAs that have finished; the last one clears cnmax and the ticket
@@ -104,6 +104,8 @@ struct Params {
     float* out_dist;
     double* inertia;      // optional: inertia[b * inertia_stride] += sum of the problem's distances
     int inertia_stride;
+    int res_c;        // alt_epi and the centroid tile stays in shared memory (loaded once per problem): the two
+                      // issuers share no ring and each works on its own row tiles only
     int* status;
 };
 
@@ -116,7 +118,7 @@ struct Ctrl {  // lives in shared memory
     uint64_t tmem_empty[2][MAX_ISSUERS];
     uint64_t auga_full[MAX_XBUF];
     uint64_t merge_full[2], merge_empty[2];
-    uint64_t turn[2];   // resident-centroid mode: issuer i may issue its next tile's MMAs (the other one has issued its own)
+    uint64_t turn[MAX_ISSUERS];   // resident-centroid mode: issuer i may issue its next tile's MMAs (the other one has issued its own)
     uint32_t tmem_base;
     int abort_flag;
     float merge_best[2][BLOCK_M];
@@ -265,17 +267,17 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         for (int i = 0; i < MAX_XBUF; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
             // MMA issuers + 4 norm warps + the 4 epilogue warps that read the row exponents
-            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), (p.res_c ? 1 : NUM_ISSUERS) + 4 + 4);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), ((XLOAD && p.res_c) ? 1 : NUM_ISSUERS) + 4 + 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1);
             for (int j = 0; j < MAX_ISSUERS; ++j)
-                ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i][j]), p.alt_epi ? NUM_EPI_WARPS / 2 : NUM_EPI_WARPS);
+                ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i][j]), (XLOAD && p.alt_epi) ? NUM_EPI_WARPS / 2 : NUM_EPI_WARPS);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_full[i]), 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_empty[i]), 4);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->turn[i]), 1);
         }
+        for (int i = 0; i < MAX_ISSUERS; ++i) ptx::mbar_init(ptx::smem_u32(&ctrl->turn[i]), 1);
         for (int i = 0; i < MAX_STAGES; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_empty[i]), NUM_ISSUERS);   // the consuming issuer and those passing over
@@ -685,7 +687,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         int dsum_b = -1;
         // one fp64 atomic per warp and problem
         auto flush_inertia = [&]() {
-            if ((wg == 0 || p.alt_epi) && p.inertia && dsum_b >= 0) {
+            if ((wg == 0 || (XLOAD && p.alt_epi)) && p.inertia && dsum_b >= 0) {
                 double t = dsum;
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
@@ -705,7 +707,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // accumulator (two passes of 128), so nothing is merged through shared memory and neither
         // warpgroup ever waits for the other; with an even number of X buffers each warpgroup sees every
         // phase of the barriers of "its" buffers.
-        for (i64 tile = blockIdx.x; p.alt_epi && ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
+        for (i64 tile = blockIdx.x; XLOAD && p.alt_epi && ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
             if ((tile_it & 1u) != static_cast<uint32_t>(wg)) continue;
             if (b != dsum_b) {
                 flush_inertia();
@@ -810,7 +812,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 dsum += static_cast<double>(dist);
             }
         }
-        for (i64 tile = blockIdx.x; !p.alt_epi && ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
+        for (i64 tile = blockIdx.x; !(XLOAD && p.alt_epi) && ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
             if (b != dsum_b) {
                 flush_inertia();
                 dsum_b = b;
