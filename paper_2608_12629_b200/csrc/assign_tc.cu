@@ -26,7 +26,10 @@
 //                      of two 256-column TMEM accumulators); tcgen05.commit frees ring slots and
 //                      publishes finished accumulators.
 //                      With one or two centroid tiles per row tile a second instantiation makes
-//                      warp 11 a producer for the X tiles alone and keeps two issuers.
+//                      warp 11 a producer for the X tiles alone and keeps two issuers.  With a single
+//                      centroid tile (K <= 256) that fits beside an even number of X buffers, the tile
+//                      stays in shared memory (loaded once per problem) and row tiles alternate between
+//                      the two issuers and between the two epilogue warpgroups (see the kernel).
 //   warps 0-7 epilogue: warp w reads TMEM lanes 32*(w%4).. (one X row per thread) and columns
 //                      128*(w/4).. of every tile with tcgen05.ld and keeps a running minimum per row.
 //                      The two column halves are merged through shared memory per row tile.
