@@ -34,9 +34,9 @@ from paper_2608_12629_b200 import inputs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel (assign_tc_kernel),
 # from the ncu capture summarised in profiles/assign_tc_kernel_c2.md (same workload, same launch shape)
-NCU_DRAM_BYTES_PER_ASSIGN_LAUNCH = {"c2": 268772352 + 8958464}
+NCU_DRAM_BYTES_PER_ASSIGN_LAUNCH = {"c2": 268921088 + 9016832}
 # the same for the dominant update kernel (slab_update_kernel), profiles/update_slab_route_c2.md
-NCU_DRAM_BYTES_PER_UPDATE_LAUNCH = {"c2": 273207040 + 4733952}
+NCU_DRAM_BYTES_PER_UPDATE_LAUNCH = {"c2": 273203712 + 4012032}
 
 METRIC = "lloyd_iters_per_sec"
 UNIT = "iter/s"
