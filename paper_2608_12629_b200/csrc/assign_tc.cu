@@ -88,7 +88,8 @@ constexpr uint32_t F32_INF = 0x7f800000u;
 // 3-6 %, whatever the order of the members.)
 struct Params {
     int B;
-    int alt_epi;      // one centroid tile per row tile: the two epilogue warpgroups take whole row tiles in turn
+    int alt_epi;      // one centroid tile per row tile: the two epilogue warpgroups take whole row tiles in turn;
+                      // the value is the number of accumulator columns in use (32..128, or 256)
     i64 N;
     int D, K;
     int nchunks;      // ceil(D / 64)
@@ -480,6 +481,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 int tb = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
                 int tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
                 const uint32_t nxb = static_cast<uint32_t>(p.n_xbuf);
+                const uint32_t idesc_aug_n = ptx::umma_idesc_bf16(BLOCK_M, p.alt_epi);
+                const uint32_t idesc_main_n = idesc_aug_n | ptx::UMMA_IDESC_NEGATE_B;
                 for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
                     const int b_now = tb;
                     tmt += static_cast<int>(gridDim.x);
@@ -516,13 +519,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         const int nk = (c == p.nchunks - 1) ? p.ksteps_last : KCHUNK / UMMA_K;
                         if (c == 0)
                             ptx::umma_bf16_lohi<false>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
-                                                       ptx::UMMA_DESC_HI_SW128, idesc_main);
+                                                       ptx::UMMA_DESC_HI_SW128, idesc_main_n);
                         else
                             ptx::umma_bf16_lohi<true>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
-                                                      ptx::UMMA_DESC_HI_SW128, idesc_main);
+                                                      ptx::UMMA_DESC_HI_SW128, idesc_main_n);
                         for (int ks = 1; ks < nk; ++ks)
                             ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
-                                                      b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main);
+                                                      b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main_n);
                     }
                     ptx::mbar_arrive(ptx::smem_u32(&ctrl->turn[iss ^ 1u]));
                     ok = wait_bar(&ctrl->auga_full[rxb], rxph, ctrl, p.status);
@@ -532,7 +535,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                               ptx::UMMA_DESC_HI_AUG,
                                               ptx::umma_desc_lo_aug(ring_base + (p.nchunks - 1) * p.stage_bytes + C_CHUNK_BYTES,
                                                                     smem_base + zero_off),
-                                              ptx::UMMA_DESC_HI_AUG, idesc_aug);
+                                              ptx::UMMA_DESC_HI_AUG, idesc_aug_n);
                     ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[iss]));
                     ptx::umma_commit(ptx::smem_u32(&ctrl->x_empty[rxb]));
                 }
@@ -729,7 +732,35 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
             float best = __uint_as_float(F32_INF);
             int bsel = 0;
-            {
+            if (p.alt_epi <= BLOCK_N / 2) {
+                // at most 128 centroids: only the 32-column groups that hold some were written
+                const int ng = p.alt_epi >> 5;
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + as * BLOCK_N;
+                uint32_t ra[32], rb[32], rc[32], rd[32];
+                ptx::tmem_ld_x32(taddr, ra);
+                if (ng > 1) ptx::tmem_ld_x32(taddr + 32, rb);
+                if (ng > 2) ptx::tmem_ld_x32(taddr + 64, rc);
+                if (ng > 3) ptx::tmem_ld_x32(taddr + 96, rd);
+                ptx::tmem_ld_wait(ra);
+                ptx::reg_dep(rb);
+                ptx::reg_dep(rc);
+                ptx::reg_dep(rd);
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][(tile_it + 2u) % n_iss]));
+                if (PACKED) {
+                    best = packed_min32(ra, 0, __uint_as_float(F32_INF));
+                    if (ng > 1) best = packed_min32(rb, 32, best);
+                    if (ng > 2) best = packed_min32(rc, 64, best);
+                    if (ng > 3) best = packed_min32(rd, 96, best);
+                    bsel = 0;
+                } else {
+                    exact_scan32(ra, 0, best, bsel);
+                    if (ng > 1) exact_scan32(rb, 32, best, bsel);
+                    if (ng > 2) exact_scan32(rc, 64, best, bsel);
+                    if (ng > 3) exact_scan32(rd, 96, best, bsel);
+                }
+            } else {
                 // lower 128 columns into registers; then every 32-column group is reduced and its
                 // registers take the matching group of the upper half at once: the accumulator goes
                 // back to its issuer after one and a half passes instead of two
@@ -1145,7 +1176,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         for (int nx = MAX_XBUF; nx >= 2; nx -= 2) {
             if (c_bytes + nx * xbuf <= budget) {
                 p.res_c = 1;
-                p.alt_epi = 1;
+                // its value: the accumulator columns the MMAs write and the epilogue reads (K <= 128: only
+                // the 32-column groups that hold centroids; the tensor pipe and the epilogue do less)
+                p.alt_epi = K <= BLOCK_N / 2 ? static_cast<int>(round_up(K, 32)) : BLOCK_N;
                 p.cps = 1;
                 p.stage_bytes = C_CHUNK_BYTES + AUG_B_BYTES;
                 p.n_stages = p.nchunks;
