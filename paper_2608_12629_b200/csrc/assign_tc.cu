@@ -719,10 +719,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 flush_inertia();
                 dsum_b = b;
             }
-            const uint32_t as = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-            ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
-            if (!ok) break;
-            ptx::tc_fence_after();
+            // the row exponents are there long before the accumulator is: fetch them while waiting for it
+            // (the X buffer is not refilled before the issuer's MMAs on it have completed either)
             const uint32_t axb = tile_it % static_cast<uint32_t>(p.n_xbuf);
             const uint32_t axph = (tile_it / static_cast<uint32_t>(p.n_xbuf)) & 1u;
             ok = wait_bar(&ctrl->auga_full[axb], axph, ctrl, p.status);
@@ -730,6 +728,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const int rowE = ctrl->row_e[axb][r];
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
+            const uint32_t as = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+            ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
+            if (!ok) break;
+            ptx::tc_fence_after();
             float best = __uint_as_float(F32_INF);
             int bsel = 0;
             if (p.alt_epi <= BLOCK_N / 2) {
