@@ -355,10 +355,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         ok = wait_bar(&ctrl->ring_empty[0], (pc & 1u) ^ 1u, ctrl, p.status);
                         if (!ok) break;
                         const uint32_t full = ptx::smem_u32(&ctrl->ring_full[0]);
-                        ptx::mbar_arrive_expect_tx(full, static_cast<uint32_t>(p.nchunks) * C_CHUNK_BYTES + AUG_B_BYTES);
+                        ptx::mbar_arrive_expect_tx(full, static_cast<uint32_t>(p.nchunks) * (p.stage_bytes - AUG_B_BYTES) + AUG_B_BYTES);
                         for (int c = 0; c < p.nchunks; ++c)
                             ptx::tma_load_3d(ring_base + c * p.stage_bytes, &tmap_c, full, c * KCHUNK, 0, tb);
-                        ptx::bulk_load(ring_base + (p.nchunks - 1) * p.stage_bytes + C_CHUNK_BYTES,
+                        ptx::bulk_load(ring_base + p.nchunks * p.stage_bytes - AUG_B_BYTES,
                                        p.caug + static_cast<size_t>(tb) * AUG_B_BYTES, AUG_B_BYTES, full);
                         cur_b = tb;
                         ++pc;
@@ -533,7 +533,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     ptx::umma_bf16_lohi<true>(d_tmem,
                                               ptx::umma_desc_lo_aug(smem_base + auga_off + rxb * AUG_A_BYTES, smem_base + zero_off),
                                               ptx::UMMA_DESC_HI_AUG,
-                                              ptx::umma_desc_lo_aug(ring_base + (p.nchunks - 1) * p.stage_bytes + C_CHUNK_BYTES,
+                                              ptx::umma_desc_lo_aug(ring_base + p.nchunks * p.stage_bytes - AUG_B_BYTES,
                                                                     smem_base + zero_off),
                                               ptx::UMMA_DESC_HI_AUG, idesc_aug_n);
                     ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[iss]));
@@ -1165,30 +1165,34 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     CUtensorMap tx, tc;
     rc = make_tmap(&tx, X, D, N, B, BLOCK_M);
     if (rc != CAKE_OK) return rc;
-    rc = make_tmap(&tc, C, D, K, B, BLOCK_N);
-    if (rc != CAKE_OK) return rc;
 
     // one or two centroid tiles per row tile: the kernel is as fast as X arrives, X gets its own producer
     const bool xload = p.n_tiles <= 2;
     p.alt_epi = 0;   // without resident centroids (D = 256) the shared epilogue measured faster
     p.res_c = 0;
+    int c_rows = BLOCK_N;   // rows of a centroid chunk in shared memory (the TMA box)
     if (p.n_tiles == 1) {
         // a single centroid tile: keep it in shared memory if an even number of X buffers fits beside it
-        const i64 c_bytes = static_cast<i64>(p.nchunks) * (C_CHUNK_BYTES + AUG_B_BYTES);
+        // (of the tile only the rows that hold centroids, in steps of 32, when there are at most 128)
+        c_rows = K <= BLOCK_N / 2 ? static_cast<int>(round_up(K, 32)) : BLOCK_N;
+        const i64 c_bytes = static_cast<i64>(p.nchunks) * (c_rows * 128 + AUG_B_BYTES);
         for (int nx = MAX_XBUF; nx >= 2; nx -= 2) {
             if (c_bytes + nx * xbuf <= budget) {
                 p.res_c = 1;
                 // its value: the accumulator columns the MMAs write and the epilogue reads (K <= 128: only
                 // the 32-column groups that hold centroids; the tensor pipe and the epilogue do less)
-                p.alt_epi = K <= BLOCK_N / 2 ? static_cast<int>(round_up(K, 32)) : BLOCK_N;
+                p.alt_epi = c_rows;
                 p.cps = 1;
-                p.stage_bytes = C_CHUNK_BYTES + AUG_B_BYTES;
+                p.stage_bytes = static_cast<uint32_t>(c_rows) * 128u + AUG_B_BYTES;
                 p.n_stages = p.nchunks;
                 p.n_xbuf = nx;
                 break;
             }
         }
     }
+    if (!p.res_c) c_rows = BLOCK_N;
+    rc = make_tmap(&tc, C, D, K, B, c_rows);
+    if (rc != CAKE_OK) return rc;
     const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf +
                               static_cast<size_t>(p.n_stages) * p.stage_bytes;
     using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const Params);
