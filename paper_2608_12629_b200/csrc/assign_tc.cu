@@ -271,7 +271,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         for (int i = 0; i < MAX_XBUF; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
             // MMA issuers + 4 norm warps + the 4 epilogue warps that read the row exponents
-            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), ((XLOAD && p.res_c) ? 1 : NUM_ISSUERS) + 4 + 4);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), ((XLOAD && p.res_c == 1) ? 1 : NUM_ISSUERS) + 4 + 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
         }
         for (int i = 0; i < 2; ++i) {
@@ -355,11 +355,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         ok = wait_bar(&ctrl->ring_empty[0], (pc & 1u) ^ 1u, ctrl, p.status);
                         if (!ok) break;
                         const uint32_t full = ptx::smem_u32(&ctrl->ring_full[0]);
-                        ptx::mbar_arrive_expect_tx(full, static_cast<uint32_t>(p.nchunks) * (p.stage_bytes - AUG_B_BYTES) + AUG_B_BYTES);
-                        for (int c = 0; c < p.nchunks; ++c)
-                            ptx::tma_load_3d(ring_base + c * p.stage_bytes, &tmap_c, full, c * KCHUNK, 0, tb);
-                        ptx::bulk_load(ring_base + p.nchunks * p.stage_bytes - AUG_B_BYTES,
-                                       p.caug + static_cast<size_t>(tb) * AUG_B_BYTES, AUG_B_BYTES, full);
+                        // (res_c = 2: two centroid tiles, one behind the other)
+                        ptx::mbar_arrive_expect_tx(full, static_cast<uint32_t>(p.res_c) *
+                                                             (static_cast<uint32_t>(p.nchunks) * (p.stage_bytes - AUG_B_BYTES) + AUG_B_BYTES));
+                        for (int j = 0; j < p.res_c; ++j) {
+                            const uint32_t tbase = ring_base + j * p.nchunks * p.stage_bytes;
+                            for (int c = 0; c < p.nchunks; ++c)
+                                ptx::tma_load_3d(tbase + c * p.stage_bytes, &tmap_c, full, c * KCHUNK, j * BLOCK_N, tb);
+                            ptx::bulk_load(tbase + p.nchunks * p.stage_bytes - AUG_B_BYTES,
+                                           p.caug + (static_cast<size_t>(tb) * p.res_c + j) * AUG_B_BYTES, AUG_B_BYTES, full);
+                        }
                         cur_b = tb;
                         ++pc;
                     }
@@ -481,7 +486,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 int tb = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
                 int tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
                 const uint32_t nxb = static_cast<uint32_t>(p.n_xbuf);
-                const uint32_t idesc_aug_n = ptx::umma_idesc_bf16(BLOCK_M, p.alt_epi);
+                const uint32_t idesc_aug_n = ptx::umma_idesc_bf16(BLOCK_M, p.alt_epi ? p.alt_epi : BLOCK_N);
                 const uint32_t idesc_main_n = idesc_aug_n | ptx::UMMA_IDESC_NEGATE_B;
                 for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
                     const int b_now = tb;
@@ -494,11 +499,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         cur_b = b_now;
                         ++pc;
                     }
-                    if ((tile_it & 1u) != iss) continue;
+                    // two resident tiles: issuer i computes centroid tile i of EVERY row tile into accumulator i
+                    // (the shared epilogue reads both and merges)
+                    const bool both = p.res_c == 2;
+                    if (!both && (tile_it & 1u) != iss) continue;
                     const uint32_t rxb = tile_it % nxb, rxph = (tile_it / nxb) & 1u;
                     ok = wait_bar(&ctrl->x_full[rxb], rxph, ctrl, p.status);
                     if (!ok) break;
-                    const uint32_t use = tile_it >> 1;          // how often this accumulator has been used before
+                    const uint32_t use = both ? tile_it : tile_it >> 1;   // how often this accumulator has been used before
                     if (use > 0u) {
                         ok = wait_bar(&ctrl->tmem_empty[iss][iss], (use - 1u) & 1u, ctrl, p.status);
                         if (!ok) break;
@@ -507,15 +515,19 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     // into step (X tiles arrive in pairs), their MMAs interleave instruction by instruction,
                     // both accumulators complete together and both epilogue warpgroups then work while
                     // the pipe idles.  In turns, one tile's MMAs run while the other tile is being reduced.
-                    if (tile_it > 0u) {
-                        ok = wait_bar(&ctrl->turn[iss], ((tile_it - 1u) >> 1) & 1u, ctrl, p.status);
+                    // (order of the groups of MMAs: one tile: t0 t1 t2 ..., issuers alternating; two tiles: t0/A t0/B
+                    // t1/A t1/B ...; issuer 0 waits for issuer 1's previous group, issuer 1 for issuer 0's current one)
+                    if (both ? (iss == 1u || tile_it > 0u) : tile_it > 0u) {
+                        const uint32_t tph = both ? (iss == 0u ? tile_it - 1u : tile_it) : (tile_it - 1u) >> 1;
+                        ok = wait_bar(&ctrl->turn[iss], tph & 1u, ctrl, p.status);
                         if (!ok) break;
                     }
                     ptx::tc_fence_after();
                     const uint32_t d_tmem = tmem_base + iss * BLOCK_N;
+                    const uint32_t c_base = ring_base + (both ? iss * p.nchunks * p.stage_bytes : 0u);   // this issuer's centroid tile
                     uint32_t a_lo = ptx::umma_desc_lo_sw128(x_base + rxb * xbuf_bytes);
                     for (int c = 0; c < p.nchunks; ++c, a_lo += X_CHUNK_BYTES >> 4) {
-                        const uint32_t b_lo = ptx::umma_desc_lo_sw128(ring_base + c * p.stage_bytes);
+                        const uint32_t b_lo = ptx::umma_desc_lo_sw128(c_base + c * p.stage_bytes);
                         const int nk = (c == p.nchunks - 1) ? p.ksteps_last : KCHUNK / UMMA_K;
                         if (c == 0)
                             ptx::umma_bf16_lohi<false>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
@@ -533,7 +545,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     ptx::umma_bf16_lohi<true>(d_tmem,
                                               ptx::umma_desc_lo_aug(smem_base + auga_off + rxb * AUG_A_BYTES, smem_base + zero_off),
                                               ptx::UMMA_DESC_HI_AUG,
-                                              ptx::umma_desc_lo_aug(ring_base + p.nchunks * p.stage_bytes - AUG_B_BYTES,
+                                              ptx::umma_desc_lo_aug(c_base + p.nchunks * p.stage_bytes - AUG_B_BYTES,
                                                                     smem_base + zero_off),
                                               ptx::UMMA_DESC_HI_AUG, idesc_aug_n);
                     ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[iss]));
@@ -1190,7 +1202,21 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             }
         }
     }
-    if (!p.res_c) c_rows = BLOCK_N;
+    if (p.n_tiles == 2) {
+        // two centroid tiles: both stay in shared memory if at least two X buffers fit beside them (D <= 128)
+        const i64 c_bytes = 2 * static_cast<i64>(p.nchunks) * (C_CHUNK_BYTES + AUG_B_BYTES);
+        for (int nx = MAX_XBUF; nx >= 2; --nx) {
+            if (2 * p.nchunks <= MAX_STAGES && c_bytes + nx * xbuf <= budget) {
+                p.res_c = 2;
+                p.cps = 1;
+                p.stage_bytes = C_CHUNK_BYTES + AUG_B_BYTES;
+                p.n_stages = 2 * p.nchunks;
+                p.n_xbuf = nx;
+                break;
+            }
+        }
+    }
+    if (p.res_c != 1) c_rows = BLOCK_N;
     rc = make_tmap(&tc, C, D, K, B, c_rows);
     if (rc != CAKE_OK) return rc;
     const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf +
