@@ -29,7 +29,8 @@
 //                      warp 11 a producer for the X tiles alone and keeps two issuers.  With a single
 //                      centroid tile (K <= 256) that fits beside an even number of X buffers, the tile
 //                      stays in shared memory (loaded once per problem) and row tiles alternate between
-//                      the two issuers and between the two epilogue warpgroups (see the kernel).
+//                      the two issuers and between the two epilogue warpgroups (see the kernel); two
+//                      centroid tiles (K <= 512, D <= 128) stay resident too, one per issuer.
 //   warps 0-7 epilogue: warp w reads TMEM lanes 32*(w%4).. (one X row per thread) and columns
 //                      128*(w/4).. of every tile with tcgen05.ld and keeps a running minimum per row.
 //                      The two column halves are merged through shared memory per row tile.
@@ -108,8 +109,9 @@ struct Params {
     float* out_dist;
     double* inertia;      // optional: inertia[b * inertia_stride] += sum of the problem's distances
     int inertia_stride;
-    int res_c;        // alt_epi and the centroid tile stays in shared memory (loaded once per problem): the two
-                      // issuers share no ring and each works on its own row tiles only
+    int res_c;        // 1: alt_epi and the centroid tile stays in shared memory (loaded once per problem): the two
+                      // issuers share no ring and each works on its own row tiles only; 2: two resident
+                      // tiles, issuer i computes tile i of every row tile (shared epilogue)
     int* status;
 };
 
