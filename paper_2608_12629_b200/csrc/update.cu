@@ -1393,7 +1393,7 @@ void slab_rows_for(int slots, int B, i64 N, int F, int* S, int* n_ctas) {
         i64 per_problem = static_cast<i64>(w) * slots / B / F * F;
         if (per_problem < F) per_problem = F;
         i64 rows = (N + per_problem - 1) / per_problem;
-        if (rows < 2048) rows = 2048;                       // tiny slabs only add launches of atomics
+        if (rows < 1024) rows = 1024;                       // smaller slabs only add atomics (measured: 512 loses)
         rows = (rows + 3) / 4 * 4;
         if (rows <= SLAB_MAX_ROWS) {
             *S = static_cast<int>(rows);
