@@ -59,7 +59,7 @@ enum {
 
 enum {
     CAKE_ASSIGN_AUTO = 0,
-    CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 256.
+    CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 512.
                                   Distances are compared as fixed-point numbers with a quantum of
                                   about 2^-19 of (|x|^2 + max |c|^2); equal ones go to the lower index */
     CAKE_ASSIGN_SIMT = 2,      /* plain CUDA-core fallback, any D                               */
@@ -71,7 +71,7 @@ enum {
                                   segmented reduction; for K > 8192 and D % 8 == 0 every cluster is
                                   summed and divided by one warp), any K                         */
     CAKE_UPDATE_SLAB = 3 << 4, /* one kernel sorts and reduces slab by slab (thread-block clusters
-                                  when K is large against the slab); D % 8 == 0, D <= 256, K <= 8192 */
+                                  when K is large against the slab); D % 8 == 0, D <= 1024, K <= 8192 */
     CAKE_UPDATE_SLAB_F1 = 4 << 4, /* the same with the cluster size forced to 1, 2 or 4 CTAs      */
     CAKE_UPDATE_SLAB_F2 = 5 << 4,
     CAKE_UPDATE_SLAB_F4 = 6 << 4,

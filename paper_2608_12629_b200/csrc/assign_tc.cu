@@ -1089,7 +1089,7 @@ extern "C" __attribute__((visibility("default"))) int cake_debug_read_trace(int 
 }
 #endif
 
-bool assign_tc_supports(int D) { return D >= 8 && D % 8 == 0 && D <= 256; }
+bool assign_tc_supports(int D) { return D >= 8 && D % 8 == 0 && D <= 512; }
 
 size_t assign_tc_aug_bytes(i64 B, int K) {
     return static_cast<size_t>(B) * (padded_k(K) / BLOCK_N) * AUG_B_BYTES;
@@ -1191,7 +1191,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         c_rows = K <= BLOCK_N / 2 ? static_cast<int>(round_up(K, 32)) : BLOCK_N;
         const i64 c_bytes = static_cast<i64>(p.nchunks) * (c_rows * 128 + AUG_B_BYTES);
         for (int nx = MAX_XBUF; nx >= 2; nx -= 2) {
-            if (c_bytes + nx * xbuf <= budget) {
+            if (p.nchunks <= MAX_STAGES && c_bytes + nx * xbuf <= budget) {
                 p.res_c = 1;
                 // its value: the accumulator columns the MMAs write and the epilogue reads (K <= 128: only
                 // the 32-column groups that hold centroids; the tensor pipe and the epilogue do less)

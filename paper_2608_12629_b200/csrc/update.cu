@@ -1017,47 +1017,50 @@ slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
     const uint32_t rowmask = (1u << rowbits) - 1u;
     const int seglen = max(SLAB_AHEAD, (mine + NGROUPS - 1) / NGROUPS);
     const int base = gid * seglen, end = min(base + seglen, mine);
-    int cur = -1;
-    float acc[8];
+    // rows wider than 32 granules (D > 256) are reduced in column blocks of 32 granules, one pass each
+    for (int sg = sl; sg - sl < G; sg += LPR) {
+        int cur = -1;
+        float acc[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-    auto flush = [&]() {
-        if (cur >= 0 && sl < G) {
-            float4* dst = reinterpret_cast<float4*>(sums_b + static_cast<size_t>(cur) * D + sl * 8);
-            atomicAdd(dst, make_float4(acc[0], acc[1], acc[2], acc[3]));
-            atomicAdd(dst + 1, make_float4(acc[4], acc[5], acc[6], acc[7]));
-        }
-    };
-    for (int q = base; q < end; q += SLAB_AHEAD) {
-        uint4 v[SLAB_AHEAD];
-        int kk[SLAB_AHEAD];
-#pragma unroll
-        for (int u = 0; u < SLAB_AHEAD; ++u) {
-            kk[u] = -1;
-            v[u] = make_uint4(0, 0, 0, 0);
-            if (q + u < end) {
-                const uint32_t rec = sorted[q + u];
-                kk[u] = static_cast<int>(rec >> rowbits);
-                if (sl < G) v[u] = __ldg(Xg + static_cast<size_t>(rec & rowmask) * G + sl);
+        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+        auto flush = [&]() {
+            if (cur >= 0 && sg < G) {
+                float4* dst = reinterpret_cast<float4*>(sums_b + static_cast<size_t>(cur) * D + sg * 8);
+                atomicAdd(dst, make_float4(acc[0], acc[1], acc[2], acc[3]));
+                atomicAdd(dst + 1, make_float4(acc[4], acc[5], acc[6], acc[7]));
             }
-        }
+        };
+        for (int q = base; q < end; q += SLAB_AHEAD) {
+            uint4 v[SLAB_AHEAD];
+            int kk[SLAB_AHEAD];
 #pragma unroll
-        for (int u = 0; u < SLAB_AHEAD; ++u) {
-            if (kk[u] >= 0) {
-                if (kk[u] != cur) {
-                    flush();
-                    cur = kk[u];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+            for (int u = 0; u < SLAB_AHEAD; ++u) {
+                kk[u] = -1;
+                v[u] = make_uint4(0, 0, 0, 0);
+                if (q + u < end) {
+                    const uint32_t rec = sorted[q + u];
+                    kk[u] = static_cast<int>(rec >> rowbits);
+                    if (sg < G) v[u] = __ldg(Xg + static_cast<size_t>(rec & rowmask) * G + sg);
                 }
-                acc[0] += bf16lo(v[u].x); acc[1] += bf16hi(v[u].x);
-                acc[2] += bf16lo(v[u].y); acc[3] += bf16hi(v[u].y);
-                acc[4] += bf16lo(v[u].z); acc[5] += bf16hi(v[u].z);
-                acc[6] += bf16lo(v[u].w); acc[7] += bf16hi(v[u].w);
+            }
+#pragma unroll
+            for (int u = 0; u < SLAB_AHEAD; ++u) {
+                if (kk[u] >= 0) {
+                    if (kk[u] != cur) {
+                        flush();
+                        cur = kk[u];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+                    }
+                    acc[0] += bf16lo(v[u].x); acc[1] += bf16hi(v[u].x);
+                    acc[2] += bf16lo(v[u].y); acc[3] += bf16hi(v[u].y);
+                    acc[4] += bf16lo(v[u].z); acc[5] += bf16hi(v[u].z);
+                    acc[6] += bf16lo(v[u].w); acc[7] += bf16hi(v[u].w);
+                }
             }
         }
+        flush();
     }
-    flush();
 }
 
 // ======================================================================= division
@@ -1354,7 +1357,7 @@ SlabKernel slab_kernel_for(int lpr, bool cluster) {
 
 int slab_lpr(int D) {
     int lpr = 4;
-    while (lpr < D / 8) lpr <<= 1;
+    while (lpr < D / 8 && lpr < 32) lpr <<= 1;
     return lpr;
 }
 
@@ -1405,7 +1408,7 @@ void slab_rows_for(int slots, int B, i64 N, int F, int* S, int* n_ctas) {
 }
 }  // namespace
 
-bool update_slab_supports(int D, int K) { return D % 8 == 0 && D >= 8 && D <= 256 && K <= SLAB_MAX_K; }
+bool update_slab_supports(int D, int K) { return D % 8 == 0 && D >= 8 && D <= 1024 && K <= SLAB_MAX_K; }
 
 static int slab_make_plan(const DeviceInfo& di, int B, i64 N, int D, int K, int force_f, SlabPlan* out) {
     const int lpr = slab_lpr(D);

@@ -33,10 +33,13 @@ def check_status(ws, want=cake.CAKE_OK):
 # ------------------------------------------------------------------------------------ assign
 
 TC_SHAPES = [
-    # N, D, K : single tile, ragged rows, ragged K, several K tiles, D tails (96, 72, 8), D=256
+    # N, D, K : single tile, ragged rows, ragged K, several K tiles, D tails (96, 72, 8), D=256, and
+    # 256 < D <= 512 (one X buffer; five to eight 64-column chunks, full and partial)
     (1, 64, 1), (127, 64, 2), (128, 64, 256), (129, 128, 257), (1000, 128, 1000), (777, 96, 65),
     (4096, 128, 300), (300, 256, 700), (257, 16, 5), (1000, 8, 3), (2000, 72, 260), (333, 192, 513),
     (20000, 64, 128), (50, 128, 2048),
+    (300, 264, 70), (1000, 288, 300), (515, 352, 1000), (2000, 480, 130), (700, 512, 600), (129, 504, 33),
+    (40000, 320, 24),
 ]
 
 
@@ -55,12 +58,12 @@ def test_assign_tcgen05_small_shapes(N, D, K, policy):
     assert rep["mismatch"] <= max(2, N // 1000), rep
 
 
-@pytest.mark.parametrize("N,D,K", [(100, 5, 7), (300, 33, 40), (64, 130, 3), (1000, 64, 100)])
+@pytest.mark.parametrize("N,D,K", [(100, 5, 7), (300, 33, 40), (64, 130, 3), (1000, 64, 100), (200, 520, 9)])
 def test_assign_simt_fallback(N, D, K):
     X, C = problem(N, D, K, seed=N * 3 + D)
     idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_SIMT)
     grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx.cpu().numpy(), dist.cpu().numpy())
-    if D % 8:  # the automatic choice must take the fallback for such D, and the tensor path must refuse
+    if D % 8 or D > 512:  # the automatic choice must take the fallback for such D, and the tensor path must refuse
         idx2, _ = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV))
         assert torch.equal(idx, idx2)
         with pytest.raises(cake.CakeError) as e:
@@ -204,10 +207,12 @@ SLAB_FLAGS = {"auto": cake.CAKE_UPDATE_SLAB, "f1": cake.CAKE_UPDATE_SLAB_F1, "f2
 
 @pytest.mark.parametrize("f", ["auto", "f1", "f2", "f4"])
 @pytest.mark.parametrize("N,D,K", [(1, 64, 1), (1000, 64, 128), (70001, 64, 100), (20000, 128, 3000), (8193, 16, 8192),
-                                   (50003, 96, 17), (300001, 128, 1024), (33000, 256, 512), (2500, 8, 3)])
+                                   (50003, 96, 17), (300001, 128, 1024), (33000, 256, 512), (2500, 8, 3),
+                                   (20001, 288, 500), (9000, 512, 100), (5000, 1000, 64), (3000, 1024, 7)])
 def test_update_slab_route(f, N, D, K):
     """Slab route: ragged last slab, N % 4 != 0, clusters of 1, 2 and 4 CTAs (also with CTAs that get no
-    rows), K at the shared-memory limit, D that does not fill the lane group."""
+    rows), K at the shared-memory limit, D that does not fill the lane group, D > 256 (several column
+    passes, the last one partial)."""
     X, C = problem(N, D, K, seed=N + D)
     g = torch.Generator().manual_seed(K)
     idx = torch.randint(0, K, (N,), generator=g, dtype=torch.int32)
@@ -425,7 +430,8 @@ def test_lloyd_handworked_example_on_gpu():
     assert out.C_bf16.float().cpu()[:, :2].tolist() == [[171 / 256, 171 / 256], [171 / 16, 171 / 16]]
 
 
-@pytest.mark.parametrize("B,N,D,K", [(1, 5000, 64, 37), (2, 3000, 128, 300), (1, 2000, 24, 9), (33, 300, 64, 5), (1, 700, 12, 6)])
+@pytest.mark.parametrize("B,N,D,K", [(1, 5000, 64, 37), (2, 3000, 128, 300), (1, 2000, 24, 9), (33, 300, 64, 5), (1, 700, 12, 6),
+                                       (1, 1500, 320, 40), (2, 900, 512, 300)])
 def test_lloyd_call_equals_stepwise_calls(B, N, D, K):
     """Inside a Lloyd call the division kernel prepares the next assign (half-norm operand, max ||c||^2,
     cleared inertia): the result must be bit-identical to assign and update called one by one, where the

@@ -25,7 +25,7 @@ def test_assign_and_lloyd_random_shapes(seed):
     rnd = random.Random(seed)
     for it in range(25):
         B = rnd.choice([1, 1, 1, 2, 3, 7, 33])
-        D = rnd.choice([8, 16, 24, 32, 40, 64, 72, 96, 128, 136, 192, 200, 256])
+        D = rnd.choice([8, 16, 24, 32, 40, 64, 72, 96, 128, 136, 192, 200, 256, 264, 320, 384, 504, 512])
         K = rnd.choice([1, 2, 3, 17, 31, 32, 33, 64, 65, 100, 127, 128, 129, 200, 255, 256, 257, 300, 511, 512, 513, 700,
                         1000, 1024, 1500])
         N = rnd.choice([1, 5, 127, 128, 129, 300, 1000, 2049, 5000, 20000, 40000, 148 * 128 + 5, 148 * 128 * 2 + 1])
@@ -79,7 +79,7 @@ def test_update_random_shapes_and_index_sets(seed):
             idx[0, 0] = -1
             idx[-1, N // 2] = K
         flag = rnd.choice([0, cake.CAKE_UPDATE_SORT, cake.CAKE_UPDATE_SORT])
-        if flag == 0 and rnd.random() < 0.3 and K <= 8192 and D % 8 == 0 and D <= 256:
+        if flag == 0 and rnd.random() < 0.3 and K <= 8192 and D % 8 == 0 and D <= 1024:
             flag = cake.CAKE_UPDATE_SLAB
         X = inputs.from_bits(rng.integers(0x3C00, 0x4100, size=(B, N, D), dtype=np.uint16))
         prev = None if rnd.random() < 0.3 else inputs.from_bits(rng.integers(0x3C00, 0x4100, size=(B, K, D), dtype=np.uint16))
