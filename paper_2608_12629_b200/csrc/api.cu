@@ -24,6 +24,8 @@ struct Workspace {
     int* rank;            // [B][N] rank of every row inside its cluster (sort route, K > 8192)
     cake_bf16* cbuf[2];   // [B][K][D] each
     float* dist;          // [B][N]
+    cake_bf16* xpad;      // [B][N][padded_d(D)] zero-padded copy of X for the tensor-core assign when D % 8 != 0
+    cake_bf16* cpad;      // [B][K][round_up(D, 64)] zero-padded copy of C it streams when D % 64 != 0
     size_t bytes;
 };
 
@@ -46,6 +48,9 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     w.cbuf[0] = reinterpret_cast<cake_bf16*>(take(kd * 2));
     w.cbuf[1] = reinterpret_cast<cake_bf16*>(take(kd * 2));
     w.dist = reinterpret_cast<float*>(take(static_cast<size_t>(B) * N * 4));
+    const size_t dpad = assign_pad_supports(D) ? static_cast<size_t>(padded_d(D)) : 0;
+    w.xpad = reinterpret_cast<cake_bf16*>(take(static_cast<size_t>(B) * N * dpad * 2));
+    w.cpad = reinterpret_cast<cake_bf16*>(take(static_cast<size_t>(B) * K * assign_cpad_columns(D) * 2));
     w.bytes = o;
     return w;
 }
@@ -70,10 +75,18 @@ int check_ws(void* ws, size_t ws_bytes, i64 B, i64 N, int D, int K, Workspace* o
 // kernel adds it up itself; the fallback needs `dist` (out_dist or scratch) and a reduction kernel.
 // zero_inertia: the entries still have to be cleared (the tensor-core prologue does it on the way).
 // aug_ready: the update ahead prepared this assign (see NextAssign): the tensor-core route skips its prologue
+// x_padded: the workspace already holds the padded copy of this X (an earlier iteration of the call made it)
 int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, int* out_idx,
               float* out_dist, double* inertia, int inertia_stride, bool zero_inertia, bool aug_ready,
-              const Workspace& w, cudaStream_t s, unsigned flags) {
+              bool x_padded, const Workspace& w, cudaStream_t s, unsigned flags) {
     unsigned path = flags & CAKE_ASSIGN_MASK;
+    int Dx = 0;   // columns of the padded copy of X, if one is used
+    if (path == CAKE_ASSIGN_AUTO && assign_pad_supports(D) && N > 0) {
+        Dx = padded_d(D);
+        if (!x_padded && launch_pad_rows(X, static_cast<i64>(B) * N, D, Dx, w.xpad, s) != cudaSuccess) return CAKE_ERR_CUDA;
+        X = w.xpad;
+        path = CAKE_ASSIGN_TCGEN05;
+    }
     if (path == CAKE_ASSIGN_AUTO) path = assign_tc_supports(D) ? CAKE_ASSIGN_TCGEN05 : CAKE_ASSIGN_SIMT;
     if (zero_inertia && inertia && (path == CAKE_ASSIGN_SIMT || N == 0)) {
         if (cudaMemset2DAsync(inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
@@ -88,7 +101,7 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
         return rc;
     }
     if (path != CAKE_ASSIGN_TCGEN05 && path != CAKE_ASSIGN_TCGEN05_EXACT) return CAKE_ERR_UNSUPPORTED;
-    if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
+    if (!assign_tc_supports(Dx ? Dx : D)) return CAKE_ERR_UNSUPPORTED;
     if (N == 0) return CAKE_OK;
     // both epilogues order by the same fixed-point values; the packed one measured as fast or faster
     // at every shape tried, so it is the automatic choice and the other stays selectable
@@ -96,7 +109,8 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
     // up to 32 problems keep max ||c||^2 in the header, which the kernel leaves zeroed: no memset per call
     const bool in_header = B <= 32;
     return launch_assign_tc(X, C, B, N, D, K, w.caug, in_header ? w.status + 16 : w.cnmax, in_header ? w.status + 1 : nullptr,
-                            exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia, aug_ready, w.status, s);
+                            exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia, aug_ready, w.status, s, Dx,
+                            assign_cpad_columns(D) ? w.cpad : nullptr);
 }
 
 // next / prepared: see launch_finalize
@@ -180,7 +194,7 @@ int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, long long
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;
-    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, false, false, w,
+    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, false, false, false, w,
                      reinterpret_cast<cudaStream_t>(stream), flags);
 }
 
@@ -248,17 +262,20 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     // The division kernel of iteration t also writes what the tensor-core assign of iteration t + 1 would
     // otherwise compute in a prologue launch of its own (while max ||c||^2 lives in the header, B <= 32).
     const unsigned apath = flags & CAKE_ASSIGN_MASK;
-    const bool tc_assign = N > 0 && assign_tc_supports(D) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
-                                                              apath == CAKE_ASSIGN_TCGEN05_EXACT);
+    const bool tc_assign = N > 0 && ((assign_tc_supports(D) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
+                                                                apath == CAKE_ASSIGN_TCGEN05_EXACT)) ||
+                                     (assign_pad_supports(D) && apath == CAKE_ASSIGN_AUTO));
+    const int cpad_columns = assign_cpad_columns(D);
     const cake_bf16* cur = C0;
     int nxt = 0;
     bool prepared = false;
     for (int t = 0; t < iters; ++t) {
         rc = do_assign(X, cur, Bi, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr, iters,
-                       true, prepared, w, s, flags);
+                       true, prepared, t > 0, w, s, flags);
         if (rc != CAKE_OK) return rc;
         cake_bf16* dst = (t == iters - 1 && out_C_bf16) ? out_C_bf16 : w.cbuf[nxt];
-        NextAssign next{w.caug, w.status + 16, out_inertia ? out_inertia + t + 1 : nullptr, iters};
+        NextAssign next{w.caug, w.status + 16, out_inertia ? out_inertia + t + 1 : nullptr, iters,
+                        cpad_columns ? w.cpad : nullptr, cpad_columns};
         const bool want = tc_assign && Bi <= 32 && t + 1 < iters;
         rc = do_update(X, out_idx, Bi, N, D, K, cur, out_C, dst, out_counts, w, s, flags, want ? &next : nullptr, &prepared);
         if (rc != CAKE_OK) return rc;

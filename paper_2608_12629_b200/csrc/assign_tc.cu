@@ -1010,7 +1010,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
 __global__ void __launch_bounds__(256)
 centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64 total_rows,
                     uint8_t* __restrict__ caug, int* __restrict__ cnmax, double* __restrict__ inertia,
-                    int inertia_stride, int B) {
+                    int inertia_stride, int B, cake_bf16* __restrict__ cpad, int Dc) {
     ptx::grid_dep_wait();      // C may come from the kernel ahead (the previous iteration's division)
     ptx::grid_dep_launch();
     // the assign kernel adds the distances up here: start from zero
@@ -1037,6 +1037,7 @@ centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64
             }
         }
         acc = aug::fold_lanes(acc);
+        if (cpad) aug::copy_row_padded(row, D, cpad + (static_cast<size_t>(b) * K + k) * Dc, Dc, lane);
     }
     if (lane == 0) aug::write_row(caug, cnmax, b, k, K, Kpad, acc);
 }
@@ -1097,17 +1098,23 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
 
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      int* cnmax, int* ticket, bool exact, int* out_idx, float* out_dist, double* inertia,
-                     int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s) {
-    if (!assign_tc_supports(D)) return CAKE_ERR_UNSUPPORTED;
+                     int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s, int Dx,
+                     cake_bf16* cpad) {
+    // D: columns of a row of C; Dk: columns of a row of X and length of the contraction (D, or D rounded up to
+    // a multiple of 8 with zeros in the copy of X); Dc: columns of a row of the centroid operand the kernel
+    // streams (C itself, or its zero-padded copy of a multiple of 64 columns, written by the prologue)
+    const int Dk = Dx ? Dx : D;
+    const int Dc = cpad ? static_cast<int>(round_up(Dk, KCHUNK)) : D;
+    if (!assign_tc_supports(Dk) || Dk < D || (!cpad && Dk != D)) return CAKE_ERR_UNSUPPORTED;
     DeviceInfo di;
     int rc = current_device_info(&di);
     if (rc != CAKE_OK) return rc;
     if (di.cc_major != 10) return CAKE_ERR_DEVICE;
 
     Params p;
-    p.B = B; p.N = N; p.D = D; p.K = K;
-    p.nchunks = (D + KCHUNK - 1) / KCHUNK;
-    p.ksteps_last = (D - (p.nchunks - 1) * KCHUNK + UMMA_K - 1) / UMMA_K;
+    p.B = B; p.N = N; p.D = Dk; p.K = K;
+    p.nchunks = (Dk + KCHUNK - 1) / KCHUNK;
+    p.ksteps_last = (Dk - (p.nchunks - 1) * KCHUNK + UMMA_K - 1) / UMMA_K;
     p.m_tiles = static_cast<int>((N + BLOCK_M - 1) / BLOCK_M);
     p.n_tiles = (K + BLOCK_N - 1) / BLOCK_N;
     p.total_tiles = static_cast<i64>(B) * p.m_tiles;
@@ -1144,7 +1151,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         cfg.numAttrs = 1;
         if (cudaLaunchKernelEx(&cfg, centroid_aug_kernel, C, K, D, Kpad, rows, static_cast<uint8_t*>(caug), cnmax,
                                (zero_inertia && B <= 256) ? inertia : static_cast<double*>(nullptr), inertia_stride,
-                               B) != cudaSuccess) {
+                               B, cpad, Dc) != cudaSuccess) {
             cudaGetLastError();
             return CAKE_ERR_CUDA;
         }
@@ -1163,7 +1170,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     // ring would then hold a single stage, X is the bound (few centroid tiles: X buffers matter more) or the
     // last chunk is a partial one (short tiles: waiting for both chunks costs more than the barriers saved)
     i64 stages = 0;
-    for (p.cps = (p.nchunks % 2 == 0 && D % KCHUNK == 0 && p.n_tiles > 2) ? 2 : 1; p.cps >= 1; --p.cps) {
+    for (p.cps = (p.nchunks % 2 == 0 && (Dk % KCHUNK == 0 || cpad) && p.n_tiles > 2) ? 2 : 1; p.cps >= 1; --p.cps) {
         p.stage_bytes = static_cast<uint32_t>(p.cps) * C_CHUNK_BYTES + AUG_B_BYTES;
         const int spt = p.nchunks / p.cps;                       // stages per centroid tile
         const i64 min_stages = p.cps == 1 ? (p.n_tiles <= 2 ? 2 : 3) : (p.n_tiles <= 2 ? 2 : 2 * spt);
@@ -1177,7 +1184,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     p.n_stages = static_cast<int>(stages > MAX_STAGES ? MAX_STAGES : stages);
 
     CUtensorMap tx, tc;
-    rc = make_tmap(&tx, X, D, N, B, BLOCK_M);
+    rc = make_tmap(&tx, X, Dk, N, B, BLOCK_M);
     if (rc != CAKE_OK) return rc;
 
     // one or two centroid tiles per row tile: the kernel is as fast as X arrives, X gets its own producer
@@ -1219,7 +1226,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         }
     }
     if (p.res_c != 1) c_rows = BLOCK_N;
-    rc = make_tmap(&tc, C, D, K, B, c_rows);
+    rc = make_tmap(&tc, cpad ? cpad : C, Dc, K, B, c_rows);
     if (rc != CAKE_OK) return rc;
     const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf +
                               static_cast<size_t>(p.n_stages) * p.stage_bytes;

@@ -60,5 +60,24 @@ __device__ __forceinline__ void write_row(uint8_t* caug, int* cnmax, i64 b, int 
         make_uint4(one | (one << 16), one | (hi << 16), mid | (lo << 16), b6 | (one << 16));
 }
 
+// The centroid rows are streamed by TMA once per row tile; rows whose pitch is not a multiple of 128
+// bytes (D % 64 != 0) measured up to twice as slow to stream, so the kernel then reads a copy whose rows
+// are padded with zeros to Dc columns (a multiple of 64).  One warp copies one row (src only 2-byte
+// aligned when D is odd; dst 16-byte aligned).
+__device__ __forceinline__ void copy_row_padded(const cake_bf16* __restrict__ src, int D, cake_bf16* __restrict__ dst,
+                                                int Dc, int lane) {
+    for (int g = lane; g < Dc / 8; g += 32) {
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = g * 8 + 2 * j;
+            const uint32_t lo = c < D ? static_cast<uint32_t>(__ldg(src + c)) : 0u;
+            const uint32_t hi = c + 1 < D ? static_cast<uint32_t>(__ldg(src + c + 1)) : 0u;
+            w[j] = lo | (hi << 16);
+        }
+        reinterpret_cast<uint4*>(dst)[g] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 }  // namespace aug
 }  // namespace cake

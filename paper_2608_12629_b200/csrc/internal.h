@@ -44,11 +44,27 @@ size_t assign_tc_aug_bytes(i64 B, int K);
 // inertia entries from zero (otherwise the caller has).
 // aug_ready: caug, cnmax and (if asked for) the cleared inertia entries are already what the prologue
 // would write for these centroids (the division kernel of the update ahead wrote them): no prologue.
+// cpad (nullable): [B][K][round_up(Dx or D, 64)] scratch; the prologue copies C there, rows padded with
+// zeros, and the kernel streams that copy (rows whose pitch is a multiple of 128 bytes stream faster).
+// Dx (0 = D): columns of a row of X when X is a copy padded with zeros to a multiple of 8 columns
+// (needs cpad).  aug_ready then also means that cpad holds the copy.
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      int* cnmax, int* ticket, bool exact, int* out_idx, float* out_dist, double* inertia,
-                     int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s);
+                     int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s,
+                     int Dx = 0, cake_bf16* cpad = nullptr);
 int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
                        int* out_idx, float* out_dist, cudaStream_t s);
+// D that is not a multiple of 8 (rows are then no multiple of 16 bytes, which TMA needs): the automatic
+// route copies X into rows of padded_d(D) columns, zeros in the padding (distances and norms do not
+// change), and runs the tensor-core kernel on the copy.
+inline int padded_d(int D) { return (int)round_up(D, 8); }
+inline bool assign_pad_supports(int D) { return D % 8 != 0 && assign_tc_supports(padded_d(D)); }
+// columns of a row of the centroid copy the tensor-core kernel streams when D is not a multiple of 64 (else 0)
+inline int assign_cpad_columns(int D) {
+    return (D % 64 != 0 && assign_tc_supports(padded_d(D))) ? (int)round_up(D, 64) : 0;
+}
+// dst[r][0..Dpad) = src[r][0..D) followed by zeros, for r < rows (Dpad % 8 == 0, dst 16-byte aligned)
+cudaError_t launch_pad_rows(const cake_bf16* src, i64 rows, int D, int Dpad, cake_bf16* dst, cudaStream_t s);
 
 // ---- update
 struct UpdateScratch {
@@ -72,7 +88,7 @@ int launch_update_smem(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
 int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K,
                        const UpdateScratch& scr, int* counts, const cake_bf16* C_prev, float* out_C,
                        cake_bf16* out_C_bf16, bool* divided, int* status, cudaStream_t s);
-// slab route (one kernel sorts and reduces slab by slab): D % 8 == 0, D <= 256, K <= 8192.
+// slab route (one kernel sorts and reduces slab by slab): D % 8 == 0, D <= 1024, K <= 8192.
 // force_f = 0 lets the launcher choose the thread-block cluster size, else 1, 2 or 4.
 bool update_slab_supports(int D, int K);
 // true when its runs of equal clusters are long enough to beat the sort route (measured threshold)
@@ -89,6 +105,8 @@ struct NextAssign {
     int* cnmax;             // zero on entry (the assign kernel ahead left it so)
     double* inertia;        // nullable: inertia[b * inertia_stride] = 0 for b < B (B <= 256)
     int inertia_stride;
+    cake_bf16* cpad;        // nullable: as for launch_assign_tc, rows of cpad_columns columns
+    int cpad_columns;
 };
 cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B,
                             int K, int D, float* out_C, cake_bf16* out_C_bf16, bool early,

@@ -99,6 +99,27 @@ inertia_kernel(const float* __restrict__ dist, i64 N, double* __restrict__ acc, 
 }
 
 // Waits on an mbarrier that nothing completes, for at most limit_ns, then reports the expiry.
+// one thread per 16-byte granule of the padded copy (the source rows are only 2-byte aligned)
+__global__ void __launch_bounds__(256)
+pad_rows_kernel(const cake_bf16* __restrict__ src, i64 rows, int D, int Gpad, uint4* __restrict__ dst) {
+    const i64 total = rows * Gpad;
+    for (i64 e = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; e < total;
+         e += static_cast<i64>(gridDim.x) * blockDim.x) {
+        const i64 r = e / Gpad;
+        const int c0 = static_cast<int>(e - r * Gpad) * 8;
+        const cake_bf16* row = src + static_cast<size_t>(r) * D;
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = c0 + 2 * j;
+            const uint32_t lo = c < D ? __ldg(row + c) : 0u;
+            const uint32_t hi = c + 1 < D ? __ldg(row + c + 1) : 0u;
+            w[j] = lo | (hi << 16);
+        }
+        dst[e] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 __global__ void bounded_wait_selftest_kernel(int* status, unsigned long long limit_ns) {
     __shared__ uint64_t bar;
     if (threadIdx.x == 0) {
@@ -135,6 +156,16 @@ cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc
     i64 ctas = (N + 256 * 8 - 1) / (256 * 8);
     if (ctas > 296) ctas = 296;
     inertia_kernel<<<dim3(static_cast<unsigned>(ctas), B), 256, 0, s>>>(dist, N, acc, acc_stride);
+    note_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pad_rows(const cake_bf16* src, i64 rows, int D, int Dpad, cake_bf16* dst, cudaStream_t s) {
+    const i64 total = rows * (Dpad / 8);
+    if (total == 0) return cudaSuccess;
+    i64 ctas = (total + 255) / 256;
+    if (ctas > 148 * 32) ctas = 148 * 32;
+    pad_rows_kernel<<<static_cast<unsigned>(ctas), 256, 0, s>>>(src, rows, D, Dpad / 8, reinterpret_cast<uint4*>(dst));
     note_launches(1);
     return cudaGetLastError();
 }

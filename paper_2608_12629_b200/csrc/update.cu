@@ -1122,7 +1122,7 @@ __global__ void __launch_bounds__(256)
 finalize_rows_kernel(const float4* __restrict__ sums, const int* __restrict__ counts,
                      const uint2* __restrict__ C_prev, i64 rows, int K, int D4, float4* __restrict__ out_C,
                      uint2* __restrict__ out_C_bf16, uint8_t* __restrict__ caug, int* __restrict__ cnmax, int Kpad,
-                     double* __restrict__ inertia, int inertia_stride, int B) {
+                     double* __restrict__ inertia, int inertia_stride, int B, uint2* __restrict__ cpad, int Dc4) {
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
     if (inertia && blockIdx.x == 0 && static_cast<int>(threadIdx.x) < B)
@@ -1130,6 +1130,8 @@ finalize_rows_kernel(const float4* __restrict__ sums, const int* __restrict__ co
     const int lane = threadIdx.x & 31;
     const i64 n_warps = static_cast<i64>(gridDim.x) * (blockDim.x >> 5);
     for (i64 row = static_cast<i64>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); row < rows; row += n_warps) {
+        if (cpad)   // the zero padding of the row's copy for the assign kernel
+            for (int j = D4 + lane; j < Dc4; j += 32) cpad[row * Dc4 + j] = make_uint2(0u, 0u);
         const int n = counts[row];
         const float fn = static_cast<float>(n);
         float acc = 0.f;
@@ -1150,6 +1152,7 @@ finalize_rows_kernel(const float4* __restrict__ sums, const int* __restrict__ co
             o.x = static_cast<uint32_t>(f32_to_bf16_rne(v.x)) | (static_cast<uint32_t>(f32_to_bf16_rne(v.y)) << 16);
             o.y = static_cast<uint32_t>(f32_to_bf16_rne(v.z)) | (static_cast<uint32_t>(f32_to_bf16_rne(v.w)) << 16);
             out_C_bf16[e] = o;
+            if (cpad) cpad[row * Dc4 + j] = o;
             acc = aug::add_squares(acc, o.x, o.y);
         }
         acc = aug::fold_lanes(acc);
@@ -1510,7 +1513,7 @@ cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf1
                                      reinterpret_cast<const float4*>(sums), counts, reinterpret_cast<const uint2*>(C_prev), rows,
                                      K, D / 4, reinterpret_cast<float4*>(out_C), reinterpret_cast<uint2*>(out_C_bf16),
                                      static_cast<uint8_t*>(next->caug), next->cnmax, padded_k(K), next->inertia,
-                                     next->inertia_stride, B);
+                                     next->inertia_stride, B, reinterpret_cast<uint2*>(next->cpad), next->cpad_columns / 4);
         note_launches(1);
         if (e == cudaSuccess && prepared) *prepared = true;
         return e;

@@ -63,12 +63,40 @@ def test_assign_simt_fallback(N, D, K):
     X, C = problem(N, D, K, seed=N * 3 + D)
     idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_SIMT)
     grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx.cpu().numpy(), dist.cpu().numpy())
-    if D % 8 or D > 512:  # the automatic choice must take the fallback for such D, and the tensor path must refuse
-        idx2, _ = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV))
-        assert torch.equal(idx, idx2)
+    if D % 8 or D > 512:  # the tensor path must refuse such D when asked for by name
         with pytest.raises(cake.CakeError) as e:
             cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_TCGEN05)
         assert e.value.code == cake.CAKE_ERR_UNSUPPORTED
+    if D > 512:           # and the automatic choice takes the fallback
+        idx2, _ = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV))
+        assert torch.equal(idx, idx2)
+
+
+@pytest.mark.parametrize("B,N,D,K", [(1, 100, 5, 7), (1, 3000, 33, 40), (2, 640, 130, 300), (1, 20000, 100, 1000),
+                                     (3, 257, 1, 2), (1, 1000, 12, 6), (1, 500, 509, 77), (1, 129, 255, 257)])
+def test_assign_feature_count_not_multiple_of_8(B, N, D, K):
+    """The automatic route copies X and C into zero-padded rows and runs the tensor-core kernel on them:
+    same grading as any other shape, and a Lloyd call (which pads X once) agrees with step-by-step calls."""
+    g = torch.Generator().manual_seed(N + D)
+    X = torch.randint(-4, 5, (B, N, D), generator=g).to(torch.bfloat16)   # small integers: sums exact in any order
+    C = torch.randint(-4, 5, (B, K, D), generator=g).to(torch.bfloat16) + 0.25
+    ws = cake.alloc_workspace(B, N, D, K, DEV)
+    Xd, Cd = X.to(DEV), C.to(DEV)
+    launches = cake.cake_kmeans_kernel_launches()
+    idx, dist = cake.cake_kmeans_assign(Xd, Cd, ws=ws)
+    assert cake.cake_kmeans_kernel_launches() - launches == 3      # copy of X, prologue, tensor-core kernel
+    check_status(ws)
+    for b in range(B):
+        grading.grade_assign(inputs.to_bits(X[b]), inputs.to_bits(C[b]), idx[b].cpu().numpy(), dist[b].cpu().numpy())
+    out = cake.cake_kmeans_lloyd(Xd, Cd, 3, ws=ws)
+    check_status(ws)
+    Cc = Cd
+    for _ in range(3):
+        i2, d2 = cake.cake_kmeans_assign(Xd, Cc, ws=ws)
+        Cf, Cb, counts = cake.cake_kmeans_update(Xd, i2, K, C_prev=Cc, ws=ws)
+        Cc = Cb
+    assert torch.equal(out.idx, i2) and torch.equal(out.dist, d2) and torch.equal(out.counts, counts)
+    assert torch.equal(out.C, Cf) and torch.equal(out.C_bf16, Cb)
 
 
 @pytest.mark.parametrize("policy", sorted(TC_POLICIES))
