@@ -191,7 +191,7 @@ def run_sweep(args):
     torch.cuda.set_device(dev)
     peaks = measured_peaks()
     Ns = [1 << 16, 1 << 20, 1 << 24] if not args.sweep_full else [1 << e for e in range(16, 25)]
-    Ds = [64, 96, 128, 256]
+    Ds = [64, 96, 100, 128, 256, 384]
     Ks = [64, 256, 1000, 1024, 4096, 65536] if not args.sweep_full else [64, 128, 256, 512, 1000, 1024, 2048, 4096,
                                                                           8192, 16384, 32768, 65536]
     print("| N | D | K | lloyd it/s | assign ms | TFLOP/s | update ms | GB/s | roofline it/s | fraction |")

@@ -38,7 +38,8 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     w.status = reinterpret_cast<int*>(take(256));
     w.caug = take(assign_tc_aug_bytes(B, K));
     w.cnmax = reinterpret_cast<int*>(take(static_cast<size_t>(B) * 4));
-    w.sums = reinterpret_cast<float*>(take(kd * 4));
+    // rows of padded_d(D) columns: for D % 8 != 0 the update may add up the padded copy of X
+    w.sums = reinterpret_cast<float*>(take(static_cast<size_t>(B) * K * padded_d(D) * 4));
     w.nvalid = reinterpret_cast<int*>(take(static_cast<size_t>(B) * 4));
     w.cursor = reinterpret_cast<int*>(take(static_cast<size_t>(B) * K * 4));
     w.pairs = reinterpret_cast<int2*>(take(static_cast<size_t>(B) * N * 8));
@@ -75,15 +76,16 @@ int check_ws(void* ws, size_t ws_bytes, i64 B, i64 N, int D, int K, Workspace* o
 // kernel adds it up itself; the fallback needs `dist` (out_dist or scratch) and a reduction kernel.
 // zero_inertia: the entries still have to be cleared (the tensor-core prologue does it on the way).
 // aug_ready: the update ahead prepared this assign (see NextAssign): the tensor-core route skips its prologue
-// x_padded: the workspace already holds the padded copy of this X (an earlier iteration of the call made it)
+// x_padded (in/out): the workspace already holds the padded copy of this X (an earlier step of the call made it)
 int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, int* out_idx,
               float* out_dist, double* inertia, int inertia_stride, bool zero_inertia, bool aug_ready,
-              bool x_padded, const Workspace& w, cudaStream_t s, unsigned flags) {
+              bool* x_padded, const Workspace& w, cudaStream_t s, unsigned flags) {
     unsigned path = flags & CAKE_ASSIGN_MASK;
     int Dx = 0;   // columns of the padded copy of X, if one is used
     if (path == CAKE_ASSIGN_AUTO && assign_pad_supports(D) && N > 0) {
         Dx = padded_d(D);
-        if (!x_padded && launch_pad_rows(X, static_cast<i64>(B) * N, D, Dx, w.xpad, s) != cudaSuccess) return CAKE_ERR_CUDA;
+        if (!*x_padded && launch_pad_rows(X, static_cast<i64>(B) * N, D, Dx, w.xpad, s) != cudaSuccess) return CAKE_ERR_CUDA;
+        *x_padded = true;
         X = w.xpad;
         path = CAKE_ASSIGN_TCGEN05;
     }
@@ -116,13 +118,23 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
 // next / prepared: see launch_finalize
 int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, const cake_bf16* C_prev,
               float* out_C, cake_bf16* out_C_bf16, int* out_counts, const Workspace& w, cudaStream_t s,
-              unsigned flags, const NextAssign* next = nullptr, bool* prepared = nullptr) {
+              unsigned flags, bool* x_padded, const NextAssign* next = nullptr, bool* prepared = nullptr) {
     if (prepared) *prepared = false;
     DeviceInfo di;
     int rc = current_device_info(&di);
     if (rc != CAKE_OK) return rc;
     unsigned path = flags & CAKE_UPDATE_MASK;
     bool divided = false;
+    int Ds = D;   // columns of a row of sums
+    if (path == CAKE_UPDATE_AUTO && assign_pad_supports(D) && update_slab_preferred(B, N, padded_d(D), K)) {
+        // D % 8 != 0: the slab route on the zero-padded copy of X (its padding columns add up to zero and are
+        // dropped by the division kernel); faster than the element-wise reduction even when the copy has to be made
+        Ds = padded_d(D);
+        if (!*x_padded && launch_pad_rows(X, static_cast<i64>(B) * N, D, Ds, w.xpad, s) != cudaSuccess) return CAKE_ERR_CUDA;
+        *x_padded = true;
+        X = w.xpad;
+        path = CAKE_UPDATE_SLAB;
+    }
     if (path == CAKE_UPDATE_AUTO) {
         // the slab route while a slab holds several rows per cluster, else the global sort; the
         // shared-memory table never measured faster than either and is only taken on request
@@ -136,14 +148,14 @@ int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, co
     } else if (path == CAKE_UPDATE_SLAB || path == CAKE_UPDATE_SLAB_F1 || path == CAKE_UPDATE_SLAB_F2 ||
                path == CAKE_UPDATE_SLAB_F4) {
         const int force_f = path == CAKE_UPDATE_SLAB ? 0 : path == CAKE_UPDATE_SLAB_F1 ? 1 : path == CAKE_UPDATE_SLAB_F2 ? 2 : 4;
-        rc = launch_update_slab(X, idx, B, N, D, K, w.sums, out_counts, w.status, force_f, s);
+        rc = launch_update_slab(X, idx, B, N, Ds, K, w.sums, out_counts, w.status, force_f, s);
     } else {
         rc = CAKE_ERR_UNSUPPORTED;
     }
     if (rc != CAKE_OK) return rc;
     if (divided) return CAKE_OK;
     const bool slab = path != CAKE_UPDATE_SMEM && path != CAKE_UPDATE_SORT;
-    if (launch_finalize(w.sums, out_counts, C_prev, B, K, D, out_C, out_C_bf16, slab, next, prepared, s) != cudaSuccess)
+    if (launch_finalize(w.sums, out_counts, C_prev, B, K, D, out_C, out_C_bf16, slab, next, prepared, s, Ds) != cudaSuccess)
         return CAKE_ERR_CUDA;
     return CAKE_OK;
 }
@@ -194,7 +206,8 @@ int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, long long
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;
-    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, false, false, false, w,
+    bool x_padded = false;
+    return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, false, false, &x_padded, w,
                      reinterpret_cast<cudaStream_t>(stream), flags);
 }
 
@@ -216,8 +229,9 @@ int cake_kmeans_update_batched(const cake_bf16* X, const int* idx, long long B, 
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;
+    bool x_padded = false;
     return do_update(X, idx, static_cast<int>(B), N, D, K, C_prev, out_C, out_C_bf16, out_counts, w,
-                     reinterpret_cast<cudaStream_t>(stream), flags);
+                     reinterpret_cast<cudaStream_t>(stream), flags, &x_padded);
 }
 
 int cake_kmeans_update(const cake_bf16* X, const int* idx, long long N, int D, int K,
@@ -269,15 +283,16 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     const cake_bf16* cur = C0;
     int nxt = 0;
     bool prepared = false;
+    bool x_padded = false;   // the workspace holds the padded copy of X (D % 8 != 0), made by the first step that needs it
     for (int t = 0; t < iters; ++t) {
         rc = do_assign(X, cur, Bi, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr, iters,
-                       true, prepared, t > 0, w, s, flags);
+                       true, prepared, &x_padded, w, s, flags);
         if (rc != CAKE_OK) return rc;
         cake_bf16* dst = (t == iters - 1 && out_C_bf16) ? out_C_bf16 : w.cbuf[nxt];
         NextAssign next{w.caug, w.status + 16, out_inertia ? out_inertia + t + 1 : nullptr, iters,
                         cpad_columns ? w.cpad : nullptr, cpad_columns};
         const bool want = tc_assign && Bi <= 32 && t + 1 < iters;
-        rc = do_update(X, out_idx, Bi, N, D, K, cur, out_C, dst, out_counts, w, s, flags, want ? &next : nullptr, &prepared);
+        rc = do_update(X, out_idx, Bi, N, D, K, cur, out_C, dst, out_counts, w, s, flags, &x_padded, want ? &next : nullptr, &prepared);
         if (rc != CAKE_OK) return rc;
         cur = dst;
         nxt ^= 1;

@@ -100,6 +100,7 @@ int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
 // next (nullable): also prepare the tensor-core assign of the centroids being written (its half-norm
 // operand, max ||c||^2, cleared inertia entries), so that that assign needs no prologue.  Needs
 // D % 4 == 0 and out_C_bf16; *prepared tells whether it was done.
+// sums_columns (0 = D): columns of a row of sums, when they were added up from the padded copy of X.
 struct NextAssign {
     void* caug;             // as for launch_assign_tc
     int* cnmax;             // zero on entry (the assign kernel ahead left it so)
@@ -110,7 +111,7 @@ struct NextAssign {
 };
 cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B,
                             int K, int D, float* out_C, cake_bf16* out_C_bf16, bool early,
-                            const NextAssign* next, bool* prepared, cudaStream_t s);
+                            const NextAssign* next, bool* prepared, cudaStream_t s, int sums_columns = 0);
 
 // ---- inertia: acc[b] += sum_i dist[b][i] (fp64 atomics); acc stride given in elements
 cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc_stride,

@@ -868,7 +868,7 @@ constexpr int SLAB_MAX_K = 8192;
 constexpr int SLAB_AHEAD = 4;                              // rows in flight per lane group
 constexpr int SLAB_MAX_F = 4;
 constexpr int SLAB_GROW_RUN = 8;                           // clusters grow until a run has this many rows
-constexpr int SLAB_MIN_RUN = 4;                            // rows per run below which the sort route is faster
+constexpr int SLAB_MIN_RUN = 4;                            // rows per run below which the sort route is faster (K > 4096)
 
 // sums and counts start at zero; the kernel behind it may begin at once (it waits before its first add)
 __global__ void __launch_bounds__(256)
@@ -1017,8 +1017,11 @@ slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
     const uint32_t rowmask = (1u << rowbits) - 1u;
     const int seglen = max(SLAB_AHEAD, (mine + NGROUPS - 1) / NGROUPS);
     const int base = gid * seglen, end = min(base + seglen, mine);
-    // rows wider than 32 granules (D > 256) are reduced in column blocks of 32 granules, one pass each
-    for (int sg = sl; sg - sl < G; sg += LPR) {
+    // rows wider than 32 granules (D > 256) are reduced in equal column blocks of at most 32 granules, one
+    // pass over the records each (G <= LPR: one pass, sg = sl)
+    const int n_pass = (G + LPR - 1) / LPR, pass_w = (G + n_pass - 1) / n_pass;
+    for (int pass = 0; pass < n_pass; ++pass) {
+        const int sg = sl < pass_w ? pass * pass_w + sl : G;   // this lane's granule (G: none)
         int cur = -1;
         float acc[8];
 #pragma unroll
@@ -1067,7 +1070,7 @@ slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
 
 __global__ void __launch_bounds__(256)
 finalize_kernel(const float* __restrict__ sums, const int* __restrict__ counts,
-                const cake_bf16* __restrict__ C_prev, i64 total, int D, float* __restrict__ out_C,
+                const cake_bf16* __restrict__ C_prev, i64 total, int D, int Ds, float* __restrict__ out_C,
                 cake_bf16* __restrict__ out_C_bf16) {
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
@@ -1076,7 +1079,7 @@ finalize_kernel(const float* __restrict__ sums, const int* __restrict__ counts,
         const i64 row = e / D;  // b*K + k
         const int n = counts[row];
         float v;
-        if (n > 0) v = sums[e] / static_cast<float>(n);
+        if (n > 0) v = sums[row * Ds + (e - row * D)] / static_cast<float>(n);
         else v = C_prev ? __uint_as_float(static_cast<uint32_t>(C_prev[e]) << 16) : 0.f;
         out_C[e] = v;
         if (out_C_bf16) out_C_bf16[e] = f32_to_bf16_rne(v);
@@ -1086,16 +1089,17 @@ finalize_kernel(const float* __restrict__ sums, const int* __restrict__ counts,
 // D % 4 == 0: four columns per thread, 16-byte loads and stores
 __global__ void __launch_bounds__(256)
 finalize4_kernel(const float4* __restrict__ sums, const int* __restrict__ counts,
-                 const uint2* __restrict__ C_prev, i64 total4, int D4, float4* __restrict__ out_C,
+                 const uint2* __restrict__ C_prev, i64 total4, int D4, int Ds4, float4* __restrict__ out_C,
                  uint2* __restrict__ out_C_bf16) {
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
     for (i64 e = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; e < total4;
          e += static_cast<i64>(gridDim.x) * blockDim.x) {
-        const int n = counts[e / D4];
+        const i64 row = e / D4;
+        const int n = counts[row];
         float4 v;
         if (n > 0) {
-            const float4 sv = sums[e];
+            const float4 sv = sums[row * Ds4 + (e - row * D4)];
             const float fn = static_cast<float>(n);
             v = make_float4(sv.x / fn, sv.y / fn, sv.z / fn, sv.w / fn);
         } else if (C_prev) {
@@ -1122,7 +1126,8 @@ __global__ void __launch_bounds__(256)
 finalize_rows_kernel(const float4* __restrict__ sums, const int* __restrict__ counts,
                      const uint2* __restrict__ C_prev, i64 rows, int K, int D4, float4* __restrict__ out_C,
                      uint2* __restrict__ out_C_bf16, uint8_t* __restrict__ caug, int* __restrict__ cnmax, int Kpad,
-                     double* __restrict__ inertia, int inertia_stride, int B, uint2* __restrict__ cpad, int Dc4) {
+                     double* __restrict__ inertia, int inertia_stride, int B, uint2* __restrict__ cpad, int Dc4,
+                     int Ds4) {
     ptx::grid_dep_wait();
     ptx::grid_dep_launch();
     if (inertia && blockIdx.x == 0 && static_cast<int>(threadIdx.x) < B)
@@ -1139,7 +1144,7 @@ finalize_rows_kernel(const float4* __restrict__ sums, const int* __restrict__ co
             const i64 e = row * D4 + j;
             float4 v;
             if (n > 0) {
-                const float4 sv = sums[e];
+                const float4 sv = sums[row * Ds4 + j];
                 v = make_float4(sv.x / fn, sv.y / fn, sv.z / fn, sv.w / fn);
             } else if (C_prev) {
                 const uint2 pv = C_prev[e];
@@ -1439,8 +1444,11 @@ bool update_slab_preferred(int B, i64 N, int D, int K) {
     SlabPlan pl;
     if (N < 1 || !update_slab_supports(D, K) || current_device_info(&di) != CAKE_OK) return false;
     if (slab_make_plan(di, B, N, D, K, 0, &pl) != CAKE_OK) return false;
+    // measured against the sort route: up to 4,096 clusters the slab route wins from 1.5 rows per run on
+    // (equal at 1.7, 17-45 % faster at 2-3.5); above, its per-CTA scan of K counters needs 4 rows per run
     const i64 rows = static_cast<i64>(pl.S) * pl.F;
-    return (rows < N ? rows : N) >= static_cast<i64>(SLAB_MIN_RUN) * K;
+    const i64 have = rows < N ? rows : N;
+    return K <= 4096 ? 2 * have >= 3 * static_cast<i64>(K) : have >= static_cast<i64>(SLAB_MIN_RUN) * K;
 }
 
 int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, float* sums, int* counts,
@@ -1501,8 +1509,9 @@ int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
 
 cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B, int K,
                             int D, float* out_C, cake_bf16* out_C_bf16, bool early, const NextAssign* next,
-                            bool* prepared, cudaStream_t s) {
+                            bool* prepared, cudaStream_t s, int sums_columns) {
     const i64 total = static_cast<i64>(B) * K * D;
+    const int Ds = sums_columns ? sums_columns : D;   // columns of a row of sums (a multiple of 4 when D is)
     if (prepared) *prepared = false;
     if (next && out_C_bf16 && D % 4 == 0 && B <= 256) {
         const i64 rows = static_cast<i64>(B) * K;
@@ -1513,7 +1522,8 @@ cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf1
                                      reinterpret_cast<const float4*>(sums), counts, reinterpret_cast<const uint2*>(C_prev), rows,
                                      K, D / 4, reinterpret_cast<float4*>(out_C), reinterpret_cast<uint2*>(out_C_bf16),
                                      static_cast<uint8_t*>(next->caug), next->cnmax, padded_k(K), next->inertia,
-                                     next->inertia_stride, B, reinterpret_cast<uint2*>(next->cpad), next->cpad_columns / 4);
+                                     next->inertia_stride, B, reinterpret_cast<uint2*>(next->cpad), next->cpad_columns / 4,
+                                     Ds / 4);
         note_launches(1);
         if (e == cudaSuccess && prepared) *prepared = true;
         return e;
@@ -1534,7 +1544,7 @@ cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf1
         cfg.gridDim = dim3(static_cast<unsigned>(ctas));
         note_launches(1);
         return cudaLaunchKernelEx(&cfg, finalize4_kernel, reinterpret_cast<const float4*>(sums), counts,
-                                  reinterpret_cast<const uint2*>(C_prev), total / 4, D / 4,
+                                  reinterpret_cast<const uint2*>(C_prev), total / 4, D / 4, Ds / 4,
                                   reinterpret_cast<float4*>(out_C), reinterpret_cast<uint2*>(out_C_bf16));
     }
     i64 ctas = (total + 256 * 4 - 1) / (256 * 4);
@@ -1542,7 +1552,7 @@ cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf1
     if (ctas < 1) ctas = 1;
     cfg.gridDim = dim3(static_cast<unsigned>(ctas));
     note_launches(1);
-    return cudaLaunchKernelEx(&cfg, finalize_kernel, sums, counts, C_prev, total, D, out_C, out_C_bf16);
+    return cudaLaunchKernelEx(&cfg, finalize_kernel, sums, counts, C_prev, total, D, Ds, out_C, out_C_bf16);
 }
 
 }  // namespace cake
