@@ -15,8 +15,8 @@
  *   - cake_bf16 is a raw bfloat16 bit pattern.  Matrices are row-major and contiguous:
  *     X[B][N][D], C[B][K][D], idx[B][N], counts[B][K].  The un-batched calls are B = 1.
  *     Base pointers must be 16-byte aligned.  Inputs must be finite.
- *   - `ws` is caller-provided scratch of at least cake_kmeans_workspace_bytes(...) bytes,
- *     256-byte aligned.  Its first word is a sticky device status (see cake_kmeans_device_status);
+ *   - `ws` is caller-provided scratch of at least cake_kmeans_workspace_bytes(...) bytes
+ *     (for D % 8 != 0 that includes room for a zero-padded copy of X), 256-byte aligned.  Its first word is a sticky device status (see cake_kmeans_device_status);
  *     the caller zeroes the first 256 bytes once, before the first call that uses the buffer.
  *     Calls that run concurrently must use distinct workspaces.
  *   - Work is enqueued on `stream` (a cudaStream_t; NULL = the legacy default stream) and the
@@ -58,7 +58,8 @@ enum {
 };
 
 enum {
-    CAKE_ASSIGN_AUTO = 0,
+    CAKE_ASSIGN_AUTO = 0,      /* the tensor-core pipeline for D <= 512 (for D % 8 != 0 on a zero-padded
+                                  copy of X kept in the workspace: same results), else the fallback  */
     CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 512.
                                   Distances are compared as fixed-point numbers with a quantum of
                                   about 2^-19 of (|x|^2 + max |c|^2); equal ones go to the lower index */
