@@ -246,6 +246,30 @@ __device__ __forceinline__ void exact_scan32(const uint32_t (&r)[32], int col_ba
 
 // XLOAD: warp 11 loads the X tiles and two warps issue MMAs (few centroid tiles per row tile);
 // otherwise the centroid producer also loads X and three warps issue MMAs.
+// Row tiles of a CTA.  Interleaved over the CTAs (blockIdx.x, blockIdx.x + gridDim.x, ...), except for a batch
+// of problems with resident centroids: there the CTA takes as many row tiles as interleaving would give it,
+// but consecutive ones, so that it meets few problems (every change of problem reloads the resident tile:
+// 32 problems of 512 row tiles on 148 CTAs change problem every 3.5 tiles when interleaved).
+// first_tile: (problem, row tile) of the CTA's first tile; tile_step: distance to its next one.
+template <bool XLOAD>
+__device__ __forceinline__ bool tiles_consecutive(const Params& p) { return XLOAD && p.res_c && p.B > 1; }
+template <bool XLOAD>
+__device__ __forceinline__ void first_tile(const Params& p, int& tb, int& tmt) {
+    if (tiles_consecutive<XLOAD>(p)) {
+        const i64 q = p.total_tiles / gridDim.x, r = p.total_tiles - q * gridDim.x;
+        const i64 first = blockIdx.x * q + (static_cast<i64>(blockIdx.x) < r ? static_cast<i64>(blockIdx.x) : r);
+        tb = static_cast<int>(first / p.m_tiles);
+        tmt = static_cast<int>(first - static_cast<i64>(tb) * p.m_tiles);
+    } else {
+        tb = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
+        tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
+    }
+}
+template <bool XLOAD>
+__device__ __forceinline__ int tile_step(const Params& p) {
+    return tiles_consecutive<XLOAD>(p) ? 1 : static_cast<int>(gridDim.x);
+}
+
 template <bool PACKED, bool XLOAD>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
@@ -350,8 +374,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 // this CTA meets; "stage 0" of the ring stands for the whole buffer
                 int cur_b = -1;
                 uint32_t pc = 0;
-                int tb = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
-                int tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
+                int tb, tmt;
+                first_tile<XLOAD>(p, tb, tmt);
+                const int tmt_step = tile_step<XLOAD>(p);
                 for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                     if (tb != cur_b) {
                         ok = wait_bar(&ctrl->ring_empty[0], (pc & 1u) ^ 1u, ctrl, p.status);
@@ -370,7 +395,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         cur_b = tb;
                         ++pc;
                     }
-                    tmt += static_cast<int>(gridDim.x);
+                    tmt += tmt_step;
                     while (tmt >= p.m_tiles) { tmt -= p.m_tiles; ++tb; }
                 }
                 if (!ok || pc == 0) {
@@ -434,8 +459,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // late: here the X loads have a thread of their own, at the price of the third MMA issuer.
         if (lane == 0) {
             uint32_t ixb = 0, ixph = 0;
-            int tb = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
-            int tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
+            int tb, tmt;
+            first_tile<XLOAD>(p, tb, tmt);
+                const int tmt_step = tile_step<XLOAD>(p);
             bool ok = true;
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 ok = wait_bar(&ctrl->x_empty[ixb], ixph ^ 1u, ctrl, p.status);
@@ -446,7 +472,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     ptx::tma_load_3d(x_base + ixb * xbuf_bytes + c * X_CHUNK_BYTES, &tmap_x, xfull,
                                      c * KCHUNK, tmt * BLOCK_M, tb);
                 if (++ixb == static_cast<uint32_t>(p.n_xbuf)) { ixb = 0; ixph ^= 1u; }
-                tmt += static_cast<int>(gridDim.x);
+                tmt += tmt_step;
                 while (tmt >= p.m_tiles) { tmt -= p.m_tiles; ++tb; }
             }
             if (!ok) {   // aborting: a bounded time for the X loads in flight to land
@@ -485,14 +511,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 // on it are done, and waits for the next problem's centroids.
                 int cur_b = -1;
                 uint32_t pc = 0, tile_it = 0;
-                int tb = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
-                int tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
+                int tb, tmt;
+                first_tile<XLOAD>(p, tb, tmt);
+                const int tmt_step = tile_step<XLOAD>(p);
                 const uint32_t nxb = static_cast<uint32_t>(p.n_xbuf);
                 const uint32_t idesc_aug_n = ptx::umma_idesc_bf16(BLOCK_M, p.alt_epi ? p.alt_epi : BLOCK_N);
                 const uint32_t idesc_main_n = idesc_aug_n | ptx::UMMA_IDESC_NEGATE_B;
                 for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
                     const int b_now = tb;
-                    tmt += static_cast<int>(gridDim.x);
+                    tmt += tmt_step;
                     while (tmt >= p.m_tiles) { tmt -= p.m_tiles; ++tb; }
                     if (b_now != cur_b) {
                         if (cur_b >= 0) ptx::umma_commit(ptx::smem_u32(&ctrl->ring_empty[0]));
@@ -648,6 +675,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int r = (warp - AUX_WARP0) * 32 + lane;
         uint32_t xb = 0, xph = 0;
         bool ok = true;
+        int nb = 0, nmt = 0;   // (problem, row tile), stepped: only where the CTA's tiles may be consecutive
+        if (XLOAD) first_tile<XLOAD>(p, nb, nmt);
+        const int nmt_step = tile_step<XLOAD>(p);
         for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
             ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);
             if (!ok) break;
@@ -671,7 +701,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             // offset M = 2^(E-127): the smallest power of two >= 2 (||x||^2 + max ||c||^2) whose biased
             // exponent E is 0 or 1 modulo 4 (then bits(M) * 128 is 0 or 2^30 modulo 2^32 and the keys
             // of the row are positive floats); m = M / 4096
-            const int tb = static_cast<int>(tile / p.m_tiles);
+            int tb;
+            if (XLOAD) {
+                tb = nb;
+                nmt += nmt_step;
+                while (nmt >= p.m_tiles) { nmt -= p.m_tiles; ++nb; }
+            } else {
+                tb = static_cast<int>(tile / p.m_tiles);
+            }
             const float bound = 2.f * (xn + __int_as_float(__ldg(p.cnmax + tb)));
             const uint32_t bb = __float_as_uint(bound);
             uint32_t E = (bb >> 23) + ((bb & 0x7FFFFFu) ? 1u : 0u);
@@ -716,10 +753,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             dsum = 0.0;
         };
         // (problem, row tile) of the current tile, stepped instead of divided
-        int b = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.m_tiles));
-        int mt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
+        int b, mt;
+        first_tile<XLOAD>(p, b, mt);
+        const int mt_step = tile_step<XLOAD>(p);
         auto next_tile = [&]() {
-            mt += static_cast<int>(gridDim.x);
+            mt += mt_step;
             while (mt >= p.m_tiles) { mt -= p.m_tiles; ++b; }
         };
         // One centroid tile per row tile: accumulator, X buffer and warpgroup all alternate with the row

@@ -883,7 +883,8 @@ zero_sums_counts_kernel(float4* __restrict__ sums4, i64 n4, int* __restrict__ co
     for (i64 e = t; e < nc; e += stride) counts[e] = 0;
 }
 
-template <int LPR, bool CLUSTER>
+// WIDE: rows of more than 32 granules (D > 256), reduced in several column passes
+template <int LPR, bool CLUSTER, bool WIDE = false>
 __global__ void __launch_bounds__(SLAB_THREADS, 1)
 slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx, i64 N, int D, int K, int S,
                    int rowbits, float* __restrict__ sums, int* __restrict__ counts, int* status) {
@@ -1018,10 +1019,10 @@ slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
     const int seglen = max(SLAB_AHEAD, (mine + NGROUPS - 1) / NGROUPS);
     const int base = gid * seglen, end = min(base + seglen, mine);
     // rows wider than 32 granules (D > 256) are reduced in equal column blocks of at most 32 granules, one
-    // pass over the records each (G <= LPR: one pass, sg = sl)
-    const int n_pass = (G + LPR - 1) / LPR, pass_w = (G + n_pass - 1) / n_pass;
+    // pass over the records each
+    const int n_pass = WIDE ? (G + LPR - 1) / LPR : 1, pass_w = WIDE ? (G + n_pass - 1) / n_pass : LPR;
     for (int pass = 0; pass < n_pass; ++pass) {
-        const int sg = sl < pass_w ? pass * pass_w + sl : G;   // this lane's granule (G: none)
+        const int sg = WIDE ? (sl < pass_w ? pass * pass_w + sl : G) : sl;   // this lane's granule (>= G: none)
         int cur = -1;
         float acc[8];
 #pragma unroll
@@ -1354,7 +1355,8 @@ struct SlabPlan {
 
 using SlabKernel = void (*)(const cake_bf16*, const int*, i64, int, int, int, int, float*, int*, int*);
 
-SlabKernel slab_kernel_for(int lpr, bool cluster) {
+SlabKernel slab_kernel_for(int lpr, bool cluster, bool wide) {
+    if (wide) return cluster ? slab_update_kernel<32, true, true> : slab_update_kernel<32, false, true>;
     switch (lpr) {
         case 4: return cluster ? slab_update_kernel<4, true> : slab_update_kernel<4, false>;
         case 8: return cluster ? slab_update_kernel<8, true> : slab_update_kernel<8, false>;
@@ -1425,7 +1427,7 @@ static int slab_make_plan(const DeviceInfo& di, int B, i64 N, int D, int K, int 
         if (force_f && F != force_f) continue;
         SlabPlan pl;
         pl.F = F;
-        const int slots = slab_slots(di, slab_kernel_for(lpr, F > 1), F, slab_smem_bytes(K, SLAB_MAX_ROWS));
+        const int slots = slab_slots(di, slab_kernel_for(lpr, F > 1, D > 256), F, slab_smem_bytes(K, SLAB_MAX_ROWS));
         if (slots < F) continue;
         slab_rows_for(slots, B, N, F, &pl.S, &pl.n_ctas);
         pl.rowbits = 1;
@@ -1482,7 +1484,7 @@ int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
     rc = slab_make_plan(di, B, N, D, K, force_f, &pl);
     if (rc != CAKE_OK) return rc;
     const int lpr = slab_lpr(D);
-    SlabKernel kernel = slab_kernel_for(lpr, pl.F > 1);
+    SlabKernel kernel = slab_kernel_for(lpr, pl.F > 1, D > 256);
     const size_t smem = slab_smem_bytes(K, pl.S);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(pl.n_ctas), static_cast<unsigned>(B));
