@@ -443,6 +443,19 @@ def test_lloyd_small_all_paths(flags):
     teacher_forced(X, C0, 4, flags=flags)
 
 
+@pytest.mark.parametrize("flags", [0, cake.CAKE_ASSIGN_SIMT, cake.CAKE_UPDATE_SORT, cake.CAKE_ASSIGN_SIMT | cake.CAKE_UPDATE_SORT])
+@pytest.mark.parametrize("N,D,K", [(3000, 50, 40), (2500, 7, 9), (1200, 300, 33)])
+def test_lloyd_feature_count_not_multiple_of_8_all_paths(N, D, K, flags):
+    """Real-valued data, graded against the oracle step by step: padded tensor-core assign + slab update on the
+    padded copy (automatic), and every mix with the fallback assign and the sort route (where the update
+    has to make the padded copy itself, or none is made at all)."""
+    X, C0 = problem(N, D, K, seed=N + D, comps=K, mean_std=2.0, sigma=1.0)
+    cur, inertia, near = teacher_forced(X, C0, 3, flags=flags)
+    assert near <= 3
+    out = cake.cake_kmeans_lloyd(X.to(DEV), C0.to(DEV), 3, flags=flags)
+    np.testing.assert_allclose(out.inertia.cpu().numpy(), inertia, rtol=1e-3)
+
+
 def test_lloyd_handworked_example_on_gpu():
     """The six-point example (golden/handworked_2d.json), padded to D=8 with zero columns."""
     pts = [[0, 0], [0, 2], [2, 0], [10, 10], [10, 12], [12, 10]]
