@@ -155,6 +155,28 @@ CAKE_API int cake_kmeans_update_batched(const cake_bf16* X, const int* idx, long
                                cake_stream_t stream, unsigned flags);
 
 /*
+ * centroid_update in two halves, for rows of X that are spread over several devices (the paper
+ * describes one device; the reduction "into per-cluster sums and counts" of the same paragraph is what
+ * has to cross devices).  Each device adds up its own rows, the caller adds the sums and counts of all
+ * devices (an all-reduce), and every device divides.  K <= 8192.
+ *   update_partial: out_sums[B][K][D] fp32 and out_counts[B][K] int32 of the rows given (overwritten,
+ *                   not accumulated); other arguments as for update.  flags: 0, CAKE_UPDATE_SLAB or
+ *                   CAKE_UPDATE_SORT.
+ *   update_finish:  out_C = sums / counts where counts > 0, else C_prev (zeros if NULL); out_C_bf16
+ *                   (may be NULL) its rounding.  No workspace.
+ */
+CAKE_API int cake_kmeans_update_partial_batched(const cake_bf16* X, const int* idx, long long B, long long N,
+                               int D, int K, float* out_sums, int* out_counts, void* ws,
+                               size_t ws_bytes, cake_stream_t stream, unsigned flags);
+/* out_inertia[b * inertia_stride] = sum_i dist[b][i] in fp64 (overwritten), the inertia of an assignment:
+ * what lloyd reports per iteration, for callers that run the steps one by one.                        */
+CAKE_API int cake_kmeans_inertia_batched(const float* dist, long long B, long long N, double* out_inertia,
+                               int inertia_stride, cake_stream_t stream);
+CAKE_API int cake_kmeans_update_finish_batched(const float* sums, const int* counts, const cake_bf16* C_prev,
+                               long long B, int K, int D, float* out_C, cake_bf16* out_C_bf16,
+                               cake_stream_t stream);
+
+/*
  * lloyd (same paragraph: a Lloyd iteration is assign followed by centroid_update).
  * For t = 0 .. iters-1: assign against C_t (C_0 = C0), out_inertia[t] = sum_i out_dist_t[i],
  * then update -> C_{t+1}; the next assign reads C_{t+1} rounded to bf16.  Exactly `iters`

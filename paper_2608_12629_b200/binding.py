@@ -28,6 +28,7 @@ EXPORTS = [
     "cake_kmeans_assign_batched", "cake_kmeans_update", "cake_kmeans_update_batched", "cake_kmeans_lloyd",
     "cake_kmeans_lloyd_batched", "cake_kmeans_lloyd_host_device_bytes", "cake_kmeans_lloyd_host",
     "cake_kmeans_device_status", "cake_kmeans_selftest_bounded_wait", "cake_kmeans_assign_static",
+    "cake_kmeans_update_partial_batched", "cake_kmeans_update_finish_batched", "cake_kmeans_inertia_batched",
 ]
 
 _lib = None
@@ -63,6 +64,9 @@ def lib() -> ctypes.CDLL:
         L.cake_kmeans_device_status.argtypes = [vp, vp, ctypes.POINTER(i)]
         L.cake_kmeans_selftest_bounded_wait.argtypes = [vp, sz, i, vp]
         L.cake_kmeans_assign_static.argtypes = [vp, vp, ll, i, i, vp, vp, vp]
+        L.cake_kmeans_update_partial_batched.argtypes = [vp, vp, ll, ll, i, i, vp, vp, vp, sz, vp, u]
+        L.cake_kmeans_update_finish_batched.argtypes = [vp, vp, vp, ll, i, i, vp, vp, vp]
+        L.cake_kmeans_inertia_batched.argtypes = [vp, ll, ll, vp, i, vp]
         for name in EXPORTS:
             if name not in ("cake_strerror", "cake_kmeans_kernel_launches"):
                 getattr(L, name).restype = i
@@ -174,6 +178,60 @@ def cake_kmeans_update(X, idx, K, C_prev=None, out_C=None, out_C_bf16=None, out_
                                           _ptr(out_counts), _ptr(ws), ws.numel(), _stream(stream, X.device), flags)
     _check(rc, "cake_kmeans_update")
     return out_C, out_C_bf16, out_counts
+
+
+def cake_kmeans_update_partial(X, idx, K, out_sums=None, out_counts=None, ws=None, stream=None, flags=0):
+    """Sums and counts of the rows given: X bf16 [N,D] / [B,N,D], idx int32 -> (sums fp32 [..,K,D], counts int32 [..,K])."""
+    _want(X, torch.bfloat16, "X"), _want(idx, torch.int32, "idx")
+    batched = X.dim() == 3
+    B = X.shape[0] if batched else 1
+    N, D = X.shape[-2], X.shape[-1]
+    shape = (B, K, D) if batched else (K, D)
+    if out_sums is None:
+        out_sums = torch.empty(shape, dtype=torch.float32, device=X.device)
+    if out_counts is None:
+        out_counts = torch.empty(shape[:-1], dtype=torch.int32, device=X.device)
+    _want(out_sums, torch.float32, "out_sums"), _want(out_counts, torch.int32, "out_counts")
+    if ws is None:
+        ws = alloc_workspace(B, N, D, K, X.device)
+    with torch.cuda.device(X.device):
+        rc = lib().cake_kmeans_update_partial_batched(_ptr(X), _ptr(idx), B, N, D, K, _ptr(out_sums), _ptr(out_counts),
+                                                      _ptr(ws), ws.numel(), _stream(stream, X.device), flags)
+    _check(rc, "cake_kmeans_update_partial")
+    return out_sums, out_counts
+
+
+def cake_kmeans_update_finish(sums, counts, C_prev=None, out_C=None, out_C_bf16=None, stream=None):
+    """Division: sums fp32 [..,K,D], counts int32 [..,K] -> (C fp32, C bf16); empty clusters keep C_prev."""
+    _want(sums, torch.float32, "sums"), _want(counts, torch.int32, "counts")
+    K, D = sums.shape[-2], sums.shape[-1]
+    B = sums.shape[0] if sums.dim() == 3 else 1
+    if C_prev is not None:
+        _want(C_prev, torch.bfloat16, "C_prev")
+    if out_C is None:
+        out_C = torch.empty_like(sums)
+    if out_C_bf16 is None:
+        out_C_bf16 = torch.empty(sums.shape, dtype=torch.bfloat16, device=sums.device)
+    with torch.cuda.device(sums.device):
+        rc = lib().cake_kmeans_update_finish_batched(_ptr(sums), _ptr(counts), _ptr(C_prev), B, K, D, _ptr(out_C),
+                                                     _ptr(out_C_bf16), _stream(stream, sums.device))
+    _check(rc, "cake_kmeans_update_finish")
+    return out_C, out_C_bf16
+
+
+def cake_kmeans_inertia(dist, out_inertia=None, stride=1, stream=None):
+    """Sum of the distances of an assignment in fp64: dist fp32 [N] / [B,N] -> out_inertia[b * stride] (fp64)."""
+    _want(dist, torch.float32, "dist")
+    B = dist.shape[0] if dist.dim() == 2 else 1
+    N = dist.shape[-1]
+    if out_inertia is None:
+        out_inertia = torch.empty(B * stride, dtype=torch.float64, device=dist.device)
+    if out_inertia.dtype != torch.float64:
+        raise TypeError("out_inertia must be float64")
+    with torch.cuda.device(dist.device):
+        rc = lib().cake_kmeans_inertia_batched(_ptr(dist), B, N, _ptr(out_inertia), stride, _stream(stream, dist.device))
+    _check(rc, "cake_kmeans_inertia")
+    return out_inertia
 
 
 @dataclass

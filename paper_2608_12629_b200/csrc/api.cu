@@ -241,6 +241,59 @@ int cake_kmeans_update(const cake_bf16* X, const int* idx, long long N, int D, i
                                       ws_bytes, stream, flags);
 }
 
+int cake_kmeans_update_partial_batched(const cake_bf16* X, const int* idx, long long B, long long N, int D,
+                                       int K, float* out_sums, int* out_counts, void* ws, size_t ws_bytes,
+                                       cake_stream_t stream, unsigned flags) {
+    int rc = check_shape(B, N, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (!out_sums || !out_counts || !ws || (N > 0 && (!X || !idx))) return CAKE_ERR_NULL;
+    if (misaligned(X, 16) || misaligned(idx, 4) || misaligned(out_sums, 16) || misaligned(out_counts, 4))
+        return CAKE_ERR_ALIGN;
+    if (K > 8192) return CAKE_ERR_UNSUPPORTED;   // above, the sort route writes means, not sums
+    Workspace w;
+    rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
+    if (rc != CAKE_OK) return rc;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int Bi = static_cast<int>(B);
+    unsigned path = flags & CAKE_UPDATE_MASK;
+    if (path == CAKE_UPDATE_AUTO) path = update_slab_supports(D, K) ? CAKE_UPDATE_SLAB : CAKE_UPDATE_SORT;
+    if (path == CAKE_UPDATE_SLAB)
+        return launch_update_slab(X, idx, Bi, N, D, K, out_sums, out_counts, w.status, 0, s);
+    if (path == CAKE_UPDATE_SORT) {
+        UpdateScratch scr{out_sums, w.nvalid, w.cursor, w.pairs, w.part, w.done, w.rank};
+        bool divided = false;
+        rc = launch_update_sort(X, idx, Bi, N, D, K, scr, out_counts, nullptr, nullptr, nullptr, &divided, w.status, s);
+        return (rc == CAKE_OK && divided) ? CAKE_ERR_UNSUPPORTED : rc;
+    }
+    return CAKE_ERR_UNSUPPORTED;
+}
+
+int cake_kmeans_update_finish_batched(const float* sums, const int* counts, const cake_bf16* C_prev, long long B,
+                                      int K, int D, float* out_C, cake_bf16* out_C_bf16, cake_stream_t stream) {
+    int rc = check_shape(B, 0, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (!sums || !counts || !out_C) return CAKE_ERR_NULL;
+    if (misaligned(sums, 16) || misaligned(counts, 4) || misaligned(C_prev, 16) || misaligned(out_C, 16) ||
+        misaligned(out_C_bf16, 16))
+        return CAKE_ERR_ALIGN;
+    if (launch_finalize(sums, counts, C_prev, static_cast<int>(B), K, D, out_C, out_C_bf16, false, nullptr, nullptr,
+                        reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return CAKE_ERR_CUDA;
+    return CAKE_OK;
+}
+
+int cake_kmeans_inertia_batched(const float* dist, long long B, long long N, double* out_inertia, int inertia_stride,
+                                cake_stream_t stream) {
+    if (B < 1 || B > 65535 || N < 0 || inertia_stride < 1) return CAKE_ERR_SHAPE;
+    if (!out_inertia || (N > 0 && !dist)) return CAKE_ERR_NULL;
+    if (misaligned(dist, 4) || misaligned(out_inertia, 8)) return CAKE_ERR_ALIGN;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemset2DAsync(out_inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
+                          static_cast<size_t>(B), s) != cudaSuccess)
+        return CAKE_ERR_CUDA;
+    return launch_inertia(dist, static_cast<int>(B), N, out_inertia, inertia_stride, s) == cudaSuccess ? CAKE_OK : CAKE_ERR_CUDA;
+}
+
 int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long B, long long N, int D,
                               int K, int iters, float* out_C, cake_bf16* out_C_bf16, int* out_idx,
                               float* out_dist, int* out_counts, double* out_inertia, void* ws,
