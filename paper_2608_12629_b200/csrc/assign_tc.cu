@@ -1203,7 +1203,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     const i64 budget = static_cast<i64>(di.smem_optin) - fixed;
     const i64 xbuf = static_cast<i64>(p.nchunks) * X_CHUNK_BYTES + AUG_A_BYTES;
     int want_xbuf = p.n_tiles <= 2 ? MAX_XBUF : 2;
-    if (p.nchunks >= 4 && p.n_tiles >= 8) want_xbuf = 1;
+    if ((p.nchunks >= 4 && p.n_tiles >= 8) || (p.nchunks == 3 && p.n_tiles >= 16)) want_xbuf = 1;   // measured
     // two chunks per ring stage when the chunk count is even (one wait and one commit per stage), unless the
     // ring would then hold a single stage, X is the bound (few centroid tiles: X buffers matter more) or the
     // last chunk is a partial one (short tiles: waiting for both chunks costs more than the barriers saved)
