@@ -251,11 +251,9 @@ __device__ __forceinline__ void exact_scan32(const uint32_t (&r)[32], int col_ba
 // but consecutive ones, so that it meets few problems (every change of problem reloads the resident tile:
 // 32 problems of 512 row tiles on 148 CTAs change problem every 3.5 tiles when interleaved).
 // first_tile: (problem, row tile) of the CTA's first tile; tile_step: distance to its next one.
-template <bool XLOAD>
-__device__ __forceinline__ bool tiles_consecutive(const Params& p) { return XLOAD && p.res_c && p.B > 1; }
-template <bool XLOAD>
+template <bool CONSEC>
 __device__ __forceinline__ void first_tile(const Params& p, int& tb, int& tmt) {
-    if (tiles_consecutive<XLOAD>(p)) {
+    if (CONSEC) {
         const i64 q = p.total_tiles / gridDim.x, r = p.total_tiles - q * gridDim.x;
         const i64 first = blockIdx.x * q + (static_cast<i64>(blockIdx.x) < r ? static_cast<i64>(blockIdx.x) : r);
         tb = static_cast<int>(first / p.m_tiles);
@@ -265,12 +263,11 @@ __device__ __forceinline__ void first_tile(const Params& p, int& tb, int& tmt) {
         tmt = static_cast<int>(blockIdx.x % static_cast<unsigned>(p.m_tiles));
     }
 }
-template <bool XLOAD>
-__device__ __forceinline__ int tile_step(const Params& p) {
-    return tiles_consecutive<XLOAD>(p) ? 1 : static_cast<int>(gridDim.x);
-}
+template <bool CONSEC>
+__device__ __forceinline__ int tile_step() { return CONSEC ? 1 : static_cast<int>(gridDim.x); }
 
-template <bool PACKED, bool XLOAD>
+// CONSEC: consecutive row tiles per CTA (a batch of problems with resident centroids: see first_tile)
+template <bool PACKED, bool XLOAD, bool CONSEC = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
                  const Params p) {
@@ -375,8 +372,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 int cur_b = -1;
                 uint32_t pc = 0;
                 int tb, tmt;
-                first_tile<XLOAD>(p, tb, tmt);
-                const int tmt_step = tile_step<XLOAD>(p);
+                first_tile<CONSEC>(p, tb, tmt);
+                const int tmt_step = tile_step<CONSEC>();
                 for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                     if (tb != cur_b) {
                         ok = wait_bar(&ctrl->ring_empty[0], (pc & 1u) ^ 1u, ctrl, p.status);
@@ -460,8 +457,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (lane == 0) {
             uint32_t ixb = 0, ixph = 0;
             int tb, tmt;
-            first_tile<XLOAD>(p, tb, tmt);
-                const int tmt_step = tile_step<XLOAD>(p);
+            first_tile<CONSEC>(p, tb, tmt);
+                const int tmt_step = tile_step<CONSEC>();
             bool ok = true;
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 ok = wait_bar(&ctrl->x_empty[ixb], ixph ^ 1u, ctrl, p.status);
@@ -512,8 +509,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 int cur_b = -1;
                 uint32_t pc = 0, tile_it = 0;
                 int tb, tmt;
-                first_tile<XLOAD>(p, tb, tmt);
-                const int tmt_step = tile_step<XLOAD>(p);
+                first_tile<CONSEC>(p, tb, tmt);
+                const int tmt_step = tile_step<CONSEC>();
                 const uint32_t nxb = static_cast<uint32_t>(p.n_xbuf);
                 const uint32_t idesc_aug_n = ptx::umma_idesc_bf16(BLOCK_M, p.alt_epi ? p.alt_epi : BLOCK_N);
                 const uint32_t idesc_main_n = idesc_aug_n | ptx::UMMA_IDESC_NEGATE_B;
@@ -676,8 +673,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         uint32_t xb = 0, xph = 0;
         bool ok = true;
         int nb = 0, nmt = 0;   // (problem, row tile), stepped: only where the CTA's tiles may be consecutive
-        if (XLOAD) first_tile<XLOAD>(p, nb, nmt);
-        const int nmt_step = tile_step<XLOAD>(p);
+        if (CONSEC) first_tile<CONSEC>(p, nb, nmt);
+        const int nmt_step = tile_step<CONSEC>();
         for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
             ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);
             if (!ok) break;
@@ -702,7 +699,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             // exponent E is 0 or 1 modulo 4 (then bits(M) * 128 is 0 or 2^30 modulo 2^32 and the keys
             // of the row are positive floats); m = M / 4096
             int tb;
-            if (XLOAD) {
+            if (CONSEC) {
                 tb = nb;
                 nmt += nmt_step;
                 while (nmt >= p.m_tiles) { nmt -= p.m_tiles; ++nb; }
@@ -754,8 +751,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         };
         // (problem, row tile) of the current tile, stepped instead of divided
         int b, mt;
-        first_tile<XLOAD>(p, b, mt);
-        const int mt_step = tile_step<XLOAD>(p);
+        first_tile<CONSEC>(p, b, mt);
+        const int mt_step = tile_step<CONSEC>();
         auto next_tile = [&]() {
             mt += mt_step;
             while (mt >= p.m_tiles) { mt -= p.m_tiles; ++b; }
@@ -1269,14 +1266,17 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf +
                               static_cast<size_t>(p.n_stages) * p.stage_bytes;
     using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const Params);
-    Kernel kernel = exact ? (xload ? assign_tc_kernel<false, true> : assign_tc_kernel<false, false>)
-                          : (xload ? assign_tc_kernel<true, true> : assign_tc_kernel<true, false>);
+    const bool consec = xload && p.res_c && B > 1;
+    Kernel kernel = exact ? (consec ? assign_tc_kernel<false, true, true> : xload ? assign_tc_kernel<false, true> : assign_tc_kernel<false, false>)
+                          : (consec ? assign_tc_kernel<true, true, true> : xload ? assign_tc_kernel<true, true> : assign_tc_kernel<true, false>);
     static int attr_done_for_device = -1;  // benign race: the attribute calls are idempotent
     if (attr_done_for_device != di.device) {
         if (cudaFuncSetAttribute(assign_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
-            cudaFuncSetAttribute(assign_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
+            cudaFuncSetAttribute(assign_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
             return CAKE_ERR_CUDA;
         attr_done_for_device = di.device;
     }
