@@ -887,14 +887,21 @@ zero_sums_counts_kernel(float4* __restrict__ sums4, i64 n4, int* __restrict__ co
 template <int LPR, bool CLUSTER, bool WIDE = false>
 __global__ void __launch_bounds__(SLAB_THREADS, 1)
 slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx, i64 N, int D, int K, int S,
-                   int rowbits, float* __restrict__ sums, int* __restrict__ counts, int* status) {
+                   int rowbits, float* __restrict__ sums, int* __restrict__ counts, int* status, i64 Nprob,
+                   int Kidx) {
     extern __shared__ int sm[];
     int* h = sm;                                                   // [K] this CTA's rows per cluster
     int* off = sm + K;                                             // [K] first position of this CTA's rows of a cluster
     uint32_t* sorted = reinterpret_cast<uint32_t*>(sm + 2 * K);    // [S] this CTA's share of the order
     __shared__ int warp_tot[SLAB_THREADS / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int b = blockIdx.y;
+    // Nprob > 0 (never with thread-block clusters): the problems of a batch as one run of N = B * Nprob rows,
+    // dealt to the CTAs without regard to where a problem ends (B problems seldom divide the SMs evenly).  A
+    // slab is at most one problem long, so it holds rows of problem b and, from row `split` on, of problem
+    // b + 1: those count as clusters Kidx .. 2 Kidx - 1 (K = 2 Kidx), which is where they lie in sums and
+    // counts seen from problem b.  Otherwise Kidx = K, blockIdx.y is the problem and split is never reached.
+    const bool flat = !CLUSTER && Nprob > 0;
+    int b = blockIdx.y;
     unsigned F = 1, c = 0;
     if constexpr (CLUSTER) {
         F = cg::this_cluster().num_blocks();
@@ -903,8 +910,14 @@ slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
     const i64 super_row0 = static_cast<i64>(blockIdx.x / F) * F * S;   // first row of the cluster's rows
     const i64 r0 = super_row0 + static_cast<i64>(c) * S;
     const int rows = r0 >= N ? 0 : static_cast<int>(r0 + S <= N ? S : N - r0);
-    const int* idx_b = idx + static_cast<size_t>(b) * N + (rows ? r0 : 0);
-    int* counts_b = counts + static_cast<size_t>(b) * K;
+    int split = S;
+    if (flat) {
+        b = static_cast<int>(r0 / Nprob);
+        const i64 left = static_cast<i64>(b + 1) * Nprob - r0;      // rows up to the end of problem b
+        split = left < S ? static_cast<int>(left) : S;
+    }
+    const int* idx_b = idx + (flat ? 0 : static_cast<size_t>(b) * N) + (rows ? r0 : 0);
+    int* counts_b = counts + static_cast<size_t>(b) * Kidx;
 
     for (int e = tid; e < K; e += SLAB_THREADS) h[e] = 0;
     __syncthreads();
@@ -929,9 +942,10 @@ slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
 #pragma unroll
     for (int u = 0; u < SLAB_VPT; ++u) {
         const int i = ((u >> 2) * SLAB_THREADS + tid) * 4 + (u & 3);
-        const bool ok = static_cast<unsigned>(kv[u]) < static_cast<unsigned>(K);
+        const bool ok = static_cast<unsigned>(kv[u]) < static_cast<unsigned>(Kidx);
         if (!ok && i < rows) bad = true;
         if (!ok || i >= rows) kv[u] = -1;
+        else if (i >= split) kv[u] += Kidx;
         rk[u] = kv[u] >= 0 ? atomicAdd(&h[kv[u]], 1) : 0;
     }
     if (bad) atomicCAS(status, CAKE_OK, CAKE_ERR_BAD_INDEX);
@@ -1013,8 +1027,8 @@ slab_update_kernel(const cake_bf16* __restrict__ X, const int* __restrict__ idx,
     const int G = D >> 3;
     const int sl = lane % LPR;
     const int gid = warp * GROUPS + lane / LPR;
-    const uint4* Xg = reinterpret_cast<const uint4*>(X) + (static_cast<size_t>(b) * N + super_row0) * G;
-    float* sums_b = sums + static_cast<size_t>(b) * K * D;
+    const uint4* Xg = reinterpret_cast<const uint4*>(X) + ((flat ? 0 : static_cast<size_t>(b) * N) + super_row0) * G;
+    float* sums_b = sums + static_cast<size_t>(b) * Kidx * D;
     const uint32_t rowmask = (1u << rowbits) - 1u;
     const int seglen = max(SLAB_AHEAD, (mine + NGROUPS - 1) / NGROUPS);
     const int base = gid * seglen, end = min(base + seglen, mine);
@@ -1351,9 +1365,10 @@ struct SlabPlan {
     int n_ctas;    // CTAs per problem (multiple of F)
     int F;         // CTAs per thread-block cluster
     int rowbits;   // bits of a row number inside a cluster's F*S rows
+    bool flat;     // slabs dealt over the rows of all problems (n_ctas is then the total)
 };
 
-using SlabKernel = void (*)(const cake_bf16*, const int*, i64, int, int, int, int, float*, int*, int*);
+using SlabKernel = void (*)(const cake_bf16*, const int*, i64, int, int, int, int, float*, int*, int*, i64, int);
 
 SlabKernel slab_kernel_for(int lpr, bool cluster, bool wide) {
     if (wide) return cluster ? slab_update_kernel<32, true, true> : slab_update_kernel<32, false, true>;
@@ -1437,6 +1452,31 @@ static int slab_make_plan(const DeviceInfo& di, int B, i64 N, int D, int K, int 
         if (static_cast<i64>(pl.S) * F >= static_cast<i64>(SLAB_GROW_RUN) * K || pl.n_ctas <= F) break;
     }
     if (best.F == 0) return CAKE_ERR_UNSUPPORTED;
+    best.flat = false;
+    // A batch whose problems leave SMs idle (32 problems on 148 SMs: 4 CTAs each, 20 SMs without work): deal
+    // the rows of all problems to the CTAs instead.  Needs no thread-block clusters, a slab no longer than a
+    // problem, and twice K counters in shared memory.
+    if (B > 1 && best.F == 1 && !force_f && 2 * static_cast<i64>(K) <= SLAB_MAX_K) {
+        const i64 total = static_cast<i64>(B) * N;
+        const int slots = di.sm_count;
+        for (int w = 1; w <= 64; ++w) {
+            i64 rows = (total + static_cast<i64>(w) * slots - 1) / (static_cast<i64>(w) * slots);
+            if (rows < 1024) rows = 1024;
+            rows = (rows + 3) / 4 * 4;
+            if (rows > SLAB_MAX_ROWS) continue;
+            const i64 n = (total + rows - 1) / rows;
+            const i64 waves = (n + slots - 1) / slots, waves_now = (static_cast<i64>(best.n_ctas) * B + slots - 1) / slots;
+            // taken when it runs as many rows per run and fewer or equally many, fuller waves
+            if (rows <= N && rows >= static_cast<i64>(SLAB_GROW_RUN) * K && waves * rows < waves_now * best.S) {
+                best.flat = true;
+                best.S = static_cast<int>(rows);
+                best.n_ctas = static_cast<int>(n);
+                best.rowbits = 1;
+                while ((static_cast<i64>(1) << best.rowbits) < rows) ++best.rowbits;
+            }
+            break;
+        }
+    }
     *out = best;
     return CAKE_OK;
 }
@@ -1485,9 +1525,11 @@ int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
     if (rc != CAKE_OK) return rc;
     const int lpr = slab_lpr(D);
     SlabKernel kernel = slab_kernel_for(lpr, pl.F > 1, D > 256);
-    const size_t smem = slab_smem_bytes(K, pl.S);
+    const int Kh = pl.flat ? 2 * K : K;                      // counters per CTA
+    const i64 Nk = pl.flat ? static_cast<i64>(B) * N : N;    // rows the grid's x dimension is dealt over
+    const size_t smem = slab_smem_bytes(Kh, pl.S);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(pl.n_ctas), static_cast<unsigned>(B));
+    cfg.gridDim = dim3(static_cast<unsigned>(pl.n_ctas), pl.flat ? 1u : static_cast<unsigned>(B));
     cfg.blockDim = dim3(SLAB_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
@@ -1501,7 +1543,8 @@ int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
     at[1].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = pl.F > 1 ? 2 : 1;
-    if (cudaLaunchKernelEx(&cfg, kernel, X, idx, N, D, K, pl.S, pl.rowbits, sums, counts, status) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kernel, X, idx, Nk, D, Kh, pl.S, pl.rowbits, sums, counts, status,
+                           pl.flat ? N : static_cast<i64>(0), K) != cudaSuccess) {
         cudaGetLastError();
         return CAKE_ERR_CUDA;
     }

@@ -275,6 +275,32 @@ def test_update_batched_unaligned_problem_size(flag):
                              inputs.to_bits(Cb[b]), counts[b].cpu().numpy())
 
 
+@pytest.mark.parametrize("B,N,D,K", [(5, 40000, 64, 100), (32, 65536, 128, 256), (7, 20001, 24, 33), (3, 70001, 128, 1000),
+                                     (9, 16385, 8, 2000)])
+def test_update_batch_dealt_over_all_ctas(B, N, D, K):
+    """Batches whose problems do not divide the SMs evenly: the slab route deals the rows of all problems to the
+    CTAs, so slabs straddle the end of a problem (also with N % 4 != 0, bad indices next to the boundary, an empty
+    cluster).  Graded per problem against the oracle, and equal to the route with one grid row per problem."""
+    g = torch.Generator().manual_seed(B * N + K)
+    X = torch.randint(-4, 5, (B, N, D), generator=g).to(torch.bfloat16)       # integers: any summation order is exact
+    C = torch.randint(-4, 5, (B, K, D), generator=g).to(torch.bfloat16)
+    idx = torch.randint(0, K, (B, N), generator=g, dtype=torch.int32)
+    idx[idx == 1] = 0
+    idx[0, N - 1] = K          # last row of problem 0 and first row of problem 1: skipped, status raised
+    idx[1, 0] = -5
+    Xd, idxd, Cd = X.to(DEV), idx.to(DEV), C.to(DEV)
+    ws = cake.alloc_workspace(B, N, D, K, DEV)
+    Cf, Cb, counts = cake.cake_kmeans_update(Xd, idxd, K, C_prev=Cd, ws=ws)
+    check_status(ws, cake.CAKE_ERR_BAD_INDEX)
+    ws2 = cake.alloc_workspace(B, N, D, K, DEV)
+    Cf1, Cb1, counts1 = cake.cake_kmeans_update(Xd, idxd, K, C_prev=Cd, ws=ws2, flags=cake.CAKE_UPDATE_SLAB_F1)
+    assert torch.equal(Cf, Cf1) and torch.equal(Cb, Cb1) and torch.equal(counts, counts1)
+    for b in range(B if B * N * D < 5e7 else 3):
+        keep = (idx[b] >= 0) & (idx[b] < K)
+        grading.grade_update(inputs.to_bits(X[b])[keep.numpy()], idx[b][keep].numpy(), K, inputs.to_bits(C[b]),
+                             Cf[b].cpu().numpy(), inputs.to_bits(Cb[b]), counts[b].cpu().numpy())
+
+
 @pytest.mark.parametrize("D", [8, 64, 256])
 def test_update_many_clusters_few_rows_with_and_without_prev(D):
     """K > 8192 with a few rows per cluster: the sort route hands every cluster to one warp, which writes
