@@ -78,6 +78,7 @@ constexpr uint32_t AUG_B_BYTES = kAssignAugTileBytes;    // 4 KiB
 constexpr uint32_t AUG_ZERO_BYTES = BLOCK_N * 16;        // 4 KiB of zeros
 constexpr int MAX_STAGES = 6;
 constexpr int MAX_XBUF = 4;
+constexpr int MAX_XCHUNKS = 8;                           // 64-column chunks of an X tile (D <= 512)
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t CTRL_BYTES = 6144;  // barriers, TMEM pointer, abort flag, merge scratch, row exponents
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
@@ -117,6 +118,9 @@ struct Params {
 
 struct Ctrl {  // lives in shared memory
     uint64_t x_full[MAX_XBUF], x_empty[MAX_XBUF];
+    // split X buffer (a single buffer whose 64-column chunks are filled and handed back one by one): chunk
+    // c < nchunks - 1 has these barriers, the last chunk x_full[0] / x_empty[0]
+    uint64_t xc_full[MAX_XCHUNKS], xc_empty[MAX_XCHUNKS];
     uint64_t ring_full[MAX_STAGES], ring_empty[MAX_STAGES];
     uint64_t tmem_full[2];
     // release of accumulator a, one barrier per issuer that may take it next: each barrier has a
@@ -267,7 +271,9 @@ template <bool CONSEC>
 __device__ __forceinline__ int tile_step() { return CONSEC ? 1 : static_cast<int>(gridDim.x); }
 
 // CONSEC: consecutive row tiles per CTA (a batch of problems with resident centroids: see first_tile)
-template <bool PACKED, bool XLOAD, bool CONSEC = false>
+// XSPLIT: one X buffer (all that fits beside the centroid ring when D > 256) whose chunks are loaded, consumed
+// and handed back one by one, so that the next row tile's first chunks arrive while this one's last are in use
+template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
                  const Params p) {
@@ -296,6 +302,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             // MMA issuers + 4 norm warps + the 4 epilogue warps that read the row exponents
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), ((XLOAD && p.res_c == 1) ? 1 : NUM_ISSUERS) + 4 + 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
+        }
+        for (int i = 0; i < MAX_XCHUNKS; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&ctrl->xc_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->xc_empty[i]), NUM_ISSUERS + 4);   // MMA issuers + 4 norm warps
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1);
@@ -461,6 +471,18 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const int tmt_step = tile_step<CONSEC>();
             bool ok = true;
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                if (XSPLIT) {
+                    // chunk by chunk, each as soon as the previous row tile is done with it
+                    for (int c = 0; ok && c < p.nchunks; ++c) {
+                        const bool lastc = c == p.nchunks - 1;
+                        ok = wait_bar(lastc ? &ctrl->x_empty[0] : &ctrl->xc_empty[c], ixph ^ 1u, ctrl, p.status);
+                        if (!ok) break;
+                        const uint32_t full = ptx::smem_u32(lastc ? &ctrl->x_full[0] : &ctrl->xc_full[c]);
+                        ptx::mbar_arrive_expect_tx(full, X_CHUNK_BYTES);
+                        ptx::tma_load_3d(x_base + c * X_CHUNK_BYTES, &tmap_x, full, c * KCHUNK, tmt * BLOCK_M, tb);
+                    }
+                    if (!ok) break;
+                } else {
                 ok = wait_bar(&ctrl->x_empty[ixb], ixph ^ 1u, ctrl, p.status);
                 if (!ok) break;
                 const uint32_t xfull = ptx::smem_u32(&ctrl->x_full[ixb]);
@@ -468,6 +490,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 for (int c = 0; c < p.nchunks; ++c)
                     ptx::tma_load_3d(x_base + ixb * xbuf_bytes + c * X_CHUNK_BYTES, &tmap_x, xfull,
                                      c * KCHUNK, tmt * BLOCK_M, tb);
+                }
                 if (++ixb == static_cast<uint32_t>(p.n_xbuf)) { ixb = 0; ixph ^= 1u; }
                 tmt += tmt_step;
                 while (tmt >= p.m_tiles) { tmt -= p.m_tiles; ++tb; }
@@ -581,9 +604,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 // every phase of the shared barriers is observed, also in row / centroid tiles this
                 // issuer has no work in: a parity wait must never fall two phases behind
-                ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);
+                if (!XSPLIT) ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);   // (split: chunk by chunk, below)
                 if (!ok) break;
                 bool have_aug = false;
+                bool owned = false;   // this issuer had a centroid tile of this row tile (at most one when XSPLIT)
                 const uint32_t a_lo_tile = ptx::umma_desc_lo_sw128(x_base + xb * xbuf_bytes);
                 const uint32_t auga_lo = ptx::umma_desc_lo_aug(smem_base + auga_off + xb * AUG_A_BYTES,
                                                                smem_base + zero_off);
@@ -611,8 +635,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         if (acc) ++rel1; else ++rel0;
                     }
                     ptx::tc_fence_after();
+                    owned = true;
                     uint32_t a_lo = a_lo_tile;
                     for (int c0 = 0; c0 < p.nchunks; c0 += p.cps) {
+                        if (XSPLIT) {   // (one chunk per stage in this mode) this chunk of X has landed
+                            ok = wait_bar(c0 == p.nchunks - 1 ? &ctrl->x_full[0] : &ctrl->xc_full[c0], xph, ctrl, p.status);
+                            if (!ok) break;
+                        }
                         ok = wait_bar(&ctrl->ring_full[s], ph, ctrl, p.status);
                         if (!ok) break;
                         const uint32_t stage = ring_base + s * p.stage_bytes;
@@ -650,10 +679,21 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                                       ptx::UMMA_DESC_HI_AUG, idesc_aug);
                         }
                         ptx::umma_commit(ptx::smem_u32(&ctrl->ring_empty[s]));
+                        // split X buffer: this issuer's only tile of the row tile is done with the chunk
+                        if (XSPLIT && c0 < p.nchunks - 1) ptx::umma_commit(ptx::smem_u32(&ctrl->xc_empty[c0]));
                         if (++s == nstg) { s = 0; ph ^= 1u; }
                     }
                     if (!ok) break;
                     ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[acc]));
+                }
+                if (XSPLIT && ok && !owned) {
+                    // no tile of this row tile: see every chunk filled (a parity wait must not fall two phases
+                    // behind) and hand it back at once
+                    for (int c = 0; ok && c < p.nchunks - 1; ++c) {
+                        ok = wait_bar(&ctrl->xc_full[c], xph, ctrl, p.status);
+                        if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->xc_empty[c]));
+                    }
+                    if (ok) ok = wait_bar(&ctrl->x_full[0], xph, ctrl, p.status);
                 }
                 if (ok && !have_aug) ok = wait_bar(&ctrl->auga_full[xb], xph, ctrl, p.status);
                 // this issuer's MMAs on the X buffer are done when this commit fires (it fires at once
@@ -676,11 +716,20 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         if (CONSEC) first_tile<CONSEC>(p, nb, nmt);
         const int nmt_step = tile_step<CONSEC>();
         for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
-            ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);
+            if (!XSPLIT) ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);
             if (!ok) break;
             const uint8_t* xrow = smem + xb * xbuf_bytes + r * 128;
             float xn0 = 0.f, xn1 = 0.f, xn2 = 0.f, xn3 = 0.f;
             for (int c = 0; c < p.nchunks; ++c) {
+                if (XSPLIT) {
+                    // chunk by chunk: the one before is handed back once the whole warp has read it
+                    if (c > 0) {
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->xc_empty[c - 1]));
+                    }
+                    ok = wait_bar(c == p.nchunks - 1 ? &ctrl->x_full[0] : &ctrl->xc_full[c], xph, ctrl, p.status);
+                    if (!ok) break;
+                }
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
                     const uint4 w = *reinterpret_cast<const uint4*>(xrow + c * X_CHUNK_BYTES +
@@ -692,6 +741,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     a = bf16lo(w.w); xn2 = fmaf(a, a, xn2); a = bf16hi(w.w); xn3 = fmaf(a, a, xn3);
                 }
             }
+            if (!ok) break;
             const float xn = (xn0 + xn1) + (xn2 + xn3);
             uint32_t hi, mid, lo;
             split3(0.5f * xn, hi, mid, lo);
@@ -1267,8 +1317,12 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
                               static_cast<size_t>(p.n_stages) * p.stage_bytes;
     using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const Params);
     const bool consec = xload && p.res_c && B > 1;
-    Kernel kernel = exact ? (consec ? assign_tc_kernel<false, true, true> : xload ? assign_tc_kernel<false, true> : assign_tc_kernel<false, false>)
-                          : (consec ? assign_tc_kernel<true, true, true> : xload ? assign_tc_kernel<true, true> : assign_tc_kernel<true, false>);
+    // a single X buffer (D > 256) is filled and handed back chunk by chunk
+    const bool xsplit = xload && !p.res_c && p.n_xbuf == 1 && p.cps == 1 && p.nchunks <= MAX_XCHUNKS;
+    Kernel kernel = exact ? (consec ? assign_tc_kernel<false, true, true> : xsplit ? assign_tc_kernel<false, true, false, true>
+                             : xload ? assign_tc_kernel<false, true> : assign_tc_kernel<false, false>)
+                          : (consec ? assign_tc_kernel<true, true, true> : xsplit ? assign_tc_kernel<true, true, false, true>
+                             : xload ? assign_tc_kernel<true, true> : assign_tc_kernel<true, false>);
     static int attr_done_for_device = -1;  // benign race: the attribute calls are idempotent
     if (attr_done_for_device != di.device) {
         if (cudaFuncSetAttribute(assign_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
@@ -1276,7 +1330,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             cudaFuncSetAttribute(assign_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
-            cudaFuncSetAttribute(assign_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
+            cudaFuncSetAttribute(assign_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<false, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
             return CAKE_ERR_CUDA;
         attr_done_for_device = di.device;
     }
