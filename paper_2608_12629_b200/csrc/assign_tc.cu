@@ -305,7 +305,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         }
         for (int i = 0; i < MAX_XCHUNKS; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->xc_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->xc_empty[i]), NUM_ISSUERS + 4);   // MMA issuers + 4 norm warps
+            ptx::mbar_init(ptx::smem_u32(&ctrl->xc_empty[i]), ((XLOAD && p.res_c == 1) ? 1 : NUM_ISSUERS) + 4);   // MMA issuers + 4 norm warps
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1);
@@ -553,7 +553,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     const bool both = p.res_c == 2;
                     if (!both && (tile_it & 1u) != iss) continue;
                     const uint32_t rxb = tile_it % nxb, rxph = (tile_it / nxb) & 1u;
-                    ok = wait_bar(&ctrl->x_full[rxb], rxph, ctrl, p.status);
+                    // (split X buffer: both issuers share the one buffer, so an issuer sees only every other
+                    // phase of its barriers and may look at them only once it has the turn: the other issuer
+                    // has then seen all of the previous row tile's phases complete)
+                    if (!XSPLIT) ok = wait_bar(&ctrl->x_full[rxb], rxph, ctrl, p.status);
                     if (!ok) break;
                     const uint32_t use = both ? tile_it : tile_it >> 1;   // how often this accumulator has been used before
                     if (use > 0u) {
@@ -576,6 +579,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     const uint32_t c_base = ring_base + (both ? iss * p.nchunks * p.stage_bytes : 0u);   // this issuer's centroid tile
                     uint32_t a_lo = ptx::umma_desc_lo_sw128(x_base + rxb * xbuf_bytes);
                     for (int c = 0; c < p.nchunks; ++c, a_lo += X_CHUNK_BYTES >> 4) {
+                        if (XSPLIT) {
+                            ok = wait_bar(c == p.nchunks - 1 ? &ctrl->x_full[0] : &ctrl->xc_full[c], rxph, ctrl, p.status);
+                            if (!ok) break;
+                        }
                         const uint32_t b_lo = ptx::umma_desc_lo_sw128(c_base + c * p.stage_bytes);
                         const int nk = (c == p.nchunks - 1) ? p.ksteps_last : KCHUNK / UMMA_K;
                         if (c == 0)
@@ -587,7 +594,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         for (int ks = 1; ks < nk; ++ks)
                             ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
                                                       b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main_n);
+                        if (XSPLIT && c < p.nchunks - 1) ptx::umma_commit(ptx::smem_u32(&ctrl->xc_empty[c]));
                     }
+                    if (!ok) break;
                     ptx::mbar_arrive(ptx::smem_u32(&ctrl->turn[iss ^ 1u]));
                     ok = wait_bar(&ctrl->auga_full[rxb], rxph, ctrl, p.status);
                     if (!ok) break;
@@ -822,14 +831,24 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             // (the X buffer is not refilled before the issuer's MMAs on it have completed either)
             const uint32_t axb = tile_it % static_cast<uint32_t>(p.n_xbuf);
             const uint32_t axph = (tile_it / static_cast<uint32_t>(p.n_xbuf)) & 1u;
-            ok = wait_bar(&ctrl->auga_full[axb], axph, ctrl, p.status);
-            if (!ok) break;
-            const int rowE = ctrl->row_e[axb][r];
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
+            int rowE = 0;
+            if (!XSPLIT) {
+                ok = wait_bar(&ctrl->auga_full[axb], axph, ctrl, p.status);
+                if (!ok) break;
+                rowE = ctrl->row_e[axb][r];
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
+            }
             const uint32_t as = tile_it & 1u, aph = (tile_it >> 1) & 1u;
             ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
             if (!ok) break;
+            if (XSPLIT) {
+                // one X buffer for both warpgroups: this one sees only every other phase of its barriers, so it
+                // reads the exponents once its accumulator is complete (the issuer waited for them)
+                rowE = ctrl->row_e[0][r];
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[0]));
+            }
             ptx::tc_fence_after();
             float best = __uint_as_float(F32_INF);
             int bsel = 0;
@@ -1295,6 +1314,15 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
                 break;
             }
         }
+        // D > 256: one X buffer beside the resident tile, filled and handed back chunk by chunk
+        if (!p.res_c && p.nchunks <= MAX_STAGES && p.nchunks <= MAX_XCHUNKS && c_bytes + xbuf <= budget) {
+            p.res_c = 1;
+            p.alt_epi = c_rows;
+            p.cps = 1;
+            p.stage_bytes = static_cast<uint32_t>(c_rows) * 128u + AUG_B_BYTES;
+            p.n_stages = p.nchunks;
+            p.n_xbuf = 1;
+        }
     }
     if (p.n_tiles == 2) {
         // two centroid tiles: both stay in shared memory if at least two X buffers fit beside them (D <= 128)
@@ -1318,11 +1346,16 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const Params);
     const bool consec = xload && p.res_c && B > 1;
     // a single X buffer (D > 256) is filled and handed back chunk by chunk
-    const bool xsplit = xload && !p.res_c && p.n_xbuf == 1 && p.cps == 1 && p.nchunks <= MAX_XCHUNKS;
-    Kernel kernel = exact ? (consec ? assign_tc_kernel<false, true, true> : xsplit ? assign_tc_kernel<false, true, false, true>
-                             : xload ? assign_tc_kernel<false, true> : assign_tc_kernel<false, false>)
-                          : (consec ? assign_tc_kernel<true, true, true> : xsplit ? assign_tc_kernel<true, true, false, true>
-                             : xload ? assign_tc_kernel<true, true> : assign_tc_kernel<true, false>);
+    const bool xsplit = xload && p.res_c != 2 && p.n_xbuf == 1 && p.cps == 1 && p.nchunks <= MAX_XCHUNKS;
+    Kernel kernel;
+    if (!xload)
+        kernel = exact ? assign_tc_kernel<false, false> : assign_tc_kernel<true, false>;
+    else if (exact)
+        kernel = consec ? (xsplit ? assign_tc_kernel<false, true, true, true> : assign_tc_kernel<false, true, true, false>)
+                        : (xsplit ? assign_tc_kernel<false, true, false, true> : assign_tc_kernel<false, true, false, false>);
+    else
+        kernel = consec ? (xsplit ? assign_tc_kernel<true, true, true, true> : assign_tc_kernel<true, true, true, false>)
+                        : (xsplit ? assign_tc_kernel<true, true, false, true> : assign_tc_kernel<true, true, false, false>);
     static int attr_done_for_device = -1;  // benign race: the attribute calls are idempotent
     if (attr_done_for_device != di.device) {
         if (cudaFuncSetAttribute(assign_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
@@ -1332,7 +1365,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             cudaFuncSetAttribute(assign_tc_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
-            cudaFuncSetAttribute(assign_tc_kernel<false, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
+            cudaFuncSetAttribute(assign_tc_kernel<false, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<false, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
             return CAKE_ERR_CUDA;
         attr_done_for_device = di.device;
     }

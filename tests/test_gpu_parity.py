@@ -39,7 +39,7 @@ TC_SHAPES = [
     (4096, 128, 300), (300, 256, 700), (257, 16, 5), (1000, 8, 3), (2000, 72, 260), (333, 192, 513),
     (20000, 64, 128), (50, 128, 2048),
     (300, 264, 70), (1000, 288, 300), (515, 352, 1000), (2000, 480, 130), (700, 512, 600), (129, 504, 33),
-    (40000, 320, 24),
+    (40000, 320, 24), (30000, 384, 100), (25000, 264, 128),
 ]
 
 
@@ -129,7 +129,8 @@ def test_assign_batched_matches_per_problem_and_oracle():
         assert torch.equal(i1, idx[b]) and torch.equal(d1, dist[b])
 
 
-@pytest.mark.parametrize("B,N,D,K", [(200, 300, 64, 100), (150, 513, 128, 256), (67, 700, 192, 7), (90, 400, 96, 200)])
+@pytest.mark.parametrize("B,N,D,K", [(200, 300, 64, 100), (150, 513, 128, 256), (67, 700, 192, 7), (90, 400, 96, 200),
+                                     (40, 700, 320, 60), (35, 900, 384, 128)])
 def test_assign_many_small_problems_single_centroid_tile(B, N, D, K):
     """One centroid tile per row tile with the tile resident in shared memory: every CTA meets several
     problems (the resident tile is reloaded, both MMA issuers hand it back), row tiles alternate between
