@@ -101,7 +101,8 @@ struct Params {
     i64 total_tiles;  // B * m_tiles
     int n_stages;     // ring depth (stages)
     int cps;          // centroid chunks per ring stage: 2 when nchunks is even (half the barrier traffic), else 1
-    uint32_t stage_bytes;   // cps * 32 KiB + 4 KiB
+    uint32_t stage_bytes;   // cps * 32 KiB + 4 KiB; resident centroids: bytes of one chunk of the tile (rows * 128),
+                            // the tile's chunks lie one behind the other, its 4 KiB half-norm block after them
     int n_xbuf;       // X buffers (1..4)
     const uint8_t* caug;  // [B][n_tiles][4 KiB] centroid-side operand of the extra k-step
     int* cnmax;           // [B] bit pattern of max_k ||c_k||^2 (fp32, >= 0)
@@ -287,7 +288,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t x_base = smem_base;
     const uint32_t ring_off = static_cast<uint32_t>(p.n_xbuf) * xbuf_bytes;
     const uint32_t ring_base = smem_base + ring_off;
-    const uint32_t auga_off = ring_off + static_cast<uint32_t>(p.n_stages) * p.stage_bytes;
+    // bytes of one resident centroid tile (chunks, then its half-norm block)
+    const uint32_t res_tile_bytes = static_cast<uint32_t>(p.nchunks) * p.stage_bytes + AUG_B_BYTES;
+    const uint32_t auga_off = ring_off + ((XLOAD && p.res_c) ? static_cast<uint32_t>(p.res_c) * res_tile_bytes
+                                                             : static_cast<uint32_t>(p.n_stages) * p.stage_bytes);
     const uint32_t zero_off = auga_off + static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES;
     const uint32_t ctrl_off = zero_off + AUG_ZERO_BYTES;
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ctrl_off);
@@ -391,12 +395,12 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         const uint32_t full = ptx::smem_u32(&ctrl->ring_full[0]);
                         // (res_c = 2: two centroid tiles, one behind the other)
                         ptx::mbar_arrive_expect_tx(full, static_cast<uint32_t>(p.res_c) *
-                                                             (static_cast<uint32_t>(p.nchunks) * (p.stage_bytes - AUG_B_BYTES) + AUG_B_BYTES));
+                                                             res_tile_bytes);
                         for (int j = 0; j < p.res_c; ++j) {
-                            const uint32_t tbase = ring_base + j * p.nchunks * p.stage_bytes;
+                            const uint32_t tbase = ring_base + j * res_tile_bytes;
                             for (int c = 0; c < p.nchunks; ++c)
                                 ptx::tma_load_3d(tbase + c * p.stage_bytes, &tmap_c, full, c * KCHUNK, j * BLOCK_N, tb);
-                            ptx::bulk_load(tbase + p.nchunks * p.stage_bytes - AUG_B_BYTES,
+                            ptx::bulk_load(tbase + res_tile_bytes - AUG_B_BYTES,
                                            p.caug + (static_cast<size_t>(tb) * p.res_c + j) * AUG_B_BYTES, AUG_B_BYTES, full);
                         }
                         cur_b = tb;
@@ -576,7 +580,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     }
                     ptx::tc_fence_after();
                     const uint32_t d_tmem = tmem_base + iss * BLOCK_N;
-                    const uint32_t c_base = ring_base + (both ? iss * p.nchunks * p.stage_bytes : 0u);   // this issuer's centroid tile
+                    const uint32_t c_base = ring_base + (both ? iss * res_tile_bytes : 0u);   // this issuer's centroid tile
                     uint32_t a_lo = ptx::umma_desc_lo_sw128(x_base + rxb * xbuf_bytes);
                     for (int c = 0; c < p.nchunks; ++c, a_lo += X_CHUNK_BYTES >> 4) {
                         if (XSPLIT) {
@@ -603,7 +607,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     ptx::umma_bf16_lohi<true>(d_tmem,
                                               ptx::umma_desc_lo_aug(smem_base + auga_off + rxb * AUG_A_BYTES, smem_base + zero_off),
                                               ptx::UMMA_DESC_HI_AUG,
-                                              ptx::umma_desc_lo_aug(c_base + p.nchunks * p.stage_bytes - AUG_B_BYTES,
+                                              ptx::umma_desc_lo_aug(c_base + res_tile_bytes - AUG_B_BYTES,
                                                                     smem_base + zero_off),
                                               ptx::UMMA_DESC_HI_AUG, idesc_aug_n);
                     ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[iss]));
@@ -1300,7 +1304,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         // a single centroid tile: keep it in shared memory if an even number of X buffers fits beside it
         // (of the tile only the rows that hold centroids, in steps of 32, when there are at most 128)
         c_rows = K <= BLOCK_N / 2 ? static_cast<int>(round_up(K, 32)) : BLOCK_N;
-        const i64 c_bytes = static_cast<i64>(p.nchunks) * (c_rows * 128 + AUG_B_BYTES);
+        const i64 c_bytes = static_cast<i64>(p.nchunks) * c_rows * 128 + AUG_B_BYTES;
         for (int nx = MAX_XBUF; nx >= 2; nx -= 2) {
             if (p.nchunks <= MAX_STAGES && c_bytes + nx * xbuf <= budget) {
                 p.res_c = 1;
@@ -1308,30 +1312,31 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
                 // the 32-column groups that hold centroids; the tensor pipe and the epilogue do less)
                 p.alt_epi = c_rows;
                 p.cps = 1;
-                p.stage_bytes = static_cast<uint32_t>(c_rows) * 128u + AUG_B_BYTES;
+                p.stage_bytes = static_cast<uint32_t>(c_rows) * 128u;
                 p.n_stages = p.nchunks;
                 p.n_xbuf = nx;
                 break;
             }
         }
         // D > 256: one X buffer beside the resident tile, filled and handed back chunk by chunk
-        if (!p.res_c && p.nchunks <= MAX_STAGES && p.nchunks <= MAX_XCHUNKS && c_bytes + xbuf <= budget) {
+        // (the ring's stage count only sizes the buffer here: the resident tile has one barrier pair)
+        if (!p.res_c && p.nchunks <= MAX_XCHUNKS && c_bytes + xbuf <= budget) {
             p.res_c = 1;
             p.alt_epi = c_rows;
             p.cps = 1;
-            p.stage_bytes = static_cast<uint32_t>(c_rows) * 128u + AUG_B_BYTES;
+            p.stage_bytes = static_cast<uint32_t>(c_rows) * 128u;
             p.n_stages = p.nchunks;
             p.n_xbuf = 1;
         }
     }
     if (p.n_tiles == 2) {
         // two centroid tiles: both stay in shared memory if at least two X buffers fit beside them (D <= 128)
-        const i64 c_bytes = 2 * static_cast<i64>(p.nchunks) * (C_CHUNK_BYTES + AUG_B_BYTES);
+        const i64 c_bytes = 2 * (static_cast<i64>(p.nchunks) * C_CHUNK_BYTES + AUG_B_BYTES);
         for (int nx = MAX_XBUF; nx >= 2; --nx) {
             if (2 * p.nchunks <= MAX_STAGES && c_bytes + nx * xbuf <= budget) {
                 p.res_c = 2;
                 p.cps = 1;
-                p.stage_bytes = C_CHUNK_BYTES + AUG_B_BYTES;
+                p.stage_bytes = C_CHUNK_BYTES;
                 p.n_stages = 2 * p.nchunks;
                 p.n_xbuf = nx;
                 break;
@@ -1341,8 +1346,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     if (p.res_c != 1) c_rows = BLOCK_N;
     rc = make_tmap(&tc, cpad ? cpad : C, Dc, K, B, c_rows);
     if (rc != CAKE_OK) return rc;
-    const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf +
-                              static_cast<size_t>(p.n_stages) * p.stage_bytes;
+    const size_t ring_bytes = p.res_c ? static_cast<size_t>(p.res_c) * (static_cast<size_t>(p.nchunks) * p.stage_bytes + AUG_B_BYTES)
+                                      : static_cast<size_t>(p.n_stages) * p.stage_bytes;
+    const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf + ring_bytes;
     using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const Params);
     const bool consec = xload && p.res_c && B > 1;
     // a single X buffer (D > 256) is filled and handed back chunk by chunk
