@@ -636,7 +636,8 @@ def test_assign_many_row_tiles_few_centroid_tiles(N, D, K):
 
 
 @pytest.mark.parametrize("N,D,K", [(1 << 21, 64, 64), (1 << 21, 128, 300), (1 << 20, 256, 600), (1 << 21, 96, 1000),
-                                   (1 << 20, 128, 1300)])
+                                   (1 << 20, 128, 1300), (1 << 20, 384, 64), (1 << 20, 512, 32), (1 << 19, 288, 300),
+                                   (1 << 20, 256, 256), (1 << 20, 100, 200)])
 def test_assign_repeatable_over_many_launches(N, D, K):
     """The assign kernel has no data-dependent order (no atomics on its outputs): repeated launches must
     return identical bits.  A role that gets ahead of a buffer it must not yet reuse (X tile, row
