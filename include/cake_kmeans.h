@@ -158,7 +158,7 @@ CAKE_API int cake_kmeans_update_batched(const cake_bf16* X, const int* idx, long
  * centroid_update in two halves, for rows of X that are spread over several devices (the paper
  * describes one device; the per-cluster sums and counts of the same paragraph are what has to cross
  * devices).  Each device adds up its own rows, the caller adds the sums and counts of all devices (an
- * all-reduce), and every device divides.  K <= 8192.
+ * all-reduce), and every device divides.
  *   update_partial: out_sums[B][K][D] fp32 and out_counts[B][K] int32 of the rows given (overwritten,
  *                   not accumulated); other arguments as for update.  flags: 0, CAKE_UPDATE_SLAB or
  *                   CAKE_UPDATE_SORT.

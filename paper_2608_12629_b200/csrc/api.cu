@@ -249,7 +249,6 @@ int cake_kmeans_update_partial_batched(const cake_bf16* X, const int* idx, long 
     if (!out_sums || !out_counts || !ws || (N > 0 && (!X || !idx))) return CAKE_ERR_NULL;
     if (misaligned(X, 16) || misaligned(idx, 4) || misaligned(out_sums, 16) || misaligned(out_counts, 4))
         return CAKE_ERR_ALIGN;
-    if (K > 8192) return CAKE_ERR_UNSUPPORTED;   // above, the sort route writes means, not sums
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;

@@ -1275,7 +1275,8 @@ int launch_update_sort(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
     const size_t kd = static_cast<size_t>(B) * K * D;
     const SortPlan pl = sort_plan(N, K);
     // large K, rows of whole 16-byte granules: the last kernel writes the means itself (no partial sums)
-    const bool means = N > 0 && !pl.blocked && D % 8 == 0 && D >= 24 && D <= 1024;
+    // (only where the caller wants centroids: without out_C the sums themselves are the result)
+    const bool means = out_C && N > 0 && !pl.blocked && D % 8 == 0 && D >= 24 && D <= 1024;
     const bool zero_in_hist = N > 0 && !pl.blocked && !means && (static_cast<i64>(K) * D) % 4 == 0;
     if (N == 0 || !pl.blocked) {
         if (!means && !zero_in_hist && cudaMemsetAsync(scr.sums, 0, kd * sizeof(float), s) != cudaSuccess)

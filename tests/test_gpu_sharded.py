@@ -29,10 +29,11 @@ def int_problem(N, D, K, seed):
 
 
 @pytest.mark.parametrize("flags", [0, cake.CAKE_UPDATE_SLAB, cake.CAKE_UPDATE_SORT])
-@pytest.mark.parametrize("N,D,K", [(5000, 64, 37), (70001, 128, 1000), (3000, 24, 8192), (900, 12, 5), (4097, 320, 100)])
+@pytest.mark.parametrize("N,D,K", [(5000, 64, 37), (70001, 128, 1000), (3000, 24, 8192), (900, 12, 5), (4097, 320, 100),
+                                   (30000, 64, 20000), (9000, 12, 9000)])
 def test_update_partial_of_two_halves_adds_up_to_the_update(N, D, K, flags):
-    if flags == cake.CAKE_UPDATE_SLAB and D % 8:
-        pytest.skip("slab route needs D % 8 == 0")
+    if flags == cake.CAKE_UPDATE_SLAB and (D % 8 or K > 8192):
+        pytest.skip("slab route needs D % 8 == 0 and K <= 8192")
     X, C0 = int_problem(N, D, K, N + D)
     g = torch.Generator().manual_seed(K)
     idx = torch.randint(0, K, (N,), generator=g, dtype=torch.int32)
@@ -43,7 +44,11 @@ def test_update_partial_of_two_halves_adds_up_to_the_update(N, D, K, flags):
     s1, c1 = cake.cake_kmeans_update_partial(Xd[h:].clone(), idxd[h:].clone(), K, flags=flags)
     Cf, Cb = cake.cake_kmeans_update_finish(s0 + s1, c0 + c1, C_prev=Cd)
     Cf_ref, Cb_ref, counts_ref = cake.cake_kmeans_update(Xd, idxd, K, C_prev=Cd)
-    assert torch.equal(c0 + c1, counts_ref) and torch.equal(Cf, Cf_ref) and torch.equal(Cb, Cb_ref)
+    assert torch.equal(c0 + c1, counts_ref)
+    if K <= 8192 or D % 8:
+        assert torch.equal(Cf, Cf_ref) and torch.equal(Cb, Cb_ref)
+    else:   # the one-call route for many clusters multiplies by a reciprocal instead of dividing: last-bit differences
+        np.testing.assert_allclose(Cf.cpu().numpy(), Cf_ref.cpu().numpy(), rtol=3e-7, atol=0)
     grading.grade_update(inputs.to_bits(X), idx.numpy(), K, inputs.to_bits(C0), Cf.cpu().numpy(), inputs.to_bits(Cb),
                          (c0 + c1).cpu().numpy())
 
@@ -51,8 +56,8 @@ def test_update_partial_of_two_halves_adds_up_to_the_update(N, D, K, flags):
 def test_update_partial_limits_and_empty_input():
     X, C0 = int_problem(100, 16, 9000, 1)
     idx = torch.zeros(100, dtype=torch.int32)
-    with pytest.raises(cake.CakeError) as e:
-        cake.cake_kmeans_update_partial(X.to(DEV), idx.to(DEV), 9000)
+    with pytest.raises(cake.CakeError) as e:       # the slab route by name stops at 8,192 clusters
+        cake.cake_kmeans_update_partial(X.to(DEV), idx.to(DEV), 9000, flags=cake.CAKE_UPDATE_SLAB)
     assert e.value.code == cake.CAKE_ERR_UNSUPPORTED
     s, c = cake.cake_kmeans_update_partial(X[:0].to(DEV), idx[:0].to(DEV), 7)
     assert int(c.sum()) == 0 and float(s.abs().sum()) == 0.0
