@@ -61,10 +61,13 @@ enum {
     CAKE_ASSIGN_AUTO = 0,      /* the tensor-core pipeline for D <= 512 (for D % 8 != 0 on a zero-padded
                                   copy of X kept in the workspace: same results), else the fallback  */
     CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 512.
-                                  Distances are compared as fixed-point numbers with a quantum of
-                                  about 2^-19 of (|x|^2 + max |c|^2); equal ones go to the lower index */
+                                  Each distance is an fp32 number whose error follows |x|^2 + |c|^2 of
+                                  its own centroid (other centroids' norms do not matter); distances are
+                                  compared with 17 significant bits (2^-16 of the distance), equal ones
+                                  go to the lower index; out_dist carries the same 17 bits.  Squared
+                                  norms must stay below 2^120                                      */
     CAKE_ASSIGN_SIMT = 2,      /* plain CUDA-core fallback, any D                               */
-    CAKE_ASSIGN_TCGEN05_EXACT = 3, /* same pipeline, full-precision comparison (slower epilogue) */
+    CAKE_ASSIGN_TCGEN05_EXACT = 3, /* same pipeline, all 24 bits compared and returned (slower epilogue) */
     CAKE_ASSIGN_MASK = 0xF,
     CAKE_UPDATE_AUTO = 0,
     CAKE_UPDATE_SMEM = 1 << 4, /* shared-memory partial sums; needs K*D*4 + K*4 bytes of smem   */

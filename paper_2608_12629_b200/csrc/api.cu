@@ -11,10 +11,8 @@ constexpr size_t kAlign = 256;
 inline size_t up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Workspace {
-    int* status;          // [64] header, zeroed by the caller once: word 0 = sticky device status, word 1 =
-                          // ticket of the assign kernel, words 16..47 = max ||c||^2 of up to 32 problems
+    int* status;          // [64] header, zeroed by the caller once: word 0 = sticky device status
     void* caug;           // [B][Kpad/256][4 KiB] half-norm operand of the tensor-core assign
-    int* cnmax;           // [B] max ||c||^2 per problem (fp32 bits)
     float* sums;          // [B][K][D]
     int* nvalid;          // [B]
     int* cursor;          // [B][K]
@@ -37,7 +35,6 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     const size_t kd = static_cast<size_t>(B) * K * D;
     w.status = reinterpret_cast<int*>(take(256));
     w.caug = take(assign_tc_aug_bytes(B, K));
-    w.cnmax = reinterpret_cast<int*>(take(static_cast<size_t>(B) * 4));
     // rows of padded_d(D) columns: for D % 8 != 0 the update may add up the padded copy of X
     w.sums = reinterpret_cast<float*>(take(static_cast<size_t>(B) * K * padded_d(D) * 4));
     w.nvalid = reinterpret_cast<int*>(take(static_cast<size_t>(B) * 4));
@@ -105,13 +102,11 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
     if (path != CAKE_ASSIGN_TCGEN05 && path != CAKE_ASSIGN_TCGEN05_EXACT) return CAKE_ERR_UNSUPPORTED;
     if (!assign_tc_supports(Dx ? Dx : D)) return CAKE_ERR_UNSUPPORTED;
     if (N == 0) return CAKE_OK;
-    // both epilogues order by the same fixed-point values; the packed one measured as fast or faster
-    // at every shape tried, so it is the automatic choice and the other stays selectable
+    // the packed epilogue (values compared with 17 significant bits) is the automatic choice; the exact
+    // one compares full fp32 values and is slower
     const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT;
-    // up to 32 problems keep max ||c||^2 in the header, which the kernel leaves zeroed: no memset per call
-    const bool in_header = B <= 32;
-    return launch_assign_tc(X, C, B, N, D, K, w.caug, in_header ? w.status + 16 : w.cnmax, in_header ? w.status + 1 : nullptr,
-                            exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia, aug_ready, w.status, s, Dx,
+    return launch_assign_tc(X, C, B, N, D, K, w.caug, exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia,
+                            aug_ready, w.status, s, Dx,
                             assign_cpad_columns(D) ? w.cpad : nullptr);
 }
 
@@ -326,7 +321,7 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     // workspace buffers and the last iteration writes the caller's buffer directly.  Each iteration's
     // inertia entries are cleared by its own assign step.
     // The division kernel of iteration t also writes what the tensor-core assign of iteration t + 1 would
-    // otherwise compute in a prologue launch of its own (while max ||c||^2 lives in the header, B <= 32).
+    // otherwise compute in a prologue launch of its own.
     const unsigned apath = flags & CAKE_ASSIGN_MASK;
     const bool tc_assign = N > 0 && ((assign_tc_supports(D) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
                                                                 apath == CAKE_ASSIGN_TCGEN05_EXACT)) ||
@@ -341,9 +336,9 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
                        true, prepared, &x_padded, w, s, flags);
         if (rc != CAKE_OK) return rc;
         cake_bf16* dst = (t == iters - 1 && out_C_bf16) ? out_C_bf16 : w.cbuf[nxt];
-        NextAssign next{w.caug, w.status + 16, out_inertia ? out_inertia + t + 1 : nullptr, iters,
+        NextAssign next{w.caug, out_inertia ? out_inertia + t + 1 : nullptr, iters,
                         cpad_columns ? w.cpad : nullptr, cpad_columns};
-        const bool want = tc_assign && Bi <= 32 && t + 1 < iters;
+        const bool want = tc_assign && t + 1 < iters;
         rc = do_update(X, out_idx, Bi, N, D, K, cur, out_C, dst, out_counts, w, s, flags, &x_padded, want ? &next : nullptr, &prepared);
         if (rc != CAKE_OK) return rc;
         cur = dst;

@@ -70,7 +70,6 @@ extern "C" int cake_kmeans_assign_static(const cake_bf16* X, const cake_bf16* C,
     // half-norm operand is rewritten in full (all ceil(K/256) tiles, padding rows included) by the
     // prologue that launch_assign_tc runs first
     if (cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) return CAKE_ERR_CUDA;
-    // header: word 0 = status, word 16 = max ||c||^2 (cleared by the prologue launch)
-    return launch_assign_tc(X, C, 1, N, D, K, scratch + kStaticHeader, status + 16, nullptr, false, out_idx, out_dist, nullptr, 0,
+    return launch_assign_tc(X, C, 1, N, D, K, scratch + kStaticHeader, false, out_idx, out_dist, nullptr, 0,
                             false, false, status, s);
 }

@@ -2,17 +2,18 @@
 //
 // Operation (paper Section 5, "Flash-KMeans clean-start workload"): for every point the squared
 // Euclidean distance to all K centroids and the arg-min.  The whole expansion
-//     M + m + d(x,c)/2 = M + m + ||x||^2/2 - x.c + ||c||^2/2
-// is accumulated in tensor memory: the D-long contraction -x.c runs with the B operand negated, and
-// one extra 16-wide k-step adds the two half-norms and a per-row offset (the X side carries
-// [xh xm xl 1 1 1 M m 0..], the centroid side [1 1 1 ch cm cl 1 1 0..], each half-norm split into
-// three bf16 terms so that nothing of its fp32 value is lost).  M is a power of two at least twice
-// ||x||^2 + max||c||^2 >= d/2, m = M/4096 keeps rounding noise positive: every accumulator of a row
-// lies in the binade [M, 2M), so its fp32 bit pattern minus that of M is the distance in FIXED POINT
-// (quantum ulp(M), about 2^-20 of the row's scale), and `bits * 128 + column` is an order-preserving
-// key that a single integer multiply-add forms.  Padded centroid rows carry 1.5 M instead of M and
-// lose to every real one.  The epilogue therefore only has to find a row minimum; the N x K matrix
-// never exists outside tensor memory.
+//     m + d(x,c)/2 = m + ||x||^2/2 - x.c + ||c||^2/2
+// is accumulated in tensor memory in fp32: the D-long contraction -x.c runs with the B operand
+// negated, and one extra 16-wide k-step adds the two half-norms (the X side carries
+// [xh xm xl 1 1 1 0..], the centroid side [1 1 1 ch cm cl 0..], each half-norm split into three bf16
+// terms so that nothing of its fp32 value is lost).  m is a per-row margin, a power of two between
+// 2^-12 and 2^-11 of ||x||^2, added to ||x||^2/2 before the split: it keeps every accumulator of the
+// row positive when the true distance is zero and rounding noise is not (a point that is its own
+// centroid), so that accumulators order like their bit patterns.  Every accumulator is a plain fp32
+// number whose error follows ||x||^2 + ||c_k||^2 of ITS OWN centroid: one centroid of huge norm
+// does not touch the resolution of the others.  Padded centroid rows carry a half-norm of 2^120
+// and lose to every real one.  The epilogue only has to find a row minimum; the N x K matrix never
+// exists outside tensor memory.
 //
 // One persistent CTA per SM, 16 warps, four roles:
 //   warp 8  producer : TMA.  A 128-row X tile (whole D) into one of the X buffers per row tile (up to
@@ -38,11 +39,14 @@
 //                      the X-side operand of the extra k-step, one row tile ahead of the MMA warps.
 // Barrier discipline: every mbarrier has waiters that see each of its phases, and whoever refills a
 // buffer waits for every reader of it (a parity wait that falls two phases behind never returns).
-// Two epilogue policies (both order by the fixed-point value, ties to the lowest index):
-//   packed : key = bits * 128 + column (one shift-and-add) and a plain 3-input float
-//            minimum over the keys finds value and position at once; no branch.
-//   exact  : minimum of the values; the position is looked up only when a 32-column group beats the
-//            running best (cheaper when there are many centroid tiles per row).
+// Two epilogue policies (ties to the lowest index):
+//   packed : key = the accumulator's bits with the low 7 replaced by the column (one logic
+//            instruction); a plain 3-input float minimum over the keys finds value and position at
+//            once, no branch.  Values are compared with 17 significant bits, i.e. to 2^-16 of the
+//            half-distance itself: far inside the tolerance of 1e-3 (||x||^2 + ||c||^2), whatever the
+//            norms of the other centroids.
+//   exact  : minimum of the full fp32 values; the position is looked up only when a 32-column group
+//            beats the running best.
 // Every wait is bounded: on expiry the CTA raises CAKE_ERR_TIMEOUT in the status word, all roles
 // leave their loops, TMEM is freed and the kernel returns.
 #include "aug.cuh"
@@ -80,7 +84,7 @@ constexpr int MAX_STAGES = 6;
 constexpr int MAX_XBUF = 4;
 constexpr int MAX_XCHUNKS = 8;                           // 64-column chunks of an X tile (D <= 512)
 constexpr int TMEM_COLS = 512;
-constexpr uint32_t CTRL_BYTES = 6144;  // barriers, TMEM pointer, abort flag, merge scratch, row exponents
+constexpr uint32_t CTRL_BYTES = 6144;  // barriers, TMEM pointer, abort flag, merge scratch, row margins
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 constexpr uint32_t WAIT_SLICE_NS = 20000;   // longest single sleep inside a wait
 constexpr uint32_t COL_MASK = 0x7Fu;   // packed policy: 7 bits address the 128 columns of a half tile
@@ -105,8 +109,6 @@ struct Params {
                             // the tile's chunks lie one behind the other, its 4 KiB half-norm block after them
     int n_xbuf;       // X buffers (1..4)
     const uint8_t* caug;  // [B][n_tiles][4 KiB] centroid-side operand of the extra k-step
-    int* cnmax;           // [B] bit pattern of max_k ||c_k||^2 (fp32, >= 0)
-    int* ticket;          // optional: CTAs that have finished; the last one clears cnmax and the ticket
     int* out_idx;
     float* out_dist;
     double* inertia;      // optional: inertia[b * inertia_stride] += sum of the problem's distances
@@ -134,7 +136,7 @@ struct Ctrl {  // lives in shared memory
     int abort_flag;
     float merge_best[2][BLOCK_M];
     int merge_idx[2][BLOCK_M];
-    int row_e[MAX_XBUF][BLOCK_M];   // biased exponent of each row's offset M
+    float row_m[MAX_XBUF][BLOCK_M];   // each row's margin m
 #ifdef CAKE_ASSIGN_TRACE
     int trace_n[NUM_WARPS];
 #endif
@@ -219,14 +221,14 @@ __device__ __forceinline__ float min32(const float (&v)[32]) {
     return fminf(ptx::fmin3(u0, u1, u2), u3);
 }
 
-// packed policy: key = bits * 128 + column (0..127 inside the half tile), modulo 2^32.  All values of a
-// row share the binade of M, whose exponent is chosen so that the keys stay below 0x7F800000: as float
-// bit patterns they are positive and finite, and float order == (fixed-point value, column) order.
-__device__ __forceinline__ float packed_min32(const uint32_t (&r)[32], int col_base, float run) {
+// packed policy: key = the accumulator with its low 7 bits replaced by the column (0..127 inside the half
+// tile).  Accumulators are positive finite floats (margin m), so the keys are too, and float order ==
+// (value truncated to 17 significant bits, column) order.
+__device__ __forceinline__ float packed_min32(const uint32_t (&r)[32], int col_base, float run, uint32_t kmask) {
     float v[32];
 #pragma unroll
     for (int j = 0; j < 32; ++j)
-        v[j] = __uint_as_float(r[j] * (COL_MASK + 1u) + static_cast<uint32_t>(col_base + j));
+        v[j] = __uint_as_float(ptx::and_or(r[j], kmask, static_cast<uint32_t>(col_base + j)));
     return fminf(run, min32(v));
 }
 
@@ -303,7 +305,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAX_XBUF; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
-            // MMA issuers + 4 norm warps + the 4 epilogue warps that read the row exponents
+            // MMA issuers + 4 norm warps + the 4 epilogue warps that read the row margins
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), ((XLOAD && p.res_c == 1) ? 1 : NUM_ISSUERS) + 4 + 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
         }
@@ -725,9 +727,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         const int r = (warp - AUX_WARP0) * 32 + lane;
         uint32_t xb = 0, xph = 0;
         bool ok = true;
-        int nb = 0, nmt = 0;   // (problem, row tile), stepped: only where the CTA's tiles may be consecutive
-        if (CONSEC) first_tile<CONSEC>(p, nb, nmt);
-        const int nmt_step = tile_step<CONSEC>();
         for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
             if (!XSPLIT) ok = wait_bar(&ctrl->x_full[xb], xph, ctrl, p.status);
             if (!ok) break;
@@ -756,30 +755,17 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             }
             if (!ok) break;
             const float xn = (xn0 + xn1) + (xn2 + xn3);
+            // margin m = 2^(e-11) for ||x||^2 in [2^e, 2^(e+1)), at least 2^-100: above the rounding noise of a
+            // zero distance (D * 2^-24 of ||x||^2 at worst), and a power of two so that it disturbs no exact sum
+            const uint32_t xe = __float_as_uint(xn) >> 23;
+            const uint32_t mbits = (xe > 38u ? xe - 11u : 27u) << 23;
             uint32_t hi, mid, lo;
-            split3(0.5f * xn, hi, mid, lo);
-            // offset M = 2^(E-127): the smallest power of two >= 2 (||x||^2 + max ||c||^2) whose biased
-            // exponent E is 0 or 1 modulo 4 (then bits(M) * 128 is 0 or 2^30 modulo 2^32 and the keys
-            // of the row are positive floats); m = M / 4096
-            int tb;
-            if (CONSEC) {
-                tb = nb;
-                nmt += nmt_step;
-                while (nmt >= p.m_tiles) { nmt -= p.m_tiles; ++nb; }
-            } else {
-                tb = static_cast<int>(tile / p.m_tiles);
-            }
-            const float bound = 2.f * (xn + __int_as_float(__ldg(p.cnmax + tb)));
-            const uint32_t bb = __float_as_uint(bound);
-            uint32_t E = (bb >> 23) + ((bb & 0x7FFFFFu) ? 1u : 0u);
-            E += (E & 3u) == 2u ? 2u : ((E & 3u) == 3u ? 1u : 0u);
-            E = E < 36u ? 36u : (E > 248u ? 248u : E);
-            ctrl->row_e[xb][r] = static_cast<int>(E);
-            // interleaved (no-swizzle) K-major layout, columns 0..7 only: one 16-byte row per X row;
-            // a power of two is exact in bf16: its bits are the top half of the fp32 pattern
+            split3(fmaf(0.5f, xn, __uint_as_float(mbits)), hi, mid, lo);
+            ctrl->row_m[xb][r] = __uint_as_float(mbits);
+            // interleaved (no-swizzle) K-major layout, columns 0..7 only: one 16-byte row per X row
             const uint32_t one = 0x3F80u;
             *reinterpret_cast<uint4*>(smem + auga_off + xb * AUG_A_BYTES + r * 16) =
-                make_uint4(hi | (mid << 16), lo | (one << 16), one | (one << 16), (E << 7) | ((E - 12u) << 23));
+                make_uint4(hi | (mid << 16), lo | (one << 16), one | (one << 16), 0u);
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
@@ -798,7 +784,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         uint32_t tile_it = 0, acc_it = 0;
         constexpr uint32_t n_iss = NUM_ISSUERS;
         uint32_t next_iss = 2 % n_iss;         // (acc_it + 2) mod n_iss
-        uint32_t exb = 0, exph = 0;          // X buffer (slot of the row exponents) and its phase
+        uint32_t exb = 0, exph = 0;          // X buffer (slot of the row margins) and its phase
+        // all ones but the 7 column bits; formed from a run-time value (K < 2^31) so that it stays in a register
+        // and each key is ONE logic instruction (register, register, immediate column)
+        const uint32_t kmask = ~COL_MASK | (static_cast<uint32_t>(p.K) >> 31);
         bool ok = true;
         double dsum = 0.0;                   // this thread's share of the current problem's inertia
         int dsum_b = -1;
@@ -831,15 +820,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 flush_inertia();
                 dsum_b = b;
             }
-            // the row exponents are there long before the accumulator is: fetch them while waiting for it
+            // the row margins are there long before the accumulator is: fetch them while waiting for it
             // (the X buffer is not refilled before the issuer's MMAs on it have completed either)
             const uint32_t axb = tile_it % static_cast<uint32_t>(p.n_xbuf);
             const uint32_t axph = (tile_it / static_cast<uint32_t>(p.n_xbuf)) & 1u;
-            int rowE = 0;
+            float rowM = 0.f;
             if (!XSPLIT) {
                 ok = wait_bar(&ctrl->auga_full[axb], axph, ctrl, p.status);
                 if (!ok) break;
-                rowE = ctrl->row_e[axb][r];
+                rowM = ctrl->row_m[axb][r];
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
             }
@@ -848,8 +837,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             if (!ok) break;
             if (XSPLIT) {
                 // one X buffer for both warpgroups: this one sees only every other phase of its barriers, so it
-                // reads the exponents once its accumulator is complete (the issuer waited for them)
-                rowE = ctrl->row_e[0][r];
+                // reads the margins once its accumulator is complete (the issuer waited for them)
+                rowM = ctrl->row_m[0][r];
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[0]));
             }
@@ -873,10 +862,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][(tile_it + 2u) % n_iss]));
                 if (PACKED) {
-                    best = packed_min32(ra, 0, __uint_as_float(F32_INF));
-                    if (ng > 1) best = packed_min32(rb, 32, best);
-                    if (ng > 2) best = packed_min32(rc, 64, best);
-                    if (ng > 3) best = packed_min32(rd, 96, best);
+                    best = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
+                    if (ng > 1) best = packed_min32(rb, 32, best, kmask);
+                    if (ng > 2) best = packed_min32(rc, 64, best, kmask);
+                    if (ng > 3) best = packed_min32(rd, 96, best, kmask);
                     bsel = 0;
                 } else {
                     exact_scan32(ra, 0, best, bsel);
@@ -900,13 +889,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 ptx::reg_dep(rd);
                 float lo_min = 0.f;
                 if (PACKED) {
-                    lo_min = packed_min32(ra, 0, __uint_as_float(F32_INF));
+                    lo_min = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
                     ptx::tmem_ld_x32(taddr + 128, ra);
-                    lo_min = packed_min32(rb, 32, lo_min);
+                    lo_min = packed_min32(rb, 32, lo_min, kmask);
                     ptx::tmem_ld_x32(taddr + 160, rb);
-                    lo_min = packed_min32(rc, 64, lo_min);
+                    lo_min = packed_min32(rc, 64, lo_min, kmask);
                     ptx::tmem_ld_x32(taddr + 192, rc);
-                    lo_min = packed_min32(rd, 96, lo_min);
+                    lo_min = packed_min32(rd, 96, lo_min, kmask);
                     ptx::tmem_ld_x32(taddr + 224, rd);
                 } else {
                     exact_scan32(ra, 0, best, bsel);
@@ -927,10 +916,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 // to the issuer of row tile tile_it + 2, which takes this accumulator next
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][(tile_it + 2u) % n_iss]));
                 if (PACKED) {
-                    float hi_min = packed_min32(ra, 0, __uint_as_float(F32_INF));
-                    hi_min = packed_min32(rb, 32, hi_min);
-                    hi_min = packed_min32(rc, 64, hi_min);
-                    hi_min = packed_min32(rd, 96, hi_min);
+                    float hi_min = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
+                    hi_min = packed_min32(rb, 32, hi_min, kmask);
+                    hi_min = packed_min32(rc, 64, hi_min, kmask);
+                    hi_min = packed_min32(rd, 96, hi_min, kmask);
                     // across the halves only the (truncated) value decides: an equal value keeps the lower half
                     best = lo_min;
                     bsel = 0;
@@ -959,12 +948,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const i64 row = static_cast<i64>(mt) * BLOCK_M + r;
             if (row < p.N) {
                 const size_t o = static_cast<size_t>(b) * static_cast<size_t>(p.N) + row;
-                const uint32_t E = static_cast<uint32_t>(rowE);
-                const uint32_t fx = PACKED ? (__float_as_uint(bval) >> 7) - ((E & 3u) << 23)
-                                           : __float_as_uint(bval) - (E << 23);
-                const float half = fmaf(static_cast<float>(fx), __uint_as_float((E - 23u) << 23),
-                                        -__uint_as_float((E - 12u) << 23));
-                const float dist = fmaxf(0.f, 2.f * half);
+                const float dist = fmaxf(0.f, 2.f * (bval - rowM));   // the accumulator is m + d/2
                 p.out_idx[o] = bidx;
                 if (p.out_dist) p.out_dist[o] = dist;
                 dsum += static_cast<double>(dist);
@@ -977,7 +961,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             }
             float best = __uint_as_float(F32_INF);   // packed: a key; exact: a value
             int bsel = 0;                            // packed: tile number; exact: global column
-            int rowE = 0;                            // biased exponent of this row's offset M (wg 0 only)
+            float rowM = 0.f;                        // this row's margin m (wg 0 only)
             for (int nt = 0; nt < p.n_tiles; ++nt, ++acc_it) {
                 const uint32_t as = acc_it & 1u, aph = (acc_it >> 1) & 1u;
                 ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
@@ -988,10 +972,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     // it this slot and the next phase of this barrier -- is handed to a later row tile
                     // only after these warps have arrived on x_empty: without that, with one centroid
                     // tile per row tile, the norm warps can get two row tiles of this buffer ahead,
-                    // overwrite the exponents and leave this parity wait behind for good.
+                    // overwrite the margins and leave this parity wait behind for good.
                     ok = wait_bar(&ctrl->auga_full[exb], exph, ctrl, p.status);
                     if (!ok) break;
-                    rowE = ctrl->row_e[exb][r];
+                    rowM = ctrl->row_m[exb][r];
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[exb]));
                 }
@@ -1015,10 +999,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 next_iss = (next_iss + 1 == n_iss) ? 0 : next_iss + 1;
                 trace_mark(ctrl, 100);
                 if (PACKED) {
-                    float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF));
-                    tmin = packed_min32(rb, 32, tmin);
-                    tmin = packed_min32(rc, 64, tmin);
-                    tmin = packed_min32(rd, 96, tmin);
+                    float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
+                    tmin = packed_min32(rb, 32, tmin, kmask);
+                    tmin = packed_min32(rc, 64, tmin, kmask);
+                    tmin = packed_min32(rd, 96, tmin, kmask);
                     // across tiles only the (truncated) value decides: an equal value keeps the earlier tile
                     if (__uint_as_float(__float_as_uint(tmin) & ~COL_MASK) <
                         __uint_as_float(__float_as_uint(best) & ~COL_MASK)) {
@@ -1037,7 +1021,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             trace_mark(ctrl, 102);
             if (++exb == static_cast<uint32_t>(p.n_xbuf)) { exb = 0; exph ^= 1u; }
             // (value, index) of this half; the value is a key with its column bits cleared (packed) or
-            // the accumulator itself (exact): both compare like the fixed-point distance
+            // the accumulator itself (exact)
             float bval;
             int bidx;
             if (PACKED) {
@@ -1071,13 +1055,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const i64 row = static_cast<i64>(mt) * BLOCK_M + r;
                 if (row < p.N) {
                     const size_t o = static_cast<size_t>(b) * static_cast<size_t>(p.N) + row;
-                    // back from fixed point: d/2 = fx * ulp(M) - m
-                    const uint32_t E = static_cast<uint32_t>(rowE);
-                    const uint32_t fx = PACKED ? (__float_as_uint(bval) >> 7) - ((E & 3u) << 23)
-                                               : __float_as_uint(bval) - (E << 23);
-                    const float half = fmaf(static_cast<float>(fx), __uint_as_float((E - 23u) << 23),
-                                            -__uint_as_float((E - 12u) << 23));
-                    const float dist = fmaxf(0.f, 2.f * half);
+                    const float dist = fmaxf(0.f, 2.f * (bval - rowM));   // the accumulator is m + d/2
                     p.out_idx[o] = bidx;
                     if (p.out_dist) p.out_dist[o] = dist;
                     dsum += static_cast<double>(dist);
@@ -1096,28 +1074,17 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, TMEM_COLS);
     }
-    // cnmax lives in memory that is zero between calls: the last CTA to get here (none reads cnmax any
-    // more) clears it for the next call
-    if (p.ticket && threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(p.ticket, 1) == static_cast<int>(gridDim.x) - 1) {
-            for (int b = 0; b < p.B; ++b) p.cnmax[b] = 0;
-            __threadfence();
-            *p.ticket = 0;
-        }
-    }
 }
 
 // Prologue: the centroid-side operand of the extra k-step.  One warp per padded centroid row k:
-// h = ||c_k||^2 / 2 split into three bf16 terms, written as the 16-byte row [1 1 1 h_hi h_mid h_lo 1 1]
+// h = ||c_k||^2 / 2 split into three bf16 terms, written as the 16-byte row [1 1 1 h_hi h_mid h_lo 0 0]
 // (columns 0..7 of the operand in the interleaved K-major layout the MMA reads: 256 rows x 16 B = 4 KiB
-// per tile; columns 8..15 are zeros the kernel supplies itself).  Rows k >= K are [1 1 1 0 0 0 1.5 1]:
-// their accumulator is 1.5 M + ... and can never win.  cnmax[b] collects max_k ||c_k||^2 (the bit
-// patterns of non-negative floats order like integers); it must be zero on entry.  With `inertia` the
-// kernel also zeroes inertia[b * inertia_stride] for the B <= 256 problems (what the assign kernel adds to).
+// per tile; columns 8..15 are zeros the kernel supplies itself).  Rows k >= K carry h = 2^120 and can
+// never win.  With `inertia` the kernel also zeroes inertia[b * inertia_stride] for the B <= 256
+// problems (what the assign kernel adds to).
 __global__ void __launch_bounds__(256)
 centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64 total_rows,
-                    uint8_t* __restrict__ caug, int* __restrict__ cnmax, double* __restrict__ inertia,
+                    uint8_t* __restrict__ caug, double* __restrict__ inertia,
                     int inertia_stride, int B, cake_bf16* __restrict__ cpad, int Dc) {
     ptx::grid_dep_wait();      // C may come from the kernel ahead (the previous iteration's division)
     ptx::grid_dep_launch();
@@ -1147,7 +1114,7 @@ centroid_aug_kernel(const cake_bf16* __restrict__ C, int K, int D, int Kpad, i64
         acc = aug::fold_lanes(acc);
         if (cpad) aug::copy_row_padded(row, D, cpad + (static_cast<size_t>(b) * K + k) * Dc, Dc, lane);
     }
-    if (lane == 0) aug::write_row(caug, cnmax, b, k, K, Kpad, acc);
+    if (lane == 0) aug::write_row(caug, b, k, K, Kpad, acc);
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time libcuda dependency)
@@ -1205,7 +1172,7 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
 }
 
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
-                     int* cnmax, int* ticket, bool exact, int* out_idx, float* out_dist, double* inertia,
+                     bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s, int Dx,
                      cake_bf16* cpad) {
     // D: columns of a row of C; Dk: columns of a row of X and length of the contraction (D, or D rounded up to
@@ -1227,8 +1194,6 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     p.n_tiles = (K + BLOCK_N - 1) / BLOCK_N;
     p.total_tiles = static_cast<i64>(B) * p.m_tiles;
     p.caug = static_cast<const uint8_t*>(caug);
-    p.cnmax = cnmax;
-    p.ticket = ticket;
     p.out_idx = out_idx; p.out_dist = out_dist; p.status = status;
     p.inertia = inertia; p.inertia_stride = inertia_stride;
     if (p.total_tiles == 0) return CAKE_OK;
@@ -1242,10 +1207,6 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     if (!aug_ready) {
         const i64 rows = static_cast<i64>(B) * Kpad;
         const i64 ctas = (rows * 32 + 255) / 256;
-        // cnmax must start at zero: either it lives where the last CTA of the previous call cleared it
-        // (ticket), or it is cleared here
-        if (!ticket && cudaMemsetAsync(cnmax, 0, static_cast<size_t>(B) * sizeof(int), s) != cudaSuccess)
-            return CAKE_ERR_CUDA;
         if (zero_inertia && inertia && B > 256) {   // more problems than the prologue's first CTA has threads
             if (cudaMemset2DAsync(inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
                                   static_cast<size_t>(B), s) != cudaSuccess)
@@ -1257,7 +1218,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         cfg.stream = s;
         cfg.attrs = pdl;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, centroid_aug_kernel, C, K, D, Kpad, rows, static_cast<uint8_t*>(caug), cnmax,
+        if (cudaLaunchKernelEx(&cfg, centroid_aug_kernel, C, K, D, Kpad, rows, static_cast<uint8_t*>(caug),
                                (zero_inertia && B <= 256) ? inertia : static_cast<double*>(nullptr), inertia_stride,
                                B, cpad, Dc) != cudaSuccess) {
             cudaGetLastError();

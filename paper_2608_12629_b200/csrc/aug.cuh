@@ -1,5 +1,5 @@
 // The centroid-side operand of the assign kernel's extra k-step, one 16-byte row per centroid:
-// [1 1 1 h_hi h_mid h_lo 1 1] with h = ||c||^2 / 2 split into three bf16 terms (paper Section 5,
+// [1 1 1 h_hi h_mid h_lo 0 0] with h = ||c||^2 / 2 split into three bf16 terms (paper Section 5,
 // "Flash-KMeans clean-start workload": the ||c||^2 term of the distance expansion).  Shared by the
 // assign prologue and by the division kernel of the update, which writes the operand of the next
 // iteration's centroids while it has them in registers: both sum the squares in the same order, so
@@ -43,21 +43,16 @@ __device__ __forceinline__ float fold_lanes(float acc) {
     return acc;
 }
 
-// Lane 0 of the warp that holds ||c_k||^2 (`norm`) of centroid k of problem b writes the row and
-// raises the problem's running maximum (bit patterns of non-negative floats order like integers).
-// k >= K: a padded row [1 1 1 0 0 0 1.5 1], whose accumulator is 1.5 M + ... and can never win.
-__device__ __forceinline__ void write_row(uint8_t* caug, int* cnmax, i64 b, int k, int K, int Kpad, float norm) {
-    uint32_t hi = 0, mid = 0, lo = 0, b6 = 0x3FC0u;
-    if (k < K) {
-        split3(0.5f * norm, hi, mid, lo);
-        b6 = 0x3F80u;
-        atomicMax(cnmax + b, __float_as_int(norm));
-    }
+// Lane 0 of the warp that holds ||c_k||^2 (`norm`) of centroid k of problem b writes the row.
+// k >= K: a padded row [1 1 1 2^120 0 0 0 0], whose accumulator is about 2^120 and can never win
+// (norms are assumed to stay below that).
+__device__ __forceinline__ void write_row(uint8_t* caug, i64 b, int k, int K, int Kpad, float norm) {
+    uint32_t hi = 0x7B80u, mid = 0, lo = 0;   // 2^120 as bf16
+    if (k < K) split3(0.5f * norm, hi, mid, lo);
     const uint32_t one = 0x3F80u;
     const int tile = k / static_cast<int>(kAssignBlockN), rr = k % static_cast<int>(kAssignBlockN);
     uint8_t* blk = caug + (static_cast<size_t>(b) * (Kpad / static_cast<int>(kAssignBlockN)) + tile) * kAssignAugTileBytes;
-    *reinterpret_cast<uint4*>(blk + rr * 16) =
-        make_uint4(one | (one << 16), one | (hi << 16), mid | (lo << 16), b6 | (one << 16));
+    *reinterpret_cast<uint4*>(blk + rr * 16) = make_uint4(one | (one << 16), one | (hi << 16), mid | (lo << 16), 0u);
 }
 
 // The centroid rows are streamed by TMA once per row tile; rows whose pitch is not a multiple of 128

@@ -27,7 +27,7 @@ unsigned long long launches_so_far();
 inline i64 round_up(i64 a, i64 b) { return (a + b - 1) / b * b; }
 
 // Centroid tiles of the tensor-core assign kernel are 256 wide; K is padded to that (padding rows
-// carry an infinite half-norm).  Per tile the kernel's prologue writes a 4 KiB operand block.
+// carry a half-norm of 2^120).  Per tile the kernel's prologue writes a 4 KiB operand block.
 constexpr int kAssignBlockN = 256;
 constexpr unsigned kAssignAugTileBytes = kAssignBlockN * 16;
 inline int padded_k(int K) { return (int)round_up(K, kAssignBlockN); }
@@ -36,20 +36,17 @@ inline int padded_k(int K) { return (int)round_up(K, kAssignBlockN); }
 bool assign_tc_supports(int D);
 // bytes of scratch (`caug`) the tensor-core assign needs for B problems of K centroids
 size_t assign_tc_aug_bytes(i64 B, int K);
-// prologue (half-norm operand into caug, max ||c||^2 into cnmax[B]) + the assign kernel; exact selects
-// the exact epilogue; inertia (nullable): inertia[b * inertia_stride] += sum_i dist[b][i], fp64, must
-// be zeroed by the caller
-// ticket (nullable): cnmax and *ticket lie in memory that is zero between calls (the kernel's last CTA
-// clears them again); without it cnmax is cleared by a memset.  zero_inertia: the prologue starts the
-// inertia entries from zero (otherwise the caller has).
-// aug_ready: caug, cnmax and (if asked for) the cleared inertia entries are already what the prologue
+// prologue (half-norm operand into caug) + the assign kernel; exact selects the exact epilogue;
+// inertia (nullable): inertia[b * inertia_stride] += sum_i dist[b][i], fp64.  zero_inertia: the prologue
+// starts the inertia entries from zero (otherwise the caller has).
+// aug_ready: caug and (if asked for) the cleared inertia entries are already what the prologue
 // would write for these centroids (the division kernel of the update ahead wrote them): no prologue.
 // cpad (nullable): [B][K][round_up(Dx or D, 64)] scratch; the prologue copies C there, rows padded with
 // zeros, and the kernel streams that copy (rows whose pitch is a multiple of 128 bytes stream faster).
 // Dx (0 = D): columns of a row of X when X is a copy padded with zeros to a multiple of 8 columns
 // (needs cpad).  aug_ready then also means that cpad holds the copy.
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
-                     int* cnmax, int* ticket, bool exact, int* out_idx, float* out_dist, double* inertia,
+                     bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s,
                      int Dx = 0, cake_bf16* cpad = nullptr);
 int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
@@ -98,12 +95,11 @@ int launch_update_slab(const cake_bf16* X, const int* idx, int B, i64 N, int D, 
 // out_C = counts>0 ? sums/counts : C_prev (or 0); optional bf16 copy.  early: launched so that it may
 // start before the kernel ahead of it in the stream has drained (it waits for that kernel itself)
 // next (nullable): also prepare the tensor-core assign of the centroids being written (its half-norm
-// operand, max ||c||^2, cleared inertia entries), so that that assign needs no prologue.  Needs
+// operand, cleared inertia entries), so that that assign needs no prologue.  Needs
 // D % 4 == 0 and out_C_bf16; *prepared tells whether it was done.
 // sums_columns (0 = D): columns of a row of sums, when they were added up from the padded copy of X.
 struct NextAssign {
     void* caug;             // as for launch_assign_tc
-    int* cnmax;             // zero on entry (the assign kernel ahead left it so)
     double* inertia;        // nullable: inertia[b * inertia_stride] = 0 for b < B (B <= 256)
     int inertia_stride;
     cake_bf16* cpad;        // nullable: as for launch_assign_tc, rows of cpad_columns columns

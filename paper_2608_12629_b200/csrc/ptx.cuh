@@ -202,6 +202,13 @@ __device__ __forceinline__ float fmin3(float a, float b, float c) {
     return d;
 }
 
+// (a & mask) | c as one three-input logic instruction
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t mask, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(c));
+    return d;
+}
+
 // ------------------------------------------------------------------ UMMA descriptors
 // Shared-memory operand descriptor for a K-major bf16 tile stored as rows of 128 bytes with the
 // 128-byte swizzle (what a TMA box of 64 bf16 x R rows with SWIZZLE_128B writes):

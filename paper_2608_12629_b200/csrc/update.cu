@@ -1136,11 +1136,11 @@ finalize4_kernel(const float4* __restrict__ sums, const int* __restrict__ counts
 // D % 4 == 0, one warp per centroid row (lanes stride the row in quads of columns): the division as in
 // finalize4_kernel and, on the way, what the tensor-core assign of these centroids needs as its
 // prologue: ||c||^2 of the bf16-rounded row (summed as the assign prologue sums it), split into the
-// k-step operand row, the problem's max ||c||^2 and cleared inertia entries.
+// k-step operand row, and cleared inertia entries.
 __global__ void __launch_bounds__(256)
 finalize_rows_kernel(const float4* __restrict__ sums, const int* __restrict__ counts,
                      const uint2* __restrict__ C_prev, i64 rows, int K, int D4, float4* __restrict__ out_C,
-                     uint2* __restrict__ out_C_bf16, uint8_t* __restrict__ caug, int* __restrict__ cnmax, int Kpad,
+                     uint2* __restrict__ out_C_bf16, uint8_t* __restrict__ caug, int Kpad,
                      double* __restrict__ inertia, int inertia_stride, int B, uint2* __restrict__ cpad, int Dc4,
                      int Ds4) {
     ptx::grid_dep_wait();
@@ -1176,7 +1176,7 @@ finalize_rows_kernel(const float4* __restrict__ sums, const int* __restrict__ co
             acc = aug::add_squares(acc, o.x, o.y);
         }
         acc = aug::fold_lanes(acc);
-        if (lane == 0) aug::write_row(caug, cnmax, row / K, static_cast<int>(row % K), K, Kpad, acc);
+        if (lane == 0) aug::write_row(caug, row / K, static_cast<int>(row % K), K, Kpad, acc);
     }
 }
 
@@ -1567,7 +1567,7 @@ cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf1
         cudaError_t e = launch_early(finalize_rows_kernel, dim3(static_cast<unsigned>(ctas)), dim3(256), 0, s,
                                      reinterpret_cast<const float4*>(sums), counts, reinterpret_cast<const uint2*>(C_prev), rows,
                                      K, D / 4, reinterpret_cast<float4*>(out_C), reinterpret_cast<uint2*>(out_C_bf16),
-                                     static_cast<uint8_t*>(next->caug), next->cnmax, padded_k(K), next->inertia,
+                                     static_cast<uint8_t*>(next->caug), padded_k(K), next->inertia,
                                      next->inertia_stride, B, reinterpret_cast<uint2*>(next->cpad), next->cpad_columns / 4,
                                      Ds / 4);
         note_launches(1);
