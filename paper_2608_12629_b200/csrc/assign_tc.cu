@@ -276,7 +276,10 @@ __device__ __forceinline__ int tile_step() { return CONSEC ? 1 : static_cast<int
 // CONSEC: consecutive row tiles per CTA (a batch of problems with resident centroids: see first_tile)
 // XSPLIT: one X buffer (all that fits beside the centroid ring when D > 256) whose chunks are loaded, consumed
 // and handed back one by one, so that the next row tile's first chunks arrive while this one's last are in use
-template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false>
+// BULK: the many-tile epilogue loads a whole 128-column slice, releases the accumulator and then reduces; otherwise
+// it reduces each 32-column group while the next one is being loaded (a template parameter and not a run-time
+// choice: with both epilogues in one kernel every shape measured 3-8 % slower)
+template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false, bool BULK = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
                  const Params p) {
@@ -981,41 +984,89 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 }
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                        as * BLOCK_N + wg * (BLOCK_N / 2);
-                // all four 32-column groups are requested at once; as soon as they are in registers
-                // the accumulator goes back to the MMA issuer and the reduction runs on registers
-                uint32_t ra[32], rb[32], rc[32], rd[32];
-                ptx::tmem_ld_x32(taddr, ra);
-                ptx::tmem_ld_x32(taddr + 32, rb);
-                ptx::tmem_ld_x32(taddr + 64, rc);
-                ptx::tmem_ld_x32(taddr + 96, rd);
-                ptx::tmem_ld_wait(ra);
-                ptx::reg_dep(rb);
-                ptx::reg_dep(rc);
-                ptx::reg_dep(rd);
-                ptx::tc_fence_before();
-                __syncwarp();
-                // to the issuer of tile acc_it + 2, which takes this accumulator next
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
-                next_iss = (next_iss + 1 == n_iss) ? 0 : next_iss + 1;
-                trace_mark(ctrl, 100);
-                if (PACKED) {
-                    float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
-                    tmin = packed_min32(rb, 32, tmin, kmask);
-                    tmin = packed_min32(rc, 64, tmin, kmask);
-                    tmin = packed_min32(rd, 96, tmin, kmask);
-                    // across tiles only the (truncated) value decides: an equal value keeps the earlier tile
-                    if (__uint_as_float(__float_as_uint(tmin) & ~COL_MASK) <
-                        __uint_as_float(__float_as_uint(best) & ~COL_MASK)) {
-                        best = tmin;
-                        bsel = nt;
+                if (!BULK) {
+                    // The four 32-column groups go through two register buffers: the load of group g + 1 is in
+                    // flight while group g is reduced (a warp that first loads everything and then reduces
+                    // leaves the TMEM path idle half of the time and the ALU pipe the other half: both warps
+                    // of a scheduler wait for the same accumulator and run in step).  The accumulator goes
+                    // back to its MMA issuer when the last group has landed.
+                    uint32_t ra[32], rb[32];
+                    ptx::tmem_ld_x32(taddr, ra);
+                    ptx::tmem_ld_wait(ra);
+                    ptx::tmem_ld_x32_before(taddr + 32, rb, ra);
+                    if (PACKED) {
+                        float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
+                        ptx::tmem_ld_wait_after(rb, tmin);
+                        ptx::tmem_ld_x32_before(taddr + 64, ra, rb);
+                        tmin = packed_min32(rb, 32, tmin, kmask);
+                        ptx::tmem_ld_wait_after(ra, tmin);
+                        ptx::tmem_ld_x32_before(taddr + 96, rb, ra);
+                        tmin = packed_min32(ra, 64, tmin, kmask);
+                        ptx::tmem_ld_wait_after(rb, tmin);
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        // to the issuer of tile acc_it + 2, which takes this accumulator next
+                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
+                        trace_mark(ctrl, 100);
+                        tmin = packed_min32(rb, 96, tmin, kmask);
+                        // across tiles only the (truncated) value decides: an equal value keeps the earlier tile
+                        if (__uint_as_float(__float_as_uint(tmin) & ~COL_MASK) <
+                            __uint_as_float(__float_as_uint(best) & ~COL_MASK)) {
+                            best = tmin;
+                            bsel = nt;
+                        }
+                    } else {
+                        const int col0 = nt * BLOCK_N + wg * (BLOCK_N / 2);
+                        exact_scan32(ra, col0, best, bsel);
+                        ptx::tmem_ld_wait_after(rb, best);
+                        ptx::tmem_ld_x32_before(taddr + 64, ra, rb);
+                        exact_scan32(rb, col0 + 32, best, bsel);
+                        ptx::tmem_ld_wait_after(ra, best);
+                        ptx::tmem_ld_x32_before(taddr + 96, rb, ra);
+                        exact_scan32(ra, col0 + 64, best, bsel);
+                        ptx::tmem_ld_wait_after(rb, best);
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
+                        trace_mark(ctrl, 100);
+                        exact_scan32(rb, col0 + 96, best, bsel);
                     }
                 } else {
-                    const int col0 = nt * BLOCK_N + wg * (BLOCK_N / 2);
-                    exact_scan32(ra, col0, best, bsel);
-                    exact_scan32(rb, col0 + 32, best, bsel);
-                    exact_scan32(rc, col0 + 64, best, bsel);
-                    exact_scan32(rd, col0 + 96, best, bsel);
+                    // (D = 128 with many centroid tiles per row tile measured 3-6 % faster when the accumulator is
+                    // handed back at once: all four groups are requested together, the accumulator is released as
+                    // soon as they have landed, and the reduction runs on registers afterwards)
+                    uint32_t ra[32], rb[32], rc[32], rd[32];
+                    ptx::tmem_ld_x32(taddr, ra);
+                    ptx::tmem_ld_x32(taddr + 32, rb);
+                    ptx::tmem_ld_x32(taddr + 64, rc);
+                    ptx::tmem_ld_x32(taddr + 96, rd);
+                    ptx::tmem_ld_wait(ra);
+                    ptx::reg_dep(rb);
+                    ptx::reg_dep(rc);
+                    ptx::reg_dep(rd);
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
+                    trace_mark(ctrl, 100);
+                    if (PACKED) {
+                        float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
+                        tmin = packed_min32(rb, 32, tmin, kmask);
+                        tmin = packed_min32(rc, 64, tmin, kmask);
+                        tmin = packed_min32(rd, 96, tmin, kmask);
+                        if (__uint_as_float(__float_as_uint(tmin) & ~COL_MASK) <
+                            __uint_as_float(__float_as_uint(best) & ~COL_MASK)) {
+                            best = tmin;
+                            bsel = nt;
+                        }
+                    } else {
+                        const int col0 = nt * BLOCK_N + wg * (BLOCK_N / 2);
+                        exact_scan32(ra, col0, best, bsel);
+                        exact_scan32(rb, col0 + 32, best, bsel);
+                        exact_scan32(rc, col0 + 64, best, bsel);
+                        exact_scan32(rd, col0 + 96, best, bsel);
+                    }
                 }
+                next_iss = (next_iss + 1 == n_iss) ? 0 : next_iss + 1;
             }
             if (!ok) break;
             trace_mark(ctrl, 102);
@@ -1315,20 +1366,27 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     // a single X buffer (D > 256) is filled and handed back chunk by chunk
     const bool xsplit = xload && p.res_c != 2 && p.n_xbuf == 1 && p.cps == 1 && p.nchunks <= MAX_XCHUNKS;
     Kernel kernel;
+    // D = 128 (two chunks) with many centroid tiles per row tile measured 3-6 % faster when the accumulator is handed
+    // back before the reduction; every other shape gains from reducing while loading (D = 64 up to 8 %)
+    const bool bulk = p.nchunks == 2 && p.n_tiles >= 8;
     if (!xload)
-        kernel = exact ? assign_tc_kernel<false, false> : assign_tc_kernel<true, false>;
+        kernel = exact ? (bulk ? assign_tc_kernel<false, false, false, false, true> : assign_tc_kernel<false, false>)
+                       : (bulk ? assign_tc_kernel<true, false, false, false, true> : assign_tc_kernel<true, false>);
     else if (exact)
         kernel = consec ? (xsplit ? assign_tc_kernel<false, true, true, true> : assign_tc_kernel<false, true, true, false>)
                         : (xsplit ? assign_tc_kernel<false, true, false, true> : assign_tc_kernel<false, true, false, false>);
     else
         kernel = consec ? (xsplit ? assign_tc_kernel<true, true, true, true> : assign_tc_kernel<true, true, true, false>)
                         : (xsplit ? assign_tc_kernel<true, true, false, true> : assign_tc_kernel<true, true, false, false>);
-    static int attr_done_for_device = -1;  // benign race: the attribute calls are idempotent
-    if (attr_done_for_device != di.device) {
+    static bool attr_done[64] = {false};   // per device; benign race: the attribute calls are idempotent
+    const bool attr_known = di.device >= 0 && di.device < 64;
+    if (!attr_known || !attr_done[di.device]) {
         if (cudaFuncSetAttribute(assign_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<false, false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
@@ -1336,7 +1394,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             cudaFuncSetAttribute(assign_tc_kernel<true, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
             return CAKE_ERR_CUDA;
-        attr_done_for_device = di.device;
+        if (attr_known) attr_done[di.device] = true;
     }
     const unsigned grid = static_cast<unsigned>(p.total_tiles < di.sm_count ? p.total_tiles : di.sm_count);
     cudaLaunchConfig_t cfg = {};

@@ -168,6 +168,35 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
         :
         : "memory");
 }
+// The same, and the wait also takes `after` as an in/out operand: whatever computes `after` is scheduled
+// ahead of the wait (work on registers that overlaps the loads in flight).
+__device__ __forceinline__ void tmem_ld_wait_after(uint32_t (&r)[32], float& after) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
+          "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]),
+          "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]),
+          "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]),
+          "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31]), "+f"(after)
+        :
+        : "memory");
+}
+// tcgen05.ld that is also ordered ahead of every later use of `held` (registers of an earlier load that are
+// about to be reduced): the load is issued first and runs while they are worked on.
+__device__ __forceinline__ void tmem_ld_x32_before(uint32_t taddr, uint32_t (&r)[32], uint32_t (&held)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%36];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+          "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]),
+          "+r"(held[0]), "+r"(held[8]), "+r"(held[16]), "+r"(held[24])
+        : "r"(taddr)
+        : "memory");
+}
 // Pure scheduling dependency (no instruction): pins a second register group behind a wait.
 __device__ __forceinline__ void reg_dep(uint32_t (&r)[32]) {
     asm volatile(""

@@ -29,7 +29,8 @@ def shard_rows(N: int, rank: int, world: int) -> tuple[int, int]:
     return first, first + q + (1 if rank < r else 0)
 
 
-def cake_kmeans_lloyd_sharded(X_local: torch.Tensor, C0: torch.Tensor, iters: int, group=None, flags: int = 0) -> LloydOutput:
+def cake_kmeans_lloyd_sharded(X_local: torch.Tensor, C0: torch.Tensor, iters: int, group=None, flags: int = 0,
+                              out: LloydOutput | None = None, ws: torch.Tensor | None = None) -> LloydOutput:
     """iters Lloyd iterations; X_local bf16 [N_local, D] are this rank's rows, C0 bf16 [K, D] the same on all ranks.
 
     Returns this rank's idx / dist (for its own rows) and the global C, counts and inertia.  Without an
@@ -43,8 +44,10 @@ def cake_kmeans_lloyd_sharded(X_local: torch.Tensor, C0: torch.Tensor, iters: in
     exchange = dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1
     if iters == 0:
         return binding.cake_kmeans_lloyd(X_local, C0, 0)
-    ws = binding.alloc_workspace(1, N, D, K, dev)
-    out = binding.alloc_lloyd_outputs(X_local, C0, iters)
+    if ws is None:
+        ws = binding.alloc_workspace(1, N, D, K, dev)
+    if out is None:
+        out = binding.alloc_lloyd_outputs(X_local, C0, iters)
     sums = torch.empty(K, D, dtype=torch.float32, device=dev)
     cbuf = [torch.empty_like(C0), torch.empty_like(C0)]
     cur = C0

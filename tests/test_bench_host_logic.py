@@ -23,6 +23,36 @@ def test_algorithmic_bytes_and_peaks():
     assert p["hbm_gbs"] > 1000 and p["bf16_tflops"] > 100 and p["source"] in ("measured", "fallback")
 
 
+def test_repeats_and_clock_bins():
+    assert bench.repeats_for(6.0, 1000.0) == 167 and bench.repeats_for(2000.0, 1000.0) == 1 and bench.repeats_for(0.0, 1000.0) == 1
+    assert bench.repeats_for(1e-4, 1000.0) == 4000                       # capped
+    peaks = {"bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0}
+    chunks = [(1965, [1.0, 1.0]), (1650, [2.0]), (None, [4.0])]
+    b = bench.bin_by_clock(chunks, peaks, unit_work=1.6e12, peak_key_burst="bf16_tflops",
+                           peak_key_settled="bf16_tflops_sustained", scale=1e-12)
+    assert b["burst"]["samples"] == 2 and b["burst"]["frac"] == pytest.approx(1.0)          # 1.6e12 FLOP in 1 ms = 1600 TF
+    assert b["settled"]["sm_mhz"] == 1650 and b["settled"]["frac"] == pytest.approx(800.0 / 1400.0)
+    assert b["unknown"]["rate"] == pytest.approx(400.0)
+    from paper_2608_12629_b200 import inputs
+    assert "c2: N=1048576 D=128 K=1024 B=1" in bench.workload_string(inputs.WORKLOADS["c2"])
+    assert "WARM" in bench.l2_note(inputs.WORKLOADS["c1"], False) and "COLD" in bench.l2_note(inputs.WORKLOADS["c1"], True)
+    assert "larger than" in bench.l2_note(inputs.WORKLOADS["c2"], False)
+
+
+def test_parity_on_sample_counts_near_ties_and_unexcused():
+    import numpy as np
+    from oracle import kmeans_oracle as orc
+    from paper_2608_12629_b200 import inputs
+    X = torch.tensor([[0.0, 0.0], [1.0, 0.0], [10.0, 0.0], [5.0, 0.0]]).to(torch.bfloat16)
+    C = torch.tensor([[0.0, 0.0], [10.0, 0.0], [10.0078125, 0.0]]).to(torch.bfloat16)   # centroids 1 and 2 nearly coincide
+    Xb, Cb = inputs.to_bits(X), inputs.to_bits(C)
+    idx_o, dist_o, _ = orc.assign(Xb, Cb)
+    sel = np.arange(4)
+    gpu = np.array([0, 1, 2, 0], dtype=np.int32)            # row 1: plainly wrong; row 2: the near twin; row 3: exact tie broken right
+    rep = bench.parity_on_sample(Xb, Cb, sel, idx_o, dist_o, gpu, orc.pair_sqdist(Xb, Cb, gpu).astype(np.float32))
+    assert rep == {"rows": 4, "mismatch": 2, "near_ties": 1, "unexcused": 1, "max_dist_err_rel": 0.0}
+
+
 def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():
     env = dict(os.environ, OMP_NUM_THREADS="4")
     cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c1", "--steps", "2",
