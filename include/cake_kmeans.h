@@ -132,10 +132,16 @@ CAKE_API int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, 
  * outside any stream capture.  All calls on a device share the one array, which keeps the
  * previous call's contents: the call itself clears what must start at zero, but two calls whose
  * work overlaps on the GPU (different streams, no ordering between them) race on it -- order them.
- * The device status word is not readable through this entry point.
+ * For D % 64 != 0 the centroid rows are streamed as they are (the workspace calls stream a zero-padded
+ * copy, which this call has no room for): same results, up to twice the time.
+ *
+ * cake_kmeans_assign_static_status reads the array's sticky device status word (CAKE_OK, or
+ * CAKE_ERR_TIMEOUT if a bounded in-kernel wait of an earlier static call expired): it synchronises
+ * `stream`, copies the word to *host_out (host pointer) and clears it.  Allocates nothing either.
  */
 CAKE_API int cake_kmeans_assign_static(const cake_bf16* X, const cake_bf16* C, long long N, int D, int K,
                                        int* out_idx, float* out_dist, cake_stream_t stream);
+CAKE_API int cake_kmeans_assign_static_status(cake_stream_t stream, int* host_out);
 
 /*
  * centroid_update (same paragraph: per-cluster sums and counts), followed by the division.

@@ -29,6 +29,7 @@ EXPORTS = [
     "cake_kmeans_lloyd_batched", "cake_kmeans_lloyd_host_device_bytes", "cake_kmeans_lloyd_host",
     "cake_kmeans_device_status", "cake_kmeans_selftest_bounded_wait", "cake_kmeans_assign_static",
     "cake_kmeans_update_partial_batched", "cake_kmeans_update_finish_batched", "cake_kmeans_inertia_batched",
+    "cake_kmeans_assign_static_status",
 ]
 
 _lib = None
@@ -64,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.cake_kmeans_device_status.argtypes = [vp, vp, ctypes.POINTER(i)]
         L.cake_kmeans_selftest_bounded_wait.argtypes = [vp, sz, i, vp]
         L.cake_kmeans_assign_static.argtypes = [vp, vp, ll, i, i, vp, vp, vp]
+        L.cake_kmeans_assign_static_status.argtypes = [vp, ctypes.POINTER(i)]
         L.cake_kmeans_update_partial_batched.argtypes = [vp, vp, ll, ll, i, i, vp, vp, vp, sz, vp, u]
         L.cake_kmeans_update_finish_batched.argtypes = [vp, vp, vp, ll, i, i, vp, vp, vp]
         L.cake_kmeans_inertia_batched.argtypes = [vp, ll, ll, vp, i, vp]
@@ -331,3 +333,12 @@ def cake_kmeans_assign_static(X, C, out_idx=None, out_dist=None, stream=None, wa
                                              _stream(stream, X.device))
     _check(rc, "cake_kmeans_assign_static")
     return out_idx, out_dist
+
+
+def cake_kmeans_assign_static_status(device, stream=None) -> int:
+    """Sticky device status of the workspace-free assign's fixed scratch on `device` (read and cleared)."""
+    v = ctypes.c_int(0)
+    with torch.cuda.device(device):
+        _check(lib().cake_kmeans_assign_static_status(_stream(stream, device), ctypes.byref(v)),
+               "cake_kmeans_assign_static_status")
+    return int(v.value)

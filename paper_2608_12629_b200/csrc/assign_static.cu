@@ -58,6 +58,7 @@ extern "C" int cake_kmeans_assign_static(const cake_bf16* X, const cake_bf16* C,
     if (K > kStaticMaxK) return CAKE_ERR_UNSUPPORTED;      // beyond the fixed scratch: use cake_kmeans_assign
     if (!C || (N > 0 && (!X || !out_idx))) return CAKE_ERR_NULL;
     if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(C)) % 16 != 0) return CAKE_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(out_idx) | reinterpret_cast<uintptr_t>(out_dist)) % 4 != 0) return CAKE_ERR_ALIGN;
     if (N == 0) return CAKE_OK;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (!assign_tc_supports(D)) return launch_assign_simt(X, C, 1, N, D, K, out_idx, out_dist, s);
@@ -65,11 +66,25 @@ extern "C" int cake_kmeans_assign_static(const cake_bf16* X, const cake_bf16* C,
     unsigned char* scratch = nullptr;
     int rc = scratch_for_current_device(&scratch);
     if (rc != CAKE_OK) return rc;
-    int* status = reinterpret_cast<int*>(scratch);
-    // the array keeps whatever the previous call left: the status word must start at zero; the
-    // half-norm operand is rewritten in full (all ceil(K/256) tiles, padding rows included) by the
-    // prologue that launch_assign_tc runs first
-    if (cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) return CAKE_ERR_CUDA;
+    // Word 0 of the array is the sticky device status: zero when the library is loaded, raised by a kernel
+    // whose bounded wait expired, read and cleared by cake_kmeans_assign_static_status.  The half-norm operand
+    // behind the header is rewritten in full (all ceil(K/256) tiles, padding rows included) by the prologue
+    // that launch_assign_tc runs first, so nothing of an earlier call survives where this one reads.
+    // (launch_assign_tc makes its host-side checks before it enqueues anything.)
     return launch_assign_tc(X, C, 1, N, D, K, scratch + kStaticHeader, false, out_idx, out_dist, nullptr, 0,
-                            false, false, status, s);
+                            false, false, reinterpret_cast<int*>(scratch), s);
+}
+
+extern "C" int cake_kmeans_assign_static_status(cake_stream_t stream, int* host_out) {
+    if (!host_out) return CAKE_ERR_NULL;
+    unsigned char* scratch = nullptr;
+    int rc = scratch_for_current_device(&scratch);
+    if (rc != CAKE_OK) return rc;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    int v = 0;
+    if (cudaMemcpyAsync(&v, scratch, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return CAKE_ERR_CUDA;
+    if (cudaMemsetAsync(scratch, 0, sizeof(int), s) != cudaSuccess) return CAKE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return CAKE_ERR_CUDA;
+    *host_out = v;
+    return CAKE_OK;
 }

@@ -1255,29 +1255,6 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     cudaLaunchAttribute pdl[1];
     pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl[0].val.programmaticStreamSerializationAllowed = 1;
-    if (!aug_ready) {
-        const i64 rows = static_cast<i64>(B) * Kpad;
-        const i64 ctas = (rows * 32 + 255) / 256;
-        if (zero_inertia && inertia && B > 256) {   // more problems than the prologue's first CTA has threads
-            if (cudaMemset2DAsync(inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
-                                  static_cast<size_t>(B), s) != cudaSuccess)
-                return CAKE_ERR_CUDA;
-        }
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(static_cast<unsigned>(ctas));
-        cfg.blockDim = dim3(256);
-        cfg.stream = s;
-        cfg.attrs = pdl;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, centroid_aug_kernel, C, K, D, Kpad, rows, static_cast<uint8_t*>(caug),
-                               (zero_inertia && B <= 256) ? inertia : static_cast<double*>(nullptr), inertia_stride,
-                               B, cpad, Dc) != cudaSuccess) {
-            cudaGetLastError();
-            return CAKE_ERR_CUDA;
-        }
-        note_launches(1);
-    }
-
     // Shared memory: X buffers (each with its 4 KiB norm operand), the centroid ring, fixed parts.
     // Few centroid tiles per row tile make row tiles short, so X has to run further ahead: up to four
     // X buffers then, two otherwise; a single one only if the ring would drop below three stages.
@@ -1396,6 +1373,30 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             return CAKE_ERR_CUDA;
         if (attr_known) attr_done[di.device] = true;
     }
+    // every host-side check has passed: from here on work is enqueued
+    if (!aug_ready) {
+        const i64 rows = static_cast<i64>(B) * Kpad;
+        const i64 ctas = (rows * 32 + 255) / 256;
+        if (zero_inertia && inertia && B > 256) {   // more problems than the prologue's first CTA has threads
+            if (cudaMemset2DAsync(inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
+                                  static_cast<size_t>(B), s) != cudaSuccess)
+                return CAKE_ERR_CUDA;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(ctas));
+        cfg.blockDim = dim3(256);
+        cfg.stream = s;
+        cfg.attrs = pdl;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, centroid_aug_kernel, C, K, D, Kpad, rows, static_cast<uint8_t*>(caug),
+                               (zero_inertia && B <= 256) ? inertia : static_cast<double*>(nullptr), inertia_stride,
+                               B, cpad, Dc) != cudaSuccess) {
+            cudaGetLastError();
+            return CAKE_ERR_CUDA;
+        }
+        note_launches(1);
+    }
+
     const unsigned grid = static_cast<unsigned>(p.total_tiles < di.sm_count ? p.total_tiles : di.sm_count);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
