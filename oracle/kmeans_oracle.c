@@ -24,8 +24,9 @@
  * integer-valued cases, K=1 / C=X / 1-D midpoint special cases, permutation and translation
  * invariances, mean / mass-conservation / Huygens identities for update, monotone inertia and
  * fixed point for Lloyd, a hand-worked 2-D example in exact rationals, and a scikit-learn
- * cross-check.  No function here is "parity unpinned" against the mathematics; the paper itself
- * prints no numeric K-means result to pin against.
+ * cross-check; oracle_knn: numpy lexsort brute force, exact integer ties, k = 1 against
+ * oracle_assign, k >= M.  No function here is "parity unpinned" against the mathematics; the paper
+ * itself prints no numeric K-means or KNN result to pin against.
  */
 #include <math.h>
 #include <stdint.h>
@@ -221,6 +222,53 @@ int oracle_lloyd(const uint16_t* X, const uint16_t* C0, i64 N, int D, int K, int
     free(Ct);
     if (!dist) free(dloc);
     return rc;
+}
+
+/*
+ * Exact k-nearest-neighbour search (the paper's Section 6 names a "KNN search" family with recall 1.0,
+ * i.e. the exact result; the distance is the squared Euclidean one of the K-means workload).
+ *   Q    [N,D] bf16 bits: queries          X [M,D] bf16 bits: database rows
+ *   idx  [N,k] the k database rows nearest to each query, ascending by (distance, row number):
+ *              among equal distances the lower row number comes first
+ *   dist [N,k] their squared distances (direct differences, fp64)
+ * When M < k the tail of each row is idx = -1, dist = +inf.
+ * Plain statement: every distance is computed, and a row enters the sorted list of the k best only if
+ * its distance is strictly smaller than the current k-th best (rows come in ascending order, so an equal
+ * later row never displaces an earlier one) and is placed behind every entry that is not larger.
+ */
+int oracle_knn(const uint16_t* Q, const uint16_t* X, i64 N, i64 M, int D, int k, int32_t* idx, double* dist) {
+    if (!Q || !X || !idx || !dist || N < 0 || M < 0 || D < 1 || k < 1) return -1;
+#pragma omp parallel
+    {
+        double* q = (double*)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(static)
+        for (i64 i = 0; i < N; ++i) {
+            for (int d = 0; d < D; ++d) q[d] = bf16_bits_to_f64(Q[i * D + d]);
+            int32_t* bi = idx + i * k;
+            double* bd = dist + i * k;
+            int cnt = 0;
+            for (int s = 0; s < k; ++s) { bi[s] = -1; bd[s] = INFINITY; }
+            for (i64 j = 0; j < M; ++j) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d) {
+                    double t = q[d] - bf16_bits_to_f64(X[j * D + d]);
+                    acc += t * t;
+                }
+                if (cnt == k && !(acc < bd[k - 1])) continue;
+                int pos = cnt < k ? cnt : k - 1;          /* slot that opens up (the last one is dropped when full) */
+                while (pos > 0 && bd[pos - 1] > acc) {    /* entries strictly larger move down one place */
+                    bd[pos] = bd[pos - 1];
+                    bi[pos] = bi[pos - 1];
+                    --pos;
+                }
+                bd[pos] = acc;
+                bi[pos] = (int32_t)j;
+                if (cnt < k) ++cnt;
+            }
+        }
+        free(q);
+    }
+    return 0;
 }
 
 int oracle_num_threads(void) {

@@ -48,6 +48,7 @@ def _load():
         lib.oracle_pair_sqdist.argtypes = [vp, vp, i64, i32, i32, vp, vp]
         lib.oracle_update.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp]
         lib.oracle_lloyd.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_knn.argtypes = [vp, vp, i64, i64, i32, i32, vp, vp]
         lib.oracle_num_threads.restype = i32
         _lib = lib
     return _lib
@@ -146,6 +147,21 @@ def update(X: np.ndarray, idx: np.ndarray, K: int, C_prev: np.ndarray | None = N
     if rc != 0:
         raise RuntimeError(f"oracle_update failed: {rc}")
     return (C_new, counts, sums) if return_sums else (C_new, counts)
+
+
+def knn(Q: np.ndarray, X: np.ndarray, k: int):
+    """The k database rows nearest to every query: Q [N,D], X [M,D] bf16 bits -> (idx int32 [N,k], dist f64 [N,k]),
+    ascending by (distance, row number); idx -1 / dist +inf where M < k."""
+    Q, X = _bits(Q, "Q"), _bits(X, "X")
+    if Q.shape[1] != X.shape[1] or k < 1:
+        raise ValueError("Q and X need the same D, k >= 1")
+    N, D = Q.shape
+    idx = np.empty((N, k), dtype=np.int32)
+    dist = np.empty((N, k), dtype=np.float64)
+    rc = _load().oracle_knn(_p(Q), _p(X), N, X.shape[0], D, k, _p(idx), _p(dist))
+    if rc != 0:
+        raise RuntimeError(f"oracle_knn failed: {rc}")
+    return idx, dist
 
 
 @dataclass

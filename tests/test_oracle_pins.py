@@ -314,3 +314,53 @@ def test_lloyd_teacher_forced_composition():
         C_new, counts = orc.update(Xb, idx, 7, cur)
         cur = orc.f64_to_bf16(C_new)
     assert np.array_equal(cur, r.C_bits) and np.array_equal(idx, r.idx) and np.array_equal(counts, r.counts)
+
+
+# ------------------------------------------------------------------------------------ k nearest neighbours
+
+def _knn_brute(Q, X, k):
+    q, x = Q.double().numpy(), X.double().numpy()
+    d = ((q[:, None, :] - x[None, :, :]) ** 2).sum(-1)
+    order = np.stack([np.lexsort((np.arange(x.shape[0]), row)) for row in d])      # by distance, then row number
+    idx = np.full((q.shape[0], k), -1, dtype=np.int64)
+    dist = np.full((q.shape[0], k), np.inf)
+    kk = min(k, x.shape[0])
+    idx[:, :kk] = order[:, :kk]
+    dist[:, :kk] = np.take_along_axis(d, order[:, :kk], 1)
+    return idx, dist
+
+
+@pytest.mark.parametrize("N,M,D,k", [(7, 50, 3, 1), (20, 200, 5, 8), (5, 64, 16, 32), (9, 10, 2, 10), (4, 6, 4, 9)])
+def test_knn_vs_numpy_bruteforce(N, M, D, k):
+    g = torch.Generator().manual_seed(N * M + k)
+    Q = torch.randn(N, D, generator=g).to(torch.bfloat16)
+    X = torch.randn(M, D, generator=g).to(torch.bfloat16)
+    idx, dist = orc.knn(inputs.to_bits(Q), inputs.to_bits(X), k)
+    bi, bd = _knn_brute(Q, X, k)
+    assert np.array_equal(idx, bi)
+    np.testing.assert_allclose(dist, bd, rtol=1e-13)
+    # a second, independent selection: partition, then order the k survivors
+    d = ((Q.double().numpy()[:, None] - X.double().numpy()[None]) ** 2).sum(-1)
+    kk = min(k, M)
+    part = np.argpartition(d, kk - 1, axis=1)[:, :kk]
+    assert all(set(part[i]) == set(idx[i, :kk]) for i in range(N))          # random reals: no ties
+    assert (np.diff(dist[:, :kk], axis=1) >= 0).all()
+
+
+def test_knn_integer_ties_go_to_the_lower_row_and_k1_is_assign():
+    g = torch.Generator().manual_seed(2)
+    Q = torch.randint(-2, 3, (40, 6), generator=g).to(torch.bfloat16)
+    X = torch.randint(-2, 3, (300, 6), generator=g).to(torch.bfloat16)
+    X[100:200] = X[0:100]                                    # every one of these rows exists twice
+    idx, dist = orc.knn(inputs.to_bits(Q), inputs.to_bits(X), 12)
+    bi, bd = _knn_brute(Q, X, 12)
+    assert np.array_equal(idx, bi) and np.array_equal(dist, bd)       # integers: exact, ties included
+    d = dist
+    tied = d[:, 1:] == d[:, :-1]
+    assert tied.any() and (idx[:, 1:][tied] > idx[:, :-1][tied]).all()
+    i1, d1 = orc.knn(inputs.to_bits(Q), inputs.to_bits(X), 1)
+    ia, da, _ = orc.assign(inputs.to_bits(Q), inputs.to_bits(X))
+    assert np.array_equal(i1[:, 0], ia) and np.array_equal(d1[:, 0], da)
+    # a point that is in the database finds itself first, at distance 0
+    i2, d2 = orc.knn(inputs.to_bits(X[:50]), inputs.to_bits(X), 3)
+    assert np.array_equal(i2[:, 0], np.arange(50)) and (d2[:, 0] == 0).all()
