@@ -335,6 +335,60 @@ def run_sweep(args):
             torch.cuda.empty_cache()
 
 
+def run_knn(args):
+    """k-nearest-neighbour search: one markdown row per shape with the fraction of the same tensor roofline the
+    assign kernel is measured against (2 N M D FLOP at the measured bf16 peak, or the bytes at HBM bandwidth)."""
+    import paper_2608_12629_b200 as cake
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = measured_peaks()
+    print("| queries N | database M | D | k | ms | TFLOP/s | fraction of roofline | rows graded | mismatch | unexcused |")
+    print("|---|---|---|---|---|---|---|---|---|---|", flush=True)
+    shapes = [(65536, 1 << 20, 128), (65536, 1 << 20, 64), (16384, 1 << 22, 128), (1 << 20, 4096, 128), (65536, 1 << 18, 256),
+              (8192, 65536, 96)]
+    for N, M, D in shapes:
+        w = inputs.sweep_workload(M, D, 64)
+        X, _ = inputs.gaussian_mixture(M, D, 4096, w.mean_std, w.sigma, w.seed, device=dev)
+        Q, _ = inputs.gaussian_mixture(N, D, 4096, w.mean_std, w.sigma, w.seed + 1, device=dev)
+        for k in (1, 8, 32):
+            ws = torch.zeros(cake.cake_knn_workspace_bytes(N, M, D, k), dtype=torch.uint8, device=dev)
+            idx, dist = cake.cake_knn_search(Q, X, k, ws=ws)
+            torch.cuda.synchronize()
+            reps = 5
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+            ev[0].record()
+            for i in range(reps):
+                cake.cake_knn_search(Q, X, k, out_idx=idx, out_dist=dist, ws=ws)
+                ev[i + 1].record()
+            torch.cuda.synchronize()
+            if cake.cake_kmeans_device_status(ws) != cake.CAKE_OK:
+                raise SystemExit("device status raised")
+            ms = statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(reps))
+            flop = 2.0 * N * M * D
+            byts = 2.0 * (N + M) * D + 8.0 * N * k
+            floor_ms = max(flop / (peaks["bf16_tflops"] * 1e12), byts / (peaks["hbm_gbs"] * 1e9)) * 1e3
+            row = f"| {N} | {M} | {D} | {k} | {ms:.3f} | {flop / ms / 1e9:.0f} | {floor_ms / ms:.3f} |"
+            if not args.no_cpu_baseline:
+                from oracle import kmeans_oracle as orc
+                sel = np.sort(np.random.default_rng(k).choice(N, 64 if M > (1 << 20) else 128, replace=False))
+                sel_t = torch.from_numpy(sel).to(dev)
+                Qb, Xb = inputs.to_bits(Q[sel_t]), inputs.to_bits(X)
+                io, do = orc.knn(Qb, Xb, k)
+                g = idx[sel_t].cpu().numpy()
+                Xf, Qf = orc.bf16_to_f64(Xb), orc.bf16_to_f64(Qb)
+                qn, xn = (Qf * Qf).sum(1), (Xf * Xf).sum(1)
+                d_g = np.stack([orc.pair_sqdist(Qb, Xf, np.ascontiguousarray(g[:, p_])) for p_ in range(k)], 1)
+                mism = g != io
+                unexc = mism & ~(np.abs(d_g - do) < 1e-3 * (qn[:, None] + xn[io]))
+                row += f" {len(sel)} | {int(mism.sum())} | {int(unexc.sum())} |"
+            else:
+                row += " - | - | - |"
+            print(row, flush=True)
+            del ws
+        del X, Q
+        torch.cuda.empty_cache()
+
+
 class Runner:
     """One workload on this rank: buffers, the Lloyd call being timed and the per-kernel calls."""
 
@@ -557,9 +611,13 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="print the shape-sweep table instead of the JSON line")
     ap.add_argument("--sweep-full", action="store_true", help="with --sweep: every power of two in N and K")
     ap.add_argument("--sweep-grade", action="store_true", help="with --sweep: grade every shape on sampled rows with the CPU oracle")
+    ap.add_argument("--knn", action="store_true", help="print the k-nearest-neighbour search table instead of the JSON line")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.knn:
+        run_knn(args)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

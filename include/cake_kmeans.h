@@ -224,6 +224,25 @@ CAKE_API int cake_kmeans_lloyd_host(const cake_bf16* X_host, const cake_bf16* C0
                            size_t dev_bytes, cake_stream_t stream, unsigned flags);
 
 /*
+ * Exact k-nearest-neighbour search (Section 6 names a KNN search family beside K-means, with recall 1.0:
+ * the exact result; Appendix F lists its routes by name only).  Same distance and same tensor-core
+ * pipeline as assign, with the database rows in the place of the centroids and a top-k epilogue.
+ *   Q        [N][D] bf16, in: queries           X [M][D] bf16, in: database rows
+ *   k        neighbours per query, 1..32 (more: CAKE_ERR_UNSUPPORTED)
+ *   out_idx  [N][k] int32, out: the k nearest database rows, ascending by (distance, row number): among
+ *            equal distances the lower row comes first; -1 where M < k
+ *   out_dist [N][k] fp32, out, may be NULL: max(0, squared distance); +inf where M < k
+ *   ws       scratch of at least cake_knn_workspace_bytes(...) bytes, 256-byte aligned, first 256 bytes
+ *            zeroed once by the caller; word 0 is the sticky device status (cake_kmeans_device_status)
+ * D <= 512 (D % 8 != 0 runs on zero-padded copies kept in ws); larger D: CAKE_ERR_UNSUPPORTED.
+ * Distances are fp32 numbers compared with all their bits; their error follows |q|^2 + |x|^2 of the pair.
+ * Asynchronous on `stream`; N = 0 does nothing.
+ */
+CAKE_API int cake_knn_workspace_bytes(long long N, long long M, int D, int k, size_t* out_bytes);
+CAKE_API int cake_knn_search(const cake_bf16* Q, const cake_bf16* X, long long N, long long M, int D, int k,
+                             int* out_idx, float* out_dist, void* ws, size_t ws_bytes, cake_stream_t stream);
+
+/*
  * Reads the sticky device status word of a workspace: synchronises `stream`, copies the word to
  * *host_out (host pointer) and clears it.  *host_out is CAKE_OK, CAKE_ERR_BAD_INDEX or
  * CAKE_ERR_TIMEOUT.  No paper counterpart.

@@ -9,7 +9,7 @@ from .binding import (  # noqa: F401
     CAKE_UPDATE_SLAB_F2, CAKE_UPDATE_SLAB_F4, CAKE_UPDATE_SMEM, CAKE_UPDATE_SORT, EXPORTS, LIB_PATH, CakeError, LloydOutput,
     alloc_lloyd_outputs, alloc_workspace, cake_kmeans_assign, cake_kmeans_assign_static, cake_kmeans_assign_static_status, cake_kmeans_device_status, cake_kmeans_inertia, cake_kmeans_lloyd,
     cake_kmeans_lloyd_host, cake_kmeans_kernel_launches, cake_kmeans_lloyd_host_device_bytes, cake_kmeans_selftest_bounded_wait,
-    cake_kmeans_update, cake_kmeans_update_finish, cake_kmeans_update_partial, cake_kmeans_workspace_bytes, cake_version, lib,
+    cake_kmeans_update, cake_kmeans_update_finish, cake_kmeans_update_partial, cake_kmeans_workspace_bytes, cake_knn_search, cake_knn_workspace_bytes, cake_version, lib,
     strerror,
 )
 from .sharded import cake_kmeans_lloyd_sharded, shard_rows  # noqa: F401

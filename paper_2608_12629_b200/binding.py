@@ -29,7 +29,7 @@ EXPORTS = [
     "cake_kmeans_lloyd_batched", "cake_kmeans_lloyd_host_device_bytes", "cake_kmeans_lloyd_host",
     "cake_kmeans_device_status", "cake_kmeans_selftest_bounded_wait", "cake_kmeans_assign_static",
     "cake_kmeans_update_partial_batched", "cake_kmeans_update_finish_batched", "cake_kmeans_inertia_batched",
-    "cake_kmeans_assign_static_status",
+    "cake_kmeans_assign_static_status", "cake_knn_workspace_bytes", "cake_knn_search",
 ]
 
 _lib = None
@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.cake_kmeans_selftest_bounded_wait.argtypes = [vp, sz, i, vp]
         L.cake_kmeans_assign_static.argtypes = [vp, vp, ll, i, i, vp, vp, vp]
         L.cake_kmeans_assign_static_status.argtypes = [vp, ctypes.POINTER(i)]
+        L.cake_knn_workspace_bytes.argtypes = [ll, ll, i, i, ctypes.POINTER(sz)]
+        L.cake_knn_search.argtypes = [vp, vp, ll, ll, i, i, vp, vp, vp, sz, vp]
         L.cake_kmeans_update_partial_batched.argtypes = [vp, vp, ll, ll, i, i, vp, vp, vp, sz, vp, u]
         L.cake_kmeans_update_finish_batched.argtypes = [vp, vp, vp, ll, i, i, vp, vp, vp]
         L.cake_kmeans_inertia_batched.argtypes = [vp, ll, ll, vp, i, vp]
@@ -342,3 +344,29 @@ def cake_kmeans_assign_static_status(device, stream=None) -> int:
         _check(lib().cake_kmeans_assign_static_status(_stream(stream, device), ctypes.byref(v)),
                "cake_kmeans_assign_static_status")
     return int(v.value)
+
+
+def cake_knn_workspace_bytes(N: int, M: int, D: int, k: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().cake_knn_workspace_bytes(N, M, D, k, ctypes.byref(out)), "cake_knn_workspace_bytes")
+    return int(out.value)
+
+
+def cake_knn_search(Q, X, k, out_idx=None, out_dist=None, ws=None, stream=None, want_dist=True):
+    """Q bf16 [N,D] queries, X bf16 [M,D] database -> (idx int32 [N,k], dist fp32 [N,k] or None), nearest first."""
+    _want(Q, torch.bfloat16, "Q"), _want(X, torch.bfloat16, "X")
+    if Q.dim() != 2 or X.dim() != 2 or Q.shape[1] != X.shape[1]:
+        raise ValueError("Q must be [N,D] and X [M,D]")
+    N, D, M = Q.shape[0], Q.shape[1], X.shape[0]
+    if out_idx is None:
+        out_idx = torch.empty(N, k, dtype=torch.int32, device=Q.device)
+    if out_dist is None and want_dist:
+        out_dist = torch.empty(N, k, dtype=torch.float32, device=Q.device)
+    if ws is None:
+        ws = torch.empty(cake_knn_workspace_bytes(N, M, D, k), dtype=torch.uint8, device=Q.device)
+        ws[:256].zero_()
+    with torch.cuda.device(Q.device):
+        rc = lib().cake_knn_search(_ptr(Q), _ptr(X), N, M, D, k, _ptr(out_idx), _ptr(out_dist), _ptr(ws), ws.numel(),
+                                   _stream(stream, Q.device))
+    _check(rc, "cake_knn_search")
+    return out_idx, out_dist

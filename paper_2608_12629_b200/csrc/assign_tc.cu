@@ -113,6 +113,8 @@ struct Params {
     float* out_dist;
     double* inertia;      // optional: inertia[b * inertia_stride] += sum of the problem's distances
     int inertia_stride;
+    int knn_k;        // TOPK instantiations (unused otherwise); out_idx / out_dist are then [N][2][TOPK]: one sorted list per
+                      // column half, merged by a small kernel afterwards
     int res_c;        // 1: alt_epi and the centroid tile stays in shared memory (loaded once per problem): the two
                       // issuers share no ring and each works on its own row tiles only; 2: two resident
                       // tiles, issuer i computes tile i of every row tile (shared epilogue)
@@ -251,6 +253,24 @@ __device__ __forceinline__ void exact_scan32(const uint32_t (&r)[32], int col_ba
     }
 }
 
+// Top-k epilogue (k-nearest-neighbour search): a row's list of its KMAX smallest values so far, in registers, sorted
+// ascending; candidates come in ascending column order, so one that equals an entry goes behind it (strict <) and
+// equal distances end up ordered by column.  x = +inf is a no-op (lanes without a candidate in a warp-wide step).
+template <int KMAX>
+__device__ __forceinline__ void topk_insert_sorted(float (&lv)[KMAX], int (&li)[KMAX], float x, int col) {
+#pragma unroll
+    for (int s = KMAX - 1; s >= 1; --s) {
+        const bool shift = x < lv[s - 1];          // the entry above moves down one place
+        const bool here = !shift && x < lv[s];     // x lands here
+        lv[s] = shift ? lv[s - 1] : (here ? x : lv[s]);
+        li[s] = shift ? li[s - 1] : (here ? col : li[s]);
+    }
+    if (x < lv[0]) {
+        lv[0] = x;
+        li[0] = col;
+    }
+}
+
 // XLOAD: warp 11 loads the X tiles and two warps issue MMAs (few centroid tiles per row tile);
 // otherwise the centroid producer also loads X and three warps issue MMAs.
 // Row tiles of a CTA.  Interleaved over the CTAs (blockIdx.x, blockIdx.x + gridDim.x, ...), except for a batch
@@ -279,7 +299,9 @@ __device__ __forceinline__ int tile_step() { return CONSEC ? 1 : static_cast<int
 // BULK: the many-tile epilogue loads a whole 128-column slice, releases the accumulator and then reduces; otherwise
 // it reduces each 32-column group while the next one is being loaded (a template parameter and not a run-time
 // choice: with both epilogues in one kernel every shape measured 3-8 % slower)
-template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false, bool BULK = false>
+// TOPK (0, 8 or 32): instead of the arg-min each epilogue thread keeps the TOPK smallest accumulators of its row and
+// column half (k-nearest-neighbour search: the "centroids" are the database rows); many-tile structure, packed gate.
+template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false, bool BULK = false, int TOPK = 0>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
                  const Params p) {
@@ -309,7 +331,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         for (int i = 0; i < MAX_XBUF; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
             // MMA issuers + 4 norm warps + the 4 epilogue warps that read the row margins
-            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), ((XLOAD && p.res_c == 1) ? 1 : NUM_ISSUERS) + 4 + 4);
+            // (TOPK: the upper column half reads the margins as well)
+            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), ((XLOAD && p.res_c == 1) ? 1 : NUM_ISSUERS) + 4 + 4 + (TOPK ? 4 : 0));
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
         }
         for (int i = 0; i < MAX_XCHUNKS; ++i) {
@@ -957,7 +980,42 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 dsum += static_cast<double>(dist);
             }
         }
+        // ---- TOPK: the row's sorted list (registers) of the smallest accumulators seen so far in this column half;
+        // its last entry is the threshold a candidate has to beat (+inf until the list is full)
+        constexpr int KL = TOPK ? TOPK : 1;
+        float lv[KL] = {};
+        int li[KL] = {};
+        float stash[TOPK ? 32 : 1];                      // a group's values, parked in local memory while it is walked
+        // One 32-column group.  Its smallest (truncated) value is compared with the threshold first; if any row of the
+        // warp may have a candidate, the group is walked: every lane marks its candidates, then all lanes insert their
+        // next candidate together, step by step (one copy of the insertion code, no lane waits for another lane's column).
+        auto topk_group = [&](const uint32_t (&rg)[32], int col0) {
+            const float gmin = packed_min32(rg, 0, __uint_as_float(F32_INF), kmask);
+            const bool want = __uint_as_float(__float_as_uint(gmin) & ~COL_MASK) < lv[KL - 1];
+            if (__any_sync(0xffffffffu, want)) {
+                uint32_t m = 0;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float v = __uint_as_float(rg[j]);
+                    stash[j] = v;
+                    m |= (v < lv[KL - 1] && col0 + j < p.K) ? (1u << j) : 0u;   // (columns behind the last row: padding)
+                }
+                while (__any_sync(0xffffffffu, m != 0u)) {
+                    const int j = m ? __ffs(static_cast<int>(m)) - 1 : 0;
+                    const float x = m ? stash[j] : __uint_as_float(F32_INF);
+                    m &= m - 1u;
+                    topk_insert_sorted<KL>(lv, li, x, col0 + j);
+                }
+            }
+        };
         for (i64 tile = blockIdx.x; !(XLOAD && p.alt_epi) && ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
+            if (TOPK) {
+#pragma unroll
+                for (int s = 0; s < KL; ++s) {
+                    lv[s] = __uint_as_float(F32_INF);
+                    li[s] = -1;
+                }
+            }
             if (b != dsum_b) {
                 flush_inertia();
                 dsum_b = b;
@@ -970,7 +1028,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
                 if (!ok) break;
                 ptx::tc_fence_after();
-                if (nt == 0 && wg == 0) {
+                if (nt == 0 && (wg == 0 || TOPK)) {
                     // Written by the norm warps before they completed auga_full.  The X buffer -- and with
                     // it this slot and the next phase of this barrier -- is handed to a later row tile
                     // only after these warps have arrived on x_empty: without that, with one centroid
@@ -984,7 +1042,29 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 }
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                        as * BLOCK_N + wg * (BLOCK_N / 2);
-                if (!BULK) {
+                if (TOPK) {
+                    // two sites of the group code (ra, rb), run twice: the list lives in registers and its insertion
+                    // is long, so the code is kept small
+                    const int col0 = nt * BLOCK_N + wg * (BLOCK_N / 2);
+                    uint32_t ra[32], rb[32];
+                    ptx::tmem_ld_x32(taddr, ra);
+                    ptx::tmem_ld_wait(ra);
+#pragma unroll 1
+                    for (int h = 0; h < 2; ++h) {
+                        ptx::tmem_ld_x32_before(taddr + 64 * h + 32, rb, ra);
+                        topk_group(ra, col0 + 64 * h);
+                        ptx::tmem_ld_wait_after(rb, lv[KL - 1]);
+                        if (h == 0) {
+                            ptx::tmem_ld_x32_before(taddr + 64, ra, rb);
+                        } else {
+                            ptx::tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
+                        }
+                        topk_group(rb, col0 + 64 * h + 32);
+                        if (h == 0) ptx::tmem_ld_wait_after(ra, lv[KL - 1]);
+                    }
+                } else if (!BULK) {
                     // The four 32-column groups go through two register buffers: the load of group g + 1 is in
                     // flight while group g is reduced (a warp that first loads everything and then reduces
                     // leaves the TMEM path idle half of the time and the ALU pipe the other half: both warps
@@ -1071,6 +1151,20 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             if (!ok) break;
             trace_mark(ctrl, 102);
             if (++exb == static_cast<uint32_t>(p.n_xbuf)) { exb = 0; exph ^= 1u; }
+            if (TOPK) {
+                // the list is sorted by (value, column): write it out, out_idx / out_dist [row][half][TOPK]; the two
+                // halves are merged by a small kernel afterwards.  Unused places: index -1, distance +inf.
+                const i64 row = static_cast<i64>(mt) * BLOCK_M + r;
+                if (row < p.N) {
+                    const size_t o = ((static_cast<size_t>(b) * static_cast<size_t>(p.N) + row) * 2 + wg) * KL;
+#pragma unroll
+                    for (int s = 0; s < KL; ++s) {
+                        p.out_idx[o + s] = li[s];
+                        p.out_dist[o + s] = fmaxf(0.f, 2.f * (lv[s] - rowM));
+                    }
+                }
+                continue;
+            }
             // (value, index) of this half; the value is a key with its column bits cleared (packed) or
             // the accumulator itself (exact)
             float bval;
@@ -1225,7 +1319,7 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s, int Dx,
-                     cake_bf16* cpad) {
+                     cake_bf16* cpad, int knn_k) {
     // D: columns of a row of C; Dk: columns of a row of X and length of the contraction (D, or D rounded up to
     // a multiple of 8 with zeros in the copy of X); Dc: columns of a row of the centroid operand the kernel
     // streams (C itself, or its zero-padded copy of a multiple of 64 columns, written by the prologue)
@@ -1247,6 +1341,8 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     p.caug = static_cast<const uint8_t*>(caug);
     p.out_idx = out_idx; p.out_dist = out_dist; p.status = status;
     p.inertia = inertia; p.inertia_stride = inertia_stride;
+    p.knn_k = knn_k;
+    if ((knn_k != 0 && knn_k != 8 && knn_k != 32) || (knn_k > 0 && (B != 1 || !out_dist || inertia))) return CAKE_ERR_UNSUPPORTED;
     if (p.total_tiles == 0) return CAKE_OK;
 
     const int Kpad = padded_k(K);
@@ -1285,11 +1381,12 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     if (rc != CAKE_OK) return rc;
 
     // one or two centroid tiles per row tile: the kernel is as fast as X arrives, X gets its own producer
-    const bool xload = p.n_tiles <= 2;
+    // (the top-k epilogue exists in the many-tile structure only)
+    const bool xload = p.n_tiles <= 2 && knn_k == 0;
     p.alt_epi = 0;   // without resident centroids (D = 256) the shared epilogue measured faster
     p.res_c = 0;
     int c_rows = BLOCK_N;   // rows of a centroid chunk in shared memory (the TMA box)
-    if (p.n_tiles == 1) {
+    if (p.n_tiles == 1 && xload) {
         // a single centroid tile: keep it in shared memory if an even number of X buffers fits beside it
         // (of the tile only the rows that hold centroids, in steps of 32, when there are at most 128)
         c_rows = K <= BLOCK_N / 2 ? static_cast<int>(round_up(K, 32)) : BLOCK_N;
@@ -1318,7 +1415,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             p.n_xbuf = 1;
         }
     }
-    if (p.n_tiles == 2) {
+    if (p.n_tiles == 2 && xload) {
         // two centroid tiles: both stay in shared memory if at least two X buffers fit beside them (D <= 128)
         const i64 c_bytes = 2 * (static_cast<i64>(p.nchunks) * C_CHUNK_BYTES + AUG_B_BYTES);
         for (int nx = MAX_XBUF; nx >= 2; --nx) {
@@ -1346,7 +1443,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     // D = 128 (two chunks) with many centroid tiles per row tile measured 3-6 % faster when the accumulator is handed
     // back before the reduction; every other shape gains from reducing while loading (D = 64 up to 8 %)
     const bool bulk = p.nchunks == 2 && p.n_tiles >= 8;
-    if (!xload)
+    if (knn_k > 0)
+        kernel = knn_k == 8 ? assign_tc_kernel<true, false, false, false, false, 8> : assign_tc_kernel<true, false, false, false, false, 32>;
+    else if (!xload)
         kernel = exact ? (bulk ? assign_tc_kernel<false, false, false, false, true> : assign_tc_kernel<false, false>)
                        : (bulk ? assign_tc_kernel<true, false, false, false, true> : assign_tc_kernel<true, false>);
     else if (exact)
@@ -1363,6 +1462,8 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             cudaFuncSetAttribute(assign_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, false, false, false, false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, false, false, false, false, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||

@@ -45,10 +45,13 @@ size_t assign_tc_aug_bytes(i64 B, int K);
 // zeros, and the kernel streams that copy (rows whose pitch is a multiple of 128 bytes stream faster).
 // Dx (0 = D): columns of a row of X when X is a copy padded with zeros to a multiple of 8 columns
 // (needs cpad).  aug_ready then also means that cpad holds the copy.
+// knn_k (0 = arg-min, else 8 or 32): k-nearest-neighbour search, B = 1; out_idx / out_dist are then [N][2][knn_k]
+// scratch, one list of the knn_k smallest distances per row and 128-column half of the tiles, each sorted by
+// (distance, column), unused places -1 / +inf; launch_knn_merge merges the two.
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s,
-                     int Dx = 0, cake_bf16* cpad = nullptr);
+                     int Dx = 0, cake_bf16* cpad = nullptr, int knn_k = 0);
 int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
                        int* out_idx, float* out_dist, cudaStream_t s);
 // D that is not a multiple of 8 (rows are then no multiple of 16 bytes, which TMA needs): the automatic
@@ -112,6 +115,10 @@ cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf1
 // ---- inertia: acc[b] += sum_i dist[b][i] (fp64 atomics); acc stride given in elements
 cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc_stride,
                            cudaStream_t s);
+
+// ---- k nearest neighbours: out[row][0..k) = the k smallest of the two sorted lists half[row][0..2)[0..kl), k <= kl
+cudaError_t launch_knn_merge(const int* half_idx, const float* half_dist, i64 N, int kl, int k, int* out_idx,
+                             float* out_dist, cudaStream_t s);
 
 // ---- bounded-wait self test
 cudaError_t launch_bounded_wait_selftest(int* status, int limit_ms, cudaStream_t s);
