@@ -164,6 +164,41 @@ def knn(Q: np.ndarray, X: np.ndarray, k: int):
     return idx, dist
 
 
+def kmeanspp_step(mind: np.ndarray, u_k: float):
+    """One draw of the seeding below: the first row whose running sum of `mind` exceeds u_k * sum(mind)
+    (a uniform row if every entry is zero).  Returns (row, running sums)."""
+    N = mind.shape[0]
+    cum = np.cumsum(mind)
+    total = cum[-1]
+    if not total > 0.0:
+        return min(int(u_k * N), N - 1), cum
+    return min(int(np.searchsorted(cum, u_k * total, side="right")), N - 1), cum
+
+
+def kmeanspp(X: np.ndarray, K: int, u: np.ndarray) -> np.ndarray:
+    """k-means++ seeding (D^2 sampling) with the random numbers passed in: u [K] uniforms in [0, 1).
+
+    Row 0 of the result is floor(u[0] * N); for k >= 1, with mind[i] the squared distance (direct differences,
+    fp64) from x_i to the nearest of the k rows chosen so far, row k is the first i whose running sum
+    mind[0] + ... + mind[i] exceeds u[k] * sum(mind).  The paper's K-means workload starts from sampled rows and
+    names no seeding; this is the textbook procedure, offered as an initialiser.  Returns the K row numbers.
+    """
+    X = _bits(X, "X")
+    N = X.shape[0]
+    u = np.asarray(u, dtype=np.float64)
+    if K < 1 or u.shape != (K,) or N < 1:
+        raise ValueError("need K >= 1 uniforms and N >= 1 rows")
+    Xf = bf16_to_f64(X)
+    rows = [min(int(u[0] * N), N - 1)]
+    mind = np.full(N, np.inf)
+    for k in range(1, K):
+        diff = Xf - Xf[rows[-1]]
+        mind = np.minimum(mind, (diff * diff).sum(1))
+        r, _ = kmeanspp_step(mind, float(u[k]))
+        rows.append(r)
+    return np.asarray(rows, dtype=np.int64)
+
+
 @dataclass
 class LloydResult:
     C: np.ndarray          # [K,D] f64, means of the last update (unrounded)

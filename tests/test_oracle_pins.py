@@ -364,3 +364,38 @@ def test_knn_integer_ties_go_to_the_lower_row_and_k1_is_assign():
     # a point that is in the database finds itself first, at distance 0
     i2, d2 = orc.knn(inputs.to_bits(X[:50]), inputs.to_bits(X), 3)
     assert np.array_equal(i2[:, 0], np.arange(50)) and (d2[:, 0] == 0).all()
+
+
+# ------------------------------------------------------------------------------------ k-means++ seeding
+
+def test_kmeanspp_hand_example_and_brute_force():
+    # points 0, 1, 10 on a line: first row floor(0.1 * 3) = 0; then mind = (0, 1, 100), running sums (0, 1, 101):
+    # u = 0.5 -> target 50.5 -> row 2; then mind = (0, 1, 0), sums (0, 1, 1): u = 0.999 -> target 0.999 -> row 1
+    X = torch.tensor([[0.0], [1.0], [10.0]]).to(torch.bfloat16)
+    assert orc.kmeanspp(inputs.to_bits(X), 3, np.array([0.1, 0.5, 0.999])).tolist() == [0, 2, 1]
+    # u just below 1/101 still lands on row 1 (sum 1 > target), row 0 has no mass and can never be drawn again
+    assert orc.kmeanspp(inputs.to_bits(X), 2, np.array([0.1, 0.009])).tolist() == [0, 1]
+    # brute force with python floats and exact fractions of the bf16 values
+    g = torch.Generator().manual_seed(5)
+    Xr = torch.randint(-3, 4, (40, 3), generator=g).to(torch.bfloat16)
+    u = np.random.default_rng(1).random(8)
+    rows = orc.kmeanspp(inputs.to_bits(Xr), 8, u)
+    pts = [[Fraction(float(v)) for v in row] for row in Xr.tolist()]
+    want = [int(u[0] * 40)]
+    for k in range(1, 8):
+        mind = [min(sum((a - b) ** 2 for a, b in zip(p, pts[r])) for r in want) for p in pts]
+        total, run, pick = sum(mind), Fraction(0), None
+        for i, m in enumerate(mind):
+            run += m
+            if run > Fraction(u[k]) * total:
+                pick = i
+                break
+        want.append(pick)
+    assert rows.tolist() == want
+    assert len(set(rows.tolist())) == 8                       # a chosen row has mind = 0: never drawn twice
+
+
+def test_kmeanspp_degenerate_inputs():
+    X = torch.ones(5, 4).to(torch.bfloat16)                    # all points coincide: draws fall back to uniform rows
+    assert orc.kmeanspp(inputs.to_bits(X), 3, np.array([0.0, 0.5, 0.99])).tolist() == [0, 2, 4]
+    assert orc.kmeanspp(inputs.to_bits(X[:1]), 1, np.array([0.7])).tolist() == [0]
