@@ -207,6 +207,34 @@ CAKE_API int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, 
                               void* ws, size_t ws_bytes, cake_stream_t stream, unsigned flags);
 
 /*
+ * lloyd with a convergence test (the paper fixes iteration counts and has no stopping rule; this is a reading of
+ * this library).  Iterations run in blocks of `check_every`; after each block the host reads the block's inertia
+ * values (one stream synchronisation per block) and stops once some iteration t >= 1 of the run had
+ * inertia[t-1] - inertia[t] <= tol * inertia[t-1].  At most max_iters iterations; *out_iters (host) receives the
+ * number run, a multiple of check_every unless max_iters cut the last block.  One problem (no batch).
+ * out_C_bf16, out_inertia ([max_iters]) and out_iters are required; the other outputs as for cake_kmeans_lloyd
+ * with iters = *out_iters.  Returns after the last block's synchronisation.
+ */
+CAKE_API int cake_kmeans_lloyd_tol(const cake_bf16* X, const cake_bf16* C0, long long N, int D, int K, int max_iters,
+                      double tol, int check_every, float* out_C, cake_bf16* out_C_bf16, int* out_idx,
+                      float* out_dist, int* out_counts, double* out_inertia, int* out_iters, void* ws,
+                      size_t ws_bytes, cake_stream_t stream, unsigned flags);
+
+/*
+ * k-means++ seeding (the paper's workload starts from sampled rows and names no seeding; this is the textbook
+ * D^2 sampling, offered as an initialiser).  The random numbers are the caller's:
+ *   u        [K] fp32 uniforms in [0,1), device, in
+ *   out_C0   [K][D] bf16, out: row 0 is X[floor(u[0] N)]; row k >= 1 is X[i] for the first i whose running sum
+ *            mind[0] + ... + mind[i] exceeds u[k] * sum(mind), mind[i] being the squared distance from x_i to
+ *            the nearest of the k rows chosen so far (a uniform row if that sum is zero)
+ *   out_rows [K] int32, out, may be NULL: the chosen row numbers
+ * Distances come from the assign kernel (fp32), the sums are fp64.  Asynchronous on `stream`, no host
+ * synchronisation; 3 to 4 kernel launches per centroid.  `ws` as for the other calls (same size).
+ */
+CAKE_API int cake_kmeans_init_plusplus(const cake_bf16* X, long long N, int D, int K, const float* u,
+                      cake_bf16* out_C0, int* out_rows, void* ws, size_t ws_bytes, cake_stream_t stream);
+
+/*
  * lloyd with HOST buffers (same operation; measures the end-to-end cost a caller with data in
  * host memory sees).  X_host, C0_host and every out_*_host pointer are HOST pointers (pinned
  * memory makes the copies asynchronous); `dev` is device scratch of at least

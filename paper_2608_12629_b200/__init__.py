@@ -7,7 +7,7 @@ from .binding import (  # noqa: F401
     CAKE_ERR_DEVICE, CAKE_ERR_NULL, CAKE_ERR_SHAPE, CAKE_ERR_TIMEOUT, CAKE_ERR_UNSUPPORTED, CAKE_ERR_WORKSPACE,
     CAKE_OK, CAKE_UPDATE_AUTO, CAKE_UPDATE_SLAB, CAKE_UPDATE_SLAB_F1,
     CAKE_UPDATE_SLAB_F2, CAKE_UPDATE_SLAB_F4, CAKE_UPDATE_SMEM, CAKE_UPDATE_SORT, EXPORTS, LIB_PATH, CakeError, LloydOutput,
-    alloc_lloyd_outputs, alloc_workspace, cake_kmeans_assign, cake_kmeans_assign_static, cake_kmeans_assign_static_status, cake_kmeans_device_status, cake_kmeans_inertia, cake_kmeans_lloyd,
+    alloc_lloyd_outputs, alloc_workspace, cake_kmeans_assign, cake_kmeans_assign_static, cake_kmeans_assign_static_status, cake_kmeans_device_status, cake_kmeans_inertia, cake_kmeans_lloyd, cake_kmeans_lloyd_tol, cake_kmeans_init_plusplus,
     cake_kmeans_lloyd_host, cake_kmeans_kernel_launches, cake_kmeans_lloyd_host_device_bytes, cake_kmeans_selftest_bounded_wait,
     cake_kmeans_update, cake_kmeans_update_finish, cake_kmeans_update_partial, cake_kmeans_workspace_bytes, cake_knn_search, cake_knn_workspace_bytes, cake_version, lib,
     strerror,

@@ -30,6 +30,7 @@ EXPORTS = [
     "cake_kmeans_device_status", "cake_kmeans_selftest_bounded_wait", "cake_kmeans_assign_static",
     "cake_kmeans_update_partial_batched", "cake_kmeans_update_finish_batched", "cake_kmeans_inertia_batched",
     "cake_kmeans_assign_static_status", "cake_knn_workspace_bytes", "cake_knn_search",
+    "cake_kmeans_lloyd_tol", "cake_kmeans_init_plusplus",
 ]
 
 _lib = None
@@ -68,6 +69,9 @@ def lib() -> ctypes.CDLL:
         L.cake_kmeans_assign_static_status.argtypes = [vp, ctypes.POINTER(i)]
         L.cake_knn_workspace_bytes.argtypes = [ll, ll, i, i, ctypes.POINTER(sz)]
         L.cake_knn_search.argtypes = [vp, vp, ll, ll, i, i, vp, vp, vp, sz, vp]
+        L.cake_kmeans_lloyd_tol.argtypes = [vp, vp, ll, i, i, i, ctypes.c_double, i, vp, vp, vp, vp, vp, vp,
+                                            ctypes.POINTER(i), vp, sz, vp, u]
+        L.cake_kmeans_init_plusplus.argtypes = [vp, ll, i, i, vp, vp, vp, vp, sz, vp]
         L.cake_kmeans_update_partial_batched.argtypes = [vp, vp, ll, ll, i, i, vp, vp, vp, sz, vp, u]
         L.cake_kmeans_update_finish_batched.argtypes = [vp, vp, vp, ll, i, i, vp, vp, vp]
         L.cake_kmeans_inertia_batched.argtypes = [vp, ll, ll, vp, i, vp]
@@ -370,3 +374,41 @@ def cake_knn_search(Q, X, k, out_idx=None, out_dist=None, ws=None, stream=None, 
                                    _stream(stream, Q.device))
     _check(rc, "cake_knn_search")
     return out_idx, out_dist
+
+
+def cake_kmeans_lloyd_tol(X, C0, max_iters, tol, check_every=1, ws=None, stream=None, flags=0):
+    """Lloyd iterations until the relative inertia decrease falls to `tol` (looked at every `check_every`
+    iterations) or max_iters; X bf16 [N,D], C0 bf16 [K,D].  Returns (LloydOutput with inertia[:iters], iters)."""
+    _want(X, torch.bfloat16, "X"), _want(C0, torch.bfloat16, "C0")
+    if X.dim() != 2 or C0.dim() != 2:
+        raise ValueError("one problem: X [N,D], C0 [K,D]")
+    B, N, D, K = _dims(X, C0)
+    out = alloc_lloyd_outputs(X, C0, max_iters)
+    if ws is None:
+        ws = alloc_workspace(1, N, D, K, X.device)
+    n = ctypes.c_int(0)
+    with torch.cuda.device(X.device):
+        rc = lib().cake_kmeans_lloyd_tol(_ptr(X), _ptr(C0), N, D, K, max_iters, float(tol), check_every, _ptr(out.C),
+                                         _ptr(out.C_bf16), _ptr(out.idx), _ptr(out.dist), _ptr(out.counts),
+                                         _ptr(out.inertia), ctypes.byref(n), _ptr(ws), ws.numel(),
+                                         _stream(stream, X.device), flags)
+    _check(rc, "cake_kmeans_lloyd_tol")
+    out.inertia = out.inertia[: n.value]
+    return out, int(n.value)
+
+
+def cake_kmeans_init_plusplus(X, K, u, ws=None, stream=None):
+    """k-means++ seeding: X bf16 [N,D], u fp32 [K] uniforms in [0,1) on the device -> (C0 bf16 [K,D], rows int32 [K])."""
+    _want(X, torch.bfloat16, "X"), _want(u, torch.float32, "u")
+    if X.dim() != 2 or u.shape != (K,):
+        raise ValueError("X must be [N,D] and u [K]")
+    N, D = X.shape
+    C0 = torch.empty(K, D, dtype=torch.bfloat16, device=X.device)
+    rows = torch.empty(K, dtype=torch.int32, device=X.device)
+    if ws is None:
+        ws = alloc_workspace(1, N, D, K, X.device)
+    with torch.cuda.device(X.device):
+        rc = lib().cake_kmeans_init_plusplus(_ptr(X), N, D, K, _ptr(u), _ptr(C0), _ptr(rows), _ptr(ws), ws.numel(),
+                                             _stream(stream, X.device))
+    _check(rc, "cake_kmeans_init_plusplus")
+    return C0, rows

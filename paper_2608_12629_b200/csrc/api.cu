@@ -24,6 +24,8 @@ struct Workspace {
     float* dist;          // [B][N]
     cake_bf16* xpad;      // [B][N][padded_d(D)] zero-padded copy of X for the tensor-core assign when D % 8 != 0
     cake_bf16* cpad;      // [B][K][round_up(D, 64)] zero-padded copy of C it streams when D % 64 != 0
+    cake_bf16* ccont;     // [B][K][D] centroids a Lloyd run continues from (convergence test between blocks of iterations)
+    double* pp_part;      // [kPlusPlusMaxSlabs] slab sums of the k-means++ seeding
     size_t bytes;
 };
 
@@ -49,6 +51,8 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     const size_t dpad = assign_pad_supports(D) ? static_cast<size_t>(padded_d(D)) : 0;
     w.xpad = reinterpret_cast<cake_bf16*>(take(static_cast<size_t>(B) * N * dpad * 2));
     w.cpad = reinterpret_cast<cake_bf16*>(take(static_cast<size_t>(B) * K * assign_cpad_columns(D) * 2));
+    w.ccont = reinterpret_cast<cake_bf16*>(take(kd * 2));
+    w.pp_part = reinterpret_cast<double*>(take(static_cast<size_t>(kPlusPlusMaxSlabs) * 8));
     w.bytes = o;
     return w;
 }
@@ -352,6 +356,89 @@ int cake_kmeans_lloyd(const cake_bf16* X, const cake_bf16* C0, long long N, int 
                       double* out_inertia, void* ws, size_t ws_bytes, cake_stream_t stream, unsigned flags) {
     return cake_kmeans_lloyd_batched(X, C0, 1, N, D, K, iters, out_C, out_C_bf16, out_idx, out_dist,
                                      out_counts, out_inertia, ws, ws_bytes, stream, flags);
+}
+
+int cake_kmeans_lloyd_tol(const cake_bf16* X, const cake_bf16* C0, long long N, int D, int K, int max_iters, double tol,
+                          int check_every, float* out_C, cake_bf16* out_C_bf16, int* out_idx, float* out_dist,
+                          int* out_counts, double* out_inertia, int* out_iters, void* ws, size_t ws_bytes,
+                          cake_stream_t stream, unsigned flags) {
+    int rc = check_shape(1, N, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (max_iters < 1 || check_every < 1 || !(tol >= 0.0)) return CAKE_ERR_SHAPE;
+    if (!out_C_bf16 || !out_inertia || !out_iters) return CAKE_ERR_NULL;
+    Workspace w;
+    rc = check_ws(ws, ws_bytes, 1, N, D, K, &w);
+    if (rc != CAKE_OK) return rc;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t kd = static_cast<size_t>(K) * D;
+    const cake_bf16* cur = C0;
+    int done = 0;
+    double prev = 0.0;
+    bool have_prev = false;
+    while (done < max_iters) {
+        const int block = max_iters - done < check_every ? max_iters - done : check_every;
+        rc = cake_kmeans_lloyd_batched(X, cur, 1, N, D, K, block, out_C, out_C_bf16, out_idx, out_dist, out_counts,
+                                       out_inertia + done, ws, ws_bytes, stream, flags);
+        if (rc != CAKE_OK) return rc;
+        // the host looks at the block's inertia values: the one synchronisation per block
+        double host[64];
+        bool stop = false;
+        for (int o = 0; o < block && !stop; o += 64) {
+            const int n = block - o < 64 ? block - o : 64;
+            if (cudaMemcpyAsync(host, out_inertia + done + o, static_cast<size_t>(n) * 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+                cudaStreamSynchronize(s) != cudaSuccess)
+                return CAKE_ERR_CUDA;
+            for (int j = 0; j < n; ++j) {
+                if (have_prev && prev - host[j] <= tol * prev) stop = true;   // looked at only at the block's end
+                prev = host[j];
+                have_prev = true;
+            }
+        }
+        done += block;
+        if (stop) break;
+        if (done < max_iters) {
+            if (cudaMemcpyAsync(w.ccont, out_C_bf16, kd * 2, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return CAKE_ERR_CUDA;
+            cur = w.ccont;
+        }
+    }
+    *out_iters = done;
+    return CAKE_OK;
+}
+
+int cake_kmeans_init_plusplus(const cake_bf16* X, long long N, int D, int K, const float* u, cake_bf16* out_C0,
+                              int* out_rows, void* ws, size_t ws_bytes, cake_stream_t stream) {
+    int rc = check_shape(1, N, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (N < 1) return CAKE_ERR_SHAPE;
+    if (!X || !u || !out_C0 || !ws) return CAKE_ERR_NULL;
+    if (misaligned(X, 16) || misaligned(out_C0, 16) || misaligned(u, 4) || misaligned(out_rows, 4)) return CAKE_ERR_ALIGN;
+    Workspace w;
+    rc = check_ws(ws, ws_bytes, 1, N, D, K, &w);
+    if (rc != CAKE_OK) return rc;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // scratch: the (row, cluster) pairs of the sort route hold an index per row (unused result of the one-centroid
+    // assign) and the running minimum; `dist` the distances to the row chosen last
+    int* idx_scr = reinterpret_cast<int*>(w.pairs);
+    float* mind = reinterpret_cast<float*>(w.pairs) + N;
+    if (launch_pp_pick(X, mind, w.pp_part, N, D, u, 0, out_C0, out_rows, s) != cudaSuccess) return CAKE_ERR_CUDA;
+    bool x_padded = false;
+    // the centroid of a one-centroid assign must start on a 16-byte boundary: rows of D % 8 != 0 columns go through
+    // the continuation buffer
+    const bool via_copy = (static_cast<size_t>(D) * 2) % 16 != 0;
+    for (int k = 1; k < K; ++k) {
+        const cake_bf16* c = out_C0 + static_cast<size_t>(k - 1) * D;
+        if (via_copy) {
+            if (cudaMemcpyAsync(w.ccont, c, static_cast<size_t>(D) * 2, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return CAKE_ERR_CUDA;
+            c = w.ccont;
+        }
+        rc = do_assign(X, c, 1, N, D, 1, idx_scr, w.dist, nullptr, 0, false, false, &x_padded, w, s,
+                       assign_tc_supports(D) ? CAKE_ASSIGN_TCGEN05_EXACT : CAKE_ASSIGN_AUTO);
+        if (rc != CAKE_OK) return rc;
+        if (launch_pp_accumulate(w.dist, mind, N, k == 1, w.pp_part, s) != cudaSuccess) return CAKE_ERR_CUDA;
+        if (launch_pp_pick(X, mind, w.pp_part, N, D, u, k, out_C0 + static_cast<size_t>(k) * D, out_rows, s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
+    }
+    return CAKE_OK;
 }
 
 namespace {

@@ -120,6 +120,15 @@ cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc
 cudaError_t launch_knn_merge(const int* half_idx, const float* half_dist, i64 N, int kl, int k, int* out_idx,
                              float* out_dist, cudaStream_t s);
 
+// ---- k-means++ seeding: running minimum of the distances and its slab sums; the draw itself
+constexpr int kPlusPlusMaxSlabs = 1024;
+// mind = first ? dist : min(mind, dist); part[slab] = sum of the slab's mind (fp64); part holds kPlusPlusMaxSlabs doubles
+cudaError_t launch_pp_accumulate(const float* dist, float* mind, i64 N, bool first, double* part, cudaStream_t s);
+// row k of the seeding: floor(u[0] N) for k = 0, else the first row whose running sum of mind exceeds u[k] * sum(mind)
+// (a uniform row if the sum is zero); copies X[row] to out_row and records the row in rows_out[k] (nullable)
+cudaError_t launch_pp_pick(const cake_bf16* X, const float* mind, const double* part, i64 N, int D, const float* u, int k,
+                           cake_bf16* out_row, int* rows_out, cudaStream_t s);
+
 // ---- bounded-wait self test
 cudaError_t launch_bounded_wait_selftest(int* status, int limit_ms, cudaStream_t s);
 
