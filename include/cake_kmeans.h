@@ -186,6 +186,26 @@ CAKE_API int cake_kmeans_update_finish_batched(const float* sums, const int* cou
                                cake_stream_t stream);
 
 /*
+ * lloyd over rows that are spread over several devices, one process per device: this call runs one rank's share.
+ * Every rank holds N_local rows and all K centroids.  Per iteration: assign and the per-cluster sums and counts of
+ * the local rows (this library's kernels), then `allreduce` -- called on the host, once per iteration, after that
+ * work has been enqueued -- must enqueue on `stream` an in-place sum over all ranks of sums[n_sums] (fp32) and
+ * counts[n_counts] (int32), both device pointers (an NCCL all-reduce, or anything ordered after the work already on
+ * the stream); then every rank divides, so all ranks hold the same centroids without a broadcast.  It returns 0, or
+ * non-zero to abort (the call then returns CAKE_ERR_CUDA).  allreduce = NULL: a single rank.
+ *   out_idx, out_dist: the local rows' last assignment; out_C, out_C_bf16, out_counts: global (same on all ranks);
+ *   out_inertia [iters]: the LOCAL rows' sums of distances (the caller adds them up over the ranks at the end).
+ * iters >= 1.  The exchange is K (D + 1) numbers per iteration whatever N is, which is why it is a collective
+ * between two launches and not a fused kernel: there is no tile-by-tile transfer to overlap with the math.
+ */
+typedef int (*cake_allreduce_fn)(void* user, float* sums, long long n_sums, int* counts, long long n_counts,
+                                 cake_stream_t stream);
+CAKE_API int cake_kmeans_lloyd_sharded(const cake_bf16* X_local, const cake_bf16* C0, long long N_local, int D, int K,
+                      int iters, float* out_C, cake_bf16* out_C_bf16, int* out_idx, float* out_dist,
+                      int* out_counts, double* out_inertia, cake_allreduce_fn allreduce, void* user, void* ws,
+                      size_t ws_bytes, cake_stream_t stream, unsigned flags);
+
+/*
  * lloyd (same paragraph: a Lloyd iteration is assign followed by centroid_update).
  * For t = 0 .. iters-1: assign against C_t (C_0 = C0), out_inertia[t] = sum_i out_dist_t[i],
  * then update -> C_{t+1}; the next assign reads C_{t+1} rounded to bf16.  Exactly `iters`

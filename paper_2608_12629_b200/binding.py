@@ -30,8 +30,12 @@ EXPORTS = [
     "cake_kmeans_device_status", "cake_kmeans_selftest_bounded_wait", "cake_kmeans_assign_static",
     "cake_kmeans_update_partial_batched", "cake_kmeans_update_finish_batched", "cake_kmeans_inertia_batched",
     "cake_kmeans_assign_static_status", "cake_knn_workspace_bytes", "cake_knn_search",
-    "cake_kmeans_lloyd_tol", "cake_kmeans_init_plusplus",
+    "cake_kmeans_lloyd_tol", "cake_kmeans_init_plusplus", "cake_kmeans_lloyd_sharded",
 ]
+
+# int (*)(void* user, float* sums, long long n_sums, int* counts, long long n_counts, cake_stream_t stream)
+ALLREDUCE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p,
+                                ctypes.c_longlong, ctypes.c_void_p)
 
 _lib = None
 
@@ -72,6 +76,7 @@ def lib() -> ctypes.CDLL:
         L.cake_kmeans_lloyd_tol.argtypes = [vp, vp, ll, i, i, i, ctypes.c_double, i, vp, vp, vp, vp, vp, vp,
                                             ctypes.POINTER(i), vp, sz, vp, u]
         L.cake_kmeans_init_plusplus.argtypes = [vp, ll, i, i, vp, vp, vp, vp, sz, vp]
+        L.cake_kmeans_lloyd_sharded.argtypes = [vp, vp, ll, i, i, i, vp, vp, vp, vp, vp, vp, ALLREDUCE_FN, vp, vp, sz, vp, u]
         L.cake_kmeans_update_partial_batched.argtypes = [vp, vp, ll, ll, i, i, vp, vp, vp, sz, vp, u]
         L.cake_kmeans_update_finish_batched.argtypes = [vp, vp, vp, ll, i, i, vp, vp, vp]
         L.cake_kmeans_inertia_batched.argtypes = [vp, ll, ll, vp, i, vp]
@@ -412,3 +417,32 @@ def cake_kmeans_init_plusplus(X, K, u, ws=None, stream=None):
                                              _stream(stream, X.device))
     _check(rc, "cake_kmeans_init_plusplus")
     return C0, rows
+
+
+def cake_kmeans_lloyd_sharded_call(X_local, C0, iters, out: LloydOutput, ws, reduce=None, stream=None, flags=0):
+    """One rank's share of a row-sharded Lloyd run through the C entry point.  `reduce(sums, counts)` (or None for a
+    single rank) is called once per iteration with the fp32 [K,D] sums and int32 [K] counts as tensors that alias the
+    library's buffers and must add them up over all ranks in place, in stream order.  out.inertia holds the LOCAL sums."""
+    _want(X_local, torch.bfloat16, "X_local"), _want(C0, torch.bfloat16, "C0")
+    N, D = X_local.shape
+    K = C0.shape[0]
+    base = ws.data_ptr()
+
+    def thunk(user, sums_ptr, n_sums, counts_ptr, n_counts, stream_ptr):
+        try:
+            off = sums_ptr - base
+            sums = ws[off:off + 4 * n_sums].view(torch.float32).view(K, D)
+            reduce(sums, out.counts)
+            return 0
+        except Exception:          # an exception must not cross the C frames
+            import traceback
+            traceback.print_exc()
+            return 1
+
+    cb = ALLREDUCE_FN(thunk) if reduce is not None else ctypes.cast(None, ALLREDUCE_FN)
+    with torch.cuda.device(X_local.device):
+        rc = lib().cake_kmeans_lloyd_sharded(_ptr(X_local), _ptr(C0), N, D, K, iters, _ptr(out.C), _ptr(out.C_bf16),
+                                             _ptr(out.idx), _ptr(out.dist), _ptr(out.counts), _ptr(out.inertia), cb, None,
+                                             _ptr(ws), ws.numel(), _stream(stream, X_local.device), flags)
+    _check(rc, "cake_kmeans_lloyd_sharded")
+    return out

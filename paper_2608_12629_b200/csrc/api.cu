@@ -240,6 +240,26 @@ int cake_kmeans_update(const cake_bf16* X, const int* idx, long long N, int D, i
                                       ws_bytes, stream, flags);
 }
 
+namespace {
+// sums and counts of the rows given (no division): the slab route while its runs are long enough (the measured
+// threshold of the one-call update; with rows spread over ranks the runs get shorter), else the sort route
+int do_update_partial(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, float* out_sums, int* out_counts,
+                      const Workspace& w, cudaStream_t s, unsigned flags) {
+    unsigned path = flags & CAKE_UPDATE_MASK;
+    if (path == CAKE_UPDATE_AUTO)
+        path = (update_slab_supports(D, K) && update_slab_preferred(B, N, D, K)) ? CAKE_UPDATE_SLAB : CAKE_UPDATE_SORT;
+    if (path == CAKE_UPDATE_SLAB)
+        return launch_update_slab(X, idx, B, N, D, K, out_sums, out_counts, w.status, 0, s);
+    if (path == CAKE_UPDATE_SORT) {
+        UpdateScratch scr{out_sums, w.nvalid, w.cursor, w.pairs, w.part, w.done, w.rank};
+        bool divided = false;
+        int rc = launch_update_sort(X, idx, B, N, D, K, scr, out_counts, nullptr, nullptr, nullptr, &divided, w.status, s);
+        return (rc == CAKE_OK && divided) ? CAKE_ERR_UNSUPPORTED : rc;
+    }
+    return CAKE_ERR_UNSUPPORTED;
+}
+}  // namespace
+
 int cake_kmeans_update_partial_batched(const cake_bf16* X, const int* idx, long long B, long long N, int D,
                                        int K, float* out_sums, int* out_counts, void* ws, size_t ws_bytes,
                                        cake_stream_t stream, unsigned flags) {
@@ -251,19 +271,52 @@ int cake_kmeans_update_partial_batched(const cake_bf16* X, const int* idx, long 
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;
+    return do_update_partial(X, idx, static_cast<int>(B), N, D, K, out_sums, out_counts, w,
+                             reinterpret_cast<cudaStream_t>(stream), flags);
+}
+
+int cake_kmeans_lloyd_sharded(const cake_bf16* X_local, const cake_bf16* C0, long long N_local, int D, int K, int iters,
+                              float* out_C, cake_bf16* out_C_bf16, int* out_idx, float* out_dist, int* out_counts,
+                              double* out_inertia, cake_allreduce_fn allreduce, void* user, void* ws, size_t ws_bytes,
+                              cake_stream_t stream, unsigned flags) {
+    int rc = check_shape(1, N_local, D, K);
+    if (rc != CAKE_OK) return rc;
+    if (iters < 1) return CAKE_ERR_SHAPE;
+    if (!C0 || !out_C || !out_counts || !ws || (N_local > 0 && (!X_local || !out_idx))) return CAKE_ERR_NULL;
+    if (misaligned(X_local, 16) || misaligned(C0, 16) || misaligned(out_C, 16) || misaligned(out_C_bf16, 16) ||
+        misaligned(out_idx, 4) || misaligned(out_dist, 4) || misaligned(out_counts, 4) || misaligned(out_inertia, 8))
+        return CAKE_ERR_ALIGN;
+    Workspace w;
+    rc = check_ws(ws, ws_bytes, 1, N_local, D, K, &w);
+    if (rc != CAKE_OK) return rc;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    const int Bi = static_cast<int>(B);
-    unsigned path = flags & CAKE_UPDATE_MASK;
-    if (path == CAKE_UPDATE_AUTO) path = update_slab_supports(D, K) ? CAKE_UPDATE_SLAB : CAKE_UPDATE_SORT;
-    if (path == CAKE_UPDATE_SLAB)
-        return launch_update_slab(X, idx, Bi, N, D, K, out_sums, out_counts, w.status, 0, s);
-    if (path == CAKE_UPDATE_SORT) {
-        UpdateScratch scr{out_sums, w.nvalid, w.cursor, w.pairs, w.part, w.done, w.rank};
-        bool divided = false;
-        rc = launch_update_sort(X, idx, Bi, N, D, K, scr, out_counts, nullptr, nullptr, nullptr, &divided, w.status, s);
-        return (rc == CAKE_OK && divided) ? CAKE_ERR_UNSUPPORTED : rc;
+    const i64 N = N_local;
+    const unsigned apath = flags & CAKE_ASSIGN_MASK;
+    const bool tc_assign = N > 0 && ((assign_tc_supports(D) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
+                                                                apath == CAKE_ASSIGN_TCGEN05_EXACT)) ||
+                                     (assign_pad_supports(D) && apath == CAKE_ASSIGN_AUTO));
+    const int cpad_columns = assign_cpad_columns(D);
+    const cake_bf16* cur = C0;
+    int nxt = 0;
+    bool prepared = false, x_padded = false;
+    for (int t = 0; t < iters; ++t) {
+        rc = do_assign(X_local, cur, 1, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr, iters, true,
+                       prepared, &x_padded, w, s, flags);
+        if (rc != CAKE_OK) return rc;
+        // this rank's sums and counts (rows of D columns: the padded copy of X is not used here)
+        rc = do_update_partial(X_local, out_idx, 1, N, D, K, w.sums, out_counts, w, s, flags);
+        if (rc != CAKE_OK) return rc;
+        // the one exchange of the iteration: the caller adds up sums and counts of all ranks, in place, in stream order
+        if (allreduce && allreduce(user, w.sums, static_cast<long long>(K) * D, out_counts, K, stream) != 0) return CAKE_ERR_CUDA;
+        cake_bf16* dst = (t == iters - 1 && out_C_bf16) ? out_C_bf16 : w.cbuf[nxt];
+        NextAssign next{w.caug, out_inertia ? out_inertia + t + 1 : nullptr, iters, cpad_columns ? w.cpad : nullptr, cpad_columns};
+        const bool want = tc_assign && t + 1 < iters;
+        if (launch_finalize(w.sums, out_counts, cur, 1, K, D, out_C, dst, false, want ? &next : nullptr, &prepared, s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
+        cur = dst;
+        nxt ^= 1;
     }
-    return CAKE_ERR_UNSUPPORTED;
+    return CAKE_OK;
 }
 
 int cake_kmeans_update_finish_batched(const float* sums, const int* counts, const cake_bf16* C_prev, long long B,

@@ -1,11 +1,10 @@
 """Lloyd iterations over rows of X that are spread over the ranks of a torch.distributed group.
 
 One process per GPU.  Every rank holds a contiguous share of the rows and all K centroids.  Per iteration
-each rank assigns its rows and adds them up per cluster with this library's kernels
-(cake_kmeans_assign, cake_kmeans_update_partial), the sums, counts and inertia are all-reduced over the
-group (NCCL on GPUs; the only exchange step of the method: K*D + K + 1 numbers per iteration, whatever
-N is), and every rank divides (cake_kmeans_update_finish), so all ranks hold the same centroids
-without a broadcast.  The paper describes the single-device iteration (Section 5, "Flash-KMeans clean-start
+each rank assigns its rows and adds them up per cluster with this library's kernels, the sums and counts are
+all-reduced over the group (NCCL on GPUs; the only exchange step of the method: K*D + K numbers per
+iteration, whatever N is), and every rank divides, so all ranks hold the same centroids without a
+broadcast; the inertia is all-reduced once at the end.  The paper describes the single-device iteration (Section 5, "Flash-KMeans clean-start
 workload"); fp32 sums of different ranks are added in the order the all-reduce chooses.
 
 Nothing here computes on tensors by itself: calls of the library and collectives only.
@@ -35,6 +34,8 @@ def cake_kmeans_lloyd_sharded(X_local: torch.Tensor, C0: torch.Tensor, iters: in
 
     Returns this rank's idx / dist (for its own rows) and the global C, counts and inertia.  Without an
     initialised process group (or with a group of one rank) it is the single-device iteration.
+    The loop itself runs inside the library (cake_kmeans_lloyd_sharded of the C ABI); this function supplies the
+    exchange: one all-reduce of the sums and one of the counts per iteration, and one of the inertia at the end.
     """
     if X_local.dim() != 2 or C0.dim() != 2 or X_local.shape[1] != C0.shape[1]:
         raise ValueError("X_local must be [N_local, D] and C0 [K, D]")
@@ -48,20 +49,12 @@ def cake_kmeans_lloyd_sharded(X_local: torch.Tensor, C0: torch.Tensor, iters: in
         ws = binding.alloc_workspace(1, N, D, K, dev)
     if out is None:
         out = binding.alloc_lloyd_outputs(X_local, C0, iters)
-    sums = torch.empty(K, D, dtype=torch.float32, device=dev)
-    cbuf = [torch.empty_like(C0), torch.empty_like(C0)]
-    cur = C0
-    for t in range(iters):
-        binding.cake_kmeans_assign(X_local, cur, out_idx=out.idx, out_dist=out.dist, ws=ws, flags=flags & 0xF)
-        binding.cake_kmeans_inertia(out.dist, out_inertia=out.inertia[t:])
-        binding.cake_kmeans_update_partial(X_local, out.idx, K, out_sums=sums, out_counts=out.counts, ws=ws,
-                                           flags=flags & 0xF0)
-        if exchange:
-            dist.all_reduce(sums, group=group)
-            dist.all_reduce(out.counts, group=group)
-        dst = out.C_bf16 if t == iters - 1 else cbuf[t & 1]
-        binding.cake_kmeans_update_finish(sums, out.counts, C_prev=cur, out_C=out.C, out_C_bf16=dst)
-        cur = dst
+
+    def reduce(sums, counts):
+        dist.all_reduce(sums, group=group)
+        dist.all_reduce(counts, group=group)
+
+    binding.cake_kmeans_lloyd_sharded_call(X_local, C0, iters, out, ws, reduce if exchange else None, flags=flags)
     if exchange:
         dist.all_reduce(out.inertia, group=group)
     return out

@@ -121,3 +121,54 @@ def test_lloyd_sharded_two_ranks_equal_the_single_device_iteration():
         assert np.array_equal(Cb, inputs.to_bits(ref.C_bf16)) and np.array_equal(C, ref.C.cpu().numpy())
         assert np.array_equal(counts, ref.counts.cpu().numpy()) and np.array_equal(idx, ref.idx.cpu().numpy()[a:b])
         np.testing.assert_allclose(inertia, ref.inertia.cpu().numpy(), rtol=1e-12)
+
+
+def _rank_real(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    torch.cuda.set_device(0)
+    X, _ = inputs.gaussian_mixture(20001, 64, 40, 2.0, 0.7, 77)
+    C0 = inputs.sample_init(X, 150, 77)
+    a, b = cake.shard_rows(X.shape[0], rank, world)
+    one = cake.cake_kmeans_lloyd_sharded(X[a:b].clone().to(DEV), C0.to(DEV), 1)
+    three = cake.cake_kmeans_lloyd_sharded(X[a:b].clone().to(DEV), C0.to(DEV), 3)
+    torch.cuda.synchronize()
+    q.put((rank, one.idx.cpu().numpy(), one.dist.cpu().numpy(), one.C.cpu().numpy(), inputs.to_bits(one.C_bf16),
+           one.counts.cpu().numpy(), one.inertia.cpu().numpy(), three.inertia.cpu().numpy()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_lloyd_sharded_two_ranks_graded_by_the_oracle():
+    """Real-valued data, two ranks: the first iteration is graded against the oracle as any single-device iteration is
+    (each rank's assignment of its rows; the update from the indices of both ranks together), three iterations against
+    the oracle's own rounded trajectory on the inertia."""
+    from oracle import kmeans_oracle as orc
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 35500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_rank_real, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = dict()
+    for _ in range(2):
+        r = q.get(timeout=300)
+        got[r[0]] = r[1:]
+    for p in procs:
+        p.join(120)
+        assert p.exitcode == 0
+    X, _ = inputs.gaussian_mixture(20001, 64, 40, 2.0, 0.7, 77)
+    C0 = inputs.sample_init(X, 150, 77)
+    Xb, Cb = inputs.to_bits(X), inputs.to_bits(C0)
+    idx_all = np.empty(X.shape[0], dtype=np.int32)
+    for rank in range(2):
+        a, b = cake.shard_rows(X.shape[0], rank, 2)
+        idx, dist_, C, Cbits, counts, inertia1, inertia3 = got[rank]
+        grading.grade_assign(Xb[a:b], Cb, idx, dist_)
+        idx_all[a:b] = idx
+    for rank in range(2):
+        idx, dist_, C, Cbits, counts, inertia1, inertia3 = got[rank]
+        grading.grade_update(Xb, idx_all, 150, Cb, C, Cbits, counts)        # the same global result on both ranks
+        ref = orc.lloyd(Xb, Cb, 3, round_centroids=True)
+        np.testing.assert_allclose(inertia3, ref.inertia, rtol=grading.INERTIA_TOL)
+        np.testing.assert_allclose(inertia1, ref.inertia[:1], rtol=grading.INERTIA_TOL)

@@ -1,7 +1,7 @@
 """Host-side logic of the row-sharded Lloyd driver, on CPU: the partition of the rows, and the driver run as two
-gloo ranks with the library calls replaced by stand-ins built on the oracle (what is checked here is the
-orchestration: what is all-reduced and when, the ping-pong of the centroid buffers, the empty-cluster rule when
-a cluster is empty on one rank only; the kernels themselves are checked on the GPU)."""
+gloo ranks with the library's per-rank call replaced by a stand-in built on the oracle (what is checked here is the
+exchange the driver supplies: what is all-reduced and when, and the empty-cluster rule when a cluster is empty on
+one rank only; the library's loop and kernels are checked on the GPU)."""
 import os
 import sys
 import types
@@ -58,9 +58,26 @@ def _oracle_binding():
         out_C_bf16.copy_(inputs.from_bits(orc.f64_to_bf16(C)))
         return out_C, out_C_bf16
 
+    def sharded_call(X, C0, iters, out, ws, reduce=None, stream=None, flags=0):
+        """What the C entry point does, stated with the stand-ins above: per iteration assign, the local inertia, the
+        local sums and counts, the caller's exchange, the division."""
+        K, D = C0.shape
+        sums = torch.empty(K, D, dtype=torch.float32)
+        cur = C0
+        for t in range(iters):
+            assign(X, cur, out.idx, out.dist)
+            inertia(out.dist, out.inertia[t:])
+            partial(X, out.idx, K, sums, out.counts)
+            if reduce is not None:
+                reduce(sums, out.counts)
+            nxt = torch.empty_like(C0)
+            finish(sums, out.counts, cur, out.C, nxt)
+            cur = nxt
+        out.C_bf16.copy_(cur)
+        return out
+
     return types.SimpleNamespace(alloc_workspace=lambda B, N, D, K, dev: torch.empty(1), alloc_lloyd_outputs=real.alloc_lloyd_outputs,
-                                 cake_kmeans_assign=assign, cake_kmeans_inertia=inertia, cake_kmeans_update_partial=partial,
-                                 cake_kmeans_update_finish=finish)
+                                 cake_kmeans_lloyd_sharded_call=sharded_call)
 
 
 def _problem():
