@@ -79,7 +79,11 @@ enum {
     CAKE_UPDATE_SLAB_F1 = 4 << 4, /* the same with the cluster size forced to 1, 2 or 4 CTAs      */
     CAKE_UPDATE_SLAB_F2 = 5 << 4,
     CAKE_UPDATE_SLAB_F4 = 6 << 4,
-    CAKE_UPDATE_MASK = 0xF << 4
+    CAKE_UPDATE_MASK = 0xF << 4,
+    CAKE_LLOYD_NO_FUSE = 1 << 8 /* lloyd: keep assign and update as two passes over X also where one problem of
+                                   K <= 128, D <= 128 (D % 8 == 0) would take the single-pass iteration, in which
+                                   the assign kernel adds each row tile to per-cluster sums on the tensor core
+                                   (sums += onehot^T X) while the tile is in shared memory                      */
 };
 
 /* Library version (major*10000 + minor*100 + patch).  No paper counterpart. */

@@ -26,6 +26,8 @@ struct Workspace {
     cake_bf16* cpad;      // [B][K][round_up(D, 64)] zero-padded copy of C it streams when D % 64 != 0
     cake_bf16* ccont;     // [B][K][D] centroids a Lloyd run continues from (convergence test between blocks of iterations)
     double* pp_part;      // [kPlusPlusMaxSlabs] slab sums of the k-means++ seeding
+    float* fpart;         // fused update (one problem, K <= 128, D <= 128): partial sums [kFuseMaxCtas][128][round_up(D, 16)]
+    int* fcnt;            // ... and partial counts [kFuseMaxCtas][128]
     size_t bytes;
 };
 
@@ -53,6 +55,12 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     w.cpad = reinterpret_cast<cake_bf16*>(take(static_cast<size_t>(B) * K * assign_cpad_columns(D) * 2));
     w.ccont = reinterpret_cast<cake_bf16*>(take(kd * 2));
     w.pp_part = reinterpret_cast<double*>(take(static_cast<size_t>(kPlusPlusMaxSlabs) * 8));
+    // (one partial per CTA of the assign kernel: at most one CTA per row tile and per SM)
+    const bool fuse = fuse_shape_ok(B, D, K);
+    const i64 row_tiles = (N + 127) / 128;
+    const size_t fctas = fuse ? static_cast<size_t>(row_tiles < kFuseMaxCtas ? row_tiles : kFuseMaxCtas) : 0;
+    w.fpart = reinterpret_cast<float*>(take(fctas * 128 * round_up(D, 16) * 4));
+    w.fcnt = reinterpret_cast<int*>(take(fctas * 128 * 4));
     w.bytes = o;
     return w;
 }
@@ -78,9 +86,12 @@ int check_ws(void* ws, size_t ws_bytes, i64 B, i64 N, int D, int K, Workspace* o
 // zero_inertia: the entries still have to be cleared (the tensor-core prologue does it on the way).
 // aug_ready: the update ahead prepared this assign (see NextAssign): the tensor-core route skips its prologue
 // x_padded (in/out): the workspace already holds the padded copy of this X (an earlier step of the call made it)
+// fuse_ctas (nullable): ask the tensor-core kernel to add the rows to per-cluster partial sums as well (fused update,
+// see launch_assign_tc); *fuse_ctas > 0 on return if it did
 int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, int* out_idx,
               float* out_dist, double* inertia, int inertia_stride, bool zero_inertia, bool aug_ready,
-              bool* x_padded, const Workspace& w, cudaStream_t s, unsigned flags) {
+              bool* x_padded, const Workspace& w, cudaStream_t s, unsigned flags, int* fuse_ctas = nullptr) {
+    if (fuse_ctas) *fuse_ctas = 0;
     unsigned path = flags & CAKE_ASSIGN_MASK;
     int Dx = 0;   // columns of the padded copy of X, if one is used
     if (path == CAKE_ASSIGN_AUTO && assign_pad_supports(D) && N > 0) {
@@ -109,9 +120,11 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
     // the packed epilogue (values compared with 17 significant bits) is the automatic choice; the exact
     // one compares full fp32 values and is slower
     const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT;
+    const bool fuse = fuse_ctas && !exact && fuse_shape_ok(B, D, K) && w.fpart && N > 0;
     return launch_assign_tc(X, C, B, N, D, K, w.caug, exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia,
                             aug_ready, w.status, s, Dx,
-                            assign_cpad_columns(D) ? w.cpad : nullptr);
+                            assign_cpad_columns(D) ? w.cpad : nullptr, 0, fuse ? w.fpart : nullptr, fuse ? w.fcnt : nullptr,
+                            fuse ? fuse_ctas : nullptr);
 }
 
 // next / prepared: see launch_finalize
@@ -388,16 +401,28 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     int nxt = 0;
     bool prepared = false;
     bool x_padded = false;   // the workspace holds the padded copy of X (D % 8 != 0), made by the first step that needs it
+    // One problem of at most 128 clusters and 128 features: a single pass over X per iteration.  The assign kernel adds
+    // the rows of every tile to per-cluster partial sums while the tile is in shared memory, and one small kernel adds
+    // the partials up and divides (two launches per iteration instead of four).
+    const bool try_fuse = tc_assign && !(flags & CAKE_LLOYD_NO_FUSE) && (flags & CAKE_UPDATE_MASK) == CAKE_UPDATE_AUTO &&
+                          apath != CAKE_ASSIGN_TCGEN05_EXACT && fuse_shape_ok(B, D, K);
     for (int t = 0; t < iters; ++t) {
+        int fuse_ctas = 0;
         rc = do_assign(X, cur, Bi, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr, iters,
-                       true, prepared, &x_padded, w, s, flags);
+                       true, prepared, &x_padded, w, s, flags, try_fuse ? &fuse_ctas : nullptr);
         if (rc != CAKE_OK) return rc;
         cake_bf16* dst = (t == iters - 1 && out_C_bf16) ? out_C_bf16 : w.cbuf[nxt];
         NextAssign next{w.caug, out_inertia ? out_inertia + t + 1 : nullptr, iters,
                         cpad_columns ? w.cpad : nullptr, cpad_columns};
         const bool want = tc_assign && t + 1 < iters;
-        rc = do_update(X, out_idx, Bi, N, D, K, cur, out_C, dst, out_counts, w, s, flags, &x_padded, want ? &next : nullptr, &prepared);
-        if (rc != CAKE_OK) return rc;
+        if (fuse_ctas > 0) {
+            if (launch_finalize_partials(w.fpart, w.fcnt, fuse_ctas, cur, K, D, out_C, dst, out_counts, want ? &next : nullptr,
+                                         &prepared, s) != cudaSuccess)
+                return CAKE_ERR_CUDA;
+        } else {
+            rc = do_update(X, out_idx, Bi, N, D, K, cur, out_C, dst, out_counts, w, s, flags, &x_padded, want ? &next : nullptr, &prepared);
+            if (rc != CAKE_OK) return rc;
+        }
         cur = dst;
         nxt ^= 1;
     }

@@ -80,8 +80,10 @@ constexpr uint32_t AUG_B_BYTES = kAssignAugTileBytes;    // 4 KiB
 // a ring stage: one or two centroid chunks plus room for the tile's half-norm block, which rides with the
 // last chunk (Params::cps, Params::stage_bytes)
 constexpr uint32_t AUG_ZERO_BYTES = BLOCK_N * 16;        // 4 KiB of zeros
+constexpr uint32_t OH_BYTES = 128 * 128 * 2;             // FUSE: the one-hot operand, 128 clusters x 128 rows of a tile, bf16
 constexpr int MAX_STAGES = 6;
-constexpr int MAX_XBUF = 4;
+constexpr int MAX_XBUF = 6;                              // (more than four only in the fused mode)
+constexpr int MAX_XBUF_PLAIN = 4;
 constexpr int MAX_XCHUNKS = 8;                           // 64-column chunks of an X tile (D <= 512)
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t CTRL_BYTES = 6144;  // barriers, TMEM pointer, abort flag, merge scratch, row margins
@@ -90,36 +92,42 @@ constexpr uint32_t WAIT_SLICE_NS = 20000;   // longest single sleep inside a wai
 constexpr uint32_t COL_MASK = 0x7Fu;   // packed policy: 7 bits address the 128 columns of a half tile
 constexpr uint32_t F32_INF = 0x7f800000u;
 
-// (The two flags sit in what would be padding: a larger Params measurably slowed the many-tile kernel down,
-// 3-6 %, whatever the order of the members.)
+// Kept as small as it gets (112 bytes; with the two tensor maps 368 bytes of kernel parameters): a larger parameter
+// block measurably slows the many-tile kernel down although not one instruction of it reads the extra members -- 24 more
+// bytes cost 5-10 % (D = 64, K = 16,384: 1.22 -> 1.34 ms; D = 128, K = 4,096: 0.87 -> 0.94 ms), whatever their position.
+// Hence the narrow integer types.
 struct Params {
-    int B;
-    int alt_epi;      // one centroid tile per row tile: the two epilogue warpgroups take whole row tiles in turn;
-                      // the value is the number of accumulator columns in use (32..128, or 256)
     i64 N;
-    int D, K;
-    int nchunks;      // ceil(D / 64)
-    int ksteps_last;  // UMMA k-steps in the last chunk
-    int m_tiles;      // ceil(N / 128)
-    int n_tiles;      // ceil(K / 256)
-    i64 total_tiles;  // B * m_tiles
-    int n_stages;     // ring depth (stages)
-    int cps;          // centroid chunks per ring stage: 2 when nchunks is even (half the barrier traffic), else 1
-    uint32_t stage_bytes;   // cps * 32 KiB + 4 KiB; resident centroids: bytes of one chunk of the tile (rows * 128),
-                            // the tile's chunks lie one behind the other, its 4 KiB half-norm block after them
-    int n_xbuf;       // X buffers (1..4)
+    i64 total_tiles;      // B * m_tiles
     const uint8_t* caug;  // [B][n_tiles][4 KiB] centroid-side operand of the extra k-step
     int* out_idx;
     float* out_dist;
     double* inertia;      // optional: inertia[b * inertia_stride] += sum of the problem's distances
-    int inertia_stride;
-    int knn_k;        // TOPK instantiations (unused otherwise); out_idx / out_dist are then [N][2][TOPK]: one sorted list per
-                      // column half, merged by a small kernel afterwards
-    int res_c;        // 1: alt_epi and the centroid tile stays in shared memory (loaded once per problem): the two
-                      // issuers share no ring and each works on its own row tiles only; 2: two resident
-                      // tiles, issuer i computes tile i of every row tile (shared epilogue)
     int* status;
+    float* fuse_sums;     // FUSE: [gridDim.x][128][round_up(D, 16)] partial sums per CTA; fuse_counts [gridDim.x][128]
+    int* fuse_counts;
+    int B, K;
+    int m_tiles;          // ceil(N / 128)
+    int n_tiles;          // ceil(K / 256)
+    uint32_t stage_bytes; // cps * 32 KiB + 4 KiB; resident centroids: bytes of one chunk of the tile (rows * 128),
+                          // the tile's chunks lie one behind the other, its 4 KiB half-norm block after them
+    int inertia_stride;
+    uint16_t D;
+    uint16_t alt_epi;     // one centroid tile per row tile: the two epilogue warpgroups take whole row tiles in turn;
+                          // the value is the number of accumulator columns in use (32..128, or 256)
+    uint8_t nchunks;      // ceil(D / 64)
+    uint8_t ksteps_last;  // UMMA k-steps in the last chunk
+    uint8_t n_stages;     // ring depth (stages)
+    uint8_t cps;          // centroid chunks per ring stage: 2 when nchunks is even (half the barrier traffic), else 1
+    uint8_t n_xbuf;       // X buffers (1..6)
+    uint8_t res_c;        // 1: alt_epi and the centroid tile stays in shared memory (loaded once per problem): the two
+                          // issuers share no ring and each works on its own row tiles only; 2: two resident
+                          // tiles, issuer i computes tile i of every row tile (shared epilogue)
+    uint8_t knn_k;        // TOPK instantiations (unused otherwise); out_idx / out_dist are then [N][2][TOPK]: one sorted
+                          // list per column half, merged by a small kernel afterwards
+    uint8_t fuse_oh2;     // FUSE: 1 = one one-hot buffer per epilogue warpgroup (else both share one)
 };
+static_assert(sizeof(Params) == 112, "kernel parameter block grew");
 
 struct Ctrl {  // lives in shared memory
     uint64_t x_full[MAX_XBUF], x_empty[MAX_XBUF];
@@ -133,6 +141,9 @@ struct Ctrl {  // lives in shared memory
     uint64_t tmem_empty[2][MAX_ISSUERS];
     uint64_t auga_full[MAX_XBUF];
     uint64_t merge_full[2], merge_empty[2];
+    // FUSE: the one-hot operand of row tile t is written (by the epilogue warpgroup t % 2) / has been read by the MMAs
+    // that add tile t to the sums (barrier t % 2); upd_done: the last such MMAs have completed
+    uint64_t oh_full[2], oh_empty[2], upd_done[2];   // (upd_done[0] only)
     uint64_t turn[MAX_ISSUERS];   // resident-centroid mode: issuer i may issue its next tile's MMAs (the other one has issued its own)
     uint32_t tmem_base;
     int abort_flag;
@@ -301,7 +312,10 @@ __device__ __forceinline__ int tile_step() { return CONSEC ? 1 : static_cast<int
 // choice: with both epilogues in one kernel every shape measured 3-8 % slower)
 // TOPK (0, 8 or 32): instead of the arg-min each epilogue thread keeps the TOPK smallest accumulators of its row and
 // column half (k-nearest-neighbour search: the "centroids" are the database rows); many-tile structure, packed gate.
-template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false, bool BULK = false, int TOPK = 0>
+// FUSE (resident mode with at most 128 centroids and D <= 128, one problem): the kernel also adds every row tile to
+// per-cluster sums while the tile is still in shared memory -- on the tensor core, as sums += onehot^T X with the
+// assignment written as a one-hot bf16 operand -- so that the centroid update needs no second pass over X.
+template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false, bool BULK = false, int TOPK = 0, bool FUSE = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
                  const Params p) {
@@ -317,8 +331,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     const uint32_t ring_base = smem_base + ring_off;
     // bytes of one resident centroid tile (chunks, then its half-norm block)
     const uint32_t res_tile_bytes = static_cast<uint32_t>(p.nchunks) * p.stage_bytes + AUG_B_BYTES;
+    // FUSE: the one-hot operand sits behind the resident tile (a multiple of 4 KiB: 1024-byte aligned as the swizzle needs)
+    const uint32_t oh_off = ring_off + res_tile_bytes;
     const uint32_t auga_off = ring_off + ((XLOAD && p.res_c) ? static_cast<uint32_t>(p.res_c) * res_tile_bytes
-                                                             : static_cast<uint32_t>(p.n_stages) * p.stage_bytes);
+                                                             : static_cast<uint32_t>(p.n_stages) * p.stage_bytes) +
+                              (FUSE ? OH_BYTES * (p.fuse_oh2 ? 2u : 1u) : 0u);
     const uint32_t zero_off = auga_off + static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES;
     const uint32_t ctrl_off = zero_off + AUG_ZERO_BYTES;
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + ctrl_off);
@@ -347,6 +364,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             ptx::mbar_init(ptx::smem_u32(&ctrl->merge_empty[i]), 4);
         }
         for (int i = 0; i < MAX_ISSUERS; ++i) ptx::mbar_init(ptx::smem_u32(&ctrl->turn[i]), 1);
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&ctrl->oh_full[i]), NUM_EPI_WARPS / 2);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->oh_empty[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->upd_done[i]), 1);
+        }
         for (int i = 0; i < MAX_STAGES; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->ring_empty[i]), NUM_ISSUERS);   // the consuming issuer and those passing over
@@ -360,6 +382,19 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // columns 8..15 of both operands of the extra k-step: one block of zeros for the whole kernel
     for (uint32_t o = threadIdx.x * 16; o < AUG_ZERO_BYTES; o += NUM_THREADS * 16)
         *reinterpret_cast<uint4*>(smem + zero_off + o) = make_uint4(0, 0, 0, 0);
+    // FUSE: the one-hot operand starts as zeros and is kept up to date element by element (a thread clears the one it
+    // set for its row in an earlier tile: fuse_last) ; fuse_cnt counts the rows of every cluster
+    int* fuse_last = reinterpret_cast<int*>(ctrl->merge_best[0]);    // [2][128]: per one-hot buffer
+    int* fuse_cnt = ctrl->merge_idx[0];
+    if (FUSE) {
+        for (uint32_t o = threadIdx.x * 16; o < OH_BYTES * (p.fuse_oh2 ? 2u : 1u); o += NUM_THREADS * 16)
+            *reinterpret_cast<uint4*>(smem + oh_off + o) = make_uint4(0, 0, 0, 0);
+        if (threadIdx.x < BLOCK_M) {
+            fuse_last[threadIdx.x] = -1;
+            fuse_last[BLOCK_M + threadIdx.x] = -1;
+            fuse_cnt[threadIdx.x] = 0;
+        }
+    }
     ptx::fence_proxy_async_smem();
     if (warp == MMA_WARP) {
         ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), TMEM_COLS);
@@ -380,7 +415,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // The epilogue keeps a whole 128-column accumulator slice in registers; the other roles need few.
     // Registers move between warpgroups accordingly (warps 0-7 grow, warps 8-15 shrink).
     if (warp >= NUM_EPI_WARPS) {
-    ptx::setmaxnreg_dec<AUX_REGS>();
+    // (FUSE: the issuing threads carry the update's descriptors as well: eight registers more for them, eight fewer
+    // for the epilogue warps; the sum stays the same)
+    ptx::setmaxnreg_dec<FUSE ? AUX_REGS + 8 : AUX_REGS>();
     if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -444,6 +481,40 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     while (!ptx::mbar_try_wait(ptx::smem_u32(&ctrl->ring_full[0]), (pc - 1u) & 1u) &&
                            ptx::globaltimer_ns() - t0 < 100000000ull) {
                     }
+                }
+                if (FUSE && ok) {
+                    // The centroids are in (one problem): this thread now issues the MMAs of the update, tile by tile:
+                    // sums (128 clusters on the TMEM lanes x D, columns 128..) += onehot^T X once the tile's epilogue has
+                    // written the one-hot operand.  A = one-hot, K-major (the rows of the tile are the contraction);
+                    // B = the X tile as it lies in its buffer, read MN-major: 64-column atoms X_CHUNK_BYTES apart, 8-row
+                    // groups 1024 B apart.  The two MMA issuers of the assign spend all their time on their own
+                    // instruction streams; eight more MMAs per tile there halved the kernel's speed.
+                    constexpr uint32_t KSTEP = (UMMA_K * 2) >> 4;
+                    const uint32_t idesc_upd = ptx::umma_idesc_bf16(BLOCK_M, (p.D + 15) & ~15) | ptx::UMMA_IDESC_B_MN_MAJOR;
+                    const uint32_t d_sums = tmem_base + BLOCK_N / 2;
+                    const uint32_t nxb = static_cast<uint32_t>(p.n_xbuf);
+                    uint32_t t_it = 0;
+                    for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++t_it) {
+                        const uint32_t g = t_it & 1u;
+                        ok = wait_bar(&ctrl->oh_full[g], (t_it >> 1) & 1u, ctrl, p.status);
+                        if (!ok) break;
+                        ptx::tc_fence_after();
+                        const uint32_t uxb = t_it % nxb;
+                        const uint32_t a0 = ptx::umma_desc_lo_sw128(smem_base + oh_off + (p.fuse_oh2 ? g * OH_BYTES : 0u));
+                        const uint32_t b0 = (((x_base + uxb * xbuf_bytes) & 0x3FFFFu) >> 4) | ((X_CHUNK_BYTES >> 4) << 16);
+#pragma unroll
+                        for (uint32_t ks = 0; ks < BLOCK_M / UMMA_K; ++ks) {
+                            const uint32_t a_lo = a0 + (ks >> 2) * (X_CHUNK_BYTES >> 4) + (ks & 3u) * KSTEP;
+                            const uint32_t b_lo = b0 + ks * ((UMMA_K * 128u) >> 4);
+                            if (ks == 0 && t_it == 0)
+                                ptx::umma_bf16_lohi<false>(d_sums, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo, ptx::UMMA_DESC_HI_SW128, idesc_upd);
+                            else
+                                ptx::umma_bf16_lohi<true>(d_sums, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo, ptx::UMMA_DESC_HI_SW128, idesc_upd);
+                        }
+                        ptx::umma_commit(ptx::smem_u32(&ctrl->oh_empty[g]));
+                        ptx::umma_commit(ptx::smem_u32(&ctrl->x_empty[uxb]));
+                    }
+                    if (ok) ptx::umma_commit(ptx::smem_u32(&ctrl->upd_done[0]));
                 }
             } else {
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
@@ -639,7 +710,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                                                                     smem_base + zero_off),
                                               ptx::UMMA_DESC_HI_AUG, idesc_aug_n);
                     ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[iss]));
-                    ptx::umma_commit(ptx::smem_u32(&ctrl->x_empty[rxb]));
+                    // (FUSE: the X buffer is also an operand of the update, whose MMAs come after these: the thread that
+                    // issues those hands the buffer back)
+                    if (!FUSE) ptx::umma_commit(ptx::smem_u32(&ctrl->x_empty[rxb]));
                 }
             } else
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
@@ -803,7 +876,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        ptx::setmaxnreg_inc<EPI_REGS>();
+        ptx::setmaxnreg_inc<FUSE ? EPI_REGS - 8 : EPI_REGS>();
         const int wg = warp >> 2;            // column half of every tile
         const int q = warp & 3;              // TMEM lane quarter this warp may read
         const int r = q * 32 + lane;         // row inside the X tile
@@ -871,7 +944,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             ptx::tc_fence_after();
             float best = __uint_as_float(F32_INF);
             int bsel = 0;
-            if (p.alt_epi <= BLOCK_N / 2) {
+            if (FUSE || p.alt_epi <= BLOCK_N / 2) {   // (FUSE: at most 128 centroids by construction)
                 // at most 128 centroids: only the 32-column groups that hold some were written
                 const int ng = p.alt_epi >> 5;
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + as * BLOCK_N;
@@ -978,6 +1051,49 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 p.out_idx[o] = bidx;
                 if (p.out_dist) p.out_dist[o] = dist;
                 dsum += static_cast<double>(dist);
+            }
+            if (FUSE) {
+                // The one-hot operand of this tile: element [cluster][row] of a 128 x 128 bf16 tile, K-major with the
+                // 128-byte swizzle, two 64-row chunks.  The buffer is shared by both warpgroups (they alternate tiles):
+                // the MMAs that read the previous tile's operand must have completed.
+                // (one buffer per warpgroup: the MMAs on this warpgroup's previous tile)
+                if (p.fuse_oh2 ? tile_it > 1u : tile_it > 0u) {
+                    const uint32_t pt = p.fuse_oh2 ? tile_it - 2u : tile_it - 1u;
+                    ok = wait_bar(&ctrl->oh_empty[pt & 1u], (pt >> 1) & 1u, ctrl, p.status);
+                    if (!ok) break;
+                }
+                const uint32_t ohb = p.fuse_oh2 ? static_cast<uint32_t>(wg) : 0u;
+                uint8_t* oh = smem + oh_off + ohb * OH_BYTES + (r >> 6) * X_CHUNK_BYTES + ((r & 7) << 1);
+                const int g8 = (r & 63) >> 3;          // 16-byte granule of the row inside its chunk
+                int* last = fuse_last + ohb * BLOCK_M;
+                const int prev = last[r];
+                if (prev >= 0) *reinterpret_cast<uint16_t*>(oh + prev * 128 + ((g8 ^ (prev & 7)) << 4)) = 0;
+                int now = -1;
+                if (row < p.N) {
+                    now = bidx;
+                    *reinterpret_cast<uint16_t*>(oh + now * 128 + ((g8 ^ (now & 7)) << 4)) = 0x3F80;
+                    atomicAdd(fuse_cnt + now, 1);
+                }
+                last[r] = now;
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->oh_full[wg]));
+            }
+        }
+        if (FUSE && ok && wg == 0) {
+            // every tile has been added: the sums (clusters on the TMEM lanes, D columns) go out as this CTA's partial
+            ok = wait_bar(&ctrl->upd_done[0], 0u, ctrl, p.status);
+            if (ok) {
+                ptx::tc_fence_after();
+                const int ncol = (p.D + 15) & ~15;
+                float* dst = p.fuse_sums + (static_cast<size_t>(blockIdx.x) * BLOCK_M + r) * ncol;
+                for (int c0 = 0; c0 < ncol; c0 += 16) {
+                    uint32_t v[16];
+                    ptx::tmem_ld_x16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + BLOCK_N / 2 + c0, v);
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4)
+                        *reinterpret_cast<uint4*>(dst + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                }
             }
         }
         // ---- TOPK: the row's sorted list (registers) of the smallest accumulators seen so far in this column half;
@@ -1214,6 +1330,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     // ---------------------------------------------------------------- teardown
     ptx::tc_fence_before();
     __syncthreads();
+    if (FUSE && threadIdx.x < BLOCK_M) p.fuse_counts[static_cast<size_t>(blockIdx.x) * BLOCK_M + threadIdx.x] = fuse_cnt[threadIdx.x];
     if (warp == MMA_WARP) {
         __syncwarp();
         ptx::tc_fence_after();
@@ -1319,7 +1436,7 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s, int Dx,
-                     cake_bf16* cpad, int knn_k) {
+                     cake_bf16* cpad, int knn_k, float* fuse_sums, int* fuse_counts, int* fuse_ctas) {
     // D: columns of a row of C; Dk: columns of a row of X and length of the contraction (D, or D rounded up to
     // a multiple of 8 with zeros in the copy of X); Dc: columns of a row of the centroid operand the kernel
     // streams (C itself, or its zero-padded copy of a multiple of 64 columns, written by the prologue)
@@ -1342,6 +1459,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     p.out_idx = out_idx; p.out_dist = out_dist; p.status = status;
     p.inertia = inertia; p.inertia_stride = inertia_stride;
     p.knn_k = knn_k;
+    p.fuse_sums = fuse_sums;
+    p.fuse_counts = fuse_counts;
+    if (fuse_ctas) *fuse_ctas = 0;
     if ((knn_k != 0 && knn_k != 8 && knn_k != 32) || (knn_k > 0 && (B != 1 || !out_dist || inertia))) return CAKE_ERR_UNSUPPORTED;
     if (p.total_tiles == 0) return CAKE_OK;
 
@@ -1357,7 +1477,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     const i64 fixed = 1024 + CTRL_BYTES + AUG_ZERO_BYTES;
     const i64 budget = static_cast<i64>(di.smem_optin) - fixed;
     const i64 xbuf = static_cast<i64>(p.nchunks) * X_CHUNK_BYTES + AUG_A_BYTES;
-    int want_xbuf = p.n_tiles <= 2 ? MAX_XBUF : 2;
+    int want_xbuf = p.n_tiles <= 2 ? MAX_XBUF_PLAIN : 2;
     if ((p.nchunks >= 4 && p.n_tiles >= 8) || (p.nchunks == 3 && p.n_tiles >= 16)) want_xbuf = 1;   // measured
     // two chunks per ring stage when the chunk count is even (one wait and one commit per stage), unless the
     // ring would then hold a single stage, X is the bound (few centroid tiles: X buffers matter more) or the
@@ -1391,7 +1511,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         // (of the tile only the rows that hold centroids, in steps of 32, when there are at most 128)
         c_rows = K <= BLOCK_N / 2 ? static_cast<int>(round_up(K, 32)) : BLOCK_N;
         const i64 c_bytes = static_cast<i64>(p.nchunks) * c_rows * 128 + AUG_B_BYTES;
-        for (int nx = MAX_XBUF; nx >= 2; nx -= 2) {
+        for (int nx = MAX_XBUF_PLAIN; nx >= 2; nx -= 2) {
             if (p.nchunks <= MAX_STAGES && c_bytes + nx * xbuf <= budget) {
                 p.res_c = 1;
                 // its value: the accumulator columns the MMAs write and the epilogue reads (K <= 128: only
@@ -1418,7 +1538,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     if (p.n_tiles == 2 && xload) {
         // two centroid tiles: both stay in shared memory if at least two X buffers fit beside them (D <= 128)
         const i64 c_bytes = 2 * (static_cast<i64>(p.nchunks) * C_CHUNK_BYTES + AUG_B_BYTES);
-        for (int nx = MAX_XBUF; nx >= 2; --nx) {
+        for (int nx = MAX_XBUF_PLAIN; nx >= 2; --nx) {
             if (2 * p.nchunks <= MAX_STAGES && c_bytes + nx * xbuf <= budget) {
                 p.res_c = 2;
                 p.cps = 1;
@@ -1429,12 +1549,31 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             }
         }
     }
+    // fused update: the resident single-tile mode with at most 128 centroids, D <= 128, one problem, and room for the
+    // one-hot operand beside FOUR X buffers (an X buffer is held until its tile has been added to the sums, which is
+    // issued behind the MMAs of the issuer's next tile: with two buffers that would wait on itself)
+    // More X buffers than the plain kernel where they fit (a buffer is held longer), and one one-hot operand per
+    // epilogue warpgroup where two fit (with a shared one the updates of consecutive tiles wait for each other).
+    bool fuse = false;
+    p.fuse_oh2 = 0;
+    if (fuse_sums && fuse_counts && B == 1 && p.res_c == 1 && K <= BLOCK_N / 2 && Dk <= 128 && !exact && knn_k == 0 && p.n_xbuf == 4 &&
+        di.sm_count <= kFuseMaxCtas) {
+        const i64 c_bytes = static_cast<i64>(p.nchunks) * c_rows * 128 + AUG_B_BYTES;
+        for (int oh = 2; oh >= 1 && !fuse; --oh)
+            for (int nx = MAX_XBUF; nx >= 4 && !fuse; nx -= 2)
+                if (c_bytes + nx * xbuf + oh * static_cast<i64>(OH_BYTES) <= budget) {
+                    fuse = true;
+                    p.fuse_oh2 = oh == 2 ? 1 : 0;
+                    p.n_xbuf = nx;
+                }
+    }
     if (p.res_c != 1) c_rows = BLOCK_N;
     rc = make_tmap(&tc, cpad ? cpad : C, Dc, K, B, c_rows);
     if (rc != CAKE_OK) return rc;
     const size_t ring_bytes = p.res_c ? static_cast<size_t>(p.res_c) * (static_cast<size_t>(p.nchunks) * p.stage_bytes + AUG_B_BYTES)
                                       : static_cast<size_t>(p.n_stages) * p.stage_bytes;
-    const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf + ring_bytes;
+    const size_t smem_bytes = static_cast<size_t>(fixed) + static_cast<size_t>(p.n_xbuf) * xbuf + ring_bytes +
+                              (fuse ? OH_BYTES * (p.fuse_oh2 ? 2u : 1u) : 0u);
     using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const Params);
     const bool consec = xload && p.res_c && B > 1;
     // a single X buffer (D > 256) is filled and handed back chunk by chunk
@@ -1443,7 +1582,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     // D = 128 (two chunks) with many centroid tiles per row tile measured 3-6 % faster when the accumulator is handed
     // back before the reduction; every other shape gains from reducing while loading (D = 64 up to 8 %)
     const bool bulk = p.nchunks == 2 && p.n_tiles >= 8;
-    if (knn_k > 0)
+    if (fuse)
+        kernel = assign_tc_kernel<true, true, false, false, false, 0, true>;
+    else if (knn_k > 0)
         kernel = knn_k == 8 ? assign_tc_kernel<true, false, false, false, false, 8> : assign_tc_kernel<true, false, false, false, false, 32>;
     else if (!xload)
         kernel = exact ? (bulk ? assign_tc_kernel<false, false, false, false, true> : assign_tc_kernel<false, false>)
@@ -1462,6 +1603,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             cudaFuncSetAttribute(assign_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, true, false, false, false, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, false, false, false, false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, false, false, false, false, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
@@ -1511,6 +1653,7 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         return CAKE_ERR_CUDA;
     }
     note_launches(1);
+    if (fuse && fuse_ctas) *fuse_ctas = static_cast<int>(grid);
     return CAKE_OK;
 }
 

@@ -51,7 +51,17 @@ size_t assign_tc_aug_bytes(i64 B, int K);
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s,
-                     int Dx = 0, cake_bf16* cpad = nullptr, int knn_k = 0);
+                     int Dx = 0, cake_bf16* cpad = nullptr, int knn_k = 0, float* fuse_sums = nullptr,
+                     int* fuse_counts = nullptr, int* fuse_ctas = nullptr);
+// Fused update (fuse_sums / fuse_counts / fuse_ctas all given, one problem, K <= 128, D <= 128 and room in shared
+// memory): the assign kernel also adds the rows of every tile to per-cluster sums on the tensor core.  On return
+// *fuse_ctas = n > 0 says that it did: fuse_sums then holds n partial sums of [128][round_up(D, 16)] floats (one per
+// CTA) and fuse_counts n partial counts of [128]; launch_finalize_partials adds them up and divides.
+// *fuse_ctas = 0: the kernel ran without (the shape does not qualify) and the update has to be done separately.
+constexpr int kFuseMaxCtas = 160;
+constexpr int kFuseMaxK = 128, kFuseMaxD = 128;
+inline bool fuse_shape_ok(i64 B, int D, int K) { return B == 1 && K <= kFuseMaxK && D <= kFuseMaxD && D % 8 == 0; }
+
 int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K,
                        int* out_idx, float* out_dist, cudaStream_t s);
 // D that is not a multiple of 8 (rows are then no multiple of 16 bytes, which TMA needs): the automatic
@@ -111,6 +121,11 @@ struct NextAssign {
 cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf16* C_prev, int B,
                             int K, int D, float* out_C, cake_bf16* out_C_bf16, bool early,
                             const NextAssign* next, bool* prepared, cudaStream_t s, int sums_columns = 0);
+// The division of the fused update: partial sums / counts of launch_assign_tc's fused mode are added up, then as
+// launch_finalize (one problem; `next` as there; out_counts receives the total counts).
+cudaError_t launch_finalize_partials(const float* part_sums, const int* part_counts, int n_ctas, const cake_bf16* C_prev,
+                                     int K, int D, float* out_C, cake_bf16* out_C_bf16, int* out_counts,
+                                     const NextAssign* next, bool* prepared, cudaStream_t s);
 
 // ---- inertia: acc[b] += sum_i dist[b][i] (fp64 atomics); acc stride given in elements
 cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc_stride,

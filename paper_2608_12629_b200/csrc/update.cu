@@ -1180,6 +1180,77 @@ finalize_rows_kernel(const float4* __restrict__ sums, const int* __restrict__ co
     }
 }
 
+// Fused update, second half.  One CTA per centroid row k: the n_part partial rows [p][k][0..D) are added up (thread =
+// (partial stripe, column quad)), then the first warp divides, applies the keep-previous rule, writes the fp32 and
+// bf16 centroid and, if asked, the row of the next assign's half-norm operand, exactly as finalize_rows_kernel does.
+__global__ void __launch_bounds__(256)
+finalize_partials_kernel(const float* __restrict__ part_sums, const int* __restrict__ part_counts, int n_part, int n_cnt,
+                         int pitch, const uint2* __restrict__ C_prev, int K, int D4, float4* __restrict__ out_C,
+                         uint2* __restrict__ out_C_bf16, int* __restrict__ out_counts, uint8_t* __restrict__ caug, int Kpad,
+                         double* __restrict__ inertia, uint2* __restrict__ cpad, int Dc4) {
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
+    __shared__ float4 red[256];
+    __shared__ int cred[256];
+    const int k = blockIdx.x;
+    if (inertia && k == 0 && threadIdx.x == 0) inertia[0] = 0.0;
+    const int t = threadIdx.x;
+    const int stripes = 256 / D4;            // D4 <= 32: at least 8 stripes of partials
+    const int col = t % D4, stripe = t / D4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (stripe < stripes)
+        for (int p = stripe; p < n_part; p += stripes) {
+            const float4 v = *reinterpret_cast<const float4*>(part_sums + (static_cast<size_t>(p) * 128 + k) * pitch + col * 4);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+    int cnt = 0;
+    for (int p = t; p < n_cnt; p += 256) cnt += part_counts[static_cast<size_t>(p) * 128 + k];
+    red[t] = acc;
+    cred[t] = cnt;
+    __syncthreads();
+    for (int o = 128; o >= 32; o >>= 1) {
+        if (t < o) cred[t] += cred[t + o];
+        __syncthreads();
+    }
+    if (t >= 32) return;
+    int n = cred[t];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+    if (t == 0) out_counts[k] = n;
+    const float fn = static_cast<float>(n);
+    float nacc = 0.f;
+    if (cpad)
+        for (int j = D4 + t; j < Dc4; j += 32) cpad[static_cast<size_t>(k) * Dc4 + j] = make_uint2(0u, 0u);
+    if (t < D4) {
+        float4 sv = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sidx = 0; sidx < stripes; ++sidx) {
+            const float4 v = red[sidx * D4 + t];
+            sv.x += v.x; sv.y += v.y; sv.z += v.z; sv.w += v.w;
+        }
+        const size_t e = static_cast<size_t>(k) * D4 + t;
+        float4 v;
+        if (n > 0) {
+            v = make_float4(sv.x / fn, sv.y / fn, sv.z / fn, sv.w / fn);
+        } else if (C_prev) {
+            const uint2 pv = C_prev[e];
+            v = make_float4(bf16lo(pv.x), bf16hi(pv.x), bf16lo(pv.y), bf16hi(pv.y));
+        } else {
+            v = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        out_C[e] = v;
+        uint2 o;
+        o.x = static_cast<uint32_t>(f32_to_bf16_rne(v.x)) | (static_cast<uint32_t>(f32_to_bf16_rne(v.y)) << 16);
+        o.y = static_cast<uint32_t>(f32_to_bf16_rne(v.z)) | (static_cast<uint32_t>(f32_to_bf16_rne(v.w)) << 16);
+        if (out_C_bf16) out_C_bf16[e] = o;
+        if (cpad) cpad[static_cast<size_t>(k) * Dc4 + t] = o;
+        nacc = aug::add_squares(nacc, o.x, o.y);
+    }
+    if (caug) {
+        nacc = aug::fold_lanes(nacc);
+        if (t == 0) aug::write_row(caug, 0, k, K, Kpad, nacc);
+    }
+}
+
 }  // namespace
 
 // ======================================================================= host side
@@ -1599,6 +1670,25 @@ cudaError_t launch_finalize(const float* sums, const int* counts, const cake_bf1
     cfg.gridDim = dim3(static_cast<unsigned>(ctas));
     note_launches(1);
     return cudaLaunchKernelEx(&cfg, finalize_kernel, sums, counts, C_prev, total, D, Ds, out_C, out_C_bf16);
+}
+
+cudaError_t launch_finalize_partials(const float* part_sums, const int* part_counts, int n_ctas, const cake_bf16* C_prev,
+                                     int K, int D, float* out_C, cake_bf16* out_C_bf16, int* out_counts,
+                                     const NextAssign* next, bool* prepared, cudaStream_t s) {
+    if (prepared) *prepared = false;
+    const bool prep = next && out_C_bf16;
+    const int Kpad = padded_k(K);
+    // (the operand's padding rows K..Kpad-1 were written by the first iteration's prologue and never change)
+    cudaError_t e = launch_early(finalize_partials_kernel, dim3(static_cast<unsigned>(K)), dim3(256), 0, s, part_sums, part_counts,
+                                 n_ctas, n_ctas, (D + 15) & ~15, reinterpret_cast<const uint2*>(C_prev), K, D / 4,
+                                 reinterpret_cast<float4*>(out_C), reinterpret_cast<uint2*>(out_C_bf16), out_counts,
+                                 prep ? static_cast<uint8_t*>(next->caug) : static_cast<uint8_t*>(nullptr), Kpad,
+                                 prep ? next->inertia : static_cast<double*>(nullptr),
+                                 prep ? reinterpret_cast<uint2*>(next->cpad) : static_cast<uint2*>(nullptr),
+                                 prep ? next->cpad_columns / 4 : 0);
+    note_launches(1);
+    if (e == cudaSuccess && prep && prepared) *prepared = true;
+    return e;
 }
 
 }  // namespace cake

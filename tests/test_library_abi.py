@@ -42,8 +42,9 @@ def test_host_only_calls(library):
     assert "workspace" in cake.strerror(cake.CAKE_ERR_WORKSPACE)
     assert cake.strerror(12345).startswith("unknown")
     small = cake.cake_kmeans_workspace_bytes(1, 1000, 64, 16)
-    big = cake.cake_kmeans_workspace_bytes(4, 1000, 64, 16)
+    big = cake.cake_kmeans_workspace_bytes(1, 100000, 64, 16)
     assert 0 < small < big and small % 256 == 0
+    assert cake.cake_kmeans_workspace_bytes(4, 1000, 64, 16) < cake.cake_kmeans_workspace_bytes(8, 1000, 64, 16)
     assert cake.cake_kmeans_lloyd_host_device_bytes(1, 1000, 64, 16, 3) > small
     for bad in [(0, 10, 8, 2), (1, -1, 8, 2), (1, 10, 0, 2), (1, 10, 8, 0)]:
         with pytest.raises(cake.CakeError) as e:
