@@ -38,6 +38,8 @@ WORKLOADS = {
     "c3": Workload("c3", 32, 65536, 128, 256, 256, 1.0, 0.5, "dirichlet", 10, 1003),
     # large K: many sparse or empty clusters
     "c4": Workload("c4", 1, 2097152, 256, 65536, 16384, 1.0, 0.3, "uniform", 5, 1004),
+    # few clusters, one problem: the shape class of the single-pass (fused) iteration, X larger than L2
+    "f1": Workload("f1", 1, 2097152, 64, 64, 64, 1.0, 0.5, "uniform", 10, 1006),
     # the paper's own clean-start shape (assign only in the paper)
     "paper": Workload("paper", 32, 65536, 128, 1024, 1024, 1.0, 0.5, "uniform", 3, 1005),
 }
