@@ -68,6 +68,11 @@ enum {
                                   norms must stay below 2^120                                      */
     CAKE_ASSIGN_SIMT = 2,      /* plain CUDA-core fallback, any D                               */
     CAKE_ASSIGN_TCGEN05_EXACT = 3, /* same pipeline, all 24 bits compared and returned (slower epilogue) */
+    CAKE_ASSIGN_TCGEN05_PAIR = 4,  /* the arithmetic and results of CAKE_ASSIGN_TCGEN05 on pairs of CTAs
+                                      (tcgen05.mma.cta_group::2: two SMs share every 256 x 256 tile and each loads half
+                                      of the centroid tile).  Never chosen automatically: measured equal to the single-CTA
+                                      kernel at D = 128, K = 1024 and behind it elsewhere.  D % 8 == 0, D <= 512, K > 512. */
+    CAKE_ASSIGN_TCGEN05_PAIR_EXACT = 5, /* ... with the epilogue of CAKE_ASSIGN_TCGEN05_EXACT                        */
     CAKE_ASSIGN_MASK = 0xF,
     CAKE_UPDATE_AUTO = 0,
     CAKE_UPDATE_SMEM = 1 << 4, /* shared-memory partial sums; needs K*D*4 + K*4 bytes of smem   */

@@ -20,6 +20,7 @@ CAKE_OK = 0
 CAKE_ERR_NULL, CAKE_ERR_SHAPE, CAKE_ERR_ALIGN, CAKE_ERR_UNSUPPORTED = -1, -2, -3, -4
 CAKE_ERR_WORKSPACE, CAKE_ERR_CUDA, CAKE_ERR_BAD_INDEX, CAKE_ERR_TIMEOUT, CAKE_ERR_DEVICE = -5, -6, -7, -8, -9
 CAKE_ASSIGN_AUTO, CAKE_ASSIGN_TCGEN05, CAKE_ASSIGN_SIMT, CAKE_ASSIGN_TCGEN05_EXACT = 0, 1, 2, 3
+CAKE_ASSIGN_TCGEN05_PAIR, CAKE_ASSIGN_TCGEN05_PAIR_EXACT = 4, 5
 CAKE_UPDATE_AUTO, CAKE_UPDATE_SMEM, CAKE_UPDATE_SORT = 0, 1 << 4, 2 << 4
 CAKE_UPDATE_SLAB, CAKE_UPDATE_SLAB_F1, CAKE_UPDATE_SLAB_F2, CAKE_UPDATE_SLAB_F4 = 3 << 4, 4 << 4, 5 << 4, 6 << 4
 CAKE_LLOYD_NO_FUSE = 1 << 8

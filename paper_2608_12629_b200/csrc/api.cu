@@ -114,17 +114,18 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
             rc = CAKE_ERR_CUDA;
         return rc;
     }
-    if (path != CAKE_ASSIGN_TCGEN05 && path != CAKE_ASSIGN_TCGEN05_EXACT) return CAKE_ERR_UNSUPPORTED;
+    const bool pair = path == CAKE_ASSIGN_TCGEN05_PAIR || path == CAKE_ASSIGN_TCGEN05_PAIR_EXACT;
+    if (path != CAKE_ASSIGN_TCGEN05 && path != CAKE_ASSIGN_TCGEN05_EXACT && !pair) return CAKE_ERR_UNSUPPORTED;
     if (!assign_tc_supports(Dx ? Dx : D)) return CAKE_ERR_UNSUPPORTED;
     if (N == 0) return CAKE_OK;
     // the packed epilogue (values compared with 17 significant bits) is the automatic choice; the exact
     // one compares full fp32 values and is slower
-    const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT;
-    const bool fuse = fuse_ctas && !exact && fuse_shape_ok(B, D, K) && w.fpart && N > 0;
+    const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT || path == CAKE_ASSIGN_TCGEN05_PAIR_EXACT;
+    const bool fuse = fuse_ctas && !exact && fuse_shape_ok(B, D, K) && w.fpart && N > 0 && !pair;
     return launch_assign_tc(X, C, B, N, D, K, w.caug, exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia,
                             aug_ready, w.status, s, Dx,
                             assign_cpad_columns(D) ? w.cpad : nullptr, 0, fuse ? w.fpart : nullptr, fuse ? w.fcnt : nullptr,
-                            fuse ? fuse_ctas : nullptr);
+                            fuse ? fuse_ctas : nullptr, pair);
 }
 
 // next / prepared: see launch_finalize
@@ -306,7 +307,8 @@ int cake_kmeans_lloyd_sharded(const cake_bf16* X_local, const cake_bf16* C0, lon
     const i64 N = N_local;
     const unsigned apath = flags & CAKE_ASSIGN_MASK;
     const bool tc_assign = N > 0 && ((assign_tc_supports(D) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
-                                                                apath == CAKE_ASSIGN_TCGEN05_EXACT)) ||
+                                                                apath == CAKE_ASSIGN_TCGEN05_EXACT || apath == CAKE_ASSIGN_TCGEN05_PAIR ||
+                                                                apath == CAKE_ASSIGN_TCGEN05_PAIR_EXACT)) ||
                                      (assign_pad_supports(D) && apath == CAKE_ASSIGN_AUTO));
     const int cpad_columns = assign_cpad_columns(D);
     const cake_bf16* cur = C0;
@@ -394,7 +396,8 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     // otherwise compute in a prologue launch of its own.
     const unsigned apath = flags & CAKE_ASSIGN_MASK;
     const bool tc_assign = N > 0 && ((assign_tc_supports(D) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
-                                                                apath == CAKE_ASSIGN_TCGEN05_EXACT)) ||
+                                                                apath == CAKE_ASSIGN_TCGEN05_EXACT || apath == CAKE_ASSIGN_TCGEN05_PAIR ||
+                                                                apath == CAKE_ASSIGN_TCGEN05_PAIR_EXACT)) ||
                                      (assign_pad_supports(D) && apath == CAKE_ASSIGN_AUTO));
     const int cpad_columns = assign_cpad_columns(D);
     const cake_bf16* cur = C0;

@@ -1415,6 +1415,24 @@ int make_tmap(CUtensorMap* m, const void* base, int D, i64 rows, int batch, int 
 
 }  // namespace
 
+int make_tmap_bf16_rows(CUtensorMap* m, const void* base, int D, i64 rows, int batch, int box_rows) {
+    return make_tmap(m, base, D, rows, batch, box_rows);
+}
+
+// bytes viewed as rows of 16 (the half-norm operand: one 16-byte row per centroid); box = box_rows rows, no swizzle
+int make_tmap_rows16(CUtensorMap* m, const void* base, i64 rows, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return CAKE_ERR_CUDA;
+    cuuint64_t dims[2] = {16, static_cast<cuuint64_t>(rows)};
+    cuuint64_t strides[1] = {16};
+    cuuint32_t box[2] = {16, static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? CAKE_OK : CAKE_ERR_CUDA;
+}
+
 #ifdef CAKE_ASSIGN_TRACE
 // Profiling build only: copies warp `w`'s trace records (3 x int64 each, up to `cap`) to `host`.
 extern "C" __attribute__((visibility("default"))) int cake_debug_read_trace(int w, long long* host, int cap) {
@@ -1436,7 +1454,7 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s, int Dx,
-                     cake_bf16* cpad, int knn_k, float* fuse_sums, int* fuse_counts, int* fuse_ctas) {
+                     cake_bf16* cpad, int knn_k, float* fuse_sums, int* fuse_counts, int* fuse_ctas, bool pair) {
     // D: columns of a row of C; Dk: columns of a row of X and length of the contraction (D, or D rounded up to
     // a multiple of 8 with zeros in the copy of X); Dc: columns of a row of the centroid operand the kernel
     // streams (C itself, or its zero-padded copy of a multiple of 64 columns, written by the prologue)
@@ -1616,6 +1634,8 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             return CAKE_ERR_CUDA;
         if (attr_known) attr_done[di.device] = true;
     }
+    // CTA pairs (on request): many centroid tiles per row tile, the centroid operand in rows of a multiple of 64 columns
+    if (pair && (xload || knn_k != 0 || fuse || Dc % KCHUNK != 0 || !assign_pair_supports(di, Dk, K))) return CAKE_ERR_UNSUPPORTED;
     // every host-side check has passed: from here on work is enqueued
     if (!aug_ready) {
         const i64 rows = static_cast<i64>(B) * Kpad;
@@ -1640,6 +1660,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         note_launches(1);
     }
 
+    if (pair)
+        return launch_assign_pair(X, cpad ? cpad : C, B, N, Dk, Dc, K, caug, exact, out_idx, out_dist, inertia, inertia_stride,
+                                  status, di, s);
     const unsigned grid = static_cast<unsigned>(p.total_tiles < di.sm_count ? p.total_tiles : di.sm_count);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);

@@ -52,7 +52,17 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
                      bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s,
                      int Dx = 0, cake_bf16* cpad = nullptr, int knn_k = 0, float* fuse_sums = nullptr,
-                     int* fuse_counts = nullptr, int* fuse_ctas = nullptr);
+                     int* fuse_counts = nullptr, int* fuse_ctas = nullptr, bool pair = false);
+// pair: the CTA-pair kernel (tcgen05.mma.cta_group::2; assign_pair.cu) instead of the single-CTA one; needs more than
+// two centroid tiles per row tile
+bool assign_pair_supports(const DeviceInfo& di, int Dk, int K);
+int launch_assign_pair(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int Dk, int Dc, int K, const void* caug,
+                       bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride, int* status,
+                       const DeviceInfo& di, cudaStream_t s);
+// tensor maps: bf16 [batch][rows][D] viewed as (D, rows, batch), box 64 columns x box_rows rows, 128-byte swizzle;
+// and bytes viewed as [rows][16], box 16 x box_rows, no swizzle
+int make_tmap_bf16_rows(CUtensorMap* m, const void* base, int D, i64 rows, int batch, int box_rows);
+int make_tmap_rows16(CUtensorMap* m, const void* base, i64 rows, int box_rows);
 // Fused update (fuse_sums / fuse_counts / fuse_ctas all given, one problem, K <= 128, D <= 128 and room in shared
 // memory): the assign kernel also adds the rows of every tile to per-cluster sums on the tensor core.  On return
 // *fuse_ctas = n > 0 says that it did: fuse_sums then holds n partial sums of [128][round_up(D, 16)] floats (one per

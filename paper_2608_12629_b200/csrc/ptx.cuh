@@ -220,6 +220,86 @@ __device__ __forceinline__ void reg_dep(uint32_t (&r)[32]) {
         : "memory");
 }
 
+// ------------------------------------------------------------------ CTA pairs (cta_group::2)
+// Two CTAs of a thread-block cluster (ranks 0 and 1) drive both SMs' tensor cores with one
+// instruction stream: rank 0 issues, every CTA supplies its own 128 rows of A and its own half of B's
+// rows from its own shared memory (same offsets in both), and every CTA's tensor memory receives its
+// own 128 rows of D.  A shared-memory address of rank 1 differs from the same offset in rank 0 by the
+// bit below.
+constexpr uint32_t CLUSTER_PEER_BIT = 1u << 24;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// All threads of all CTAs of the cluster (unbounded: only where every thread is certain to arrive).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// One arrival on an mbarrier of any CTA of the cluster (`bar` is a shared::cluster address).  Release at CTA
+// scope: a cluster-scope release waits for the thread's earlier global stores and was measured at about 1,100
+// clocks per arrival; what the waiter reads afterwards is tensor memory (tcgen05.wait::ld has completed) or shared
+// memory of the arriving CTA behind a proxy fence.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// The same tiled loads as above, but the byte count may be reported to an mbarrier of the pair's other
+// CTA (`bar` is a shared::cluster address); the destination is the executing CTA's own shared memory.
+// No multicast.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar, int x,
+                                                 int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar, int x,
+                                                 int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+// Tensor memory of a CTA pair: the same warp of both CTAs executes each of these.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
+                 : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B over the pair (M = 256), issued by one thread of rank 0.
+template <bool ACC>
+__device__ __forceinline__ void umma_pair_bf16_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                                    uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
+    const uint32_t z = 0;
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, {%7, %7, %7, %7, %7, %7, %7, %7}, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(ACC ? 1u : 0u), "r"(z)
+        : "memory");
+}
+// One arrival on the mbarrier at this shared-memory offset in every CTA of `mask` (bit r = rank r)
+// once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_pair_commit(uint32_t bar, uint16_t mask) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(mask)
+        : "memory");
+}
+
 // warpgroup-wide register reallocation (all four warps of an aligned warpgroup execute it)
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {
