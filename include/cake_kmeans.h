@@ -58,9 +58,12 @@ enum {
 };
 
 enum {
-    CAKE_ASSIGN_AUTO = 0,      /* the tensor-core pipeline for D <= 512 (for D % 8 != 0 on a zero-padded
+    CAKE_ASSIGN_AUTO = 0,      /* the tensor-core pipeline for D <= 8192 (for D % 8 != 0 on a zero-padded
                                   copy of X kept in the workspace: same results), else the fallback  */
-    CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 512.
+    CAKE_ASSIGN_TCGEN05 = 1,   /* TMA + tcgen05.mma + TMEM pipeline; needs D % 8 == 0, D <= 8192.  Up to D = 512
+                                  a CTA keeps its 128-row X tile in shared memory; longer rows are streamed chunk
+                                  by chunk beside the centroids by pairs of CTAs (two more scratch arrays in the
+                                  workspace, 20 bytes per row, written once per call).
                                   Each distance is an fp32 number whose error follows |x|^2 + |c|^2 of
                                   its own centroid (other centroids' norms do not matter); distances are
                                   compared with 17 significant bits (2^-16 of the distance), equal ones
@@ -71,7 +74,8 @@ enum {
     CAKE_ASSIGN_TCGEN05_PAIR = 4,  /* the arithmetic and results of CAKE_ASSIGN_TCGEN05 on pairs of CTAs
                                       (tcgen05.mma.cta_group::2: two SMs share every 256 x 256 tile and each loads half
                                       of the centroid tile).  Never chosen automatically: measured equal to the single-CTA
-                                      kernel at D = 128, K = 1024 and behind it elsewhere.  D % 8 == 0, D <= 512, K > 512. */
+                                      kernel at D = 128, K = 1024 and behind it elsewhere.  D % 8 == 0; D <= 512 needs K > 512
+                                      (longer rows take the pair kernel under every tensor-core flag).                 */
     CAKE_ASSIGN_TCGEN05_PAIR_EXACT = 5, /* ... with the epilogue of CAKE_ASSIGN_TCGEN05_EXACT                        */
     CAKE_ASSIGN_MASK = 0xF,
     CAKE_UPDATE_AUTO = 0,

@@ -28,7 +28,15 @@ struct Workspace {
     double* pp_part;      // [kPlusPlusMaxSlabs] slab sums of the k-means++ seeding
     float* fpart;         // fused update (one problem, K <= 128, D <= 128): partial sums [kFuseMaxCtas][128][round_up(D, 16)]
     int* fcnt;            // ... and partial counts [kFuseMaxCtas][128]
+    void* xaug;           // rows of more than 512 columns: [B][round_up(N, 256)][16 B] X-side operand of the extra k-step
+    float* xrowm;         // ... and the rows' margins [B][round_up(N, 256)]
     size_t bytes;
+};
+
+// what an earlier step of the same call has already derived from X in the workspace
+struct XPrep {
+    bool padded = false;   // xpad holds the zero-padded copy (D % 8 != 0)
+    bool aug = false;      // xaug / xrowm are written (rows of more than 512 columns)
 };
 
 Workspace carve(void* base, i64 B, i64 N, int D, int K) {
@@ -61,6 +69,9 @@ Workspace carve(void* base, i64 B, i64 N, int D, int K) {
     const size_t fctas = fuse ? static_cast<size_t>(row_tiles < kFuseMaxCtas ? row_tiles : kFuseMaxCtas) : 0;
     w.fpart = reinterpret_cast<float*>(take(fctas * 128 * round_up(D, 16) * 4));
     w.fcnt = reinterpret_cast<int*>(take(fctas * 128 * 4));
+    const bool wide = assign_wide_supports(padded_d(D));
+    w.xaug = take(wide ? assign_wide_aug_bytes(B, N) : 0);
+    w.xrowm = reinterpret_cast<float*>(take(wide ? assign_wide_margin_bytes(B, N) : 0));
     w.bytes = o;
     return w;
 }
@@ -85,23 +96,26 @@ int check_ws(void* ws, size_t ws_bytes, i64 B, i64 N, int D, int K, Workspace* o
 // kernel adds it up itself; the fallback needs `dist` (out_dist or scratch) and a reduction kernel.
 // zero_inertia: the entries still have to be cleared (the tensor-core prologue does it on the way).
 // aug_ready: the update ahead prepared this assign (see NextAssign): the tensor-core route skips its prologue
-// x_padded (in/out): the workspace already holds the padded copy of this X (an earlier step of the call made it)
+// xprep (in/out): what the workspace already holds of this X (an earlier step of the call made it)
 // fuse_ctas (nullable): ask the tensor-core kernel to add the rows to per-cluster partial sums as well (fused update,
 // see launch_assign_tc); *fuse_ctas > 0 on return if it did
 int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, int* out_idx,
               float* out_dist, double* inertia, int inertia_stride, bool zero_inertia, bool aug_ready,
-              bool* x_padded, const Workspace& w, cudaStream_t s, unsigned flags, int* fuse_ctas = nullptr) {
+              XPrep* xprep, const Workspace& w, cudaStream_t s, unsigned flags, int* fuse_ctas = nullptr) {
     if (fuse_ctas) *fuse_ctas = 0;
     unsigned path = flags & CAKE_ASSIGN_MASK;
     int Dx = 0;   // columns of the padded copy of X, if one is used
     if (path == CAKE_ASSIGN_AUTO && assign_pad_supports(D) && N > 0) {
         Dx = padded_d(D);
-        if (!*x_padded && launch_pad_rows(X, static_cast<i64>(B) * N, D, Dx, w.xpad, s) != cudaSuccess) return CAKE_ERR_CUDA;
-        *x_padded = true;
+        if (!xprep->padded && launch_pad_rows(X, static_cast<i64>(B) * N, D, Dx, w.xpad, s) != cudaSuccess) return CAKE_ERR_CUDA;
+        xprep->padded = true;
         X = w.xpad;
         path = CAKE_ASSIGN_TCGEN05;
     }
-    if (path == CAKE_ASSIGN_AUTO) path = assign_tc_supports(D) ? CAKE_ASSIGN_TCGEN05 : CAKE_ASSIGN_SIMT;
+    // rows of more than 512 columns: the CTA-pair kernel's wide mode (X streamed beside the centroids), chosen
+    // automatically and by either tensor-core flag
+    const bool wide = assign_wide_supports(Dx ? Dx : D);
+    if (path == CAKE_ASSIGN_AUTO) path = (assign_tc_supports(D) || wide) ? CAKE_ASSIGN_TCGEN05 : CAKE_ASSIGN_SIMT;
     if (zero_inertia && inertia && (path == CAKE_ASSIGN_SIMT || N == 0)) {
         if (cudaMemset2DAsync(inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
                               static_cast<size_t>(B), s) != cudaSuccess)
@@ -116,22 +130,24 @@ int do_assign(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K
     }
     const bool pair = path == CAKE_ASSIGN_TCGEN05_PAIR || path == CAKE_ASSIGN_TCGEN05_PAIR_EXACT;
     if (path != CAKE_ASSIGN_TCGEN05 && path != CAKE_ASSIGN_TCGEN05_EXACT && !pair) return CAKE_ERR_UNSUPPORTED;
-    if (!assign_tc_supports(Dx ? Dx : D)) return CAKE_ERR_UNSUPPORTED;
+    if (!assign_tc_supports(Dx ? Dx : D) && !wide) return CAKE_ERR_UNSUPPORTED;
     if (N == 0) return CAKE_OK;
     // the packed epilogue (values compared with 17 significant bits) is the automatic choice; the exact
     // one compares full fp32 values and is slower
     const bool exact = path == CAKE_ASSIGN_TCGEN05_EXACT || path == CAKE_ASSIGN_TCGEN05_PAIR_EXACT;
     const bool fuse = fuse_ctas && !exact && fuse_shape_ok(B, D, K) && w.fpart && N > 0 && !pair;
-    return launch_assign_tc(X, C, B, N, D, K, w.caug, exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia,
-                            aug_ready, w.status, s, Dx,
-                            assign_cpad_columns(D) ? w.cpad : nullptr, 0, fuse ? w.fpart : nullptr, fuse ? w.fcnt : nullptr,
-                            fuse ? fuse_ctas : nullptr, pair);
+    const int rc = launch_assign_tc(X, C, B, N, D, K, w.caug, exact, out_idx, out_dist, inertia, inertia_stride, zero_inertia,
+                                    aug_ready, w.status, s, Dx,
+                                    assign_cpad_columns(D) ? w.cpad : nullptr, 0, fuse ? w.fpart : nullptr, fuse ? w.fcnt : nullptr,
+                                    fuse ? fuse_ctas : nullptr, pair, w.xaug, w.xrowm, xprep->aug);
+    if (rc == CAKE_OK && wide) xprep->aug = true;
+    return rc;
 }
 
 // next / prepared: see launch_finalize
 int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, const cake_bf16* C_prev,
               float* out_C, cake_bf16* out_C_bf16, int* out_counts, const Workspace& w, cudaStream_t s,
-              unsigned flags, bool* x_padded, const NextAssign* next = nullptr, bool* prepared = nullptr) {
+              unsigned flags, XPrep* xprep, const NextAssign* next = nullptr, bool* prepared = nullptr) {
     if (prepared) *prepared = false;
     DeviceInfo di;
     int rc = current_device_info(&di);
@@ -143,8 +159,8 @@ int do_update(const cake_bf16* X, const int* idx, int B, i64 N, int D, int K, co
         // D % 8 != 0: the slab route on the zero-padded copy of X (its padding columns add up to zero and are
         // dropped by the division kernel); faster than the element-wise reduction even when the copy has to be made
         Ds = padded_d(D);
-        if (!*x_padded && launch_pad_rows(X, static_cast<i64>(B) * N, D, Ds, w.xpad, s) != cudaSuccess) return CAKE_ERR_CUDA;
-        *x_padded = true;
+        if (!xprep->padded && launch_pad_rows(X, static_cast<i64>(B) * N, D, Ds, w.xpad, s) != cudaSuccess) return CAKE_ERR_CUDA;
+        xprep->padded = true;
         X = w.xpad;
         path = CAKE_UPDATE_SLAB;
     }
@@ -219,7 +235,7 @@ int cake_kmeans_assign_batched(const cake_bf16* X, const cake_bf16* C, long long
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;
-    bool x_padded = false;
+    XPrep x_padded;
     return do_assign(X, C, static_cast<int>(B), N, D, K, out_idx, out_dist, nullptr, 0, false, false, &x_padded, w,
                      reinterpret_cast<cudaStream_t>(stream), flags);
 }
@@ -242,7 +258,7 @@ int cake_kmeans_update_batched(const cake_bf16* X, const int* idx, long long B, 
     Workspace w;
     rc = check_ws(ws, ws_bytes, B, N, D, K, &w);
     if (rc != CAKE_OK) return rc;
-    bool x_padded = false;
+    XPrep x_padded;
     return do_update(X, idx, static_cast<int>(B), N, D, K, C_prev, out_C, out_C_bf16, out_counts, w,
                      reinterpret_cast<cudaStream_t>(stream), flags, &x_padded);
 }
@@ -306,14 +322,15 @@ int cake_kmeans_lloyd_sharded(const cake_bf16* X_local, const cake_bf16* C0, lon
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const i64 N = N_local;
     const unsigned apath = flags & CAKE_ASSIGN_MASK;
-    const bool tc_assign = N > 0 && ((assign_tc_supports(D) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
+    const bool tc_assign = N > 0 && (((assign_tc_supports(D) || assign_wide_supports(D)) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
                                                                 apath == CAKE_ASSIGN_TCGEN05_EXACT || apath == CAKE_ASSIGN_TCGEN05_PAIR ||
                                                                 apath == CAKE_ASSIGN_TCGEN05_PAIR_EXACT)) ||
                                      (assign_pad_supports(D) && apath == CAKE_ASSIGN_AUTO));
     const int cpad_columns = assign_cpad_columns(D);
     const cake_bf16* cur = C0;
     int nxt = 0;
-    bool prepared = false, x_padded = false;
+    bool prepared = false;
+    XPrep x_padded;
     for (int t = 0; t < iters; ++t) {
         rc = do_assign(X_local, cur, 1, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr, iters, true,
                        prepared, &x_padded, w, s, flags);
@@ -395,7 +412,7 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     // The division kernel of iteration t also writes what the tensor-core assign of iteration t + 1 would
     // otherwise compute in a prologue launch of its own.
     const unsigned apath = flags & CAKE_ASSIGN_MASK;
-    const bool tc_assign = N > 0 && ((assign_tc_supports(D) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
+    const bool tc_assign = N > 0 && (((assign_tc_supports(D) || assign_wide_supports(D)) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05 ||
                                                                 apath == CAKE_ASSIGN_TCGEN05_EXACT || apath == CAKE_ASSIGN_TCGEN05_PAIR ||
                                                                 apath == CAKE_ASSIGN_TCGEN05_PAIR_EXACT)) ||
                                      (assign_pad_supports(D) && apath == CAKE_ASSIGN_AUTO));
@@ -403,7 +420,7 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     const cake_bf16* cur = C0;
     int nxt = 0;
     bool prepared = false;
-    bool x_padded = false;   // the workspace holds the padded copy of X (D % 8 != 0), made by the first step that needs it
+    XPrep x_padded;   // what the workspace holds of X (padded copy, wide-row operand), made by the first step that needs it
     // One problem of at most 128 clusters and 128 features: a single pass over X per iteration.  The assign kernel adds
     // the rows of every tile to per-cluster partial sums while the tile is in shared memory, and one small kernel adds
     // the partials up and divides (two launches per iteration instead of four).
@@ -502,7 +519,7 @@ int cake_kmeans_init_plusplus(const cake_bf16* X, long long N, int D, int K, con
     int* idx_scr = reinterpret_cast<int*>(w.pairs);
     float* mind = reinterpret_cast<float*>(w.pairs) + N;
     if (launch_pp_pick(X, mind, w.pp_part, N, D, u, 0, out_C0, out_rows, s) != cudaSuccess) return CAKE_ERR_CUDA;
-    bool x_padded = false;
+    XPrep x_padded;
     // the centroid of a one-centroid assign must start on a 16-byte boundary: rows of D % 8 != 0 columns go through
     // the continuation buffer
     const bool via_copy = (static_cast<size_t>(D) * 2) % 16 != 0;

@@ -84,6 +84,8 @@ struct Params {
     int n_xbuf;       // 1 or 2 X buffers
     int* out_idx;
     float* out_dist;
+    const float* row_m;   // wide mode: every row's margin m, [B][Npad]
+    i64 Npad;             // ... rows per problem there (N rounded up to a multiple of 256)
     double* inertia;      // optional: inertia[b * inertia_stride] += sum of the problem's distances
     int inertia_stride;
     int* status;
@@ -219,21 +221,30 @@ __device__ __forceinline__ void exact_scan32(const uint32_t (&r)[32], int col_ba
 
 // BULK: the epilogue requests a whole 128-column slice at once, hands the accumulator back as soon as it has
 // landed and reduces from registers; otherwise the four 32-column groups go through two register buffers.
-template <bool PACKED, bool BULK>
+// WIDE (rows of more than 512 columns, which no CTA can keep resident): X is streamed like the centroids, a chunk
+// of each per ring stage, and the X-side operand of the extra k-step and the row margins come from global memory
+// (row_aug_kernel wrote them); the norm warps idle.
+template <bool PACKED, bool BULK, bool WIDE = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
-                  const __grid_constant__ CUtensorMap tmap_aug, const Params p) {
+                  const __grid_constant__ CUtensorMap tmap_aug, const __grid_constant__ CUtensorMap tmap_xaug, const Params p) {
     extern __shared__ uint8_t smem_raw[];
     // 128B-swizzled tiles need 1024-byte alignment
     const uint32_t raw_addr = ptx::smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
     uint8_t* smem = smem_raw + pad;
     const uint32_t smem_base = raw_addr + pad;
-    const uint32_t xbuf_bytes = static_cast<uint32_t>(p.nchunks) * X_CHUNK_BYTES;
+    const uint32_t xbuf_bytes = WIDE ? 0u : static_cast<uint32_t>(p.nchunks) * X_CHUNK_BYTES;
     const uint32_t x_base = smem_base;
     const uint32_t ring_off = static_cast<uint32_t>(p.n_xbuf) * xbuf_bytes;
     const uint32_t ring_base = smem_base + ring_off;
-    const uint32_t stage_bytes = static_cast<uint32_t>(p.cps) * C_HALF_BYTES + AUG_B_HALF;
+    // a chunk of a stage: this CTA's half of the centroid chunk, in the wide mode behind its X chunk
+    // Wide rows: one issuer with the whole ring.  A tile is tens of stages long there, the issuers would work one
+    // after the other anyway, and a load takes longer than the MMAs of the two or three stages a sub-ring holds.
+    constexpr int NISS = WIDE ? 1 : NUM_ISSUERS;
+    constexpr uint32_t CHUNK_STRIDE = WIDE ? X_CHUNK_BYTES + C_HALF_BYTES : C_HALF_BYTES;
+    constexpr uint32_t C_IN_CHUNK = WIDE ? X_CHUNK_BYTES : 0u;
+    const uint32_t stage_bytes = static_cast<uint32_t>(p.cps) * CHUNK_STRIDE + AUG_B_HALF;
     const uint32_t auga_off = ring_off + static_cast<uint32_t>(p.n_stages) * stage_bytes;
     const uint32_t zero_off = auga_off + static_cast<uint32_t>(p.n_xbuf) * AUG_A_BYTES;
     const uint32_t ctrl_off = zero_off + AUG_ZERO_BYTES;
@@ -250,8 +261,9 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAX_XBUF; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), NUM_ISSUERS + 4 + 4);  // MMA issuers, norm warps, one epilogue warpgroup
-            ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 8);
+            // MMA issuers, norm warps, one epilogue warpgroup (wide: the issuers alone)
+            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), WIDE ? NISS : NISS + 4 + 4);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), WIDE ? 1 : 8);   // norm warps of both CTAs (wide: rank 0's producer)
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_local[i]), 4);
         }
         for (int i = 0; i < 2; ++i) {
@@ -283,6 +295,7 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         ptx::prefetch_tensormap(&tmap_x);
         ptx::prefetch_tensormap(&tmap_c);
         ptx::prefetch_tensormap(&tmap_aug);
+        if (WIDE) ptx::prefetch_tensormap(&tmap_xaug);
     }
     ptx::tc_fence_before();
     __syncthreads();
@@ -313,11 +326,19 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             auto issue_x = [&]() {
                 const int tb = static_cast<int>(x_next / p.m_tiles);
                 const int tmt = static_cast<int>(x_next % p.m_tiles);
-                const uint32_t xfull = ptx::smem_u32(&ctrl->x_full[ixb]);
-                ptx::mbar_arrive_expect_tx(xfull, xbuf_bytes);
-                for (int c = 0; c < p.nchunks; ++c)
-                    ptx::tma_load_3d(x_base + ixb * xbuf_bytes + c * X_CHUNK_BYTES, &tmap_x, xfull,
-                                     c * KCHUNK, tmt * (2 * BLOCK_M) + static_cast<int>(rank) * BLOCK_M, tb);
+                if (WIDE) {
+                    // the row tile's X-side operand of the extra k-step (this CTA's 128 rows of it); both CTAs' bytes
+                    // are counted on rank 0's barrier, where the issuers wait
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctrl->auga_full[ixb]), 2u * AUG_A_BYTES);
+                    ptx::tma_load_2d_pair(smem_base + auga_off + ixb * AUG_A_BYTES, &tmap_xaug, at_rank0(&ctrl->auga_full[ixb]), 0,
+                                          static_cast<int>(tb * p.Npad + tmt * (2 * BLOCK_M) + static_cast<int>(rank) * BLOCK_M));
+                } else {
+                    const uint32_t xfull = ptx::smem_u32(&ctrl->x_full[ixb]);
+                    ptx::mbar_arrive_expect_tx(xfull, xbuf_bytes);
+                    for (int c = 0; c < p.nchunks; ++c)
+                        ptx::tma_load_3d(x_base + ixb * xbuf_bytes + c * X_CHUNK_BYTES, &tmap_x, xfull,
+                                         c * KCHUNK, tmt * (2 * BLOCK_M) + static_cast<int>(rank) * BLOCK_M, tb);
+                }
                 x_next += n_pairs;
                 if (++ixb == static_cast<uint32_t>(p.n_xbuf)) { ixb = 0; ixph ^= 1u; }
             };
@@ -329,13 +350,14 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             };
             for (i64 tile = pair; ok && tile < p.total_tiles; tile += n_pairs) {
                 const int b = static_cast<int>(tile / p.m_tiles);
+                const int xrow = static_cast<int>(tile % p.m_tiles) * (2 * BLOCK_M) + static_cast<int>(rank) * BLOCK_M;
                 prefetch_x();
                 if (x_next <= tile) {   // this tile's own X is still outstanding: its buffer must free up
                     ok = wait_bar(&ctrl->x_empty[ixb], ixph ^ 1u, ctrl, p.status);
                     if (!ok) break;
                     issue_x();
                 }
-                for (int nt = 0; ok && nt < p.n_tiles; ++nt, turn = (turn + 1 == NUM_ISSUERS) ? 0 : turn + 1) {
+                for (int nt = 0; ok && nt < p.n_tiles; ++nt, turn = (turn + 1 == NISS) ? 0 : turn + 1) {
                     const int crow = nt * BLOCK_N + static_cast<int>(rank) * (BLOCK_N / 2);   // this CTA's centroid rows
                     uint32_t rs = turn == 0 ? sr0 : (turn == 1 ? sr1 : sr2);
                     uint32_t rph = turn == 0 ? sp0 : (turn == 1 ? sp1 : sp2);
@@ -350,13 +372,15 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                         // both CTAs' bytes are counted on rank 0's barrier, which rank 0 arms
                         if (rank == 0)
                             ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctrl->ring_full[slot]),
-                                                       2u * (static_cast<uint32_t>(nc) * C_HALF_BYTES + (last ? AUG_B_HALF : 0u)));
+                                                       2u * (static_cast<uint32_t>(nc) * CHUNK_STRIDE + (last ? AUG_B_HALF : 0u)));
                         const uint32_t full0 = at_rank0(&ctrl->ring_full[slot]);
                         const uint32_t stage = ring_base + slot * stage_bytes;
-                        for (int j = 0; j < nc; ++j)
-                            ptx::tma_load_3d_pair(stage + j * C_HALF_BYTES, &tmap_c, full0, (c + j) * KCHUNK, crow, b);
+                        for (int j = 0; j < nc; ++j) {
+                            if (WIDE) ptx::tma_load_3d_pair(stage + j * CHUNK_STRIDE, &tmap_x, full0, (c + j) * KCHUNK, xrow, b);
+                            ptx::tma_load_3d_pair(stage + j * CHUNK_STRIDE + C_IN_CHUNK, &tmap_c, full0, (c + j) * KCHUNK, crow, b);
+                        }
                         if (last)   // the tile's half-norm operand rides with its last chunks
-                            ptx::tma_load_2d_pair(stage + static_cast<uint32_t>(p.cps) * C_HALF_BYTES, &tmap_aug, full0, 0,
+                            ptx::tma_load_2d_pair(stage + static_cast<uint32_t>(p.cps) * CHUNK_STRIDE, &tmap_aug, full0, 0,
                                                   b * p.Kpad + crow);
                         if (++rs == spi) { rs = 0; rph ^= 1u; }
                     }
@@ -370,7 +394,7 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 }
             }
         }
-    } else if (warp >= MMA_WARP && warp < MMA_WARP + NUM_ISSUERS) {
+    } else if (warp >= MMA_WARP && warp < MMA_WARP + NISS) {
         // ------------------------------------------------------------ MMA issuers (rank 0 only)
         // Three warps, one issuing thread each; centroid tiles go round robin over them (tile t to
         // issuer t mod 3, into accumulator t mod 2) because one thread's own instruction stream is too
@@ -399,7 +423,7 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 const uint32_t a_lo_tile = ptx::umma_desc_lo_sw128(x_base + xb * xbuf_bytes);
                 const uint32_t auga_lo = ptx::umma_desc_lo_aug(smem_base + auga_off + xb * AUG_A_BYTES,
                                                                smem_base + zero_off);
-                for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it, turn = (turn + 1 == NUM_ISSUERS) ? 0 : turn + 1) {
+                for (int nt = 0; ok && nt < p.n_tiles; ++nt, ++acc_it, turn = (turn + 1 == NISS) ? 0 : turn + 1) {
                     if (turn != iss) continue;   // another issuer's tile, in that issuer's sub-ring
                     const uint32_t acc = acc_it & 1u;
                     const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
@@ -420,7 +444,8 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                         const uint32_t stage = ring_base + (slot0 + s) * stage_bytes;
                         const int nc = min(p.cps, p.nchunks - c0);
                         for (int j = 0; j < nc; ++j, a_lo += X_CHUNK_BYTES >> 4) {
-                            const uint32_t b_lo = ptx::umma_desc_lo_sw128(stage + j * C_HALF_BYTES);
+                            if (WIDE) a_lo = ptx::umma_desc_lo_sw128(stage + j * CHUNK_STRIDE);   // the X chunk of this stage
+                            const uint32_t b_lo = ptx::umma_desc_lo_sw128(stage + j * CHUNK_STRIDE + C_IN_CHUNK);
                             const bool last = c0 + j == p.nchunks - 1;
                             const int nk = last ? p.ksteps_last : KCHUNK / UMMA_K;
                             if (c0 + j == 0)
@@ -442,7 +467,7 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                             // the extra k-step: + ||x||^2/2 + m + ||c||^2/2; its centroid side came with this stage
                             if (last)
                                 ptx::umma_pair_bf16_lohi<true>(d_tmem, auga_lo, ptx::UMMA_DESC_HI_AUG,
-                                                               ptx::umma_desc_lo_aug(stage + static_cast<uint32_t>(p.cps) * C_HALF_BYTES,
+                                                               ptx::umma_desc_lo_aug(stage + static_cast<uint32_t>(p.cps) * CHUNK_STRIDE,
                                                                                      smem_base + zero_off),
                                                                ptx::UMMA_DESC_HI_AUG, idesc_aug);
                         }
@@ -458,7 +483,7 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 if (++xb == static_cast<uint32_t>(p.n_xbuf)) { xb = 0; xph ^= 1u; }
             }
         }
-    } else if (warp >= AUX_WARP0) {
+    } else if (!WIDE && warp >= AUX_WARP0) {
         // ------------------------------------------------------------ norm warps
         // One thread per X row: ||x||^2/2 + m from the swizzled X tile (16-byte granule g of row r sits
         // at position g ^ (r & 7); the order of the granules does not matter for a sum), split into
@@ -511,7 +536,7 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         const int q = warp & 3;              // TMEM lane quarter this warp may read
         const int r = q * 32 + lane;         // row inside the X tile
         uint32_t tile_it = 0, acc_it = 0;
-        uint32_t next_iss = 2 % NUM_ISSUERS;   // (acc_it + 2) mod NUM_ISSUERS
+        uint32_t next_iss = 2 % NISS;   // (acc_it + 2) mod the number of issuers
         uint32_t exb = 0, exph = 0;          // X buffer (slot of the row margins) and its phase
         const uint32_t kmask = ~COL_MASK | (static_cast<uint32_t>(p.K) >> 31);   // in a register (see assign_tc.cu)
         bool ok = true;
@@ -548,14 +573,18 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 if (!ok) break;
                 ptx::tc_fence_after();
                 if (nt == 0 && wg == 0) {
-                    // written by the norm warps before they completed auga_local; read now, while the X
-                    // buffer (and with it this slot) cannot have been handed to a later row tile
-                    ok = wait_bar(&ctrl->auga_local[exb], exph, ctrl, p.status);
-                    if (!ok) break;
-                    rowM = ctrl->row_m[exb][r];
-                    // the slot of the margins goes back with the X buffer: this warpgroup has read it
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[exb]));
+                    if (WIDE) {
+                        rowM = p.row_m[static_cast<i64>(b) * p.Npad + static_cast<i64>(mt) * (2 * BLOCK_M) + rank * BLOCK_M + r];
+                    } else {
+                        // written by the norm warps before they completed auga_local; read now, while the X
+                        // buffer (and with it this slot) cannot have been handed to a later row tile
+                        ok = wait_bar(&ctrl->auga_local[exb], exph, ctrl, p.status);
+                        if (!ok) break;
+                        rowM = ctrl->row_m[exb][r];
+                        // the slot of the margins goes back with the X buffer: this warpgroup has read it
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[exb]));
+                    }
                 }
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                        as * BLOCK_N + wg * (BLOCK_N / 2);
@@ -635,7 +664,7 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                         exact_scan32(rd, col0 + 96, best, bsel);
                     }
                 }
-                next_iss = (next_iss + 1 == NUM_ISSUERS) ? 0 : next_iss + 1;
+                next_iss = (next_iss + 1 == NISS) ? 0 : next_iss + 1;
             }
             if (!ok) break;
             trace_mark(ctrl, 102);
@@ -714,6 +743,63 @@ extern "C" __attribute__((visibility("default"))) int cake_debug_read_trace_pair
 }
 #endif
 
+// ======================================================================= rows of more than 512 columns
+namespace {
+// One warp per row of X: ||x||^2 in fp32, the margin m and the X-side operand of the extra k-step
+// ([hi mid lo 1 1 1 0 0] in bf16, hi + mid + lo = ||x||^2/2 + m), as the norm warps of the kernels with a resident X
+// tile compute them in shared memory.  Rows N .. Npad-1 of a problem (the last row tile's tail) get zeros.
+__global__ void __launch_bounds__(256)
+row_aug_kernel(const cake_bf16* __restrict__ X, i64 N, int D, i64 Npad, i64 rows_total, uint4* __restrict__ aug,
+               float* __restrict__ row_m) {
+    const int lane = threadIdx.x & 31;
+    const i64 row = static_cast<i64>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows_total) return;
+    const i64 b = row / Npad, i = row - b * Npad;
+    if (i >= N) {
+        if (lane == 0) {
+            aug[row] = make_uint4(0, 0, 0, 0);
+            row_m[row] = 0.f;
+        }
+        return;
+    }
+    const uint4* x = reinterpret_cast<const uint4*>(X + (static_cast<size_t>(b) * N + i) * D);
+    float xn0 = 0.f, xn1 = 0.f, xn2 = 0.f, xn3 = 0.f;
+    for (int g = lane; g < D / 8; g += 32) {
+        const uint4 w = __ldg(x + g);
+        float a = bf16lo(w.x); xn0 = fmaf(a, a, xn0); a = bf16hi(w.x); xn1 = fmaf(a, a, xn1);
+        a = bf16lo(w.y); xn2 = fmaf(a, a, xn2); a = bf16hi(w.y); xn3 = fmaf(a, a, xn3);
+        a = bf16lo(w.z); xn0 = fmaf(a, a, xn0); a = bf16hi(w.z); xn1 = fmaf(a, a, xn1);
+        a = bf16lo(w.w); xn2 = fmaf(a, a, xn2); a = bf16hi(w.w); xn3 = fmaf(a, a, xn3);
+    }
+    float xn = (xn0 + xn1) + (xn2 + xn3);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) xn += __shfl_xor_sync(0xffffffffu, xn, o);
+    if (lane == 0) {
+        // margin m = 2^(e-11) for ||x||^2 in [2^e, 2^(e+1)), at least 2^-100 (see assign_tc.cu)
+        const uint32_t xe = __float_as_uint(xn) >> 23;
+        const uint32_t mbits = (xe > 38u ? xe - 11u : 27u) << 23;
+        uint32_t hi, mid, lo;
+        split3(fmaf(0.5f, xn, __uint_as_float(mbits)), hi, mid, lo);
+        const uint32_t one = 0x3F80u;
+        aug[row] = make_uint4(hi | (mid << 16), lo | (one << 16), one | (one << 16), 0u);
+        row_m[row] = __uint_as_float(mbits);
+    }
+}
+
+}  // namespace
+
+size_t assign_wide_aug_bytes(i64 B, i64 N) { return static_cast<size_t>(B) * round_up(N, 2 * BLOCK_M) * 16; }
+size_t assign_wide_margin_bytes(i64 B, i64 N) { return static_cast<size_t>(B) * round_up(N, 2 * BLOCK_M) * 4; }
+
+cudaError_t launch_row_aug(const cake_bf16* X, int B, i64 N, int D, void* xaug, float* xrowm, cudaStream_t s) {
+    const i64 Npad = round_up(N, 2 * BLOCK_M);
+    const i64 rows = static_cast<i64>(B) * Npad;
+    if (rows == 0) return cudaSuccess;
+    row_aug_kernel<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, s>>>(X, N, D, Npad, rows, static_cast<uint4*>(xaug), xrowm);
+    note_launches(1);
+    return cudaGetLastError();
+}
+
 // ======================================================================= host side
 namespace {
 struct PairPlan {
@@ -723,10 +809,22 @@ struct PairPlan {
 
 // Shared memory: n_xbuf X buffers and NUM_ISSUERS sub-rings of spi stages of cps chunks.  Preferred: a whole
 // centroid tile per stage (one wait and one commit per tile on the issuing thread), then more than one stage per
-// issuer; few centroid tiles per row tile want more X buffers instead.
-bool plan_pair(const DeviceInfo& di, int nchunks, int n_tiles, PairPlan* out) {
+// issuer; few centroid tiles per row tile want more X buffers instead.  Wide rows: no X buffer (two 2 KiB operands
+// of the extra k-step instead), a stage holds one chunk of X and of the centroids.
+bool plan_pair(const DeviceInfo& di, int nchunks, int n_tiles, bool wide, PairPlan* out) {
     const i64 fixed = 1024 + CTRL_BYTES + AUG_ZERO_BYTES;
     const i64 budget = static_cast<i64>(di.smem_optin) - fixed;
+    if (wide) {
+        const i64 stage = X_CHUNK_BYTES + C_HALF_BYTES + AUG_B_HALF;
+        i64 spi = (budget - 2 * AUG_A_BYTES) / stage;   // one issuer: the whole ring is its sub-ring
+        if (spi < 2) return false;
+        if (spi > MAX_STAGES) spi = MAX_STAGES;
+        out->n_xbuf = 2;
+        out->spi = static_cast<int>(spi);
+        out->cps = 1;
+        out->smem_bytes = static_cast<size_t>(fixed + 2 * AUG_A_BYTES + spi * stage);
+        return true;
+    }
     const i64 xbuf = static_cast<i64>(nchunks) * X_CHUNK_BYTES + AUG_A_BYTES;
     const int want_xbuf = n_tiles <= 2 ? MAX_XBUF : 2;
     for (int n_xbuf = want_xbuf; n_xbuf >= 1; --n_xbuf) {
@@ -756,14 +854,17 @@ bool plan_pair(const DeviceInfo& di, int nchunks, int n_tiles, PairPlan* out) {
 // whether the pair kernel has a shared-memory layout for these sizes (the caller checks before it enqueues anything)
 bool assign_pair_supports(const DeviceInfo& di, int Dk, int K) {
     PairPlan pl;
-    return plan_pair(di, (Dk + KCHUNK - 1) / KCHUNK, (K + BLOCK_N - 1) / BLOCK_N, &pl);
+    return plan_pair(di, (Dk + KCHUNK - 1) / KCHUNK, (K + BLOCK_N - 1) / BLOCK_N, Dk > kAssignResidentMaxD, &pl);
 }
 
 // X and C as for launch_assign_tc (C may be the zero-padded copy: Dc columns, a multiple of 64); the half-norm
-// operand `caug` must have been written (the caller ran the prologue).
+// operand `caug` must have been written (the caller ran the prologue).  Dk > 512 selects the wide mode: xaug and
+// xrowm as launch_row_aug wrote them for this X.
 int launch_assign_pair(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int Dk, int Dc, int K, const void* caug,
                        bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride, int* status,
-                       const DeviceInfo& di, cudaStream_t s) {
+                       const DeviceInfo& di, cudaStream_t s, const void* xaug, const float* xrowm) {
+    const bool wide = Dk > kAssignResidentMaxD;
+    if (wide && (!xaug || !xrowm)) return CAKE_ERR_NULL;
     Params p;
     p.B = B; p.N = N; p.D = Dk; p.K = K;
     p.nchunks = (Dk + KCHUNK - 1) / KCHUNK;
@@ -774,32 +875,41 @@ int launch_assign_pair(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int
     p.Kpad = padded_k(K);
     p.out_idx = out_idx; p.out_dist = out_dist; p.status = status;
     p.inertia = inertia; p.inertia_stride = inertia_stride;
+    p.row_m = xrowm;
+    p.Npad = round_up(N, 2 * BLOCK_M);
     if (p.total_tiles == 0) return CAKE_OK;
 
     PairPlan pl;
-    if (!plan_pair(di, p.nchunks, p.n_tiles, &pl)) return CAKE_ERR_UNSUPPORTED;
+    if (!plan_pair(di, p.nchunks, p.n_tiles, wide, &pl)) return CAKE_ERR_UNSUPPORTED;
     p.n_xbuf = pl.n_xbuf;
     p.spi = pl.spi;
     p.cps = pl.cps;
-    p.n_stages = pl.spi * NUM_ISSUERS;
+    p.n_stages = pl.spi * (wide ? 1 : NUM_ISSUERS);
 
-    CUtensorMap tx, tc, ta;
+    CUtensorMap tx, tc, ta, txa;
     int rc = make_tmap_bf16_rows(&tx, X, Dk, N, B, BLOCK_M);
     if (rc != CAKE_OK) return rc;
     rc = make_tmap_bf16_rows(&tc, C, Dc, K, B, BLOCK_N / 2);
     if (rc != CAKE_OK) return rc;
     rc = make_tmap_rows16(&ta, caug, static_cast<i64>(B) * p.Kpad, BLOCK_N / 2);
     if (rc != CAKE_OK) return rc;
+    if (wide) {
+        rc = make_tmap_rows16(&txa, xaug, static_cast<i64>(B) * p.Npad, BLOCK_M);
+        if (rc != CAKE_OK) return rc;
+    } else {
+        txa = ta;   // not read
+    }
 
+    using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const Params);
+    static const Kernel kernels[6] = {assign_pair_kernel<true, false>,  assign_pair_kernel<false, false>,
+                                      assign_pair_kernel<true, true>,   assign_pair_kernel<false, true>,
+                                      assign_pair_kernel<true, false, true>, assign_pair_kernel<false, false, true>};
     static bool attr_done[64] = {false};   // per device; benign race: the attribute calls are idempotent
     const bool known = di.device >= 0 && di.device < 64;
     if (!known || !attr_done[di.device]) {
-        const int sm = di.smem_optin;
-        if (cudaFuncSetAttribute(assign_pair_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm) != cudaSuccess ||
-            cudaFuncSetAttribute(assign_pair_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm) != cudaSuccess ||
-            cudaFuncSetAttribute(assign_pair_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm) != cudaSuccess ||
-            cudaFuncSetAttribute(assign_pair_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm) != cudaSuccess)
-            return CAKE_ERR_CUDA;
+        for (Kernel k : kernels)
+            if (cudaFuncSetAttribute(reinterpret_cast<const void*>(k), cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
+                return CAKE_ERR_CUDA;
         if (known) attr_done[di.device] = true;
     }
     // one CTA per SM, in pairs; no more pairs than row tiles
@@ -819,12 +929,9 @@ int launch_assign_pair(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 2;
-    const bool bulk = p.n_tiles >= 8;   // measured: 2-4 % at K >= 2048, nothing or a small loss below
-    const cudaError_t e =
-        bulk ? (exact ? cudaLaunchKernelEx(&cfg, assign_pair_kernel<false, true>, tx, tc, ta, p)
-                      : cudaLaunchKernelEx(&cfg, assign_pair_kernel<true, true>, tx, tc, ta, p))
-             : (exact ? cudaLaunchKernelEx(&cfg, assign_pair_kernel<false, false>, tx, tc, ta, p)
-                      : cudaLaunchKernelEx(&cfg, assign_pair_kernel<true, false>, tx, tc, ta, p));
+    const bool bulk = !wide && p.n_tiles >= 8;   // measured: 2-4 % at K >= 2048, nothing or a small loss below
+    const Kernel kernel = kernels[(wide ? 4 : bulk ? 2 : 0) + (exact ? 1 : 0)];
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tx, tc, ta, txa, p);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return CAKE_ERR_CUDA;

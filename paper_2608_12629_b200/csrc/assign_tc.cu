@@ -1451,20 +1451,66 @@ size_t assign_tc_aug_bytes(i64 B, int K) {
     return static_cast<size_t>(B) * (padded_k(K) / BLOCK_N) * AUG_B_BYTES;
 }
 
+// The prologue of a tensor-core assign: the centroids' half-norm operand into caug (and the zero-padded copy of C
+// into cpad, and zeros into the inertia entries when asked), with programmatic dependent launch allowed.
+static int launch_centroid_prologue(const cake_bf16* C, int B, int D, int K, void* caug, cake_bf16* cpad, int Dc,
+                                    double* inertia, int inertia_stride, bool zero_inertia, cudaStream_t s) {
+    const int Kpad = padded_k(K);
+    const i64 rows = static_cast<i64>(B) * Kpad;
+    const i64 ctas = (rows * 32 + 255) / 256;
+    if (zero_inertia && inertia && B > 256) {   // more problems than the prologue's first CTA has threads
+        if (cudaMemset2DAsync(inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
+                              static_cast<size_t>(B), s) != cudaSuccess)
+            return CAKE_ERR_CUDA;
+    }
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ctas));
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, centroid_aug_kernel, C, K, D, Kpad, rows, static_cast<uint8_t*>(caug),
+                           (zero_inertia && B <= 256) ? inertia : static_cast<double*>(nullptr), inertia_stride,
+                           B, cpad, Dc) != cudaSuccess) {
+        cudaGetLastError();
+        return CAKE_ERR_CUDA;
+    }
+    note_launches(1);
+    return CAKE_OK;
+}
+
 int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D, int K, void* caug,
                      bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s, int Dx,
-                     cake_bf16* cpad, int knn_k, float* fuse_sums, int* fuse_counts, int* fuse_ctas, bool pair) {
+                     cake_bf16* cpad, int knn_k, float* fuse_sums, int* fuse_counts, int* fuse_ctas, bool pair,
+                     void* xaug, float* xrowm, bool xaug_ready) {
     // D: columns of a row of C; Dk: columns of a row of X and length of the contraction (D, or D rounded up to
     // a multiple of 8 with zeros in the copy of X); Dc: columns of a row of the centroid operand the kernel
     // streams (C itself, or its zero-padded copy of a multiple of 64 columns, written by the prologue)
     const int Dk = Dx ? Dx : D;
     const int Dc = cpad ? static_cast<int>(round_up(Dk, KCHUNK)) : D;
-    if (!assign_tc_supports(Dk) || Dk < D || (!cpad && Dk != D)) return CAKE_ERR_UNSUPPORTED;
+    const bool wide = assign_wide_supports(Dk);
+    if ((!assign_tc_supports(Dk) && !wide) || Dk < D || (!cpad && Dk != D)) return CAKE_ERR_UNSUPPORTED;
     DeviceInfo di;
     int rc = current_device_info(&di);
     if (rc != CAKE_OK) return rc;
     if (di.cc_major != 10) return CAKE_ERR_DEVICE;
+    if (wide) {
+        // rows too long for a resident X tile: the CTA-pair kernel streams X beside the centroids
+        if (knn_k != 0 || Dc % KCHUNK != 0 || !xaug || !xrowm || !assign_pair_supports(di, Dk, K)) return CAKE_ERR_UNSUPPORTED;
+        if (fuse_ctas) *fuse_ctas = 0;
+        if (N == 0) return CAKE_OK;
+        if (!aug_ready) {
+            rc = launch_centroid_prologue(C, B, D, K, caug, cpad, Dc, inertia, inertia_stride, zero_inertia, s);
+            if (rc != CAKE_OK) return rc;
+        }
+        if (!xaug_ready && launch_row_aug(X, B, N, Dk, xaug, xrowm, s) != cudaSuccess) return CAKE_ERR_CUDA;
+        return launch_assign_pair(X, cpad ? cpad : C, B, N, Dk, Dc, K, caug, exact, out_idx, out_dist, inertia, inertia_stride,
+                                  status, di, s, xaug, xrowm);
+    }
 
     Params p;
     p.B = B; p.N = N; p.D = Dk; p.K = K;
@@ -1638,26 +1684,8 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     if (pair && (xload || knn_k != 0 || fuse || Dc % KCHUNK != 0 || !assign_pair_supports(di, Dk, K))) return CAKE_ERR_UNSUPPORTED;
     // every host-side check has passed: from here on work is enqueued
     if (!aug_ready) {
-        const i64 rows = static_cast<i64>(B) * Kpad;
-        const i64 ctas = (rows * 32 + 255) / 256;
-        if (zero_inertia && inertia && B > 256) {   // more problems than the prologue's first CTA has threads
-            if (cudaMemset2DAsync(inertia, static_cast<size_t>(inertia_stride) * sizeof(double), 0, sizeof(double),
-                                  static_cast<size_t>(B), s) != cudaSuccess)
-                return CAKE_ERR_CUDA;
-        }
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(static_cast<unsigned>(ctas));
-        cfg.blockDim = dim3(256);
-        cfg.stream = s;
-        cfg.attrs = pdl;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, centroid_aug_kernel, C, K, D, Kpad, rows, static_cast<uint8_t*>(caug),
-                               (zero_inertia && B <= 256) ? inertia : static_cast<double*>(nullptr), inertia_stride,
-                               B, cpad, Dc) != cudaSuccess) {
-            cudaGetLastError();
-            return CAKE_ERR_CUDA;
-        }
-        note_launches(1);
+        rc = launch_centroid_prologue(C, B, D, K, caug, cpad, Dc, inertia, inertia_stride, zero_inertia, s);
+        if (rc != CAKE_OK) return rc;
     }
 
     if (pair)

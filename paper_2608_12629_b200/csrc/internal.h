@@ -34,6 +34,15 @@ inline int padded_k(int K) { return (int)round_up(K, kAssignBlockN); }
 
 // ---- assign
 bool assign_tc_supports(int D);
+// Rows of up to kAssignResidentMaxD columns keep a whole X tile resident in shared memory (assign_tc.cu, and
+// assign_pair.cu on request); longer rows (D % 8 == 0, up to kAssignWideMaxD) stream X chunk by chunk beside the
+// centroids in the CTA-pair kernel's wide mode, which needs two per-row arrays written by launch_row_aug.
+constexpr int kAssignResidentMaxD = 512;
+constexpr int kAssignWideMaxD = 8192;
+inline bool assign_wide_supports(int D) { return D % 8 == 0 && D > kAssignResidentMaxD && D <= kAssignWideMaxD; }
+size_t assign_wide_aug_bytes(i64 B, i64 N);      // X-side operand of the extra k-step, 16 bytes per row
+size_t assign_wide_margin_bytes(i64 B, i64 N);   // the rows' margins m, 4 bytes per row
+cudaError_t launch_row_aug(const cake_bf16* X, int B, i64 N, int D, void* xaug, float* xrowm, cudaStream_t s);
 // bytes of scratch (`caug`) the tensor-core assign needs for B problems of K centroids
 size_t assign_tc_aug_bytes(i64 B, int K);
 // prologue (half-norm operand into caug) + the assign kernel; exact selects the exact epilogue;
@@ -52,13 +61,15 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
                      bool exact, int* out_idx, float* out_dist, double* inertia,
                      int inertia_stride, bool zero_inertia, bool aug_ready, int* status, cudaStream_t s,
                      int Dx = 0, cake_bf16* cpad = nullptr, int knn_k = 0, float* fuse_sums = nullptr,
-                     int* fuse_counts = nullptr, int* fuse_ctas = nullptr, bool pair = false);
+                     int* fuse_counts = nullptr, int* fuse_ctas = nullptr, bool pair = false, void* xaug = nullptr, float* xrowm = nullptr,
+                     bool xaug_ready = false);
 // pair: the CTA-pair kernel (tcgen05.mma.cta_group::2; assign_pair.cu) instead of the single-CTA one; needs more than
-// two centroid tiles per row tile
+// two centroid tiles per row tile.  Rows of more than kAssignResidentMaxD columns always take that kernel, in its
+// wide mode: xaug / xrowm are the scratch arrays of launch_row_aug (run here unless xaug_ready).
 bool assign_pair_supports(const DeviceInfo& di, int Dk, int K);
 int launch_assign_pair(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int Dk, int Dc, int K, const void* caug,
                        bool exact, int* out_idx, float* out_dist, double* inertia, int inertia_stride, int* status,
-                       const DeviceInfo& di, cudaStream_t s);
+                       const DeviceInfo& di, cudaStream_t s, const void* xaug = nullptr, const float* xrowm = nullptr);
 // tensor maps: bf16 [batch][rows][D] viewed as (D, rows, batch), box 64 columns x box_rows rows, 128-byte swizzle;
 // and bytes viewed as [rows][16], box 16 x box_rows, no swizzle
 int make_tmap_bf16_rows(CUtensorMap* m, const void* base, int D, i64 rows, int batch, int box_rows);
@@ -78,10 +89,12 @@ int launch_assign_simt(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int
 // route copies X into rows of padded_d(D) columns, zeros in the padding (distances and norms do not
 // change), and runs the tensor-core kernel on the copy.
 inline int padded_d(int D) { return (int)round_up(D, 8); }
-inline bool assign_pad_supports(int D) { return D % 8 != 0 && assign_tc_supports(padded_d(D)); }
+inline bool assign_pad_supports(int D) {
+    return D % 8 != 0 && (assign_tc_supports(padded_d(D)) || assign_wide_supports(padded_d(D)));
+}
 // columns of a row of the centroid copy the tensor-core kernel streams when D is not a multiple of 64 (else 0)
 inline int assign_cpad_columns(int D) {
-    return (D % 64 != 0 && assign_tc_supports(padded_d(D))) ? (int)round_up(D, 64) : 0;
+    return (D % 64 != 0 && (assign_tc_supports(padded_d(D)) || assign_wide_supports(padded_d(D)))) ? (int)round_up(D, 64) : 0;
 }
 // dst[r][0..Dpad) = src[r][0..D) followed by zeros, for r < rows (Dpad % 8 == 0, dst 16-byte aligned)
 cudaError_t launch_pad_rows(const cake_bf16* src, i64 rows, int D, int Dpad, cake_bf16* dst, cudaStream_t s);

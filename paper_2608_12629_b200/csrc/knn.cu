@@ -80,7 +80,7 @@ int check_shape(i64 N, i64 M, int D, int k) {
     if (N > INT_MAX - 1024 || M > INT_MAX - 1024) return CAKE_ERR_SHAPE;
     if (static_cast<double>(N) * D > 4.0e13 || static_cast<double>(M) * D > 4.0e13) return CAKE_ERR_SHAPE;
     if (k > kMaxK) return CAKE_ERR_UNSUPPORTED;
-    if (!assign_tc_supports(D) && !assign_pad_supports(D)) return CAKE_ERR_UNSUPPORTED;   // D > 512
+    if (padded_d(D) > kAssignResidentMaxD) return CAKE_ERR_UNSUPPORTED;   // the top-k epilogue exists for a resident X tile only
     return CAKE_OK;
 }
 

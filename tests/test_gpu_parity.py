@@ -63,13 +63,15 @@ def test_assign_simt_fallback(N, D, K):
     X, C = problem(N, D, K, seed=N * 3 + D)
     idx, dist = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_SIMT)
     grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx.cpu().numpy(), dist.cpu().numpy())
-    if D % 8 or D > 512:  # the tensor path must refuse such D when asked for by name
+    if D % 8:  # the tensor path must refuse such D when asked for by name
         with pytest.raises(cake.CakeError) as e:
             cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_TCGEN05)
         assert e.value.code == cake.CAKE_ERR_UNSUPPORTED
-    if D > 512:           # and the automatic choice takes the fallback
-        idx2, _ = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV))
-        assert torch.equal(idx, idx2)
+    if D > 512:           # rows too long for a resident X tile: the tensor cores stream them (automatically and by name)
+        idx2, dist2 = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV))
+        grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx2.cpu().numpy(), dist2.cpu().numpy())
+        idx3, dist3 = cake.cake_kmeans_assign(X.to(DEV), C.to(DEV), flags=cake.CAKE_ASSIGN_TCGEN05)
+        assert torch.equal(idx2, idx3) and torch.equal(dist2, dist3)
 
 
 @pytest.mark.parametrize("B,N,D,K", [(1, 100, 5, 7), (1, 3000, 33, 40), (2, 640, 130, 300), (1, 20000, 100, 1000),
