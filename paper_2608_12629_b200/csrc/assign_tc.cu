@@ -315,7 +315,12 @@ __device__ __forceinline__ int tile_step() { return CONSEC ? 1 : static_cast<int
 // FUSE (resident mode with at most 128 centroids and D <= 128, one problem): the kernel also adds every row tile to
 // per-cluster sums while the tile is still in shared memory -- on the tensor core, as sums += onehot^T X with the
 // assignment written as a one-hot bf16 operand -- so that the centroid update needs no second pass over X.
-template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false, bool BULK = false, int TOPK = 0, bool FUSE = false>
+// NARROW: the resident single-tile mode with at most 128 centroids (or D <= 64), packed policy, whole X buffers: the
+// epilogue for at most 128 centroids (two register buffers) in an instantiation of its own.  The shared code for such tiles (four buffers, a run-time branch
+// beside the 256-column epilogue) spills 64 registers and ran 25-35 % slower at 64 < K <= 128; it remains for the
+// exact policy, the split X buffer and the fused update (where it is the only branch and does not spill).
+template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false, bool BULK = false, int TOPK = 0, bool FUSE = false,
+          bool NARROW = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
                  const Params p) {
@@ -944,7 +949,39 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             ptx::tc_fence_after();
             float best = __uint_as_float(F32_INF);
             int bsel = 0;
-            if (FUSE || p.alt_epi <= BLOCK_N / 2) {   // (FUSE: at most 128 centroids by construction)
+            if (NARROW && p.alt_epi <= BLOCK_N / 2) {
+                // at most 128 centroids: only the 32-column groups that hold some were written; they go through two
+                // register buffers, the load of the next group in flight while one is reduced
+                const int ng = p.alt_epi >> 5;
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + as * BLOCK_N;
+                uint32_t ra[32], rb[32];
+                ptx::tmem_ld_x32(taddr, ra);
+                ptx::tmem_ld_wait(ra);
+                if (ng > 1) ptx::tmem_ld_x32_before(taddr + 32, rb, ra);
+                if (PACKED) best = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
+                else exact_scan32(ra, 0, best, bsel);
+                if (ng > 1) {
+                    ptx::tmem_ld_wait_after(rb, best);
+                    if (ng > 2) ptx::tmem_ld_x32_before(taddr + 64, ra, rb);
+                    if (PACKED) best = packed_min32(rb, 32, best, kmask);
+                    else exact_scan32(rb, 32, best, bsel);
+                    if (ng > 2) {
+                        ptx::tmem_ld_wait_after(ra, best);
+                        if (ng > 3) ptx::tmem_ld_x32_before(taddr + 96, rb, ra);
+                        if (PACKED) best = packed_min32(ra, 64, best, kmask);
+                        else exact_scan32(ra, 64, best, bsel);
+                        if (ng > 3) {
+                            ptx::tmem_ld_wait_after(rb, best);
+                            if (PACKED) best = packed_min32(rb, 96, best, kmask);
+                            else exact_scan32(rb, 96, best, bsel);
+                        }
+                    }
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][(tile_it + 2u) % n_iss]));
+                if (PACKED) bsel = 0;
+            } else if (FUSE || (!NARROW && p.alt_epi <= BLOCK_N / 2)) {   // (FUSE: at most 128 centroids by construction; else: the exact policy, split X buffer)
                 // at most 128 centroids: only the 32-column groups that hold some were written
                 const int ng = p.alt_epi >> 5;
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + as * BLOCK_N;
@@ -1656,6 +1693,11 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
     else if (exact)
         kernel = consec ? (xsplit ? assign_tc_kernel<false, true, true, true> : assign_tc_kernel<false, true, true, false>)
                         : (xsplit ? assign_tc_kernel<false, true, false, true> : assign_tc_kernel<false, true, false, false>);
+    // (with the split X buffer the shared code measured faster; the 256-column epilogue of the instantiation without the
+    // spilling branch measured 13 % faster at D = 64 and 1.5-3 % slower at D = 128)
+    else if (p.res_c == 1 && !xsplit && (p.alt_epi <= BLOCK_N / 2 || p.nchunks == 1))
+        kernel = consec ? assign_tc_kernel<true, true, true, false, false, 0, false, true>
+                        : assign_tc_kernel<true, true, false, false, false, 0, false, true>;
     else
         kernel = consec ? (xsplit ? assign_tc_kernel<true, true, true, true> : assign_tc_kernel<true, true, true, false>)
                         : (xsplit ? assign_tc_kernel<true, true, false, true> : assign_tc_kernel<true, true, false, false>);
@@ -1676,7 +1718,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             cudaFuncSetAttribute(assign_tc_kernel<true, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
-            cudaFuncSetAttribute(assign_tc_kernel<false, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
+            cudaFuncSetAttribute(assign_tc_kernel<false, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, true, true, false, false, 0, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, true, false, false, false, 0, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
             return CAKE_ERR_CUDA;
         if (attr_known) attr_done[di.device] = true;
     }
