@@ -730,7 +730,7 @@ def main():
             torch.cuda.empty_cache()
             with ClockSampler(physical_gpu_index(local)) as xclocks:
                 line["extra"] = [extra_row(cake, name, dev, peaks, xclocks, not args.no_cpu_baseline)
-                                 for name in ("c1", "c2", "c3", "c4", "paper", "f1") if name != w.name]
+                                 for name in ("c1", "c2", "c3", "c4", "paper", "f1", "w1") if name != w.name]
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()

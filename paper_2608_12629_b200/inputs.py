@@ -40,6 +40,8 @@ WORKLOADS = {
     "c4": Workload("c4", 1, 2097152, 256, 65536, 16384, 1.0, 0.3, "uniform", 5, 1004),
     # few clusters, one problem: the shape class of the single-pass (fused) iteration, X larger than L2
     "f1": Workload("f1", 1, 2097152, 64, 64, 64, 1.0, 0.5, "uniform", 10, 1006),
+    # rows of 1,024 features: no X tile stays resident, the contraction is streamed over D
+    "w1": Workload("w1", 1, 262144, 1024, 1024, 1024, 1.0, 0.5, "uniform", 5, 1007),
     # the paper's own clean-start shape (assign only in the paper)
     "paper": Workload("paper", 32, 65536, 128, 1024, 1024, 1.0, 0.5, "uniform", 3, 1005),
 }

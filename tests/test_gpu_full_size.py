@@ -91,3 +91,13 @@ def test_c3_every_problem_of_the_batch():
 
 def test_paper_shape_every_problem_of_the_batch():
     batched_one_iteration("paper", 1024)
+
+
+def test_w1_wide_rows_three_iterations_sampled():
+    """The wide-row workload (D = 1,024: X streamed over D by CTA pairs) at full size, teacher-forced, sampled rows;
+    the update of such rows (D = 1,024) graded in full."""
+    w = inputs.WORKLOADS["w1"]
+    X, C0 = inputs.make_problem(w, device=DEV)
+    reports, _ = teacher_forced_full_size(X, C0, 3, 0, 2048, w.seed)
+    for t, rep in enumerate(reports):
+        assert rep["unexcused"] == 0 and rep["mismatch"] <= 3, (t, rep)
