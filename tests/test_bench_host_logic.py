@@ -95,3 +95,13 @@ def test_max_over_ranks_and_whole_job_value_with_gloo_world_size_2():
     assert red == [11.0, 3.0, 1.0, 14.0]                            # the slowest rank decides every time
     assert line["ms_per_step"] == pytest.approx(11.0 / 4)
     assert line["value"] == pytest.approx(2 * 1000.0 / (11.0 / 4))   # units of ALL ranks / max time
+
+
+def test_roofline_denominator_follows_the_clock_bin_of_the_launches():
+    peaks = {"bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0, "source": "measured"}
+    p, src = bench.roofline_peak({"settled": {"samples": 900}, "burst": {"samples": 20}}, peaks)
+    assert p == 1400.0 and "sustained" in src
+    p, src = bench.roofline_peak({"burst": {"samples": 50}}, peaks)
+    assert p == 1600.0 and "burst" in src
+    p, src = bench.roofline_peak({"settled": {"samples": 10}}, {"bf16_tflops": 1590.0, "source": "fallback"})
+    assert p == 1590.0 and src.startswith("fallback")
