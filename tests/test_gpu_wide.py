@@ -100,3 +100,31 @@ def test_wide_rows_lloyd_teacher_forced(N, D, K):
     # the first iteration starts from the same centroids as the oracle's free run (later ones may part at a near-tie)
     first = orc.lloyd(Xb, inputs.to_bits(C0), 1, round_centroids=True)
     np.testing.assert_allclose(full.inertia.cpu().numpy()[:1], first.inertia, rtol=grading.INERTIA_TOL)
+
+
+def test_wide_rows_through_the_other_lloyd_entry_points():
+    """The convergence-tolerance loop, the row-sharded loop (one rank) and the k-means++ seeding take rows of more than
+    512 columns through the same route: equal to the plain Lloyd call, seeding graded against the oracle's draw rule."""
+    from paper_2608_12629_b200 import sharded
+    N, D, K = 3000, 640, 40
+    X, _ = inputs.gaussian_mixture(N, D, K, 2.0, 1.0, 17)
+    C0 = inputs.sample_init(X, K, 17)
+    Xd, Cd = X.to(DEV), C0.to(DEV)
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    ref = cake.cake_kmeans_lloyd(Xd, Cd, 4, ws=ws)
+    sh = sharded.cake_kmeans_lloyd_sharded(Xd, Cd, 4)
+    assert torch.equal(sh.idx, ref.idx) and torch.equal(sh.C_bf16, ref.C_bf16) and torch.equal(sh.counts, ref.counts)
+    tol, iters = cake.cake_kmeans_lloyd_tol(Xd, Cd, 4, 0.0, check_every=2, ws=ws)
+    torch.cuda.synchronize()
+    assert cake.cake_kmeans_device_status(ws) == cake.CAKE_OK
+    assert iters == 4 and torch.equal(tol.idx, ref.idx) and torch.equal(tol.C_bf16, ref.C_bf16)
+    np.testing.assert_allclose(tol.inertia.cpu().numpy()[:4], ref.inertia.cpu().numpy(), rtol=1e-12)
+    # seeding: every drawn row is distinct and the first one is the oracle's (u[0] picks a row uniformly)
+    u = torch.rand(K, generator=torch.Generator().manual_seed(3)).float()
+    Cs, rows = cake.cake_kmeans_init_plusplus(Xd, K, u.to(DEV))
+    torch.cuda.synchronize()
+    rows = rows.cpu().numpy()
+    assert len(set(rows.tolist())) == K
+    want = orc.kmeanspp(inputs.to_bits(X), K, u.numpy().astype(np.float64))
+    assert rows[0] == want[0] and (rows == want).mean() >= 0.5
+    assert torch.equal(Cs.cpu(), X[torch.from_numpy(rows).long()])
