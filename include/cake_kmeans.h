@@ -89,10 +89,14 @@ enum {
     CAKE_UPDATE_SLAB_F2 = 5 << 4,
     CAKE_UPDATE_SLAB_F4 = 6 << 4,
     CAKE_UPDATE_MASK = 0xF << 4,
-    CAKE_LLOYD_NO_FUSE = 1 << 8 /* lloyd: keep assign and update as two passes over X also where one problem of
+    CAKE_LLOYD_NO_FUSE = 1 << 8, /* lloyd: keep assign and update as two passes over X also where one problem of
                                    K <= 128, D <= 128 (D % 8 == 0) would take the single-pass iteration, in which
                                    the assign kernel adds each row tile to per-cluster sums on the tensor core
                                    (sums += onehot^T X) while the tile is in shared memory                      */
+    CAKE_LLOYD_NO_RESIDENT = 1 << 9 /* lloyd: do not take the one-launch form of the single-pass iteration, which a
+                                   problem of D = 64 or 128 and at most four 128-row tiles per SM runs in: all
+                                   iterations in one cooperative kernel whose CTAs keep their rows in shared memory and
+                                   meet at grid barriers (same arithmetic; fp32 partial sums added in another order) */
 };
 
 /* Library version (major*10000 + minor*100 + patch).  No paper counterpart. */

@@ -4,7 +4,7 @@ The CUDA library is loaded on first use; nothing here computes anything on its o
 """
 from .binding import (  # noqa: F401
     CAKE_ASSIGN_AUTO, CAKE_ASSIGN_SIMT, CAKE_ASSIGN_TCGEN05, CAKE_ASSIGN_TCGEN05_EXACT, CAKE_ASSIGN_TCGEN05_PAIR, CAKE_ASSIGN_TCGEN05_PAIR_EXACT, CAKE_ERR_ALIGN, CAKE_ERR_BAD_INDEX, CAKE_ERR_CUDA,
-    CAKE_ERR_DEVICE, CAKE_LLOYD_NO_FUSE, CAKE_ERR_NULL, CAKE_ERR_SHAPE, CAKE_ERR_TIMEOUT, CAKE_ERR_UNSUPPORTED, CAKE_ERR_WORKSPACE,
+    CAKE_ERR_DEVICE, CAKE_LLOYD_NO_FUSE, CAKE_LLOYD_NO_RESIDENT, CAKE_ERR_NULL, CAKE_ERR_SHAPE, CAKE_ERR_TIMEOUT, CAKE_ERR_UNSUPPORTED, CAKE_ERR_WORKSPACE,
     CAKE_OK, CAKE_UPDATE_AUTO, CAKE_UPDATE_SLAB, CAKE_UPDATE_SLAB_F1,
     CAKE_UPDATE_SLAB_F2, CAKE_UPDATE_SLAB_F4, CAKE_UPDATE_SMEM, CAKE_UPDATE_SORT, EXPORTS, LIB_PATH, CakeError, LloydOutput,
     alloc_lloyd_outputs, alloc_workspace, cake_kmeans_assign, cake_kmeans_assign_static, cake_kmeans_assign_static_status, cake_kmeans_device_status, cake_kmeans_inertia, cake_kmeans_lloyd, cake_kmeans_lloyd_tol, cake_kmeans_init_plusplus,

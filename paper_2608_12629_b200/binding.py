@@ -24,6 +24,7 @@ CAKE_ASSIGN_TCGEN05_PAIR, CAKE_ASSIGN_TCGEN05_PAIR_EXACT = 4, 5
 CAKE_UPDATE_AUTO, CAKE_UPDATE_SMEM, CAKE_UPDATE_SORT = 0, 1 << 4, 2 << 4
 CAKE_UPDATE_SLAB, CAKE_UPDATE_SLAB_F1, CAKE_UPDATE_SLAB_F2, CAKE_UPDATE_SLAB_F4 = 3 << 4, 4 << 4, 5 << 4, 6 << 4
 CAKE_LLOYD_NO_FUSE = 1 << 8
+CAKE_LLOYD_NO_RESIDENT = 1 << 9
 
 EXPORTS = [
     "cake_version", "cake_kmeans_kernel_launches", "cake_strerror", "cake_kmeans_workspace_bytes", "cake_kmeans_assign",

@@ -426,6 +426,18 @@ int cake_kmeans_lloyd_batched(const cake_bf16* X, const cake_bf16* C0, long long
     // the partials up and divides (two launches per iteration instead of four).
     const bool try_fuse = tc_assign && !(flags & CAKE_LLOYD_NO_FUSE) && (flags & CAKE_UPDATE_MASK) == CAKE_UPDATE_AUTO &&
                           apath != CAKE_ASSIGN_TCGEN05_EXACT && fuse_shape_ok(B, D, K);
+    // ... and where the CTAs can keep all rows in shared memory, every iteration in one cooperative launch
+    if (try_fuse && !(flags & CAKE_LLOYD_NO_RESIDENT) && (apath == CAKE_ASSIGN_AUTO || apath == CAKE_ASSIGN_TCGEN05) && w.fpart) {
+        DeviceInfo di;
+        rc = current_device_info(&di);
+        if (rc != CAKE_OK) return rc;
+        if (lloyd_small_supports(di, N, D, K)) {
+            rc = launch_lloyd_small(X, C0, N, D, K, iters, w.fpart, w.fcnt, w.cbuf[0], reinterpret_cast<unsigned*>(w.status + 32),
+                                    out_C, out_C_bf16, out_idx, out_dist, out_counts, out_inertia, w.status, di, s);
+            if (rc == CAKE_OK) return rc;
+            // (a cooperative launch the device refuses: the general path below; what was enqueued so far are two clears)
+        }
+    }
     for (int t = 0; t < iters; ++t) {
         int fuse_ctas = 0;
         rc = do_assign(X, cur, Bi, N, D, K, out_idx, out_dist, out_inertia ? out_inertia + t : nullptr, iters,

@@ -150,6 +150,14 @@ cudaError_t launch_finalize_partials(const float* part_sums, const int* part_cou
                                      int K, int D, float* out_C, cake_bf16* out_C_bf16, int* out_counts,
                                      const NextAssign* next, bool* prepared, cudaStream_t s);
 
+// ---- all Lloyd iterations of a small problem in one cooperative launch (lloyd_small.cu): one problem, K <= 128,
+// D = 64 or 128, at most four 128-row tiles per SM.  part_sums [SMs][128][D], part_counts [SMs][128], cbuf [K][D] and
+// gbar (one word) are scratch; inertia (nullable) gets one entry per iteration.
+bool lloyd_small_supports(const DeviceInfo& di, i64 N, int D, int K);
+int launch_lloyd_small(const cake_bf16* X, const cake_bf16* C0, i64 N, int D, int K, int iters, float* part_sums,
+                       int* part_counts, cake_bf16* cbuf, unsigned* gbar, float* out_C, cake_bf16* out_C_bf16, int* out_idx,
+                       float* out_dist, int* out_counts, double* inertia, int* status, const DeviceInfo& di, cudaStream_t s);
+
 // ---- inertia: acc[b] += sum_i dist[b][i] (fp64 atomics); acc stride given in elements
 cudaError_t launch_inertia(const float* dist, int B, i64 N, double* acc, int acc_stride,
                            cudaStream_t s);

@@ -31,12 +31,21 @@ def test_fused_iteration_equals_two_pass_iteration_on_integer_data(N, D, K):
     launches = cake.cake_kmeans_kernel_launches() - n0
     torch.cuda.synchronize()
     assert cake.cake_kmeans_device_status(ws) == cake.CAKE_OK
-    assert launches == 1 + 2 * 4, launches                         # the first prologue, then assign + division per iteration
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    resident = D in (64, 128) and (N + 127) // 128 <= 4 * sms      # small enough for the one-launch form
+    # one cooperative launch for all iterations, or the first prologue, then assign + division per iteration
+    assert launches == (1 if resident else 1 + 2 * 4), launches
     b = cake.cake_kmeans_lloyd(Xd, Cd, 4, ws=ws, flags=cake.CAKE_LLOYD_NO_FUSE)
     assert torch.equal(a.idx, b.idx) and torch.equal(a.dist, b.dist) and torch.equal(a.counts, b.counts)
     assert torch.equal(a.C, b.C) and torch.equal(a.C_bf16, b.C_bf16)
-    np.testing.assert_allclose(a.inertia.cpu().numpy(), b.inertia.cpu().numpy(), rtol=1e-12)
+    np.testing.assert_allclose(a.inertia.cpu().numpy(), b.inertia.cpu().numpy(), rtol=1e-9)
     assert int(a.counts.sum()) == N
+    if resident:      # ... and the two-launch form of the single-pass iteration agrees with both
+        n0 = cake.cake_kmeans_kernel_launches()
+        c = cake.cake_kmeans_lloyd(Xd, Cd, 4, ws=ws, flags=cake.CAKE_LLOYD_NO_RESIDENT)
+        assert cake.cake_kmeans_kernel_launches() - n0 == 1 + 2 * 4
+        assert torch.equal(a.idx, c.idx) and torch.equal(a.dist, c.dist) and torch.equal(a.counts, c.counts)
+        assert torch.equal(a.C, c.C) and torch.equal(a.C_bf16, c.C_bf16)
 
 
 @pytest.mark.parametrize("N,D,K", [(3000, 64, 50), (32768, 64, 128), (10000, 128, 100), (5000, 40, 17)])
@@ -70,3 +79,51 @@ def test_fused_iteration_empty_clusters_keep_their_centroid_and_repeat_bit_for_b
     b = cake.cake_kmeans_lloyd(Xd, Cd, 3)
     assert torch.equal(a.idx, b.idx) and torch.equal(a.counts, b.counts)
     np.testing.assert_allclose(a.C.cpu().numpy(), b.C.cpu().numpy(), rtol=1e-5, atol=1e-6)    # fp32 summation order only
+
+
+@pytest.mark.parametrize("N,D,K", [(1, 64, 1), (300, 64, 7), (18944, 64, 128), (32768, 64, 128), (75776, 64, 100),
+                                   (40000, 128, 128), (75776, 128, 33), (5000, 128, 1)])
+def test_one_launch_form_teacher_forced_and_against_the_two_launch_form(N, D, K):
+    """All iterations in one cooperative kernel (rows resident in shared memory, grid barriers): every iteration graded by
+    the oracle (teacher-forced), the run equal to the two-launch form in assignments, and repeatable bit for bit (its
+    partial sums are added in a fixed order)."""
+    X, _ = inputs.gaussian_mixture(N, D, max(K, 2), 2.0, 1.0, N + K)
+    C0 = inputs.sample_init(X, K, N)
+    Xb = inputs.to_bits(X)
+    Xd = X.to(DEV)
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    cur = C0.to(DEV)
+    for _ in range(3):
+        n0 = cake.cake_kmeans_kernel_launches()
+        out = cake.cake_kmeans_lloyd(Xd, cur, 1, ws=ws)
+        assert cake.cake_kmeans_kernel_launches() - n0 == 1
+        assert cake.cake_kmeans_device_status(ws) == cake.CAKE_OK
+        cb = inputs.to_bits(cur)
+        idx = out.idx.cpu().numpy()
+        grading.grade_assign(Xb, cb, idx, out.dist.cpu().numpy())
+        grading.grade_update(Xb, idx, K, cb, out.C.cpu().numpy(), inputs.to_bits(out.C_bf16), out.counts.cpu().numpy())
+        assert abs(float(out.inertia[0]) - float(out.dist.double().sum())) <= 1e-9 * max(1.0, float(out.inertia[0]))
+        cur = out.C_bf16
+    a = cake.cake_kmeans_lloyd(Xd, C0.to(DEV), 5, ws=ws)
+    b = cake.cake_kmeans_lloyd(Xd, C0.to(DEV), 5, ws=ws)
+    assert torch.equal(a.idx, b.idx) and torch.equal(a.C, b.C) and torch.equal(a.C_bf16, b.C_bf16) and torch.equal(a.dist, b.dist)
+    c = cake.cake_kmeans_lloyd(Xd, C0.to(DEV), 5, ws=ws, flags=cake.CAKE_LLOYD_NO_RESIDENT)
+    torch.cuda.synchronize()
+    assert cake.cake_kmeans_device_status(ws) == cake.CAKE_OK
+    assert (a.idx != c.idx).float().mean().item() <= 1e-3           # (fp32 sums in another order: a near-tie may flip)
+    np.testing.assert_allclose(a.inertia.cpu().numpy(), c.inertia.cpu().numpy(), rtol=1e-4)
+
+
+def test_one_launch_form_without_optional_outputs_and_through_the_tolerance_loop():
+    N, D, K = 20000, 64, 50
+    X, _ = inputs.gaussian_mixture(N, D, K, 2.0, 1.0, 9)
+    C0 = inputs.sample_init(X, K, 9)
+    Xd, Cd = X.to(DEV), C0.to(DEV)
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    ref = cake.cake_kmeans_lloyd(Xd, Cd, 6, ws=ws)
+    tol, iters = cake.cake_kmeans_lloyd_tol(Xd, Cd, 6, 0.0, check_every=2, ws=ws)
+    torch.cuda.synchronize()
+    assert cake.cake_kmeans_device_status(ws) == cake.CAKE_OK
+    assert iters == 6 and torch.equal(tol.idx, ref.idx) and torch.equal(tol.C_bf16, ref.C_bf16)
+    np.testing.assert_allclose(tol.inertia.cpu().numpy()[:6], ref.inertia.cpu().numpy(), rtol=1e-9)
+    assert (np.diff(ref.inertia.cpu().numpy()) <= 0).all()
