@@ -94,7 +94,7 @@ enum {
                                    the assign kernel adds each row tile to per-cluster sums on the tensor core
                                    (sums += onehot^T X) while the tile is in shared memory                      */
     CAKE_LLOYD_NO_RESIDENT = 1 << 9 /* lloyd: do not take the one-launch form of the single-pass iteration, which a
-                                   problem of D = 64 or 128 and at most four 128-row tiles per SM runs in: all
+                                   problem of D <= 128 (D % 8 == 0) and at most four 128-row tiles per SM runs in: all
                                    iterations in one cooperative kernel whose CTAs keep their rows in shared memory and
                                    meet at grid barriers (same arithmetic; fp32 partial sums added in another order) */
 };

@@ -151,7 +151,7 @@ cudaError_t launch_finalize_partials(const float* part_sums, const int* part_cou
                                      const NextAssign* next, bool* prepared, cudaStream_t s);
 
 // ---- all Lloyd iterations of a small problem in one cooperative launch (lloyd_small.cu): one problem, K <= 128,
-// D = 64 or 128, at most four 128-row tiles per SM.  part_sums [SMs][128][D], part_counts [SMs][128], cbuf [K][D] and
+// D <= 128 (D % 8 == 0), at most four 128-row tiles per SM.  part_sums [SMs][128][round_up(D, 16)], part_counts [SMs][128], cbuf [K][D] and
 // gbar (one word) are scratch; inertia (nullable) gets one entry per iteration.
 bool lloyd_small_supports(const DeviceInfo& di, i64 N, int D, int K);
 int launch_lloyd_small(const cake_bf16* X, const cake_bf16* C0, i64 N, int D, int K, int iters, float* part_sums,

@@ -1,7 +1,7 @@
 // Lloyd iterations of a SMALL problem in one kernel launch (paper Section 5, "Flash-KMeans clean-start workload": the
 // assignment and update steps of every iteration; Appendix F lists a single-pass "gap-fused" route for the iteration).
 //
-// One problem, at most 128 clusters, D = 64 or 128, and few enough rows that every CTA can keep its row tiles in
+// One problem, at most 128 clusters, D <= 128 (a multiple of 8), and few enough rows that every CTA can keep its row tiles in
 // shared memory for the whole call (at most four 128-row tiles per SM).  Such problems are bound by launch and set-up
 // latency, not by arithmetic: the two-kernel iteration of the general path costs about 14 us there, of which the
 // tensor pipe works for less than one.  Here one cooperative launch runs all iterations:
@@ -42,10 +42,11 @@ struct Params {
     const cake_bf16* C0;      // [K][D] initial centroids
     i64 N;
     int D, K, iters;
-    int nchunks;              // D / 64
+    int nchunks;              // ceil(D / 64): columns D .. 64 nchunks - 1 of the tiles are zeros
+    int ncol;                 // D rounded up to 16: columns of the sums (the update MMA's N), pitch of the partial sums
     int c_rows;               // K rounded up to 32: columns of an accumulator
     int tiles;                // ceil(N / 128)
-    float* part_sums;         // [grid][128][D] per-CTA partial sums
+    float* part_sums;         // [grid][128][ncol] per-CTA partial sums
     int* part_counts;         // [grid][128]
     cake_bf16* cbuf;          // [K][D] the centroids between iterations
     float* out_C;             // [K][D] fp32, may be null
@@ -65,6 +66,7 @@ struct Ctrl {
     int cnt[128];             // rows per cluster (this CTA, this iteration)
     float4 red[THREADS];      // finalize: partial rows per stripe
     int cred[THREADS];
+    double dred[4];           // the warps' shares of the iteration's inertia
 };
 static_assert(sizeof(Ctrl) <= 4096, "control block");
 
@@ -161,6 +163,9 @@ lloyd_small_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
     // zeros: columns 8..15 of the operands of the extra k-step, and the one-hot operand (kept up to date element by element)
     for (uint32_t o = tid * 16; o < ZERO_BYTES; o += THREADS * 16) *reinterpret_cast<uint4*>(smem + zero_off + o) = make_uint4(0, 0, 0, 0);
     for (uint32_t o = tid * 16; o < OH_BYTES; o += THREADS * 16) *reinterpret_cast<uint4*>(smem + oh_off + o) = make_uint4(0, 0, 0, 0);
+    // (the centroid tile too: the granules behind column D of its last chunk are never written and must read as zeros)
+    for (uint32_t o = tid * 16; o < static_cast<uint32_t>(p.nchunks) * C_CHUNK_BYTES; o += THREADS * 16)
+        *reinterpret_cast<uint4*>(smem + c_off + o) = make_uint4(0, 0, 0, 0);
     ptx::fence_proxy_async_smem();
     if (warp == 0) {
         ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), TMEM_COLS);
@@ -218,7 +223,7 @@ lloyd_small_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
     constexpr uint32_t KSTEP = (UMMA_K * 2) >> 4;
     const uint32_t idesc_aug = ptx::umma_idesc_bf16(BLOCK_M, p.c_rows);
     const uint32_t idesc_main = idesc_aug | ptx::UMMA_IDESC_NEGATE_B;   // accumulates -x.c
-    const uint32_t idesc_upd = ptx::umma_idesc_bf16(BLOCK_M, p.D) | ptx::UMMA_IDESC_B_MN_MAJOR;
+    const uint32_t idesc_upd = ptx::umma_idesc_bf16(BLOCK_M, p.ncol) | ptx::UMMA_IDESC_B_MN_MAJOR;
     uint32_t ph0 = 0, ph1 = 0, upd_n = 0;                      // completed uses of the barriers
     unsigned gb = 0;
     int prev_oh = -1;                                          // the cluster whose one-hot entry this row has set
@@ -374,8 +379,8 @@ lloyd_small_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
         wait_bar(&ctrl->bar_upd, (upd_n - 1u) & 1u, ctrl, p.status);
         ptx::tc_fence_after();
         {
-            float* dst = p.part_sums + (static_cast<size_t>(blockIdx.x) * 128 + tid) * p.D;
-            for (int c0 = 0; c0 < p.D; c0 += 16) {
+            float* dst = p.part_sums + (static_cast<size_t>(blockIdx.x) * 128 + tid) * p.ncol;
+            for (int c0 = 0; c0 < p.ncol; c0 += 16) {
                 uint32_t v[16];
                 ptx::tmem_ld_x16(tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + SUMS_COL + c0, v);
 #pragma unroll
@@ -384,25 +389,27 @@ lloyd_small_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
             p.part_counts[static_cast<size_t>(blockIdx.x) * 128 + tid] = ctrl->cnt[tid];
         }
         ptx::tc_fence_before();
-        if (p.inertia) {
+        if (p.inertia) {   // one fp64 atomic per CTA and iteration
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
-            if (lane == 0) atomicAdd(p.inertia + it, dsum);
+            if (lane == 0) ctrl->dred[warp] = dsum;
+            __syncthreads();
+            if (tid == 0) atomicAdd(p.inertia + it, (ctrl->dred[0] + ctrl->dred[1]) + (ctrl->dred[2] + ctrl->dred[3]));
         }
         grid_barrier(p.gbar, gb++, ctrl, p.status);
 
-        // ---- division: cluster k by CTA k mod grid.  Thread = (stripe of partials, column quad); the first warp adds the
-        // stripes up, divides (an empty cluster keeps its previous centroid) and writes fp32 and bf16 (RNE) centroids.
+        // ---- division: cluster k by CTA k mod grid.  Thread = (stripe of partials, column quad), the threads behind the
+        // last whole stripe idle; the first warp adds the stripes up, divides (an empty cluster keeps its previous centroid) and writes fp32 and bf16 (RNE) centroids.
         const int D4 = p.D >> 2, stripes = THREADS / D4;
         const int n_part = static_cast<int>(gridDim.x);
         for (int k = blockIdx.x; k < p.K; k += gridDim.x) {
             const int col = tid % D4, stripe = tid / D4;
             // (all loads of a stripe are requested before the first is added: the loop is a chain of L2 latencies otherwise)
             float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            const float4* prow = reinterpret_cast<const float4*>(p.part_sums + static_cast<size_t>(k) * p.D) + col;
-            const size_t pstep = static_cast<size_t>(128) * p.D / 4;
+            const float4* prow = reinterpret_cast<const float4*>(p.part_sums + static_cast<size_t>(k) * p.ncol) + col;
+            const size_t pstep = static_cast<size_t>(128) * p.ncol / 4;
             constexpr int BATCH = 20;   // (148 partials over 8 stripes: one batch)
-            for (int q0 = stripe; q0 < n_part; q0 += BATCH * stripes) {
+            for (int q0 = stripe; stripe < stripes && q0 < n_part; q0 += BATCH * stripes) {
                 float4 v[BATCH];
 #pragma unroll
                 for (int u = 0; u < BATCH; ++u) {
@@ -469,17 +476,17 @@ size_t small_smem_bytes(int R, int nchunks) {
 }
 }  // namespace
 
-// One problem of at most 128 clusters, D = 64 or 128, whose row tiles fit four to an SM.
+// One problem of at most 128 clusters, D <= 128 (a multiple of 8), whose row tiles fit four to an SM.
 bool lloyd_small_supports(const DeviceInfo& di, i64 N, int D, int K) {
-    if (di.cc_major != 10 || N < 1 || K < 1 || K > 128 || (D != 64 && D != 128)) return false;
+    if (di.cc_major != 10 || N < 1 || K < 1 || K > 128 || D < 8 || D > 128 || D % 8 != 0) return false;
     const i64 tiles = (N + BLOCK_M - 1) / BLOCK_M;
     if (tiles > static_cast<i64>(MAX_R) * di.sm_count) return false;
     const int grid = static_cast<int>(tiles < di.sm_count ? tiles : di.sm_count);
     const int R = static_cast<int>((tiles + grid - 1) / grid);
-    return small_smem_bytes(R, D / KCHUNK) <= static_cast<size_t>(di.smem_optin);
+    return small_smem_bytes(R, (D + KCHUNK - 1) / KCHUNK) <= static_cast<size_t>(di.smem_optin);
 }
 
-// part_sums [grid][128][D] fp32, part_counts [grid][128] int, cbuf [K][D] bf16 and gbar (one word) are scratch; inertia
+// part_sums [grid][128][round_up(D, 16)] fp32, part_counts [grid][128] int, cbuf [K][D] bf16 and gbar (one word) are scratch; inertia
 // (nullable) has one entry per iteration.  Everything is enqueued on `s`: two small clears and one cooperative launch.
 int launch_lloyd_small(const cake_bf16* X, const cake_bf16* C0, i64 N, int D, int K, int iters, float* part_sums,
                        int* part_counts, cake_bf16* cbuf, unsigned* gbar, float* out_C, cake_bf16* out_C_bf16, int* out_idx,
@@ -487,7 +494,8 @@ int launch_lloyd_small(const cake_bf16* X, const cake_bf16* C0, i64 N, int D, in
     if (!lloyd_small_supports(di, N, D, K) || iters < 1) return CAKE_ERR_UNSUPPORTED;
     Params p;
     p.C0 = C0; p.N = N; p.D = D; p.K = K; p.iters = iters;
-    p.nchunks = D / KCHUNK;
+    p.nchunks = (D + KCHUNK - 1) / KCHUNK;
+    p.ncol = static_cast<int>(round_up(D, 16));
     p.c_rows = static_cast<int>(round_up(K, 32));
     p.tiles = static_cast<int>((N + BLOCK_M - 1) / BLOCK_M);
     p.part_sums = part_sums; p.part_counts = part_counts; p.cbuf = cbuf;

@@ -32,7 +32,7 @@ def test_fused_iteration_equals_two_pass_iteration_on_integer_data(N, D, K):
     torch.cuda.synchronize()
     assert cake.cake_kmeans_device_status(ws) == cake.CAKE_OK
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    resident = D in (64, 128) and (N + 127) // 128 <= 4 * sms      # small enough for the one-launch form
+    resident = (N + 127) // 128 <= 4 * sms                         # small enough for the one-launch form
     # one cooperative launch for all iterations, or the first prologue, then assign + division per iteration
     assert launches == (1 if resident else 1 + 2 * 4), launches
     b = cake.cake_kmeans_lloyd(Xd, Cd, 4, ws=ws, flags=cake.CAKE_LLOYD_NO_FUSE)
@@ -82,7 +82,8 @@ def test_fused_iteration_empty_clusters_keep_their_centroid_and_repeat_bit_for_b
 
 
 @pytest.mark.parametrize("N,D,K", [(1, 64, 1), (300, 64, 7), (18944, 64, 128), (32768, 64, 128), (75776, 64, 100),
-                                   (40000, 128, 128), (75776, 128, 33), (5000, 128, 1)])
+                                   (40000, 128, 128), (75776, 128, 33), (5000, 128, 1), (9000, 8, 5), (30000, 24, 40),
+                                   (50000, 32, 128), (20000, 72, 100), (60000, 96, 77), (33333, 120, 128)])
 def test_one_launch_form_teacher_forced_and_against_the_two_launch_form(N, D, K):
     """All iterations in one cooperative kernel (rows resident in shared memory, grid barriers): every iteration graded by
     the oracle (teacher-forced), the run equal to the two-launch form in assignments, and repeatable bit for bit (its
