@@ -156,6 +156,21 @@ struct Ctrl {  // lives in shared memory
 };
 static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
 
+#ifdef CAKE_ASSIGN_ACC
+// Profiling build only (-DCAKE_ASSIGN_ACC): clocks spent in sections of CTA 0's issuing threads, added up in registers
+__device__ long long g_acc[32];
+#define ACC_DECL(v) long long v = 0
+#define ACC_T(v) const long long v = clock64()
+#define ACC_SUM(v, d) v += (d)
+#define ACC_SET(v, d) v = (d)
+#define ACC_DUMP(slot, v) do { if (blockIdx.x == 0) g_acc[slot] = v; } while (0)
+#else
+#define ACC_DECL(v) ((void)0)
+#define ACC_T(v) ((void)0)
+#define ACC_SUM(v, d) ((void)0)
+#define ACC_SET(v, d) ((void)0)
+#define ACC_DUMP(slot, v) ((void)0)
+#endif
 #ifdef CAKE_ASSIGN_TRACE
 // Profiling build only (-DCAKE_ASSIGN_TRACE): CTA 0 logs every barrier wait of its warp leaders as
 // {barrier slot in Ctrl, start clock, end clock} per warp; read back with cake_debug_read_trace.
@@ -354,7 +369,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             ptx::mbar_init(ptx::smem_u32(&ctrl->x_full[i]), 1);
             // MMA issuers + 4 norm warps + the 4 epilogue warps that read the row margins
             // (TOPK: the upper column half reads the margins as well)
-            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]), ((XLOAD && p.res_c == 1) ? 1 : NUM_ISSUERS) + 4 + 4 + (TOPK ? 4 : 0));
+            // (one resident tile, whole X buffers: the epilogue's arrival comes after the accumulator is complete and stands
+            // for the MMAs as well; FUSE: the thread that issues the update commits)
+            ptx::mbar_init(ptx::smem_u32(&ctrl->x_empty[i]),
+                           ((XLOAD && p.res_c == 1) ? ((XSPLIT || FUSE) ? 1 : 0) : NUM_ISSUERS) + 4 + 4 + (TOPK ? 4 : 0));
             ptx::mbar_init(ptx::smem_u32(&ctrl->auga_full[i]), 4);
         }
         for (int i = 0; i < MAX_XCHUNKS; ++i) {
@@ -640,11 +658,88 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 int cur_b = -1;
                 uint32_t pc = 0, tile_it = 0;
                 int tb, tmt;
+                ACC_DECL(acc_main); ACC_DECL(acc_tail); ACC_DECL(acc_n); ACC_DECL(acc_all);
+                ACC_DECL(acc_top); ACC_DECL(acc_xf); ACC_DECL(acc_pre); ACC_DECL(t_prev);
+                ACC_T(t_loop0);
                 first_tile<CONSEC>(p, tb, tmt);
                 const int tmt_step = tile_step<CONSEC>();
                 const uint32_t nxb = static_cast<uint32_t>(p.n_xbuf);
                 const uint32_t idesc_aug_n = ptx::umma_idesc_bf16(BLOCK_M, p.alt_epi ? p.alt_epi : BLOCK_N);
                 const uint32_t idesc_main_n = idesc_aug_n | ptx::UMMA_IDESC_NEGATE_B;
+                if (!XSPLIT && !FUSE && p.res_c == 1) {
+                    // One resident tile, whole X buffers (the fused update keeps the general loop below: it measured 3 % faster there): this loop is the thread's whole life and every row tile passes
+                    // through it, so it does as little as it can.  Buffer, phases and descriptors are stepped (no
+                    // divisions); one wait covers X and its half-norm operand (the norm warps arrive on it after they
+                    // have seen the X tile); the X buffer is handed back by the epilogue warpgroup once the accumulator
+                    // is complete, not by a commit of this thread.
+                    const uint32_t n_my = static_cast<uint32_t>((p.total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+                    const uint32_t d_tmem = tmem_base + iss * BLOCK_N;
+                    const uint32_t b0 = ptx::umma_desc_lo_sw128(ring_base);
+                    const uint32_t b_step = p.stage_bytes >> 4;
+                    const uint32_t augb_lo = ptx::umma_desc_lo_aug(ring_base + res_tile_bytes - AUG_B_BYTES, smem_base + zero_off);
+                    const int turn_c = (p.nchunks - 1) >> 1;   // the turn goes on after the first half of the MMAs
+                    uint32_t rxb = iss, rxph = 0, k_own = 0;   // this issuer's X buffer and phase, its own tiles so far
+                    for (; ok && tile_it < n_my; ++tile_it) {
+                        const int b_now = tb;
+                        tmt += tmt_step;
+                        while (tmt >= p.m_tiles) { tmt -= p.m_tiles; ++tb; }
+                        if (b_now != cur_b) {
+                            if (cur_b >= 0) ptx::umma_commit(ptx::smem_u32(&ctrl->ring_empty[0]));
+                            ok = wait_bar(&ctrl->ring_full[0], pc & 1u, ctrl, p.status);
+                            if (!ok) break;
+                            cur_b = b_now;
+                            ++pc;
+                        }
+                        if ((tile_it & 1u) != iss) continue;
+                        ACC_T(t_0);
+                        ACC_SUM(acc_top, t_prev ? t_0 - t_prev : 0);
+                        ok = wait_bar(&ctrl->auga_full[rxb], rxph, ctrl, p.status);
+                        if (!ok) break;
+                        ACC_T(t_1);
+                        if (k_own > 0u) {
+                            ok = wait_bar(&ctrl->tmem_empty[iss][iss], (k_own - 1u) & 1u, ctrl, p.status);
+                            if (!ok) break;
+                        }
+                        // (the issuers take turns, see below: issuer 0 waits for issuer 1's previous tile, issuer 1 for
+                        // issuer 0's current one)
+                        if (iss == 1u || k_own > 0u) {
+                            ok = wait_bar(&ctrl->turn[iss], (iss == 1u ? k_own : k_own - 1u) & 1u, ctrl, p.status);
+                            if (!ok) break;
+                        }
+                        ptx::tc_fence_after();
+                        ACC_T(t_a);
+                        uint32_t a_lo = ptx::umma_desc_lo_sw128(x_base + rxb * xbuf_bytes), b_lo = b0;
+                        for (int c = 0; c < p.nchunks; ++c, a_lo += X_CHUNK_BYTES >> 4, b_lo += b_step) {
+                            if (c == 0)
+                                ptx::umma_bf16_lohi<false>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo, ptx::UMMA_DESC_HI_SW128, idesc_main_n);
+                            else
+                                ptx::umma_bf16_lohi<true>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo, ptx::UMMA_DESC_HI_SW128, idesc_main_n);
+                            if (c < p.nchunks - 1 || p.ksteps_last == KCHUNK / UMMA_K) {   // a whole chunk: straight-line code
+#pragma unroll
+                                for (int ks = 1; ks < KCHUNK / UMMA_K; ++ks)
+                                    ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
+                                                              b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main_n);
+                            } else {
+                                for (int ks = 1; ks < p.ksteps_last; ++ks)
+                                    ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
+                                                              b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main_n);
+                            }
+                            if (c == turn_c) ptx::mbar_arrive(ptx::smem_u32(&ctrl->turn[iss ^ 1u]));
+                        }
+                        ACC_T(t_b);
+                        ptx::umma_bf16_lohi<true>(d_tmem,
+                                                  ptx::umma_desc_lo_aug(smem_base + auga_off + rxb * AUG_A_BYTES, smem_base + zero_off),
+                                                  ptx::UMMA_DESC_HI_AUG, augb_lo, ptx::UMMA_DESC_HI_AUG, idesc_aug_n);
+                        ptx::umma_commit(ptx::smem_u32(&ctrl->tmem_full[iss]));
+                        ACC_T(t_c);
+                        ACC_SUM(acc_main, t_b - t_a); ACC_SUM(acc_tail, t_c - t_b); ACC_SUM(acc_n, 1);
+                        ACC_SUM(acc_xf, t_1 - t_0); ACC_SUM(acc_pre, t_a - t_1);
+                        ACC_SET(t_prev, t_c);
+                        ++k_own;
+                        rxb += 2u;
+                        if (rxb >= nxb) { rxb -= nxb; rxph ^= 1u; }
+                    }
+                } else
                 for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it) {
                     const int b_now = tb;
                     tmt += tmt_step;
@@ -699,9 +794,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         else
                             ptx::umma_bf16_lohi<true>(d_tmem, a_lo, ptx::UMMA_DESC_HI_SW128, b_lo,
                                                       ptx::UMMA_DESC_HI_SW128, idesc_main_n);
-                        for (int ks = 1; ks < nk; ++ks)
-                            ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
-                                                      b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main_n);
+                        if (nk == KCHUNK / UMMA_K) {   // a whole chunk: straight-line code
+#pragma unroll
+                            for (int ks = 1; ks < KCHUNK / UMMA_K; ++ks)
+                                ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
+                                                          b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main_n);
+                        } else {
+                            for (int ks = 1; ks < nk; ++ks)
+                                ptx::umma_bf16_lohi<true>(d_tmem, a_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128,
+                                                          b_lo + ks * KSTEP, ptx::UMMA_DESC_HI_SW128, idesc_main_n);
+                        }
                         if (XSPLIT && c < p.nchunks - 1) ptx::umma_commit(ptx::smem_u32(&ctrl->xc_empty[c]));
                     }
                     if (!ok) break;
@@ -719,6 +821,10 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     // issues those hands the buffer back)
                     if (!FUSE) ptx::umma_commit(ptx::smem_u32(&ctrl->x_empty[rxb]));
                 }
+                ACC_T(t_loop1);
+                ACC_SUM(acc_all, t_loop1 - t_loop0);
+                ACC_DUMP(iss * 8 + 0, acc_main); ACC_DUMP(iss * 8 + 1, acc_tail); ACC_DUMP(iss * 8 + 2, acc_n); ACC_DUMP(iss * 8 + 3, acc_all);
+                ACC_DUMP(iss * 8 + 4, acc_top); ACC_DUMP(iss * 8 + 5, acc_xf); ACC_DUMP(iss * 8 + 6, acc_pre);
             } else
             for (i64 tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 // every phase of the shared barriers is observed, also in row / centroid tiles this
@@ -934,11 +1040,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 if (!ok) break;
                 rowM = ctrl->row_m[axb][r];
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
+                if (FUSE && lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
             }
             const uint32_t as = tile_it & 1u, aph = (tile_it >> 1) & 1u;
             ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
             if (!ok) break;
+            // (the MMAs that read the X buffer are complete: this arrival hands it back for them as well)
+            if (!XSPLIT && !FUSE && lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
             if (XSPLIT) {
                 // one X buffer for both warpgroups: this one sees only every other phase of its barriers, so it
                 // reads the margins once its accumulator is complete (the issuer waited for them)
@@ -1470,6 +1578,13 @@ int make_tmap_rows16(CUtensorMap* m, const void* base, i64 rows, int box_rows) {
     return r == CUDA_SUCCESS ? CAKE_OK : CAKE_ERR_CUDA;
 }
 
+#ifdef CAKE_ASSIGN_ACC
+extern "C" __attribute__((visibility("default"))) int cake_debug_read_acc(long long* host) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(host, g_acc, sizeof(long long) * 32);
+    return 32;
+}
+#endif
 #ifdef CAKE_ASSIGN_TRACE
 // Profiling build only: copies warp `w`'s trace records (3 x int64 each, up to `cap`) to `host`.
 extern "C" __attribute__((visibility("default"))) int cake_debug_read_trace(int w, long long* host, int cap) {
