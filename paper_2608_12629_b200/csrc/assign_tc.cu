@@ -84,6 +84,9 @@ constexpr uint32_t OH_BYTES = 128 * 128 * 2;             // FUSE: the one-hot op
 constexpr int MAX_STAGES = 6;
 constexpr int MAX_XBUF = 6;                              // (more than four only in the fused mode)
 constexpr int MAX_XBUF_PLAIN = 4;
+#ifndef GATE_MIN_TILES
+#define GATE_MIN_TILES 64                                 // centroid tiles per row tile from which the gated epilogue is used
+#endif
 constexpr int MAX_XCHUNKS = 8;                           // 64-column chunks of an X tile (D <= 512)
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t CTRL_BYTES = 6144;  // barriers, TMEM pointer, abort flag, merge scratch, row margins
@@ -260,6 +263,25 @@ __device__ __forceinline__ float packed_min32(const uint32_t (&r)[32], int col_b
     return fminf(run, min32(v));
 }
 
+// GATE: the group's smallest accumulator first, with 3-input minima on the raw values (half an instruction per column);
+// the keys are built and reduced (another 1.1 per column) only if some row of the warp can still improve on `thr`, the
+// truncated value of its best key before this tile.  Same result as without the gate: a group whose smallest truncated
+// value is not below thr cannot replace the best (across tiles an equal value keeps the earlier tile), and leaving it
+// out of the tile's minimum changes nothing else, since what remains is then not below thr either.  After t tiles a
+// group still passes with probability about 1 - exp(-8 / t) on unordered centroids: worth it from 64 tiles on.
+template <bool GATE>
+__device__ __forceinline__ float group_min32(const uint32_t (&r)[32], int col_base, float run, float thr, uint32_t kmask) {
+    if (GATE) {
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+        const float g = min32(v);
+        const bool want = __uint_as_float(__float_as_uint(g) & kmask) < thr;
+        if (!__any_sync(0xffffffffu, want)) return run;
+    }
+    return packed_min32(r, col_base, run, kmask);
+}
+
 // exact policy: full-precision group minimum; position looked up (lowest column first) only on a hit.
 __device__ __forceinline__ void exact_scan32(const uint32_t (&r)[32], int col_base, float& best, int& bidx) {
     float v[32];
@@ -335,7 +357,7 @@ __device__ __forceinline__ int tile_step() { return CONSEC ? 1 : static_cast<int
 // beside the 256-column epilogue) spills 64 registers and ran 25-35 % slower at 64 < K <= 128; it remains for the
 // exact policy, the split X buffer and the fused update (where it is the only branch and does not spill).
 template <bool PACKED, bool XLOAD, bool CONSEC = false, bool XSPLIT = false, bool BULK = false, int TOPK = 0, bool FUSE = false,
-          bool NARROW = false>
+          bool NARROW = false, bool GATE = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_c,
                  const Params p) {
@@ -1336,20 +1358,21 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     ptx::tmem_ld_wait(ra);
                     ptx::tmem_ld_x32_before(taddr + 32, rb, ra);
                     if (PACKED) {
-                        float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
+                        const float thr = __uint_as_float(__float_as_uint(best) & ~COL_MASK);
+                        float tmin = group_min32<GATE>(ra, 0, __uint_as_float(F32_INF), thr, kmask);
                         ptx::tmem_ld_wait_after(rb, tmin);
                         ptx::tmem_ld_x32_before(taddr + 64, ra, rb);
-                        tmin = packed_min32(rb, 32, tmin, kmask);
+                        tmin = group_min32<GATE>(rb, 32, tmin, thr, kmask);
                         ptx::tmem_ld_wait_after(ra, tmin);
                         ptx::tmem_ld_x32_before(taddr + 96, rb, ra);
-                        tmin = packed_min32(ra, 64, tmin, kmask);
+                        tmin = group_min32<GATE>(ra, 64, tmin, thr, kmask);
                         ptx::tmem_ld_wait_after(rb, tmin);
                         ptx::tc_fence_before();
                         __syncwarp();
                         // to the issuer of tile acc_it + 2, which takes this accumulator next
                         if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
                         trace_mark(ctrl, 100);
-                        tmin = packed_min32(rb, 96, tmin, kmask);
+                        tmin = group_min32<GATE>(rb, 96, tmin, thr, kmask);
                         // across tiles only the (truncated) value decides: an equal value keeps the earlier tile
                         if (__uint_as_float(__float_as_uint(tmin) & ~COL_MASK) <
                             __uint_as_float(__float_as_uint(best) & ~COL_MASK)) {
@@ -1390,10 +1413,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
                     trace_mark(ctrl, 100);
                     if (PACKED) {
-                        float tmin = packed_min32(ra, 0, __uint_as_float(F32_INF), kmask);
-                        tmin = packed_min32(rb, 32, tmin, kmask);
-                        tmin = packed_min32(rc, 64, tmin, kmask);
-                        tmin = packed_min32(rd, 96, tmin, kmask);
+                        const float thr = __uint_as_float(__float_as_uint(best) & ~COL_MASK);
+                        float tmin = group_min32<GATE>(ra, 0, __uint_as_float(F32_INF), thr, kmask);
+                        tmin = group_min32<GATE>(rb, 32, tmin, thr, kmask);
+                        tmin = group_min32<GATE>(rc, 64, tmin, thr, kmask);
+                        tmin = group_min32<GATE>(rd, 96, tmin, thr, kmask);
                         if (__uint_as_float(__float_as_uint(tmin) & ~COL_MASK) <
                             __uint_as_float(__float_as_uint(best) & ~COL_MASK)) {
                             best = tmin;
@@ -1802,6 +1826,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
         kernel = assign_tc_kernel<true, true, false, false, false, 0, true>;
     else if (knn_k > 0)
         kernel = knn_k == 8 ? assign_tc_kernel<true, false, false, false, false, 8> : assign_tc_kernel<true, false, false, false, false, 32>;
+    else if (!xload && !exact && p.n_tiles >= GATE_MIN_TILES)   // (see group_min32)
+        kernel = bulk ? assign_tc_kernel<true, false, false, false, true, 0, false, false, true>
+                      : assign_tc_kernel<true, false, false, false, false, 0, false, false, true>;
     else if (!xload)
         kernel = exact ? (bulk ? assign_tc_kernel<false, false, false, false, true> : assign_tc_kernel<false, false>)
                        : (bulk ? assign_tc_kernel<true, false, false, false, true> : assign_tc_kernel<true, false>);
@@ -1835,7 +1862,9 @@ int launch_assign_tc(const cake_bf16* X, const cake_bf16* C, int B, i64 N, int D
             cudaFuncSetAttribute(assign_tc_kernel<true, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<false, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
             cudaFuncSetAttribute(assign_tc_kernel<true, true, true, false, false, 0, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
-            cudaFuncSetAttribute(assign_tc_kernel<true, true, false, false, false, 0, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
+            cudaFuncSetAttribute(assign_tc_kernel<true, true, false, false, false, 0, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, false, false, false, true, 0, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess ||
+            cudaFuncSetAttribute(assign_tc_kernel<true, false, false, false, false, 0, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, di.smem_optin) != cudaSuccess)
             return CAKE_ERR_CUDA;
         if (attr_known) attr_done[di.device] = true;
     }

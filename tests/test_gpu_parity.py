@@ -166,6 +166,38 @@ def test_assign_many_row_tiles_few_centroids_and_single_buffer_shapes():
         grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx.cpu().numpy(), dist.cpu().numpy(), rows=rows)
 
 
+@pytest.mark.parametrize("N,D,K,order", [(3000, 64, 16384, "random"), (2500, 32, 20000, "random"), (1500, 128, 33000, "random"),
+                                         (1200, 200, 16400, "random"), (1000, 256, 16500, "random"),
+                                         (2000, 64, 16384, "closer_later"), (2000, 128, 16384, "closer_later"),
+                                         (2000, 64, 16384, "duplicates"), (1500, 128, 20000, "duplicates")])
+def test_assign_gated_epilogue_from_64_centroid_tiles(N, D, K, order):
+    """From 64 centroid tiles per row tile the epilogue first takes a 32-column group's smallest raw accumulator and
+    builds the keys only where some row can still improve.  Graded by the oracle, and bit-identical to the CTA-pair
+    kernel, which has the same arithmetic and no gate: on unordered centroids, on centroids ordered so that later tiles
+    keep winning (every group passes the gate), and with every centroid repeated half the table later (an equal value
+    in a later tile must not replace the earlier one)."""
+    both, _ = inputs.gaussian_mixture(N + K, D, 48, 1.0, 0.5, N + K + D)
+    X, C = both[:N].contiguous(), both[N:].contiguous()
+    if order == "closer_later":
+        far = ((C.float() - X.float().mean(0)) ** 2).sum(1)
+        C = C[torch.argsort(far, descending=True)].contiguous()
+    if order == "duplicates":
+        g = torch.Generator().manual_seed(K)
+        X = torch.randint(-3, 4, (N, D), generator=g).to(torch.bfloat16)
+        C = torch.randint(-3, 4, (K, D), generator=g).to(torch.bfloat16)
+        C[K // 2:] = C[:K - K // 2]
+    Xd, Cd = X.to(DEV), C.to(DEV)
+    ws = cake.alloc_workspace(1, N, D, K, DEV)
+    idx, dist = cake.cake_kmeans_assign(Xd, Cd, ws=ws, flags=cake.CAKE_ASSIGN_TCGEN05)
+    check_status(ws)
+    grading.grade_assign(inputs.to_bits(X), inputs.to_bits(C), idx.cpu().numpy(), dist.cpu().numpy())
+    ip, dp = cake.cake_kmeans_assign(Xd, Cd, ws=ws, flags=cake.CAKE_ASSIGN_TCGEN05_PAIR)
+    check_status(ws)
+    assert torch.equal(idx, ip) and torch.equal(dist, dp)
+    if order == "duplicates":
+        assert int(idx.max()) < K - K // 2                      # the first copy of the winning centroid
+
+
 def test_assign_edge_cases():
     X, C = problem(64, 64, 4, seed=1)
     # N = 0
