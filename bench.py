@@ -299,7 +299,11 @@ def run_sweep(args):
                 C0 = inputs.sample_init(X, K, w.seed)
                 ws = cake.alloc_workspace(1, N, D, K, dev)
                 out = cake.alloc_lloyd_outputs(X, C0, w.iters)
-                cake.cake_kmeans_lloyd(X, C0, 1, out=cake.alloc_lloyd_outputs(X, C0, 1), ws=ws)      # warm-up
+                wo = cake.alloc_lloyd_outputs(X, C0, 1)
+                cake.cake_kmeans_lloyd(X, C0, 1, out=wo, ws=ws)      # warm-up: the loop, and the two kernels timed one by one
+                cake.cake_kmeans_assign(X, C0, out_idx=wo.idx, out_dist=wo.dist, ws=ws)
+                cake.cake_kmeans_update(X, wo.idx, K, C_prev=C0, out_C=wo.C, out_C_bf16=wo.C_bf16, out_counts=wo.counts, ws=ws)
+                del wo
                 e[0].record()
                 cake.cake_kmeans_lloyd(X, C0, w.iters, out=out, ws=ws)
                 e[1].record()
