@@ -1046,36 +1046,38 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // accumulator (two passes of 128), so nothing is merged through shared memory and neither
         // warpgroup ever waits for the other; with an even number of X buffers each warpgroup sees every
         // phase of the barriers of "its" buffers.
-        for (i64 tile = blockIdx.x; XLOAD && p.alt_epi && ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
-            if ((tile_it & 1u) != static_cast<uint32_t>(wg)) continue;
+        // (this warpgroup's X buffer is stepped, not divided out of the tile count: the loop is the warpgroup's critical
+        // path; with a single buffer -- XSPLIT -- it is not used)
+        uint32_t axb = static_cast<uint32_t>(wg) % static_cast<uint32_t>(p.n_xbuf);
+        ACC_DECL(ea_n); ACC_DECL(ea_w1); ACC_DECL(ea_w2); ACC_DECL(ea_red); ACC_DECL(ea_st); ACC_DECL(ea_w3); ACC_DECL(ea_oh); ACC_DECL(ea_top); ACC_DECL(ea_prev);
+        // (the loop walks this warpgroup's own tiles only: every other one of the CTA's)
+        if (XLOAD && p.alt_epi) {
+        const uint32_t n_alt = static_cast<uint32_t>((p.total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+        if (wg == 1) next_tile();
+        for (tile_it = static_cast<uint32_t>(wg); ok && tile_it < n_alt; tile_it += 2u, next_tile(), next_tile()) {
+            ACC_T(e_0);
+            ACC_SUM(ea_top, ea_prev ? e_0 - ea_prev : 0);
             if (b != dsum_b) {
                 flush_inertia();
                 dsum_b = b;
             }
             // the row margins are there long before the accumulator is: fetch them while waiting for it
             // (the X buffer is not refilled before the issuer's MMAs on it have completed either)
-            const uint32_t axb = tile_it % static_cast<uint32_t>(p.n_xbuf);
-            const uint32_t axph = (tile_it / static_cast<uint32_t>(p.n_xbuf)) & 1u;
-            float rowM = 0.f;
-            if (!XSPLIT) {
-                ok = wait_bar(&ctrl->auga_full[axb], axph, ctrl, p.status);
-                if (!ok) break;
-                rowM = ctrl->row_m[axb][r];
-                __syncwarp();
-                if (FUSE && lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
-            }
+            ACC_T(e_1);
             const uint32_t as = tile_it & 1u, aph = (tile_it >> 1) & 1u;
             ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
             if (!ok) break;
-            // (the MMAs that read the X buffer are complete: this arrival hands it back for them as well)
-            if (!XSPLIT && !FUSE && lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[axb]));
-            if (XSPLIT) {
-                // one X buffer for both warpgroups: this one sees only every other phase of its barriers, so it
-                // reads the margins once its accumulator is complete (the issuer waited for them)
-                rowM = ctrl->row_m[0][r];
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[0]));
-            }
+            ACC_T(e_2);
+            // The row margins: written by the norm warps before they completed auga_full, which the issuer waited for
+            // before the tile's last MMA, so they are there once the accumulator is complete (no wait of this warp's own).
+            // The X buffer, and with it this slot, is handed to a later row tile only after this warp's arrival (the
+            // norm warps could otherwise get two row tiles of the buffer ahead and overwrite the margins); the MMAs
+            // that read the buffer are complete as well, so outside FUSE and XSPLIT (where the update's or the
+            // issuers' commits do that) the arrival also stands for them.
+            const uint32_t mxb = XSPLIT ? 0u : axb;
+            const float rowM = ctrl->row_m[mxb][r];
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[mxb]));
             ptx::tc_fence_after();
             float best = __uint_as_float(F32_INF);
             int bsel = 0;
@@ -1211,6 +1213,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 bval = best;
                 bidx = bsel;
             }
+            ACC_T(e_3);
             const i64 row = static_cast<i64>(mt) * BLOCK_M + r;
             if (row < p.N) {
                 const size_t o = static_cast<size_t>(b) * static_cast<size_t>(p.N) + row;
@@ -1219,6 +1222,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 if (p.out_dist) p.out_dist[o] = dist;
                 dsum += static_cast<double>(dist);
             }
+            if (!XSPLIT) {
+                axb += 2u;
+                if (axb >= static_cast<uint32_t>(p.n_xbuf)) axb -= static_cast<uint32_t>(p.n_xbuf);
+            }
+            ACC_T(e_4);
+            ACC_SUM(ea_n, 1); ACC_SUM(ea_w1, e_1 - e_0); ACC_SUM(ea_w2, e_2 - e_1); ACC_SUM(ea_red, e_3 - e_2); ACC_SUM(ea_st, e_4 - e_3);
+            ACC_SET(ea_prev, e_4);
             if (FUSE) {
                 // The one-hot operand of this tile: element [cluster][row] of a 128 x 128 bf16 tile, K-major with the
                 // 128-byte swizzle, two 64-row chunks.  The buffer is shared by both warpgroups (they alternate tiles):
@@ -1229,6 +1239,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     ok = wait_bar(&ctrl->oh_empty[pt & 1u], (pt >> 1) & 1u, ctrl, p.status);
                     if (!ok) break;
                 }
+                ACC_T(e_5);
                 const uint32_t ohb = p.fuse_oh2 ? static_cast<uint32_t>(wg) : 0u;
                 uint8_t* oh = smem + oh_off + ohb * OH_BYTES + (r >> 6) * X_CHUNK_BYTES + ((r & 7) << 1);
                 const int g8 = (r & 63) >> 3;          // 16-byte granule of the row inside its chunk
@@ -1245,7 +1256,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->oh_full[wg]));
+                ACC_T(e_6);
+                ACC_SUM(ea_w3, e_5 - e_4); ACC_SUM(ea_oh, e_6 - e_5);
+                ACC_SET(ea_prev, e_6);
             }
+        }
+        }
+        if (XLOAD && lane == 0 && (warp == 0 || warp == 4)) {
+            ACC_DUMP(16 + wg * 8 + 0, ea_n); ACC_DUMP(16 + wg * 8 + 1, ea_top); ACC_DUMP(16 + wg * 8 + 2, ea_w1); ACC_DUMP(16 + wg * 8 + 3, ea_w2);
+            ACC_DUMP(16 + wg * 8 + 4, ea_red); ACC_DUMP(16 + wg * 8 + 5, ea_st); ACC_DUMP(16 + wg * 8 + 6, ea_w3); ACC_DUMP(16 + wg * 8 + 7, ea_oh);
         }
         if (FUSE && ok && wg == 0) {
             // every tile has been added: the sums (clusters on the TMEM lanes, D columns) go out as this CTA's partial
