@@ -689,7 +689,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const uint32_t idesc_aug_n = ptx::umma_idesc_bf16(BLOCK_M, p.alt_epi ? p.alt_epi : BLOCK_N);
                 const uint32_t idesc_main_n = idesc_aug_n | ptx::UMMA_IDESC_NEGATE_B;
                 if (!XSPLIT && !FUSE && p.res_c == 1) {
-                    // One resident tile, whole X buffers (the fused update keeps the general loop below: it measured 3 % faster there): this loop is the thread's whole life and every row tile passes
+                    // One resident tile, whole X buffers (the fused update keeps the general loop below: it measured 3 % faster
+                    // there): this loop is the thread's whole life and every row tile passes
                     // through it, so it does as little as it can.  Buffer, phases and descriptors are stepped (no
                     // divisions); one wait covers X and its half-norm operand (the norm warps arrive on it after they
                     // have seen the X tile); the X buffer is handed back by the epilogue warpgroup once the accumulator
@@ -1049,7 +1050,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
         // (this warpgroup's X buffer is stepped, not divided out of the tile count: the loop is the warpgroup's critical
         // path; with a single buffer -- XSPLIT -- it is not used)
         uint32_t axb = static_cast<uint32_t>(wg) % static_cast<uint32_t>(p.n_xbuf);
-        ACC_DECL(ea_n); ACC_DECL(ea_w1); ACC_DECL(ea_w2); ACC_DECL(ea_red); ACC_DECL(ea_st); ACC_DECL(ea_w3); ACC_DECL(ea_oh); ACC_DECL(ea_top); ACC_DECL(ea_prev);
+        ACC_DECL(ea_n); ACC_DECL(ea_w1); ACC_DECL(ea_w2); ACC_DECL(ea_red); ACC_DECL(ea_st);
+        ACC_DECL(ea_w3); ACC_DECL(ea_oh); ACC_DECL(ea_top); ACC_DECL(ea_prev);
         // (the loop walks this warpgroup's own tiles only: every other one of the CTA's)
         if (XLOAD && p.alt_epi) {
         const uint32_t n_alt = static_cast<uint32_t>((p.total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
