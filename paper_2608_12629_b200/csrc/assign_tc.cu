@@ -1312,7 +1312,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 }
             }
         };
+        ACC_DECL(mt_n); ACC_DECL(mt_wait); ACC_DECL(mt_row0); ACC_DECL(mt_hold); ACC_DECL(mt_red); ACC_DECL(mt_end); ACC_DECL(mt_top); ACC_DECL(mt_prev);
         for (i64 tile = blockIdx.x; !(XLOAD && p.alt_epi) && ok && tile < p.total_tiles; tile += gridDim.x, ++tile_it, next_tile()) {
+            ACC_T(m_0);
+            ACC_SUM(mt_top, mt_prev ? m_0 - mt_prev : 0);
+            ACC_SUM(mt_n, 1);
             if (TOPK) {
 #pragma unroll
                 for (int s = 0; s < KL; ++s) {
@@ -1329,8 +1333,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             float rowM = 0.f;                        // this row's margin m (wg 0 only)
             for (int nt = 0; nt < p.n_tiles; ++nt, ++acc_it) {
                 const uint32_t as = acc_it & 1u, aph = (acc_it >> 1) & 1u;
+                ACC_T(m_1);
                 ok = wait_bar(&ctrl->tmem_full[as], aph, ctrl, p.status);
                 if (!ok) break;
+                ACC_T(m_2);
+                ACC_SUM(mt_wait, m_2 - m_1);
                 ptx::tc_fence_after();
                 if (nt == 0 && (wg == 0 || TOPK)) {
                     // Written by the norm warps before they completed auga_full.  The X buffer -- and with
@@ -1344,6 +1351,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->x_empty[exb]));
                 }
+                ACC_T(m_3);
+                ACC_SUM(mt_row0, m_3 - m_2);
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                        as * BLOCK_N + wg * (BLOCK_N / 2);
                 if (TOPK) {
@@ -1393,6 +1402,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         // to the issuer of tile acc_it + 2, which takes this accumulator next
                         if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
                         trace_mark(ctrl, 100);
+                        ACC_T(m_4); ACC_SUM(mt_hold, m_4 - m_3); ACC_SET(mt_prev, m_4);
                         tmin = group_min32<GATE>(rb, 96, tmin, thr, kmask);
                         // across tiles only the (truncated) value decides: an equal value keeps the earlier tile
                         if (__uint_as_float(__float_as_uint(tmin) & ~COL_MASK) <
@@ -1414,6 +1424,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
                         trace_mark(ctrl, 100);
+                        ACC_T(m_4); ACC_SUM(mt_hold, m_4 - m_3); ACC_SET(mt_prev, m_4);
                         exact_scan32(rb, col0 + 96, best, bsel);
                     }
                 } else {
@@ -1433,6 +1444,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[as][next_iss]));
                     trace_mark(ctrl, 100);
+                    ACC_T(m_4); ACC_SUM(mt_hold, m_4 - m_3); ACC_SET(mt_prev, m_4);
                     if (PACKED) {
                         const float thr = __uint_as_float(__float_as_uint(best) & ~COL_MASK);
                         float tmin = group_min32<GATE>(ra, 0, __uint_as_float(F32_INF), thr, kmask);
@@ -1453,6 +1465,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     }
                 }
                 next_iss = (next_iss + 1 == n_iss) ? 0 : next_iss + 1;
+                ACC_T(m_5);
+                ACC_SUM(mt_red, mt_prev ? m_5 - mt_prev : 0);
+                ACC_SET(mt_prev, m_5);
             }
             if (!ok) break;
             trace_mark(ctrl, 102);
@@ -1513,6 +1528,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 }
             }
             trace_mark(ctrl, 103);
+            ACC_T(m_6);
+            ACC_SUM(mt_end, mt_prev ? m_6 - mt_prev : 0);
+            ACC_SET(mt_prev, m_6);
+        }
+        if (!(XLOAD && p.alt_epi) && lane == 0 && (warp == 0 || warp == 4)) {
+            ACC_DUMP(16 + wg * 8 + 0, mt_n); ACC_DUMP(16 + wg * 8 + 1, mt_top); ACC_DUMP(16 + wg * 8 + 2, mt_wait); ACC_DUMP(16 + wg * 8 + 3, mt_row0);
+            ACC_DUMP(16 + wg * 8 + 4, mt_hold); ACC_DUMP(16 + wg * 8 + 5, mt_red); ACC_DUMP(16 + wg * 8 + 6, mt_end);
         }
         if (ok) flush_inertia();
     }
