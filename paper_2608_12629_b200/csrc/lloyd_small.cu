@@ -253,11 +253,24 @@ lloyd_small_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
         const cake_bf16* src = it == 0 ? p.C0 : p.cbuf;
         // ---- this iteration's centroids into shared memory, K-major with the 128-byte swizzle the MMA reads (rows K ..
         // c_rows - 1 are zeros).  Loads that bypass L1: after the first iteration other CTAs wrote these rows in this launch.
-        for (int e = tid; e < p.c_rows * gpr; e += THREADS) {
-            const int k = e / gpr, g = e - k * gpr;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (k < p.K) v = __ldcg(reinterpret_cast<const uint4*>(src + static_cast<size_t>(k) * p.D) + g);
-            *reinterpret_cast<uint4*>(smem + c_off + (g >> 3) * C_CHUNK_BYTES + k * 128 + (((g & 7) ^ (k & 7)) << 4)) = v;
+        // (eight loads of a thread are requested before the first is stored: one L2 latency per batch, not per load)
+        constexpr int CBATCH = 8;
+        for (int e0 = tid; e0 < p.c_rows * gpr; e0 += THREADS * CBATCH) {
+            uint4 v[CBATCH];
+#pragma unroll
+            for (int u = 0; u < CBATCH; ++u) {
+                const int e = e0 + u * THREADS;
+                const int k = e / gpr, g = e - k * gpr;
+                v[u] = make_uint4(0, 0, 0, 0);
+                if (e < p.c_rows * gpr && k < p.K) v[u] = __ldcg(reinterpret_cast<const uint4*>(src + static_cast<size_t>(k) * p.D) + g);
+            }
+#pragma unroll
+            for (int u = 0; u < CBATCH; ++u) {
+                const int e = e0 + u * THREADS;
+                const int k = e / gpr, g = e - k * gpr;
+                if (e < p.c_rows * gpr)
+                    *reinterpret_cast<uint4*>(smem + c_off + (g >> 3) * C_CHUNK_BYTES + k * 128 + (((g & 7) ^ (k & 7)) << 4)) = v[u];
+            }
         }
         ctrl->cnt[tid] = 0;
         __syncthreads();
@@ -405,6 +418,9 @@ lloyd_small_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
         for (int k = blockIdx.x; k < p.K; k += gridDim.x) {
             const int col = tid % D4, stripe = tid / D4;
             // (all loads of a stripe are requested before the first is added: the loop is a chain of L2 latencies otherwise)
+            // (the counts are requested first: their loads are in flight together with the sums')
+            int cn0 = tid < n_part ? __ldcg(p.part_counts + static_cast<size_t>(tid) * 128 + k) : 0;
+            int cn1 = tid + THREADS < n_part ? __ldcg(p.part_counts + static_cast<size_t>(tid + THREADS) * 128 + k) : 0;
             float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
             const float4* prow = reinterpret_cast<const float4*>(p.part_sums + static_cast<size_t>(k) * p.ncol) + col;
             const size_t pstep = static_cast<size_t>(128) * p.ncol / 4;
@@ -419,8 +435,8 @@ lloyd_small_kernel(const __grid_constant__ CUtensorMap tmap_x, const Params p) {
 #pragma unroll
                 for (int u = 0; u < BATCH; ++u) { acc4.x += v[u].x; acc4.y += v[u].y; acc4.z += v[u].z; acc4.w += v[u].w; }
             }
-            int cn = 0;
-            for (int q = tid; q < n_part; q += THREADS) cn += __ldcg(p.part_counts + static_cast<size_t>(q) * 128 + k);
+            int cn = cn0 + cn1;
+            for (int q = tid + 2 * THREADS; q < n_part; q += THREADS) cn += __ldcg(p.part_counts + static_cast<size_t>(q) * 128 + k);
             ctrl->red[tid] = acc4;
             ctrl->cred[tid] = cn;
             __syncthreads();

@@ -1197,14 +1197,26 @@ finalize_partials_kernel(const float* __restrict__ part_sums, const int* __restr
     const int t = threadIdx.x;
     const int stripes = 256 / D4;            // D4 <= 32: at least 8 stripes of partials
     const int col = t % D4, stripe = t / D4;
+    // (the partials come from L2: all loads of a thread are requested before the first is added -- counts first -- so
+    // that the kernel pays one L2 latency per batch and not one per partial; same order of additions)
+    int cnt = t < n_cnt ? part_counts[static_cast<size_t>(t) * 128 + k] : 0;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (stripe < stripes)
-        for (int p = stripe; p < n_part; p += stripes) {
-            const float4 v = *reinterpret_cast<const float4*>(part_sums + (static_cast<size_t>(p) * 128 + k) * pitch + col * 4);
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    if (stripe < stripes) {
+        constexpr int BATCH = 10;
+        const float* base = part_sums + static_cast<size_t>(k) * pitch + col * 4;
+        const size_t pstep = static_cast<size_t>(128) * pitch;
+        for (int p0 = stripe; p0 < n_part; p0 += BATCH * stripes) {
+            float4 v[BATCH];
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) {
+                const int p = p0 + u * stripes;
+                v[u] = p < n_part ? *reinterpret_cast<const float4*>(base + static_cast<size_t>(p) * pstep) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
         }
-    int cnt = 0;
-    for (int p = t; p < n_cnt; p += 256) cnt += part_counts[static_cast<size_t>(p) * 128 + k];
+    }
+    for (int p = t + 256; p < n_cnt; p += 256) cnt += part_counts[static_cast<size_t>(p) * 128 + k];
     red[t] = acc;
     cred[t] = cnt;
     __syncthreads();
